@@ -1,0 +1,431 @@
+/*
+ * CPU oracle for low-precision fast bilinear matrix multiplication.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what the
+ * method computes; tests, the smoke check and the benchmark's CPU-baseline leg are
+ * its only callers.  It shares no code with the CUDA library and the library never
+ * calls it.
+ *
+ * What is computed (paper Section 2.1, Eq. 1):
+ *     M_r  = ( sum_{i,l} u_{r,il} A_il ) ( sum_{l,j} v_{r,lj} B_lj ),  r = 1..R
+ *     C_ij = sum_r w_{r,ij} M_r
+ * with the block sums ROUNDED to the product dtype before they are multiplied
+ * (Section 2.3 / Appendix B.1: the schedule "rounds the block sums"), products and
+ * the final combination carried in high precision, and one rounding to the output
+ * dtype.  Sign variants and the general gauge are the coefficient transforms of
+ * Section 2.1.  The stability criteria follow Appendix B.1; the certificate
+ * constants L_A, L_B, L_W follow Section 4.2.
+ *
+ * Precision choices (each is a stated reading, the paper being silent):
+ *   - coefficients are held in fp64 and used as (double)(float)c;
+ *   - a block sum is the decision that produces a quantised code, so it is formed
+ *     in the precision the kernel uses: an fp32 fused-multiply-add chain over the
+ *     nonzero coefficients in ascending row-major (i,l) order, then ONE rounding to
+ *     the product dtype (after an exact power-of-two scale for e4m3);
+ *   - products, decode, classical and exact references accumulate in fp64, in
+ *     ascending inner index t and ascending product index r;
+ *   - with product dtype "f64" nothing is rounded at all (exact-arithmetic mode,
+ *     used to pin the Brent equations and gauge invariance).
+ *
+ * Pins (see tests): printed Strassen example values, Brent equations on integer
+ * matrices, identity/sign gauges, printed constants (L_A=L_B=4, L_W=16, Phi=1024,
+ * nnz=432), the same-offset row leak pattern, brute-force triple loops.
+ * Parity unpinned: the error-amplification ratios at the benchmark workloads (the
+ * paper prints none for synthetic inputs of these shapes).
+ *
+ * All matrices are dense row-major arrays of double.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <float.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORC_F32 = 0, ORC_BF16 = 1, ORC_E4M3 = 2, ORC_F64 = 3 };
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------- */
+/* Rounding of a real (held in a double) to a binary floating-point format,    */
+/* written from the format definitions: p significant bits (implicit bit        */
+/* included), minimum normal exponent emin, round to nearest, ties to even,    */
+/* gradual underflow.  x/q and rint(x/q)*q are exact because q is a power of    */
+/* two, so the only rounding is rint's (current mode: to nearest even).        */
+/* ------------------------------------------------------------------------- */
+static double round_to_format(double x, int p, int emin) {
+  if (x == 0.0 || isnan(x) || isinf(x)) return x;
+  int e;
+  (void)frexp(x, &e);      /* |x| = f * 2^e, f in [0.5,1)  =>  floor(log2|x|) = e-1 */
+  e -= 1;
+  if (e < emin) e = emin;  /* subnormal range: fixed quantum */
+  double q = ldexp(1.0, e - p + 1);
+  return rint(x / q) * q;
+}
+
+/* bf16: 8 significant bits, fp32 exponent range, overflow to infinity (IEEE).   */
+static double round_bf16(double x) {
+  double y = round_to_format(x, 8, -126);
+  const double maxv = (2.0 - ldexp(1.0, -7)) * ldexp(1.0, 127);
+  if (fabs(y) > maxv && !isinf(x)) return copysign(INFINITY, x);
+  return y;
+}
+
+/* fp32: 24 significant bits.                                                    */
+static double round_f32(double x) { return (double)(float)x; }
+
+/* e4m3 (OCP E4M3, finite-only): 4 significant bits (Appendix D, "p = 4"), bias 7
+ * so emin = -6 and the least subnormal is 2^-9, largest finite 448; conversions
+ * saturate to +-448 (also from infinity); NaN stays NaN.                        */
+static double round_e4m3(double x) {
+  if (isnan(x)) return x;
+  if (isinf(x)) return copysign(448.0, x);
+  double y = round_to_format(x, 4, -6);
+  if (fabs(y) > 448.0) return copysign(448.0, x);
+  return y;
+}
+
+double orc_round(double x, int fmt) {
+  switch (fmt) {
+    case ORC_F32: return round_f32(x);
+    case ORC_BF16: return round_bf16(x);
+    case ORC_E4M3: return round_e4m3(x);
+    default: return x;
+  }
+}
+
+void orc_round_array(const double* x, double* y, int64_t n, int fmt) {
+  for (int64_t i = 0; i < n; ++i) y[i] = orc_round(x[i], fmt);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Coefficient algebra (host fp64).  U is [R][m][k], V is [R][k][n], W is       */
+/* [R][m][n]; w is indexed by the C block it feeds (Eq. 1).                     */
+/* ------------------------------------------------------------------------- */
+
+/* Largest violation of the Brent equations
+ *   sum_r u_{r,il} v_{r,l'j} w_{r,i'j'} = [i=i'][l=l'][j=j'],
+ * which is what "every unwanted cross term cancels" (Section 2.1) means.       */
+double orc_brent_max_residual(int m, int k, int n, int R, const double* U, const double* V,
+                              const double* W) {
+  double worst = 0.0;
+  for (int i = 0; i < m; ++i)
+    for (int l = 0; l < k; ++l)
+      for (int l2 = 0; l2 < k; ++l2)
+        for (int j = 0; j < n; ++j)
+          for (int i2 = 0; i2 < m; ++i2)
+            for (int j2 = 0; j2 < n; ++j2) {
+              double s = 0.0;
+              for (int r = 0; r < R; ++r)
+                s += U[(r * m + i) * k + l] * V[(r * k + l2) * n + j] * W[(r * m + i2) * n + j2];
+              double want = (i == i2 && l == l2 && j == j2) ? 1.0 : 0.0;
+              double d = fabs(s - want);
+              if (d > worst) worst = d;
+            }
+  return worst;
+}
+
+/* Nesting: the outer algorithm applied to blocks that are themselves multiplied by
+ * the inner one ("Strassen's algorithm applied to its own blocks", Section 1).
+ * Block rows are contiguous: global block index = outer*inner_dim + inner
+ * (Section 3.2: rows split into four contiguous blocks); product index
+ * r = r1*R2 + r2.                                                               */
+void orc_kron(int m1, int k1, int n1, int R1, const double* U1, const double* V1, const double* W1,
+              int m2, int k2, int n2, int R2, const double* U2, const double* V2, const double* W2,
+              double* U, double* V, double* W) {
+  int m = m1 * m2, k = k1 * k2, n = n1 * n2;
+  for (int r1 = 0; r1 < R1; ++r1)
+    for (int r2 = 0; r2 < R2; ++r2) {
+      int r = r1 * R2 + r2;
+      for (int I = 0; I < m1; ++I) for (int i = 0; i < m2; ++i)
+        for (int L = 0; L < k1; ++L) for (int l = 0; l < k2; ++l)
+          U[(r * m + I * m2 + i) * k + L * k2 + l] = U1[(r1 * m1 + I) * k1 + L] * U2[(r2 * m2 + i) * k2 + l];
+      for (int L = 0; L < k1; ++L) for (int l = 0; l < k2; ++l)
+        for (int J = 0; J < n1; ++J) for (int j = 0; j < n2; ++j)
+          V[(r * k + L * k2 + l) * n + J * n2 + j] = V1[(r1 * k1 + L) * n1 + J] * V2[(r2 * k2 + l) * n2 + j];
+      for (int I = 0; I < m1; ++I) for (int i = 0; i < m2; ++i)
+        for (int J = 0; J < n1; ++J) for (int j = 0; j < n2; ++j)
+          W[(r * m + I * m2 + i) * n + J * n2 + j] = W1[(r1 * m1 + I) * n1 + J] * W2[(r2 * m2 + i) * n2 + j];
+    }
+}
+
+/* Inverse of a small d x d matrix by Gauss-Jordan elimination with partial
+ * pivoting.  Returns 0 on success, 1 if a pivot vanishes.                       */
+static int invert_small(int d, const double* X, double* Xi) {
+  double a[16 * 32];
+  if (d > 16) return 1;
+  for (int i = 0; i < d; ++i)
+    for (int j = 0; j < d; ++j) {
+      a[i * 2 * d + j] = X[i * d + j];
+      a[i * 2 * d + d + j] = (i == j) ? 1.0 : 0.0;
+    }
+  for (int c = 0; c < d; ++c) {
+    int piv = c;
+    for (int i = c + 1; i < d; ++i)
+      if (fabs(a[i * 2 * d + c]) > fabs(a[piv * 2 * d + c])) piv = i;
+    if (a[piv * 2 * d + c] == 0.0) return 1;
+    if (piv != c)
+      for (int j = 0; j < 2 * d; ++j) {
+        double t = a[c * 2 * d + j]; a[c * 2 * d + j] = a[piv * 2 * d + j]; a[piv * 2 * d + j] = t;
+      }
+    double inv = 1.0 / a[c * 2 * d + c];
+    for (int j = 0; j < 2 * d; ++j) a[c * 2 * d + j] *= inv;
+    for (int i = 0; i < d; ++i) {
+      if (i == c) continue;
+      double f = a[i * 2 * d + c];
+      if (f == 0.0) continue;
+      for (int j = 0; j < 2 * d; ++j) a[i * 2 * d + j] -= f * a[c * 2 * d + j];
+    }
+  }
+  for (int i = 0; i < d; ++i)
+    for (int j = 0; j < d; ++j) Xi[i * d + j] = a[i * 2 * d + d + j];
+  return 0;
+}
+
+/* Gauge transform.  AB = P^-1 (P A Q^-1)(Q B S^-1) S with P, Q, S acting on block
+ * indices: running the algorithm on A' = P A Q^-1, B' = Q B S^-1 and mapping the
+ * result back is the algorithm with coefficients
+ *     U'_r = P^T U_r Q^-T,   V'_r = Q^T V_r S^-T,   W'_r = P^-1 W_r S
+ * (U_r read as an m x k matrix, and so on).  For diagonal sign matrices D, E, F this
+ * is d_i e_l u, e_l f_j v, d_i f_j w — the sign variants of Section 2.1; the general
+ * invertible case is the "larger set of equivalences" the same section mentions.
+ * Returns 1 if P, Q or S is singular.                                           */
+int orc_gauge(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+              const double* P, const double* Q, const double* S, double* Ug, double* Vg, double* Wg) {
+  double Pi[256], Qi[256], Si[256];
+  if (m > 16 || k > 16 || n > 16) return 1;
+  if (invert_small(m, P, Pi) || invert_small(k, Q, Qi) || invert_small(n, S, Si)) return 1;
+  for (int r = 0; r < R; ++r) {
+    /* U'_r[a][b] = sum_{i,l} P[i][a] U_r[i][l] Qi[b][l] */
+    for (int a = 0; a < m; ++a)
+      for (int b = 0; b < k; ++b) {
+        double s = 0.0;
+        for (int i = 0; i < m; ++i)
+          for (int l = 0; l < k; ++l) s += P[i * m + a] * U[(r * m + i) * k + l] * Qi[b * k + l];
+        Ug[(r * m + a) * k + b] = s;
+      }
+    /* V'_r[a][b] = sum_{l,j} Q[l][a] V_r[l][j] Si[b][j] */
+    for (int a = 0; a < k; ++a)
+      for (int b = 0; b < n; ++b) {
+        double s = 0.0;
+        for (int l = 0; l < k; ++l)
+          for (int j = 0; j < n; ++j) s += Q[l * k + a] * V[(r * k + l) * n + j] * Si[b * n + j];
+        Vg[(r * k + a) * n + b] = s;
+      }
+    /* W'_r[a][b] = sum_{i,j} Pi[a][i] W_r[i][j] S[j][b] */
+    for (int a = 0; a < m; ++a)
+      for (int b = 0; b < n; ++b) {
+        double s = 0.0;
+        for (int i = 0; i < m; ++i)
+          for (int j = 0; j < n; ++j) s += Pi[a * m + i] * W[(r * m + i) * n + j] * S[j * n + b];
+        Wg[(r * m + a) * n + b] = s;
+      }
+  }
+  return 0;
+}
+
+/* Criteria and certificate constants.
+ * meta[0]=L_A = max_r sum|u_r|, meta[1]=L_B, meta[2]=L_W = max_ij sum_r |w_{r,ij}|
+ * (Section 4.2); meta[3]=Phi = sum_r |u_r|_2^2 |v_r|_2^2 |w_r|_2^2, meta[4]=number of
+ * nonzero coefficients over U,V,W, meta[5]=largest |coefficient|,
+ * meta[6]=Q = max_ij( gamma_ij + max_{r: w!=0}(alpha_r+beta_r) ),
+ * meta[7]=E = max_ij sum_r a_r b_r |w_{r,ij}|  (Appendix B.1).                  */
+void orc_criteria(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                  double* meta) {
+  double LA = 0, LB = 0, LW = 0, Phi = 0, nnz = 0, mx = 0, Qc = 0, Ec = 0;
+  double* a1 = (double*)calloc(R, sizeof(double));
+  double* b1 = (double*)calloc(R, sizeof(double));
+  double* al = (double*)calloc(R, sizeof(double));
+  double* be = (double*)calloc(R, sizeof(double));
+  for (int r = 0; r < R; ++r) {
+    double u2 = 0, v2 = 0, w2 = 0;
+    for (int x = 0; x < m * k; ++x) {
+      double c = U[r * m * k + x];
+      a1[r] += fabs(c); u2 += c * c; if (c != 0) { al[r] += 1; nnz += 1; } if (fabs(c) > mx) mx = fabs(c);
+    }
+    for (int x = 0; x < k * n; ++x) {
+      double c = V[r * k * n + x];
+      b1[r] += fabs(c); v2 += c * c; if (c != 0) { be[r] += 1; nnz += 1; } if (fabs(c) > mx) mx = fabs(c);
+    }
+    for (int x = 0; x < m * n; ++x) {
+      double c = W[r * m * n + x];
+      w2 += c * c; if (c != 0) nnz += 1; if (fabs(c) > mx) mx = fabs(c);
+    }
+    if (a1[r] > LA) LA = a1[r];
+    if (b1[r] > LB) LB = b1[r];
+    Phi += u2 * v2 * w2;
+  }
+  for (int x = 0; x < m * n; ++x) {
+    double lw = 0, gamma = 0, ab = 0, e = 0;
+    for (int r = 0; r < R; ++r) {
+      double c = W[r * m * n + x];
+      lw += fabs(c);
+      e += a1[r] * b1[r] * fabs(c);
+      if (c != 0) { gamma += 1; if (al[r] + be[r] > ab) ab = al[r] + be[r]; }
+    }
+    if (lw > LW) LW = lw;
+    if (gamma + ab > Qc) Qc = gamma + ab;
+    if (e > Ec) Ec = e;
+  }
+  meta[0] = LA; meta[1] = LB; meta[2] = LW; meta[3] = Phi; meta[4] = nnz; meta[5] = mx;
+  meta[6] = Qc; meta[7] = Ec;
+  free(a1); free(b1); free(al); free(be);
+}
+
+/* ------------------------------------------------------------------------- */
+/* The realisation: encode -> R products -> decode.                            */
+/* ------------------------------------------------------------------------- */
+
+/* One block sum, Eq. 1 inner parentheses: out[p][t] = sum_x coef[x] * blk_x[p][t] over the
+ * nonzero coefficients in ascending x (row-major over the block grid).
+ * src is the whole matrix (ld elements per row); block x = (x / gc, x % gc) of a grid with gc
+ * block columns, block size br x bc.  f32chain selects the fp32 FMA chain (quantised modes) or
+ * a plain fp64 sum (exact mode).                                                   */
+static void block_sum(const double* src, int64_t ld, int gr, int gc, int64_t br, int64_t bc,
+                      const double* coef, int f32chain, double* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < br; ++p)
+    for (int64_t t = 0; t < bc; ++t) {
+      if (f32chain) {
+        float acc = 0.0f;
+        for (int x = 0; x < gr * gc; ++x) {
+          float c = (float)coef[x];
+          if (c == 0.0f) continue;
+          float a = (float)src[((int64_t)(x / gc) * br + p) * ld + (int64_t)(x % gc) * bc + t];
+          acc = fmaf(c, a, acc);
+        }
+        out[p * bc + t] = (double)acc;
+      } else {
+        double acc = 0.0;
+        for (int x = 0; x < gr * gc; ++x) {
+          double c = coef[x];
+          if (c == 0.0) continue;
+          acc += c * src[((int64_t)(x / gc) * br + p) * ld + (int64_t)(x % gc) * bc + t];
+        }
+        out[p * bc + t] = acc;
+      }
+    }
+}
+
+/* Per-tensor power-of-two scale of an encoded operand for e4m3 (reading: one scale per
+ * encoded tensor, s = 2^ceil(log2(amax/448)), s = 1 if the tensor is all zero).   */
+static double pow2_scale_448(const double* x, int64_t n) {
+  double amax = 0.0;
+  for (int64_t i = 0; i < n; ++i) { double a = fabs(x[i]); if (a > amax) amax = a; }
+  if (amax == 0.0 || isnan(amax) || isinf(amax)) return 1.0;
+  int e;
+  double f = frexp(amax / 448.0, &e);   /* amax/448 = f*2^e, f in [0.5,1) */
+  if (f == 0.5) e -= 1;                 /* exact power of two: ceil(log2) = e-1 */
+  return ldexp(1.0, e);
+}
+
+/* C = A_hat * B_hat in fp64, ascending inner index (i-k-j loop order).             */
+static void matmul_f64(const double* A, const double* B, double* C, int64_t M, int64_t K, int64_t N) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < M; ++i) {
+    double* c = C + i * N;
+    for (int64_t j = 0; j < N; ++j) c[j] = 0.0;
+    for (int64_t t = 0; t < K; ++t) {
+      double a = A[i * K + t];
+      const double* b = B + t * N;
+      for (int64_t j = 0; j < N; ++j) c[j] += a * b[j];
+    }
+  }
+}
+
+/* Apply an algorithm <m,k,n;R> to A (M x K) and B (K x N); C is M x N.
+ * pd = product dtype the block sums are rounded to, od = output dtype,
+ * scale_mode 0: no scales; 1: per-encoded-tensor power-of-two scale (e4m3).
+ * Optional outputs (may be NULL): Ahat [R][bm][bk], Bhat [R][bk][bn] (the rounded,
+ * scaled block sums), sA[R], sB[R], Mout [R][bm][bn] (the fp64 products).
+ * Returns 0, or 1 if a dimension does not divide.                                 */
+int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                    int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                    int pd, int od, int scale_mode, double* C,
+                    double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
+                    double* M_out) {
+  if (M % m || K % k || N % n) return 1;
+  int64_t bm = M / m, bk = K / k, bn = N / n;
+  int quant = (pd != ORC_F64);
+  double* Ah = (double*)malloc(sizeof(double) * bm * bk);
+  double* Bh = (double*)malloc(sizeof(double) * bk * bn);
+  double* Mr = (double*)malloc(sizeof(double) * bm * bn);
+  double* acc = (double*)calloc((size_t)M * N, sizeof(double));
+  double* cu = (double*)malloc(sizeof(double) * m * k);
+  double* cv = (double*)malloc(sizeof(double) * k * n);
+  for (int r = 0; r < R; ++r) {
+    /* coefficients as the kernel sees them: fp32 values (exact mode keeps fp64) */
+    for (int x = 0; x < m * k; ++x) cu[x] = quant ? (double)(float)U[r * m * k + x] : U[r * m * k + x];
+    for (int x = 0; x < k * n; ++x) cv[x] = quant ? (double)(float)V[r * k * n + x] : V[r * k * n + x];
+    /* encode: block sums, scale, one rounding to the product dtype */
+    block_sum(A, K, m, k, bm, bk, cu, quant, Ah);
+    block_sum(B, N, k, n, bk, bn, cv, quant, Bh);
+    double sa = 1.0, sb = 1.0;
+    if (scale_mode == 1) { sa = pow2_scale_448(Ah, bm * bk); sb = pow2_scale_448(Bh, bk * bn); }
+    if (quant) {
+      for (int64_t x = 0; x < bm * bk; ++x) Ah[x] = orc_round(Ah[x] / sa, pd);
+      for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x] / sb, pd);
+    }
+    if (Ahat_out) memcpy(Ahat_out + (size_t)r * bm * bk, Ah, sizeof(double) * bm * bk);
+    if (Bhat_out) memcpy(Bhat_out + (size_t)r * bk * bn, Bh, sizeof(double) * bk * bn);
+    if (sA_out) sA_out[r] = sa;
+    if (sB_out) sB_out[r] = sb;
+    /* product */
+    matmul_f64(Ah, Bh, Mr, bm, bk, bn);
+    if (M_out) memcpy(M_out + (size_t)r * bm * bn, Mr, sizeof(double) * bm * bn);
+    /* decode, ascending r: C_ij += w_{r,ij} * (sA_r sB_r) * M_r */
+    for (int i = 0; i < m; ++i)
+      for (int j = 0; j < n; ++j) {
+        double w = quant ? (double)(float)W[(r * m + i) * n + j] : W[(r * m + i) * n + j];
+        if (w == 0.0) continue;
+        double ws = w * (sa * sb);
+#pragma omp parallel for schedule(static)
+        for (int64_t p = 0; p < bm; ++p)
+          for (int64_t q = 0; q < bn; ++q)
+            acc[(i * bm + p) * N + j * bn + q] += ws * Mr[p * bn + q];
+      }
+  }
+  for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x], od);
+  free(Ah); free(Bh); free(Mr); free(acc); free(cu); free(cv);
+  return 0;
+}
+
+/* Classical product at the same dtypes (the control): operands rounded to the product
+ * dtype (after a per-tensor power-of-two scale in scale_mode 1), fp64 accumulation,
+ * one rounding to the output dtype.                                                */
+int orc_classical_gemm(int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                       int pd, int od, int scale_mode, double* C) {
+  double* Ah = (double*)malloc(sizeof(double) * M * K);
+  double* Bh = (double*)malloc(sizeof(double) * K * N);
+  double* acc = (double*)malloc(sizeof(double) * M * N);
+  double sa = 1.0, sb = 1.0;
+  if (scale_mode == 1) { sa = pow2_scale_448(A, M * K); sb = pow2_scale_448(B, K * N); }
+  for (int64_t x = 0; x < M * K; ++x) Ah[x] = orc_round(A[x] / sa, pd);
+  for (int64_t x = 0; x < K * N; ++x) Bh[x] = orc_round(B[x] / sb, pd);
+  matmul_f64(Ah, Bh, acc, M, K, N);
+  for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x] * (sa * sb), od);
+  free(Ah); free(Bh); free(acc);
+  return 0;
+}
+
+/* Exact reference: the fp64 product of the stored operand values (Appendix B.1:
+ * "a float64 reference").                                                        */
+void orc_exact_gemm(int64_t M, int64_t K, int64_t N, const double* A, const double* B, double* C) {
+  matmul_f64(A, B, C, M, K, N);
+}
+
+/* Squared Frobenius error and reference norm: out[0] = sum (C-Cs)^2, out[1] = sum Cs^2. */
+void orc_fro_err(const double* C, const double* Cs, int64_t n, double* out) {
+  double e = 0.0, s = 0.0;
+  for (int64_t i = 0; i < n; ++i) { double d = C[i] - Cs[i]; e += d * d; s += Cs[i] * Cs[i]; }
+  out[0] = e; out[1] = s;
+}

@@ -1,0 +1,282 @@
+"""Python face of the CPU oracle: ctypes over ``fmm_oracle.c`` plus the few host-side
+definitions that are clearer in numpy (the printed Strassen table, the sign-variant
+formula as printed, the summary statistics).
+
+TEST INFRASTRUCTURE ONLY — see the header of ``fmm_oracle.c``.  Nothing here imports
+the CUDA library; the library never imports this.
+
+Citations are to the paper's sections / equations / tables.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fmm_oracle.c")
+_SO = os.path.join(_HERE, "libfmm_oracle.so")
+
+F32, BF16, E4M3, F64 = 0, 1, 2, 3
+_FMT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3, "f64": F64, "fp64": F64}
+
+__all__ = [
+    "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "round_to", "strassen",
+    "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
+    "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
+    "error_ratio", "summary",
+]
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FP contraction)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O3", "-march=native", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-shared", "-fPIC", "-std=c11", "-o", _SO, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+_lib = None
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        lib = C.CDLL(build())
+        dp = C.POINTER(C.c_double)
+        i64 = C.c_int64
+        lib.orc_num_threads.restype = C.c_int
+        lib.orc_round.restype = C.c_double
+        lib.orc_round.argtypes = [C.c_double, C.c_int]
+        lib.orc_round_array.argtypes = [dp, dp, i64, C.c_int]
+        lib.orc_brent_max_residual.restype = C.c_double
+        lib.orc_brent_max_residual.argtypes = [C.c_int] * 4 + [dp] * 3
+        lib.orc_kron.argtypes = [C.c_int] * 4 + [dp] * 3 + [C.c_int] * 4 + [dp] * 3 + [dp] * 3
+        lib.orc_gauge.restype = C.c_int
+        lib.orc_gauge.argtypes = [C.c_int] * 4 + [dp] * 9
+        lib.orc_criteria.argtypes = [C.c_int] * 4 + [dp] * 4
+        lib.orc_scheme_gemm.restype = C.c_int
+        lib.orc_scheme_gemm.argtypes = ([C.c_int] * 4 + [dp] * 3 + [i64] * 3 + [dp] * 2 +
+                                        [C.c_int] * 3 + [dp] * 6)
+        lib.orc_classical_gemm.restype = C.c_int
+        lib.orc_classical_gemm.argtypes = [i64] * 3 + [dp] * 2 + [C.c_int] * 3 + [dp]
+        lib.orc_exact_gemm.argtypes = [i64] * 3 + [dp] * 3
+        lib.orc_fro_err.argtypes = [dp, dp, i64, dp]
+        _lib = lib
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.POINTER(C.c_double))
+
+
+def _d(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+
+
+def _fmt(f):
+    return _FMT[f] if isinstance(f, str) else int(f)
+
+
+def num_threads() -> int:
+    return int(_L().orc_num_threads())
+
+
+def round_to(x, fmt):
+    """Round real value(s) to a storage format (round to nearest even; e4m3 saturates)."""
+    x = _d(x)
+    y = np.empty_like(x)
+    _L().orc_round_array(_p(x), _p(y), x.size, _fmt(fmt))
+    return y
+
+
+@dataclass(frozen=True)
+class Scheme:
+    """Coefficients of Eq. 1: U[R,m,k], V[R,k,n], W[R,m,n] (w indexed by the C block it feeds)."""
+    U: np.ndarray
+    V: np.ndarray
+    W: np.ndarray
+
+    @property
+    def dims(self):
+        R, m, k = self.U.shape
+        return m, k, self.V.shape[2], R
+
+
+def strassen() -> Scheme:
+    """Strassen's <2,2,2;7>, typed from the product table of Appendix A.1:
+    M1=(A11+A22)(B11+B22), M2=(A21+A22)B11, M3=A11(B12-B22), M4=A22(B21-B11),
+    M5=(A11+A12)B22, M6=(A21-A11)(B11+B12), M7=(A12-A22)(B21+B22);
+    C11=M1+M4-M5+M7, C12=M3+M5, C21=M2+M4, C22=M1-M2+M3+M6."""
+    U = np.zeros((7, 2, 2)); V = np.zeros((7, 2, 2)); W = np.zeros((7, 2, 2))
+    a = {(1, 1): (0, 0), (1, 2): (0, 1), (2, 1): (1, 0), (2, 2): (1, 1)}
+    prods = [
+        ([(1, 1, 1), (2, 2, 1)], [(1, 1, 1), (2, 2, 1)]),
+        ([(2, 1, 1), (2, 2, 1)], [(1, 1, 1)]),
+        ([(1, 1, 1)], [(1, 2, 1), (2, 2, -1)]),
+        ([(2, 2, 1)], [(2, 1, 1), (1, 1, -1)]),
+        ([(1, 1, 1), (1, 2, 1)], [(2, 2, 1)]),
+        ([(2, 1, 1), (1, 1, -1)], [(1, 1, 1), (1, 2, 1)]),
+        ([(1, 2, 1), (2, 2, -1)], [(2, 1, 1), (2, 2, 1)]),
+    ]
+    for r, (ua, vb) in enumerate(prods):
+        for (i, l, s) in ua:
+            U[(r,) + a[(i, l)]] = s
+        for (l, j, s) in vb:
+            V[(r,) + a[(l, j)]] = s
+    outs = {(1, 1): [(1, 1), (4, 1), (5, -1), (7, 1)], (1, 2): [(3, 1), (5, 1)],
+            (2, 1): [(2, 1), (4, 1)], (2, 2): [(1, 1), (2, -1), (3, 1), (6, 1)]}
+    for ij, terms in outs.items():
+        for (r, s) in terms:
+            W[(r - 1,) + a[ij]] = s
+    return Scheme(U, V, W)
+
+
+def classical_scheme(m: int, k: int, n: int) -> Scheme:
+    """The classical algorithm as a scheme: R = mkn products A_il B_lj (Section 2.1)."""
+    R = m * k * n
+    U = np.zeros((R, m, k)); V = np.zeros((R, k, n)); W = np.zeros((R, m, n))
+    r = 0
+    for i in range(m):
+        for l in range(k):
+            for j in range(n):
+                U[r, i, l] = 1; V[r, l, j] = 1; W[r, i, j] = 1
+                r += 1
+    return Scheme(U, V, W)
+
+
+def kron(outer: Scheme, inner: Scheme) -> Scheme:
+    """Nested algorithm (outer applied to blocks multiplied by inner); contiguous blocks."""
+    m1, k1, n1, R1 = outer.dims
+    m2, k2, n2, R2 = inner.dims
+    U = np.zeros((R1 * R2, m1 * m2, k1 * k2)); V = np.zeros((R1 * R2, k1 * k2, n1 * n2))
+    W = np.zeros((R1 * R2, m1 * m2, n1 * n2))
+    _L().orc_kron(m1, k1, n1, R1, _p(_d(outer.U)), _p(_d(outer.V)), _p(_d(outer.W)),
+                  m2, k2, n2, R2, _p(_d(inner.U)), _p(_d(inner.V)), _p(_d(inner.W)),
+                  _p(U), _p(V), _p(W))
+    return Scheme(U, V, W)
+
+
+def gauge(s: Scheme, P, Q, S) -> Scheme:
+    """General gauge: U'_r = P^T U_r Q^-T, V'_r = Q^T V_r S^-T, W'_r = P^-1 W_r S."""
+    m, k, n, R = s.dims
+    U = np.empty_like(_d(s.U)); V = np.empty_like(_d(s.V)); W = np.empty_like(_d(s.W))
+    rc = _L().orc_gauge(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)),
+                        _p(_d(P)), _p(_d(Q)), _p(_d(S)), _p(U), _p(V), _p(W))
+    if rc:
+        raise ValueError("singular gauge matrix")
+    return Scheme(U, V, W)
+
+
+def sign_variant(s: Scheme, d, e, f) -> Scheme:
+    """Sign variant exactly as Section 2.1 prints it: d_i e_l u, e_l f_j v, d_i f_j w."""
+    d = np.asarray(d, float); e = np.asarray(e, float); f = np.asarray(f, float)
+    U = s.U * d[None, :, None] * e[None, None, :]
+    V = s.V * e[None, :, None] * f[None, None, :]
+    W = s.W * d[None, :, None] * f[None, None, :]
+    return Scheme(U, V, W)
+
+
+def sign_variants(m: int, k: int, n: int):
+    """All (d, e, f) with d_1 = e_1 = f_1 = 1 (Section 2.1): 2^(m-1) 2^(k-1) 2^(n-1) triples."""
+    out = []
+    for a in range(2 ** (m - 1)):
+        d = [1.0] + [(-1.0 if (a >> b) & 1 else 1.0) for b in range(m - 1)]
+        for bb in range(2 ** (k - 1)):
+            e = [1.0] + [(-1.0 if (bb >> b) & 1 else 1.0) for b in range(k - 1)]
+            for c in range(2 ** (n - 1)):
+                f = [1.0] + [(-1.0 if (c >> b) & 1 else 1.0) for b in range(n - 1)]
+                out.append((np.array(d), np.array(e), np.array(f)))
+    return out
+
+
+def brent_residual(s: Scheme) -> float:
+    m, k, n, R = s.dims
+    return float(_L().orc_brent_max_residual(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W))))
+
+
+def criteria(s: Scheme) -> dict:
+    m, k, n, R = s.dims
+    meta = np.zeros(8)
+    _L().orc_criteria(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), _p(meta))
+    keys = ["L_A", "L_B", "L_W", "Phi", "nnz", "maxabs", "Q", "E"]
+    return dict(zip(keys, meta.tolist()))
+
+
+def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts: bool = False):
+    """Apply the algorithm with block sums rounded to ``pd``; returns C (values of ``od``).
+    With ``parts`` also returns dict(Ahat, Bhat, sA, sB, M)."""
+    m, k, n, R = s.dims
+    A = _d(A); B = _d(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    Cm = np.empty((M, N))
+    Ah = Bh = sA = sB = Mr = None
+    if parts:
+        bm, bk, bn = M // m, K // k, N // n
+        Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
+        sA = np.empty(R); sB = np.empty(R)
+    rc = _L().orc_scheme_gemm(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
+                              _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
+                              _p(sB), _p(Mr))
+    if rc:
+        raise ValueError("matrix dimensions are not divisible by the block grid")
+    if parts:
+        return Cm, dict(Ahat=Ah, Bhat=Bh, sA=sA, sB=sB, M=Mr)
+    return Cm
+
+
+def classical_gemm(A, B, pd="bf16", od="f32", scale_mode: int = 0):
+    A = _d(A); B = _d(B)
+    M, K = A.shape
+    N = B.shape[1]
+    Cm = np.empty((M, N))
+    _L().orc_classical_gemm(M, K, N, _p(A), _p(B), _fmt(pd), _fmt(od), int(scale_mode), _p(Cm))
+    return Cm
+
+
+def exact_gemm(A, B):
+    A = _d(A); B = _d(B)
+    M, K = A.shape
+    N = B.shape[1]
+    Cm = np.empty((M, N))
+    _L().orc_exact_gemm(M, K, N, _p(A), _p(B), _p(Cm))
+    return Cm
+
+
+def fro_err(Cm, Cs):
+    """(sum (C-C*)^2, sum C*^2) in fp64."""
+    Cm = _d(Cm); Cs = _d(Cs)
+    out = np.zeros(2)
+    _L().orc_fro_err(_p(Cm), _p(Cs), Cm.size, _p(out))
+    return float(out[0]), float(out[1])
+
+
+def rel_error(Cm, Cs) -> float:
+    """Relative error in the Frobenius norm against the float64 reference (Appendix B.1)."""
+    e, s = fro_err(Cm, Cs)
+    return math.sqrt(e / s) if s > 0 else (0.0 if e == 0 else math.inf)
+
+
+def error_ratio(E_scheme: float, E_classical: float) -> float:
+    """Error-amplification ratio rho = E_scheme / E_classical; 1 if both vanish, inf if only
+    the classical error vanishes."""
+    if E_classical == 0.0:
+        return 1.0 if E_scheme == 0.0 else math.inf
+    return E_scheme / E_classical
+
+
+def summary(ratios) -> dict:
+    """Smallest, median (upper of the two middle values when the count is even, Table 3
+    caption), largest, spread = largest/smallest, and the number of ratios above 2."""
+    r = np.sort(np.asarray(ratios, dtype=np.float64))
+    G = r.size
+    return dict(min=float(r[0]), median=float(r[G // 2]), max=float(r[-1]),
+                spread=float(r[-1] / r[0]) if r[0] > 0 else math.inf,
+                count_gt2=int(np.sum(r > 2.0)), G=int(G))
