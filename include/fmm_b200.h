@@ -1,0 +1,211 @@
+/*
+ * fmm_b200 — low-precision fast bilinear matrix multiplication on one B200 (sm_100a).
+ *
+ * C ABI.  No C++ or framework types cross this boundary: plain pointers and sizes only.
+ * Every pointer argument says whether it is HOST or DEVICE memory.
+ *
+ * The operation (paper Section 2.1, Eq. 1).  An algorithm <m,k,n;R> with coefficients
+ * U[R][m][k], V[R][k][n], W[R][m][n] splits A (M x K) into an m x k grid of blocks A_il
+ * and B (K x N) into a k x n grid B_lj (contiguous blocks, Section 3.2) and computes
+ *     Ahat_r = rnd_Pd( (sum_{i,l} u_{r,il} A_il) / sA_r )        "encode A"
+ *     Bhat_r = rnd_Pd( (sum_{l,j} v_{r,lj} B_lj) / sB_r )        "encode B"
+ *     M_r    = Ahat_r * Bhat_r                    (fp32 accumulation, tensor cores)
+ *     C_ij   = rnd_O( sum_r w_{r,ij} sA_r sB_r M_r )             "decode"
+ * The rounding of the block sums to the product dtype Pd is the step whose effect the
+ * paper studies (Section 2.3, Appendix B.1); products stay fp32 and are combined in fp32
+ * (Appendix B.1).  Coefficients are used as fp32 values of the fp64 numbers held in the
+ * handle.  Block sums are formed as an fp32 fused-multiply-add chain over the nonzero
+ * coefficients in ascending row-major (i,l) resp. (l,j) order; decode adds in ascending r.
+ *
+ * Conventions
+ *   - every call returns an fmm_status; nothing throws, aborts or prints;
+ *   - out-parameters are written only when FMM_OK is returned;
+ *   - scheme handles are created by the library (host memory only, no GPU needed),
+ *     are immutable, and are released with scheme_free; gauge/kron results are
+ *     independent objects;
+ *   - operand, result and workspace buffers are caller-owned DEVICE memory, 256-byte
+ *     aligned, row-major, leading dimensions in elements and a multiple of 16 bytes;
+ *   - calls that take a stream only enqueue work on it (no synchronisation, no device
+ *     allocation), except error_sweep, which synchronises the stream once at its end
+ *     because it returns host numbers;
+ *   - M % m, K % k, N % n must be 0, K/k must be a multiple of 16 and N/n a multiple
+ *     of 8 (FMM_ERR_SHAPE otherwise): zero padding is the caller's job, as in the paper
+ *     (Appendix B.2 pads 40 rows to 48);
+ *   - NaN/Inf in operands propagate; e4m3 conversion saturates at +-448.
+ */
+#ifndef FMM_B200_H
+#define FMM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fmm_scheme fmm_scheme; /* opaque, library-owned, immutable */
+
+typedef enum {
+  FMM_OK = 0,
+  FMM_ERR_ARG = 1,       /* null pointer, bad enum, bad size */
+  FMM_ERR_SHAPE = 2,     /* divisibility / alignment of M,K,N,ld* violated */
+  FMM_ERR_BRENT = 3,     /* coefficients do not satisfy the Brent equations within tolerance */
+  FMM_ERR_SINGULAR = 4,  /* gauge matrix singular or above the condition limit */
+  FMM_ERR_DTYPE = 5,     /* unsupported storage/product/output combination */
+  FMM_ERR_WORKSPACE = 6, /* workspace null, misaligned or too small */
+  FMM_ERR_CUDA = 7,      /* a CUDA runtime/driver call failed (incl. no device) */
+  FMM_ERR_TIMEOUT = 8,   /* a bounded device-side wait expired; results are invalid */
+  FMM_ERR_LIMIT = 9      /* scheme larger than the library's table limits */
+} fmm_status;
+
+typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
+
+/* Limits of the coefficient tables a handle may hold. */
+#define FMM_MAX_GRID 4    /* m, k, n <= 4 */
+#define FMM_MAX_R 64      /* R <= 64 */
+
+/* flags of fmm_gemm_desc */
+#define FMM_FLAG_REUSE_BHAT 1 /* the workspace already holds Bhat (and sB) written by an earlier
+                                 scheme_gemm call with the same scheme, desc and workspace: skip
+                                 "encode B".  Weights are static, so their block sums can be
+                                 formed once (the paper prepares weight block sums offline,
+                                 Section 3.1 / Appendix C).                                   */
+
+/* The float-path "quantisation specification" (Section 2.2 treats these choices as part of the
+ * operator): shapes, dtypes, layout of B, scale rule. */
+typedef struct {
+  int64_t M, K, N;       /* C[M x N] = A[M x K] * B[K x N] */
+  int64_t lda, ldb, ldc; /* leading dimensions in elements */
+  int32_t storage;       /* fmm_dtype of A and B in memory: FMM_F32 or FMM_BF16 */
+  int32_t product;       /* fmm_dtype the block sums are rounded to: FMM_BF16 or FMM_E4M3 */
+  int32_t output;        /* fmm_dtype of C: FMM_F32 or FMM_BF16 */
+  int32_t b_is_weight_layout; /* 0: B stored [K x N] (N contiguous); 1: B stored [N x K]
+                                 (K contiguous, the nn.Linear weight layout) */
+  int32_t scale_mode;    /* 0: no scales.  1 (e4m3 only): one power-of-two scale per encoded
+                            tensor, s = 2^ceil(log2(amax/448)), s = 1 for an all-zero tensor;
+                            classical_gemm uses one such scale per operand */
+  int32_t flags;         /* FMM_FLAG_* */
+} fmm_gemm_desc;
+
+/* Summary of a sweep (Table 3 caption: smallest, median = upper of the two middle values when the
+ * count is even, largest; spread = largest / smallest; number of ratios above 2). */
+typedef struct {
+  double min, median, max, spread;
+  int64_t count_gt2;
+  int64_t G;
+  double e_classical_rel; /* relative Frobenius error of the classical product vs fp64 */
+  double norm_ref;        /* Frobenius norm of the fp64 reference */
+} fmm_sweep_summary;
+
+/* ---- scheme handles (HOST only; usable without a GPU) ---------------------------------- */
+
+/* Create a handle from coefficient arrays U[R][m][k], V[R][k][n], W[R][m][n] (HOST, fp64,
+ * row-major; w indexed by the C block it feeds, Eq. 1).  The Brent equations (all unwanted
+ * cross terms cancel, Section 2.1) are checked: FMM_ERR_BRENT if the largest residual
+ * exceeds brent_tol * max(1, R * max|u| * max|v| * max|w|).  brent_tol <= 0 selects 1e-12.
+ * The arrays are copied.  FMM_ERR_LIMIT if m,k,n > FMM_MAX_GRID or R > FMM_MAX_R.       */
+fmm_status scheme_load(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                       double brent_tol, fmm_scheme** out);
+
+/* Built-in algorithms: "strassen222" (the seven products of the paper's Appendix A.1 table),
+ * "strassen444" (its nesting with itself, 49 products, Section 1), "classical111",
+ * "classical222" (the mkn-product classical algorithm written as a scheme).                */
+fmm_status scheme_builtin(const char* name, fmm_scheme** out);
+
+/* Nesting: `outer` applied to blocks multiplied by `inner`; block index = outer*dim_inner + inner
+ * (contiguous blocks, Section 3.2), product index r = r_outer * R_inner + r_inner.  The result
+ * remembers its factors (see gauge_apply, level 1).                                         */
+fmm_status scheme_kron(const fmm_scheme* outer, const fmm_scheme* inner, fmm_scheme** out);
+
+/* Gauge transform (Section 2.1).  With P[m][m], Q[k][k], S[n][n] (HOST, fp64, row-major,
+ * invertible):  U'_r = P^T U_r Q^-T,  V'_r = Q^T V_r S^-T,  W'_r = P^-1 W_r S, which for diagonal
+ * sign matrices D,E,F is the paper's sign variant d_i e_l u, e_l f_j v, d_i f_j w.
+ * level 0: P,Q,S act on the handle's own m x k x n grid.
+ * level 1: the handle must come from scheme_kron; P,Q,S have the OUTER factor's dimensions and
+ *          transform the outer factor only.
+ * FMM_ERR_SINGULAR if a matrix is singular or its 2-norm condition number exceeds cond_limit
+ * (cond_limit <= 0: no limit).  Sign gauges are exact: every operation on 0, +-1 entries is. */
+fmm_status gauge_apply(const fmm_scheme* in, int level, const double* P, const double* Q, const double* S,
+                       double cond_limit, fmm_scheme** out);
+
+/* dims[4] = {m,k,n,R}.  meta[8] = {L_A, L_B, L_W (Section 4.2), Phi, number of nonzero
+ * coefficients, largest |coefficient|, Q, E (Appendix B.1)}.  Either pointer may be NULL. */
+fmm_status scheme_info(const fmm_scheme* s, int dims[4], double meta[8]);
+
+/* Copy the coefficients out (HOST buffers of R*m*k, R*k*n, R*m*n doubles; any may be NULL). */
+fmm_status scheme_coefficients(const fmm_scheme* s, double* U, double* V, double* W);
+
+void scheme_free(fmm_scheme* s);
+
+/* ---- device work ------------------------------------------------------------------------ */
+
+/* Bytes of DEVICE workspace scheme_gemm needs for this scheme and problem (0 on bad args). */
+size_t scheme_gemm_workspace(const fmm_scheme* s, const fmm_gemm_desc* d);
+
+/* Where scheme_gemm leaves its intermediates inside the workspace (byte offsets from d_ws), so that a
+ * caller (or a test) can inspect each step of Eq. 1 after the call:
+ *   off[0] Ahat  [R][M/m][K/k]  product dtype      off[1] Bhat [R][N/n][K/k] product dtype (K-major)
+ *   off[2] M_r   [R][M/m][N/n]  fp32               off[3] sA[R] fp32    off[4] sB[R] fp32
+ * (sA, sB are written only in scale_mode 1).                                                   */
+fmm_status scheme_gemm_workspace_layout(const fmm_scheme* s, const fmm_gemm_desc* d, size_t off[5]);
+
+/* C = scheme(A, B) as defined at the top of this file (Eq. 1 with rounded block sums).
+ * dA, dB, dC: DEVICE.  d_ws: DEVICE, >= scheme_gemm_workspace bytes, 256-byte aligned; its
+ * contents are scratch except that Bhat persists for FMM_FLAG_REUSE_BHAT.  Asynchronous on
+ * `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream).  Device-side waits
+ * are bounded; a wait that expires is reported by fmm_device_status.                       */
+fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* dA, const void* dB,
+                       void* dC, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/* Read (after synchronising the stream) the device status word the kernels of the last call
+ * on this workspace left: FMM_OK or FMM_ERR_TIMEOUT.                                        */
+fmm_status fmm_device_status(const void* d_ws, void* cuda_stream);
+
+size_t classical_gemm_workspace(const fmm_gemm_desc* d);
+
+/* The classical product at the same dtypes (the paper's control, Section 3.1):
+ * C = rnd_O( sA sB * rnd_Pd(A/sA) * rnd_Pd(B/sB) ), fp32 accumulation on the same tensor-core
+ * kernel.  With storage == product == bf16 and weight layout the operands are read in place. */
+fmm_status classical_gemm(const fmm_gemm_desc* d, const void* dA, const void* dB, void* dC,
+                          void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+/* Exact reference (Appendix B.1, "a float64 reference"): dCstar[M x N] (DEVICE, fp64, ld = N)
+ * = fp64 product of the stored operand values.  desc->product/output are ignored.          */
+fmm_status exact_gemm_f64(const fmm_gemm_desc* d, const void* dA, const void* dB, double* dCstar,
+                          void* cuda_stream);
+
+size_t error_frobenius_workspace(void);
+
+/* Squared Frobenius error against the fp64 reference (Appendix B.1): d_out[0] = sum (C - C*)^2,
+ * d_out[1] = sum C*^2 (DEVICE, 2 doubles).  dC has dtype desc->output and leading dimension
+ * desc->ldc; dCstar is M x N fp64 with ld = N.  Per-block partial sums go to the workspace and are
+ * added in a fixed order, so the result is reproducible run to run.                         */
+fmm_status error_frobenius(const fmm_gemm_desc* d, const void* dC, const double* dCstar, double* d_out,
+                           void* d_ws, size_t ws_bytes, void* cuda_stream);
+
+size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int G);
+
+/* Sweep over G gauge-equivalent copies of one scheme (Section 3.3 / Table 3, model-free form of
+ * Appendix B.1).  For g = 0..G-1 the scheme gauge_apply(base, level, P_g, Q_g, S_g) is run on the
+ * same operands; its squared Frobenius error against the fp64 reference is reduced on the device
+ * (C_g is not stored).  The error-amplification ratio is
+ *     rho_g = ||C_g - C*||_F / ||C_cl - C*||_F ,
+ * C_cl the classical product at the same dtypes (rho = 1 if both errors vanish, +inf if only the
+ * classical one does).
+ * P, Q, S: HOST, G stacked row-major matrices (dimension of the gauged grid).  dCstar: DEVICE fp64
+ * M x N reference, or NULL to have it computed.  h_ratios: HOST, G doubles (may be NULL).
+ * out: HOST.  Synchronises the stream once before returning.                                */
+fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P, const double* Q,
+                       const double* S, const fmm_gemm_desc* d, const void* dA, const void* dB,
+                       const double* dCstar, double* h_ratios, fmm_sweep_summary* out, void* d_ws,
+                       size_t ws_bytes, void* cuda_stream);
+
+const char* fmm_status_string(fmm_status st);
+
+/* Number of kernels this library has launched in this process (for benchmarks' accounting). */
+int64_t fmm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FMM_B200_H */

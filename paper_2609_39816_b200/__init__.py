@@ -1,0 +1,12 @@
+"""B200-native scheme GEMM (fast bilinear matrix multiplication at low precision).
+
+Thin Python binding over the C-ABI library ``libfmm_b200.so`` (argument marshalling only;
+every step of the path runs in the library's CUDA kernels).  There is no CPU fallback: importing
+:mod:`paper_2609_39816_b200.binding` raises if the library has not been built.
+"""
+from .binding import (  # noqa: F401
+    FmmError, Scheme, GemmDesc, SweepSummary, scheme_load, scheme_builtin, scheme_kron, gauge_apply,
+    scheme_gemm, scheme_gemm_workspace, scheme_gemm_workspace_layout, classical_gemm, classical_gemm_workspace, exact_gemm_f64,
+    error_frobenius, error_sweep, error_sweep_workspace, device_status, launch_count, lib_path,
+    F32, BF16, E4M3, FLAG_REUSE_BHAT, EXPORTED_SYMBOLS,
+)

@@ -1,0 +1,244 @@
+"""ctypes binding with the same names as the C ABI declared in ``include/fmm_b200.h``.
+
+Only marshalling happens here: torch tensors are reduced to ``data_ptr()`` and the current CUDA
+stream to its handle.  The shared library is loaded at import; if it is missing the import fails
+loudly (build it with ``python -m paper_2609_39816_b200._build`` or ``__graft_entry__.build()``).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from ._build import LIB_PATH
+
+F32, BF16, E4M3 = 0, 1, 2
+FLAG_REUSE_BHAT = 1
+_DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
+
+EXPORTED_SYMBOLS = [
+    "scheme_load", "scheme_builtin", "scheme_kron", "gauge_apply", "scheme_info", "scheme_coefficients",
+    "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status", "classical_gemm_workspace",
+    "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius",
+    "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count",
+]
+
+
+class FmmError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: fmm_status {code} ({_status_string(code)})")
+        self.code = code
+
+
+class GemmDesc(C.Structure):
+    _fields_ = [("M", C.c_int64), ("K", C.c_int64), ("N", C.c_int64), ("lda", C.c_int64), ("ldb", C.c_int64),
+                ("ldc", C.c_int64), ("storage", C.c_int32), ("product", C.c_int32), ("output", C.c_int32),
+                ("b_is_weight_layout", C.c_int32), ("scale_mode", C.c_int32), ("flags", C.c_int32)]
+
+    @staticmethod
+    def make(M, K, N, storage, product, output, weight_layout=False, scale_mode=0, flags=0, lda=None, ldb=None,
+             ldc=None):
+        d = GemmDesc()
+        d.M, d.K, d.N = M, K, N
+        d.lda = K if lda is None else lda
+        d.ldb = (K if weight_layout else N) if ldb is None else ldb
+        d.ldc = N if ldc is None else ldc
+        d.storage = _DT[storage] if isinstance(storage, str) else storage
+        d.product = _DT[product] if isinstance(product, str) else product
+        d.output = _DT[output] if isinstance(output, str) else output
+        d.b_is_weight_layout = int(bool(weight_layout))
+        d.scale_mode = scale_mode
+        d.flags = flags
+        return d
+
+
+class SweepSummary(C.Structure):
+    _fields_ = [("min", C.c_double), ("median", C.c_double), ("max", C.c_double), ("spread", C.c_double),
+                ("count_gt2", C.c_int64), ("G", C.c_int64), ("e_classical_rel", C.c_double),
+                ("norm_ref", C.c_double)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build the CUDA library first (there is no CPU fallback)")
+_lib = C.CDLL(LIB_PATH)
+_vp, _dp, _sz = C.c_void_p, C.POINTER(C.c_double), C.c_size_t
+_lib.scheme_load.argtypes = [C.c_int] * 4 + [_dp] * 3 + [C.c_double, C.POINTER(_vp)]
+_lib.scheme_builtin.argtypes = [C.c_char_p, C.POINTER(_vp)]
+_lib.scheme_kron.argtypes = [_vp, _vp, C.POINTER(_vp)]
+_lib.gauge_apply.argtypes = [_vp, C.c_int, _dp, _dp, _dp, C.c_double, C.POINTER(_vp)]
+_lib.scheme_info.argtypes = [_vp, C.POINTER(C.c_int), _dp]
+_lib.scheme_coefficients.argtypes = [_vp, _dp, _dp, _dp]
+_lib.scheme_free.argtypes = [_vp]
+_lib.scheme_free.restype = None
+_lib.scheme_gemm_workspace.argtypes = [_vp, C.POINTER(GemmDesc)]
+_lib.scheme_gemm_workspace.restype = _sz
+_lib.scheme_gemm_workspace_layout.argtypes = [_vp, C.POINTER(GemmDesc), C.POINTER(_sz)]
+_lib.scheme_gemm.argtypes = [_vp, C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.fmm_device_status.argtypes = [_vp, _vp]
+_lib.classical_gemm_workspace.argtypes = [C.POINTER(GemmDesc)]
+_lib.classical_gemm_workspace.restype = _sz
+_lib.classical_gemm.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.exact_gemm_f64.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp]
+_lib.error_frobenius_workspace.argtypes = []
+_lib.error_frobenius_workspace.restype = _sz
+_lib.error_frobenius.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.error_sweep_workspace.argtypes = [_vp, C.POINTER(GemmDesc), C.c_int]
+_lib.error_sweep_workspace.restype = _sz
+_lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(GemmDesc), _vp, _vp, _vp, _dp,
+                             C.POINTER(SweepSummary), _vp, _sz, _vp]
+_lib.fmm_status_string.argtypes = [C.c_int]
+_lib.fmm_status_string.restype = C.c_char_p
+_lib.fmm_launch_count.restype = C.c_int64
+
+
+def lib_path() -> str:
+    return LIB_PATH
+
+
+def _status_string(code: int) -> str:
+    return _lib.fmm_status_string(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != 0:
+        raise FmmError(code, what)
+
+
+def _dbl(a):
+    a = np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+    return a, a.ctypes.data_as(_dp)
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+class Scheme:
+    """Owning wrapper of an ``fmm_scheme*``."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h:
+            _lib.scheme_free(h)
+
+    @property
+    def handle(self):
+        return self._h
+
+    @property
+    def dims(self):
+        d = (C.c_int * 4)()
+        _check(_lib.scheme_info(self._h, d, None), "scheme_info")
+        return tuple(d)
+
+    @property
+    def info(self) -> dict:
+        meta = np.zeros(8)
+        _check(_lib.scheme_info(self._h, None, meta.ctypes.data_as(_dp)), "scheme_info")
+        return dict(zip(["L_A", "L_B", "L_W", "Phi", "nnz", "maxabs", "Q", "E"], meta.tolist()))
+
+    def coefficients(self):
+        m, k, n, R = self.dims
+        U, V, W = np.empty((R, m, k)), np.empty((R, k, n)), np.empty((R, m, n))
+        _check(_lib.scheme_coefficients(self._h, U.ctypes.data_as(_dp), V.ctypes.data_as(_dp),
+                                        W.ctypes.data_as(_dp)), "scheme_coefficients")
+        return U, V, W
+
+
+def scheme_load(U, V, W, brent_tol: float = 0.0) -> Scheme:
+    U, pu = _dbl(U); V, pv = _dbl(V); W, pw = _dbl(W)
+    R, m, k = U.shape
+    n = V.shape[2]
+    if V.shape != (R, k, n) or W.shape != (R, m, n):
+        raise ValueError("coefficient arrays must be U[R,m,k], V[R,k,n], W[R,m,n]")
+    h = _vp()
+    _check(_lib.scheme_load(m, k, n, R, pu, pv, pw, brent_tol, C.byref(h)), "scheme_load")
+    return Scheme(h)
+
+
+def scheme_builtin(name: str) -> Scheme:
+    h = _vp()
+    _check(_lib.scheme_builtin(name.encode(), C.byref(h)), "scheme_builtin")
+    return Scheme(h)
+
+
+def scheme_kron(outer: Scheme, inner: Scheme) -> Scheme:
+    h = _vp()
+    _check(_lib.scheme_kron(outer.handle, inner.handle, C.byref(h)), "scheme_kron")
+    return Scheme(h)
+
+
+def gauge_apply(s: Scheme, P, Q, S, level: int = 0, cond_limit: float = 0.0) -> Scheme:
+    _, pp = _dbl(P); _, pq = _dbl(Q); _, ps = _dbl(S)
+    h = _vp()
+    _check(_lib.gauge_apply(s.handle, level, pp, pq, ps, cond_limit, C.byref(h)), "gauge_apply")
+    return Scheme(h)
+
+
+def scheme_gemm_workspace(s: Scheme, d: GemmDesc) -> int:
+    return int(_lib.scheme_gemm_workspace(s.handle, C.byref(d)))
+
+
+def scheme_gemm_workspace_layout(s: Scheme, d: GemmDesc) -> dict:
+    off = (_sz * 5)()
+    _check(_lib.scheme_gemm_workspace_layout(s.handle, C.byref(d), off), "scheme_gemm_workspace_layout")
+    return dict(zip(["Ahat", "Bhat", "M", "sA", "sB"], [int(x) for x in off]))
+
+
+def classical_gemm_workspace(d: GemmDesc) -> int:
+    return int(_lib.classical_gemm_workspace(C.byref(d)))
+
+
+def error_sweep_workspace(s: Scheme, d: GemmDesc, G: int) -> int:
+    return int(_lib.error_sweep_workspace(s.handle, C.byref(d), G))
+
+
+def scheme_gemm(s: Scheme, d: GemmDesc, A, B, Cout, ws) -> None:
+    _check(_lib.scheme_gemm(s.handle, C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws),
+                            ws.numel() * ws.element_size(), _stream()), "scheme_gemm")
+
+
+def classical_gemm(d: GemmDesc, A, B, Cout, ws) -> None:
+    _check(_lib.classical_gemm(C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws),
+                               ws.numel() * ws.element_size(), _stream()), "classical_gemm")
+
+
+def exact_gemm_f64(d: GemmDesc, A, B, Cstar) -> None:
+    _check(_lib.exact_gemm_f64(C.byref(d), _ptr(A), _ptr(B), _ptr(Cstar), _stream()), "exact_gemm_f64")
+
+
+def error_frobenius(d: GemmDesc, Cmat, Cstar, out2, ws) -> None:
+    _check(_lib.error_frobenius(C.byref(d), _ptr(Cmat), _ptr(Cstar), _ptr(out2), _ptr(ws),
+                                ws.numel() * ws.element_size(), _stream()), "error_frobenius")
+
+
+def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=None):
+    """Returns (ratios[G] as numpy fp64, summary dict)."""
+    P, pp = _dbl(P); Q, pq = _dbl(Q); S, ps = _dbl(S)
+    G = P.shape[0]
+    ratios = np.empty(G)
+    summ = SweepSummary()
+    _check(_lib.error_sweep(base.handle, level, G, pp, pq, ps, C.byref(d), _ptr(A), _ptr(B), _ptr(Cstar),
+                            ratios.ctypes.data_as(_dp), C.byref(summ), _ptr(ws), ws.numel() * ws.element_size(),
+                            _stream()), "error_sweep")
+    return ratios, summ.as_dict()
+
+
+def device_status(ws) -> None:
+    _check(_lib.fmm_device_status(_ptr(ws), _stream()), "fmm_device_status")
+
+
+def launch_count() -> int:
+    return int(_lib.fmm_launch_count())

@@ -1,0 +1,401 @@
+// C-ABI entry points that run on the device: scheme_gemm, classical_gemm, exact_gemm_f64,
+// error_frobenius, error_sweep.  Host code only validates, lays out the workspace and enqueues
+// kernels on the caller's stream.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "kernels_stream.cuh"
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a = 1024) { return (x + a - 1) / a * a; }
+inline int esize(int dt) { return dt == FMM_F32 ? 4 : dt == FMM_BF16 ? 2 : 1; }
+
+constexpr int kMaxStreamPartials = 148 * 8;
+
+// Workspace of one scheme GEMM.  Everything is an offset from the workspace base.
+struct GemmLayout {
+  size_t status, tabA, tabB, tabW, amaxA, amaxB, sA, sB, partials, bt, ahat, bhat, prod, total;
+  int n_partials;
+};
+
+fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
+  if (!d) return FMM_ERR_ARG;
+  if (d->M <= 0 || d->K <= 0 || d->N <= 0) return FMM_ERR_SHAPE;
+  if (d->storage != FMM_F32 && d->storage != FMM_BF16) return FMM_ERR_DTYPE;
+  if (d->product != FMM_BF16 && d->product != FMM_E4M3) return FMM_ERR_DTYPE;
+  if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
+  if (d->scale_mode != 0 && !(d->scale_mode == 1 && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
+  if (d->M % m || d->K % k || d->N % n) return FMM_ERR_SHAPE;
+  if ((d->K / k) % 16 || (d->N / n) % 8) return FMM_ERR_SHAPE;
+  const int es = esize(d->storage), eo = esize(d->output);
+  const int64_t min_ldb = d->b_is_weight_layout ? d->K : d->N;
+  if (d->lda < d->K || d->ldb < min_ldb || d->ldc < d->N) return FMM_ERR_SHAPE;
+  if ((d->lda * es) % 16 || (d->ldb * es) % 16 || (d->ldc * eo) % 16) return FMM_ERR_SHAPE;
+  return FMM_OK;
+}
+
+GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
+  GemmLayout L;
+  const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
+  const int ep = esize(d->product), es = esize(d->storage);
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.tabA = o; o += align_up(sizeof(CoefTable));
+  L.tabB = o; o += align_up(sizeof(CoefTable));
+  L.tabW = o; o += align_up(sizeof(CoefTable));
+  L.amaxA = o; o += align_up(FMM_MAX_R * 4);
+  L.amaxB = o; o += align_up(FMM_MAX_R * 4);
+  L.sA = o; o += align_up(FMM_MAX_R * 4);
+  L.sB = o; o += align_up(FMM_MAX_R * 4);
+  L.n_partials = std::max(decode_grid(bm, bn), kMaxStreamPartials);
+  L.partials = o; o += align_up((size_t)L.n_partials * 8 * 2);
+  L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
+  L.ahat = o; o += align_up((size_t)R * bm * bk * ep);
+  L.bhat = o; o += align_up((size_t)R * bn * bk * ep);
+  L.prod = o; o += align_up((size_t)R * bm * bn * 4);
+  L.total = o;
+  return L;
+}
+
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+#define FMM_CUDA(x) do { if ((x) != cudaSuccess) return FMM_ERR_CUDA; } while (0)
+#define FMM_TRY(x) do { fmm_status _s = (x); if (_s != FMM_OK) return _s; } while (0)
+
+// Encode one operand: optional amax pass, then block sums -> product dtype.
+fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
+                          const CoefTable* d_tab, void* hat, unsigned* amax, float* scale, cudaStream_t st) {
+  const bool scaled = d->scale_mode == 1;
+  if (scaled) {
+    FMM_CUDA(cudaMemsetAsync(amax, 0, FMM_MAX_R * 4, st));
+    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, hat, amax, scale, true, true, st));
+  }
+  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, hat, amax, scale, false, scaled, st));
+  return FMM_OK;
+}
+
+// The whole path for one scheme on one operand pair.  If C is null the result is not stored; if cstar32 is
+// given the squared error is reduced into err_out[0] (device).  `tables` are host tables to upload, or null
+// when the device tables at L.tab* are already in place.
+fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLayout& L, const CoefTable* hA,
+                      const CoefTable* hB, const CoefTable* hW, const CoefTable* dA_tab, const CoefTable* dB_tab,
+                      const CoefTable* dW_tab, const void* A, const void* Bsrc_kmajor, int64_t ldb_kmajor, void* C,
+                      const float* cstar32, double* err_out, void* ws, bool skip_b, cudaStream_t st) {
+  const int m = s->m, k = s->k, n = s->n, R = s->R;
+  const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
+  if (hA) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabA), hA, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  if (hB && !skip_b) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabB), hB, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  if (hW) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabW), hW, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  if (!dA_tab) dA_tab = at<CoefTable>(ws, L.tabA);
+  if (!dB_tab) dB_tab = at<CoefTable>(ws, L.tabB);
+  if (!dW_tab) dW_tab = at<CoefTable>(ws, L.tabW);
+  const bool scaled = d->scale_mode == 1;
+  float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
+  float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
+
+  FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
+  if (!skip_b)
+    FMM_TRY(encode_operand(d, Bsrc_kmajor, ldb_kmajor, n, k, bn, bk, dB_tab, at<char>(ws, L.bhat),
+                           at<unsigned>(ws, L.amaxB), sB, st));
+  BlockProductArgs g{};
+  g.product = d->product;
+  g.A = at<char>(ws, L.ahat); g.lda = bk; g.a_batch = bm * bk;
+  g.B = at<char>(ws, L.bhat); g.ldb = bk; g.b_batch = bn * bk;
+  g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = R;
+  g.out = at<char>(ws, L.prod); g.ldo = bn; g.o_batch = bm * bn; g.out_mode = 0; g.output = FMM_F32;
+  g.status = at<DeviceStatus>(ws, L.status);
+  FMM_TRY(launch_block_products(g, st));
+  int np = 0;
+  FMM_CUDA(launch_decode(d->output, at<float>(ws, L.prod), dW_tab, sA, sB, m, n, bm, bn, C, d->ldc, cstar32,
+                         at<double>(ws, L.partials), &np, st));
+  if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(ws, L.partials), np, err_out, st));
+  return FMM_OK;
+}
+
+// B as a K-major matrix [N x K]: in place for the weight layout, else transposed into the workspace.
+fmm_status kmajor_b(const fmm_gemm_desc* d, const void* B, void* ws, size_t bt_off, const void** out, int64_t* ld,
+                    bool skip, cudaStream_t st) {
+  if (d->b_is_weight_layout) { *out = B; *ld = d->ldb; return FMM_OK; }
+  void* bt = at<char>(ws, bt_off);
+  if (!skip) FMM_CUDA(launch_transpose(esize(d->storage), B, d->ldb, d->K, d->N, bt, st));
+  *out = bt; *ld = d->K;
+  return FMM_OK;
+}
+
+fmm_status check_ws(const void* ws, size_t have, size_t need) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u) || have < need) return FMM_ERR_WORKSPACE;
+  return FMM_OK;
+}
+
+fmm_scheme classical_scheme_111() {
+  fmm_scheme c;
+  c.m = c.k = c.n = c.R = 1;
+  c.U = {1.0}; c.V = {1.0}; c.W = {1.0};
+  return c;
+}
+
+// Workspace of the classical product.
+struct ClassicalLayout { size_t status, tab, amaxA, amaxB, sA, sB, bt, ahat, bhat, total; bool direct; };
+
+ClassicalLayout classical_layout(const fmm_gemm_desc* d) {
+  ClassicalLayout L;
+  const int ep = esize(d->product), es = esize(d->storage);
+  L.direct = d->storage == FMM_BF16 && d->product == FMM_BF16 && d->scale_mode == 0;
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.tab = o; o += align_up(sizeof(CoefTable));
+  L.amaxA = o; o += align_up(FMM_MAX_R * 4);
+  L.amaxB = o; o += align_up(FMM_MAX_R * 4);
+  L.sA = o; o += align_up(FMM_MAX_R * 4);
+  L.sB = o; o += align_up(FMM_MAX_R * 4);
+  L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
+  L.ahat = o; o += L.direct ? 0 : align_up((size_t)d->M * d->K * ep);
+  L.bhat = o; o += L.direct ? 0 : align_up((size_t)d->N * d->K * ep);
+  L.total = o;
+  return L;
+}
+
+fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const void* A, const void* B, void* C,
+                         void* ws, cudaStream_t st) {
+  const void* bk_ptr; int64_t bk_ld;
+  FMM_TRY(kmajor_b(d, B, ws, L.bt, &bk_ptr, &bk_ld, false, st));
+  BlockProductArgs g{};
+  g.product = d->product;
+  g.rows_a = d->M; g.rows_b = d->N; g.kdim = d->K; g.batches = 1;
+  g.out = C; g.ldo = d->ldc; g.o_batch = 0; g.out_mode = 1; g.output = d->output;
+  g.status = at<DeviceStatus>(ws, L.status);
+  if (L.direct) {
+    g.A = A; g.lda = d->lda; g.a_batch = 0;
+    g.B = bk_ptr; g.ldb = bk_ld; g.b_batch = 0;
+  } else {
+    fmm_scheme one = classical_scheme_111();
+    CoefTable t;
+    std::memset(&t, 0, sizeof(t));
+    fmm_build_tables(one, &t, nullptr, nullptr);
+    FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tab), &t, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    const bool scaled = d->scale_mode == 1;
+    float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
+    float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
+    FMM_TRY(encode_operand(d, A, d->lda, 1, 1, d->M, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.ahat),
+                           at<unsigned>(ws, L.amaxA), sA, st));
+    FMM_TRY(encode_operand(d, bk_ptr, bk_ld, 1, 1, d->N, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.bhat),
+                           at<unsigned>(ws, L.amaxB), sB, st));
+    g.A = at<char>(ws, L.ahat); g.lda = d->K; g.a_batch = 0;
+    g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
+    g.sA = sA; g.sB = sB;
+  }
+  return launch_block_products(g, st);
+}
+
+// Workspace of a sweep: the GEMM layout plus reference copies, classical result, tables and sums.
+struct SweepLayout {
+  GemmLayout g; ClassicalLayout c;
+  size_t gemm, classical, cstar, cstar32, ccl, tables, sums, total;
+};
+
+SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
+  SweepLayout L;
+  L.g = gemm_layout(s->m, s->k, s->n, s->R, d);
+  L.c = classical_layout(d);
+  size_t o = 0;
+  L.gemm = o; o += align_up(L.g.total);
+  L.classical = o; o += align_up(L.c.total);
+  L.cstar = o; o += align_up((size_t)d->M * d->N * 8);
+  L.cstar32 = o; o += align_up((size_t)d->M * d->N * 4);
+  L.ccl = o; o += align_up((size_t)d->M * d->N * esize(d->output));
+  L.tables = o; o += align_up((size_t)G * 3 * sizeof(CoefTable));
+  L.sums = o; o += align_up((size_t)(G + 8) * 8);
+  L.total = o;
+  return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t fmm_launch_count(void) { return fmm_launch_counter(); }
+
+size_t scheme_gemm_workspace(const fmm_scheme* s, const fmm_gemm_desc* d) {
+  if (!s || check_desc(d, s->m, s->k, s->n) != FMM_OK) return 0;
+  return gemm_layout(s->m, s->k, s->n, s->R, d).total;
+}
+
+fmm_status scheme_gemm_workspace_layout(const fmm_scheme* s, const fmm_gemm_desc* d, size_t off[5]) {
+  if (!s || !off) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, s->m, s->k, s->n));
+  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d);
+  off[0] = L.ahat; off[1] = L.bhat; off[2] = L.prod; off[3] = L.sA; off[4] = L.sB;
+  return FMM_OK;
+}
+
+fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* dA, const void* dB, void* dC,
+                       void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!s || !d || !dA || !dB || !dC) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, s->m, s->k, s->n));
+  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d);
+  FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool skip_b = (d->flags & FMM_FLAG_REUSE_BHAT) != 0;
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  CoefTable tA, tB, tW;
+  std::memset(&tA, 0, sizeof(tA)); std::memset(&tB, 0, sizeof(tB)); std::memset(&tW, 0, sizeof(tW));
+  fmm_build_tables(*s, &tA, &tB, &tW);
+  const void* bk_ptr; int64_t bk_ld;
+  FMM_TRY(kmajor_b(d, dB, d_ws, L.bt, &bk_ptr, &bk_ld, skip_b, st));
+  return run_scheme(s, d, L, &tA, &tB, &tW, nullptr, nullptr, nullptr, dA, bk_ptr, bk_ld, dC, nullptr, nullptr, d_ws,
+                    skip_b, st);
+}
+
+fmm_status fmm_device_status(const void* d_ws, void* cuda_stream) {
+  if (!d_ws) return FMM_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DeviceStatus h;
+  FMM_CUDA(cudaMemcpyAsync(&h, d_ws, sizeof(h), cudaMemcpyDeviceToHost, st));
+  FMM_CUDA(cudaStreamSynchronize(st));
+  return h.code == 0 ? FMM_OK : FMM_ERR_TIMEOUT;
+}
+
+size_t classical_gemm_workspace(const fmm_gemm_desc* d) {
+  if (check_desc(d, 1, 1, 1) != FMM_OK) return 0;
+  return classical_layout(d).total;
+}
+
+fmm_status classical_gemm(const fmm_gemm_desc* d, const void* dA, const void* dB, void* dC, void* d_ws,
+                          size_t ws_bytes, void* cuda_stream) {
+  if (!d || !dA || !dB || !dC) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, 1, 1, 1));
+  const ClassicalLayout L = classical_layout(d);
+  FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  return run_classical(d, L, dA, dB, dC, d_ws, st);
+}
+
+fmm_status exact_gemm_f64(const fmm_gemm_desc* d, const void* dA, const void* dB, double* dCstar, void* cuda_stream) {
+  if (!d || !dA || !dB || !dCstar) return FMM_ERR_ARG;
+  if (d->M <= 0 || d->K <= 0 || d->N <= 0) return FMM_ERR_SHAPE;
+  if (d->storage != FMM_F32 && d->storage != FMM_BF16) return FMM_ERR_DTYPE;
+  FMM_CUDA(launch_exact_f64(d->storage, dA, d->lda, dB, d->ldb, d->b_is_weight_layout, d->M, d->K, d->N, dCstar,
+                            static_cast<cudaStream_t>(cuda_stream)));
+  return FMM_OK;
+}
+
+size_t error_frobenius_workspace(void) { return align_up((size_t)kMaxStreamPartials * 8 * 2); }
+
+fmm_status error_frobenius(const fmm_gemm_desc* d, const void* dC, const double* dCstar, double* d_out, void* d_ws,
+                           size_t ws_bytes, void* cuda_stream) {
+  if (!d || !dC || !dCstar || !d_out) return FMM_ERR_ARG;
+  if (d->M <= 0 || d->N <= 0 || d->ldc < d->N) return FMM_ERR_SHAPE;
+  if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
+  FMM_TRY(check_ws(d_ws, ws_bytes, error_frobenius_workspace()));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  double* pe = at<double>(d_ws, 0);
+  double* pr = pe + kMaxStreamPartials;
+  int np = 0;
+  FMM_CUDA(launch_frob_err(d->output, dC, d->ldc, dCstar, d->M, d->N, pe, pr, &np, st));
+  FMM_CUDA(launch_sum_partials(pe, np, d_out, st));
+  FMM_CUDA(launch_sum_partials(pr, np, d_out + 1, st));
+  return FMM_OK;
+}
+
+size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int G) {
+  if (!base || G < 1 || check_desc(d, base->m, base->k, base->n) != FMM_OK) return 0;
+  return sweep_layout(base, d, G).total;
+}
+
+fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P, const double* Q, const double* S,
+                       const fmm_gemm_desc* d, const void* dA, const void* dB, const double* dCstar, double* h_ratios,
+                       fmm_sweep_summary* out, void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!base || !P || !Q || !S || !d || !dA || !dB || !out || G < 1) return FMM_ERR_ARG;
+  if (level != 0 && level != 1) return FMM_ERR_ARG;
+  if (level == 1 && (!base->outer || !base->inner)) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, base->m, base->k, base->n));
+  const SweepLayout L = sweep_layout(base, d, G);
+  FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const fmm_scheme* grid = level == 1 ? base->outer.get() : base;
+  const int gm = grid->m, gk = grid->k, gn = grid->n;
+
+  // 1. gauge-transformed coefficient tables, built on the host and uploaded once
+  std::vector<CoefTable> tabs((size_t)G * 3);
+  std::memset(tabs.data(), 0, tabs.size() * sizeof(CoefTable));
+  for (int g = 0; g < G; ++g) {
+    fmm_scheme* gs = nullptr;
+    FMM_TRY(fmm_gauge_core(*base, level, P + (size_t)g * gm * gm, Q + (size_t)g * gk * gk, S + (size_t)g * gn * gn, 0.0, &gs));
+    fmm_build_tables(*gs, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2]);
+    scheme_free(gs);
+  }
+  char* ws = static_cast<char*>(d_ws);
+  void* gws = ws + L.gemm;
+  void* cws = ws + L.classical;
+  CoefTable* d_tabs = at<CoefTable>(ws, L.tables);
+  double* sums = at<double>(ws, L.sums);  // [0]=n*, [1]=e_cl, [2]=scratch, [8..8+G) = e_g
+  FMM_CUDA(cudaMemcpyAsync(d_tabs, tabs.data(), tabs.size() * sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemsetAsync(at<char>(gws, L.g.status), 0, sizeof(DeviceStatus), st));
+  FMM_CUDA(cudaMemsetAsync(at<char>(cws, L.c.status), 0, sizeof(DeviceStatus), st));
+
+  // 2. fp64 reference, its fp32 copy and its squared norm
+  const double* cstar = dCstar;
+  if (!cstar) {
+    double* mine = at<double>(ws, L.cstar);
+    FMM_CUDA(launch_exact_f64(d->storage, dA, d->lda, dB, d->ldb, d->b_is_weight_layout, d->M, d->K, d->N, mine, st));
+    cstar = mine;
+  }
+  float* cstar32 = at<float>(ws, L.cstar32);
+  double* part = at<double>(gws, L.g.partials);
+  int np = 0;
+  FMM_CUDA(launch_cstar_prepare(cstar, d->M * d->N, cstar32, part, &np, st));
+  FMM_CUDA(launch_sum_partials(part, np, sums + 0, st));
+
+  // 3. classical product at the same dtypes and its error
+  fmm_gemm_desc dcl = *d;
+  dcl.ldc = d->N;
+  void* ccl = at<char>(ws, L.ccl);
+  FMM_TRY(run_classical(&dcl, L.c, dA, dB, ccl, cws, st));
+  FMM_CUDA(launch_frob_err(d->output, ccl, d->N, cstar, d->M, d->N, part, nullptr, &np, st));
+  FMM_CUDA(launch_sum_partials(part, np, sums + 1, st));
+
+  // 4. the sweep: per gauge encode A, encode B, R products, decode + error reduction
+  const void* bk_ptr; int64_t bk_ld;
+  FMM_TRY(kmajor_b(d, dB, gws, L.g.bt, &bk_ptr, &bk_ld, false, st));
+  for (int g = 0; g < G; ++g) {
+    FMM_TRY(run_scheme(base, d, L.g, nullptr, nullptr, nullptr, d_tabs + 3 * g, d_tabs + 3 * g + 1, d_tabs + 3 * g + 2,
+                       dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
+  }
+
+  // 5. results to the host
+  std::vector<double> h((size_t)G + 8);
+  DeviceStatus hs_g, hs_c;
+  FMM_CUDA(cudaMemcpyAsync(h.data(), sums, h.size() * 8, cudaMemcpyDeviceToHost, st));
+  FMM_CUDA(cudaMemcpyAsync(&hs_g, at<char>(gws, L.g.status), sizeof(DeviceStatus), cudaMemcpyDeviceToHost, st));
+  FMM_CUDA(cudaMemcpyAsync(&hs_c, at<char>(cws, L.c.status), sizeof(DeviceStatus), cudaMemcpyDeviceToHost, st));
+  FMM_CUDA(cudaStreamSynchronize(st));
+  if (hs_g.code != 0 || hs_c.code != 0) return FMM_ERR_TIMEOUT;
+
+  const double nref = h[0], ecl = h[1];
+  std::vector<double> rho(G);
+  for (int g = 0; g < G; ++g) {
+    const double eg = h[8 + g];
+    rho[g] = (ecl == 0.0) ? (eg == 0.0 ? 1.0 : INFINITY) : std::sqrt(eg / ecl);
+  }
+  if (h_ratios) std::copy(rho.begin(), rho.end(), h_ratios);
+  std::vector<double> sorted = rho;
+  std::sort(sorted.begin(), sorted.end());
+  out->min = sorted.front();
+  out->max = sorted.back();
+  out->median = sorted[G / 2];  // upper of the two middle values when G is even
+  out->spread = sorted.front() > 0 ? sorted.back() / sorted.front() : INFINITY;
+  out->count_gt2 = (int64_t)std::count_if(rho.begin(), rho.end(), [](double x) { return x > 2.0; });
+  out->G = G;
+  out->e_classical_rel = nref > 0 ? std::sqrt(ecl / nref) : 0.0;
+  out->norm_ref = std::sqrt(nref);
+  return FMM_OK;
+}
+
+}  // extern "C"

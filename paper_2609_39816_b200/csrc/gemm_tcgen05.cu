@@ -1,0 +1,468 @@
+// Batched block products M_r = Ahat_r * Bhat_r^T on Blackwell tensor cores (sm_100a).
+//
+// One persistent CTA per SM walks a static list of (product r, row tile, column tile).
+//   warp 0        : TMA producer  — cp.async.bulk.tensor loads of a 128 x BK tile of Ahat_r and a
+//                   BN x BK tile of Bhat_r (both K-major, 128-byte swizzle) into a shared-memory ring;
+//   warp 1        : allocates TMEM, then one lane issues tcgen05.mma (M=128, N=BN, K=32 bytes) into one
+//                   of two fp32 accumulator buffers in TMEM, and tcgen05.commit releases ring stages /
+//                   publishes the finished accumulator through mbarriers;
+//   warps 2..5    : epilogue — tcgen05.ld the accumulator (each warp its own 32-lane quadrant),
+//                   store fp32 products (or the rounded, scaled result) to global memory, and hand the
+//                   TMEM buffer back.
+// Double-buffered TMEM lets the epilogue of tile i overlap the main loop of tile i+1.
+// Every mbarrier wait is bounded: after ~2 s without progress a role raises the CTA's abort flag,
+// records FMM_ERR_TIMEOUT in the device status word, lets its outstanding copies land (bounded),
+// and the CTA frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <mutex>
+
+#include "kernels_stream.cuh"
+
+namespace {
+
+constexpr int BM = 128;             // rows of A per tile = UMMA M
+constexpr int BKB = 128;            // bytes of the inner dimension per ring stage (one swizzle span)
+constexpr int UMMA_KB = 32;         // bytes of the inner dimension per tcgen05.mma
+constexpr int kNumThreads = 192;    // 6 warps
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where,
+                                          DeviceStatus* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        if (status != nullptr) {
+          atomicExch(&status->code, (int)FMM_ERR_TIMEOUT);
+          atomicExch(&status->where, where);
+        }
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <bool kFp8>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  if (kFp8) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
+// swizzle (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B): start address (>>4), leading byte offset
+// (unused for this layout, 1), stride byte offset = 8 rows * 128 B = 1024 (>>4), descriptor version 1,
+// layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// Instruction descriptor: fp32 accumulator, A and B formats (kind::f16: 1 = bf16; kind::f8f6f4: 0 = e4m3),
+// both operands K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(bool fp8, int n) {
+  return (1u << 4) | ((fp8 ? 0u : 1u) << 7) | ((fp8 ? 0u : 1u) << 10) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(BM >> 4) << 24);
+}
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kABytes = BM * BKB;
+  static constexpr int kBBytes = BN * BKB;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
+};
+
+struct TileParams {
+  int rows_a, rows_b;       // extents of one batch entry
+  int kbytes;               // inner extent in bytes
+  int elem_bytes;           // 2 (bf16) or 1 (e4m3)
+  int batches;
+  int tiles_m, tiles_n;
+  long long ldo, o_batch;   // output strides in elements
+  int out_mode;             // 0: fp32 products; 1: scaled + rounded result
+  int out_bf16;             // out_mode 1: 1 -> bf16, 0 -> fp32
+};
+
+template <int BN, bool kFp8>
+__global__ void __launch_bounds__(kNumThreads, 1)
+block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                      void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
+                      TileParams tp, DeviceStatus* status) {
+  using L = SmemLayout<BN>;
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment of the swizzled tiles
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - raw_addr);
+  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
+  // barrier block: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2], drain, tmem base, abort flag
+  const uint32_t bar_base = smem_u32(bar_mem);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr uint32_t kTmemCols = 2 * BN;  // two accumulator buffers (256 or 512 columns)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM allocation (whole warp), address lands in shared memory
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_kb = (tp.kbytes + BKB - 1) / BKB;
+  const int tiles_per_batch = tp.tiles_m * tp.tiles_n;
+  const int total_tiles = tiles_per_batch * tp.batches;
+  const int kelems_per_stage = BKB / tp.elem_bytes;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int r = tile / tiles_per_batch;
+        const int rem = tile - r * tiles_per_batch;
+        const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status);
+          if (!ok) break;
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t sb = sa + L::kABytes;
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::kStageBytes);
+          tma_load_3d(sa, &map_a, full_bar(stage), kb * kelems_per_stage, tm * BM, r);
+          tma_load_3d(sb, &map_b, full_bar(stage), kb * kelems_per_stage, tn * BN, r);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let copies that were already issued land before the CTA's shared memory goes away:
+        // the most recent fill of every stage completes phase (fills-1)&1 of its full barrier.
+        for (int s = 0; s < L::kStages; ++s) {
+          const uint32_t last_parity = (s < stage) ? phase : (phase ^ 1u);
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(s), last_parity)) {
+            if (global_timer_ns() - t0 > 20000000ull) break;  // 20 ms
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kFp8, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + L::kABytes);
+#pragma unroll
+          for (int k = 0; k < BKB / UMMA_KB; ++k) {
+            // advance both descriptors by 32 bytes along K inside the swizzle span (address field is >>4)
+            tc_mma<kFp8>(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc,
+                         (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // stage reusable once these MMAs have read it
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) {  // wait (bounded) for MMAs in flight before TMEM is freed
+        tc_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0)) {
+          if (global_timer_ns() - t0 > 20000000ull) break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) are the ones this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    float alpha = 1.0f;
+    if (tp.out_mode == 1 && sA != nullptr && sB != nullptr) alpha = sA[0] * sB[0];
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int r = tile / tiles_per_batch;
+      const int rem = tile - r * tiles_per_batch;
+      const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
+      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = tm * BM + quad * 32 + lane;
+      const bool row_ok = row < tp.rows_a;
+      const long long row_off = (long long)r * tp.o_batch + (long long)row * tp.ldo;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c * 32);
+        tc_ld32(taddr, v);
+        tc_wait_ld();
+        const int col0 = tn * BN + c * 32;
+        if (row_ok && col0 < tp.rows_b) {
+          const int ncols = min(32, tp.rows_b - col0);
+          if (tp.out_mode == 0) {
+            float* dst = reinterpret_cast<float*>(out) + row_off + col0;
+            if (ncols == 32) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols) dst[j] = __uint_as_float(v[j]);
+            }
+          } else if (tp.out_bf16) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + row_off + col0;
+            if (ncols == 32) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 pk;
+                uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                  __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2 * h]) * alpha,
+                                                            __uint_as_float(v[j + 2 * h + 1]) * alpha);
+                  pw[h] = *reinterpret_cast<uint32_t*>(&b2);
+                }
+                *reinterpret_cast<uint4*>(dst + j) = pk;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * alpha);
+            }
+          } else {
+            float* dst = reinterpret_cast<float*>(out) + row_off + col0;
+            if (ncols == 32) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) =
+                    make_float4(__uint_as_float(v[j]) * alpha, __uint_as_float(v[j + 1]) * alpha,
+                                __uint_as_float(v[j + 2]) * alpha, __uint_as_float(v[j + 3]) * alpha);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < ncols) dst[j] = __uint_as_float(v[j]) * alpha;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// K-major operand [batches][rows][kdim] -> 3-D map, box {128 bytes of K, box_rows, 1}, 128-byte swizzle.
+bool make_operand_map(CUtensorMap* map, bool fp8, const void* ptr, int64_t rows, int64_t kdim, int64_t ld,
+                      int64_t batch_stride, int batches, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const int es = fp8 ? 1 : 2;
+  cuuint64_t dims[3] = {(cuuint64_t)kdim, (cuuint64_t)rows, (cuuint64_t)batches};
+  cuuint64_t strides[2] = {(cuuint64_t)(ld * es), (cuuint64_t)((batches > 1 ? batch_stride : rows * ld) * es)};
+  cuuint32_t box[3] = {(cuuint32_t)(BKB / es), (cuuint32_t)box_rows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult rc = fn(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                   const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+template <int BN, bool kFp8>
+fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
+  using L = SmemLayout<BN>;
+  CUtensorMap ma, mb;
+  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, BN)) return FMM_ERR_CUDA;
+  TileParams tp;
+  tp.rows_a = (int)a.rows_a; tp.rows_b = (int)a.rows_b;
+  tp.elem_bytes = kFp8 ? 1 : 2;
+  tp.kbytes = (int)a.kdim * tp.elem_bytes;
+  tp.batches = a.batches;
+  tp.tiles_m = (int)((a.rows_a + BM - 1) / BM);
+  tp.tiles_n = (int)((a.rows_b + BN - 1) / BN);
+  tp.ldo = a.ldo; tp.o_batch = a.o_batch;
+  tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
+  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
+  if (total <= 0) return FMM_OK;
+  const int sms = sm_count();
+  if (sms <= 0) return FMM_ERR_CUDA;
+  const int grid = (int)(total < sms ? total : sms);
+  auto k = block_products_kernel<BN, kFp8>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
+  k<<<grid, kNumThreads, L::kTotal, st>>>(ma, mb, a.out, a.sA, a.sB, tp, a.status);
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+}  // namespace
+
+fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
+  if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim > 0x3fffffff) return FMM_ERR_SHAPE;
+  const bool fp8 = (a.product == FMM_E4M3);
+  if (!fp8 && a.product != FMM_BF16) return FMM_ERR_DTYPE;
+  // narrow problems use the 128-column tile (less padding, more tiles in flight)
+  const bool narrow = a.rows_b <= 128;
+  if (fp8) return narrow ? launch_t<128, true>(a, st) : launch_t<256, true>(a, st);
+  return narrow ? launch_t<128, false>(a, st) : launch_t<256, false>(a, st);
+}

@@ -1,0 +1,65 @@
+// Launch wrappers of the streaming (HBM-bound) kernels and of the tensor-core block products.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "fmm_internal.h"
+
+// Device-resident status word at the start of every workspace.
+struct DeviceStatus {
+  int code;       // 0 ok, FMM_ERR_TIMEOUT when a bounded wait expired
+  int where;      // which wait gave up (role id * 16 + barrier kind), for diagnosis
+  int pad[62];
+};
+
+int64_t& fmm_launch_counter();
+
+// X: source matrix (storage dtype), rows x cols with leading dimension ldx, split into a gr x gc grid of
+// br x bc blocks.  out[R][br][bc] in the product dtype.  With amax_only the kernel only accumulates
+// max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).
+// With use_scale, scale[r] is derived from amax_bits[r] (2^ceil(log2(amax/448)), 1 if amax==0),
+// written to scale[R] and divided out before rounding.
+cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
+                          int64_t bc, const CoefTable* d_tab, void* out, unsigned* amax_bits, float* scale,
+                          bool amax_only, bool use_scale, cudaStream_t st);
+
+// Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
+cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
+                             cudaStream_t st);
+
+// Decode (+ optional error reduction).  prod[R][bm][bn] fp32.  If C != nullptr the rounded result is stored
+// (dtype `output`, leading dimension ldc).  If cstar32 != nullptr the per-block partial sums of
+// (rnd_O(c) - C*)^2 are written to partials[gridDim.x] and *n_partials receives gridDim.x.
+cudaError_t launch_decode(int output, const float* prod, const CoefTable* d_tab, const float* sA, const float* sB,
+                          int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc, const float* cstar32,
+                          double* partials, int* n_partials, cudaStream_t st);
+int decode_grid(int64_t bm, int64_t bn);
+
+// out[0] = sum of partials[0..n) in a fixed order (single block).
+cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st);
+
+// C*(fp64) -> fp32 copy, and partial sums of C*^2.
+cudaError_t launch_cstar_prepare(const double* cstar, int64_t count, float* cstar32, double* partials,
+                                 int* n_partials, cudaStream_t st);
+// partial sums of (C - C*)^2 and of C*^2 (two arrays of n_partials doubles, the second may be null).
+cudaError_t launch_frob_err(int output, const void* C, int64_t ldc, const double* cstar, int64_t M, int64_t N,
+                            double* part_err, double* part_ref, int* n_partials, cudaStream_t st);
+int stream_grid(int64_t count);
+
+cudaError_t launch_exact_f64(int storage, const void* A, int64_t lda, const void* B, int64_t ldb,
+                             int b_weight_layout, int64_t M, int64_t K, int64_t N, double* C, cudaStream_t st);
+
+// Batched block products on tcgen05 tensor cores:
+//   D_r[rows_a x rows_b] = A_r[rows_a x kdim] * B_r[rows_b x kdim]^T   (both operands K-major)
+// product dtype bf16 or e4m3, fp32 accumulation in TMEM.
+//   out_mode 0: store fp32 to out (float*, row stride ldo, batch stride ldo_batch elements)
+//   out_mode 1: store rnd(alpha * acc) as `output` dtype (alpha = sA[0]*sB[0] when given, else 1).
+struct BlockProductArgs {
+  int product;               // FMM_BF16 / FMM_E4M3
+  const void* A; int64_t lda; int64_t a_batch;   // elements
+  const void* B; int64_t ldb; int64_t b_batch;
+  int64_t rows_a, rows_b, kdim; int batches;
+  void* out; int64_t ldo; int64_t o_batch; int out_mode; int output;
+  const float* sA; const float* sB;
+  DeviceStatus* status;
+};
+fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
