@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the scheme-GEMM hot path on B200.
+
+One "step" = one pass of the whole path over one operand pair: encode A, encode B, the R block
+products on tcgen05 tensor cores, decode.  Workload (N=1): two-level Strassen <4,4,4;49>, bf16,
+M=K=N=4096, activations N(0,1) with 0.5% outlier channels x100, weights N(0,0.02) in the nn.Linear
+layout [N,K].  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N>1 (torchrun) every rank runs an independent replica of the GEMM (the path does not shard;
+weak scaling) and the gauge sweep shards its gauges over the ranks.
+`--impl reference` times the CPU oracle (a deliberately slow program) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "scheme_gemm_effective_tflops_2MNK_over_t"
+UNIT = "TFLOP/s"
+C2 = dict(M=4096, K=4096, N=4096, scheme="strassen444", R=49, grid=4)
+C3 = dict(M=2048, K=4096, N=4096, scheme="strassen222", R=7, grid=2)
+L2_FLUSH_BYTES = 256 << 20
+
+
+# ------------------------------------------------------------------ multi-rank helpers (tested on gloo)
+def shard_gauges(G: int, rank: int, world: int):
+    """Gauges are independent units: rank r takes r, r+world, r+2*world, ..."""
+    return list(range(rank, G, world))
+
+
+def gather_ratios(local, mine, G: int, rank: int, world: int, device="cuda"):
+    """All-gather the per-rank ratio vectors into one length-G vector (every rank gets it)."""
+    import torch
+    import torch.distributed as dist
+    full = torch.zeros(G, dtype=torch.float64, device=device)
+    if len(mine):
+        full[torch.tensor(mine, dtype=torch.long, device=device)] = local.to(device)
+    if world > 1:
+        dist.all_reduce(full, op=dist.ReduceOp.SUM)     # disjoint supports: sum == gather
+    return full
+
+
+# ------------------------------------------------------------------ inputs
+def c2_inputs(seed: int):
+    from fmm_inputs import generators as gen
+    A = gen.activations_outlier(seed, 1, C2["M"], C2["K"], dist="normal", frac=0.005, factor=100.0)
+    B = gen.weights(seed, 2, C2["K"], C2["N"], std=0.02)
+    At, A64 = gen.to_storage(A, "bf16")
+    Bt, B64 = gen.to_storage(B, "bf16")
+    return At, Bt.t().contiguous(), A64, B64          # B in weight layout [N,K]
+
+
+def c3_inputs(seed: int):
+    from fmm_inputs import generators as gen
+    A = gen.activations_outlier(seed, 3, C3["M"], C3["K"], dist="normal", frac=0.005, factor=100.0)
+    B = gen.weights(seed, 4, C3["K"], C3["N"], std=0.02)
+    At, _ = gen.to_storage(A, "bf16")
+    Bt, _ = gen.to_storage(B, "bf16")
+    return At, Bt.t().contiguous()
+
+
+def sweep_gauges(G: int, seed: int = 1):
+    from fmm_inputs import generators as gen
+    P = np.stack([gen.gauge_log_uniform_cond(seed, 3 * g, 2) for g in range(G)])
+    Q = np.stack([gen.gauge_log_uniform_cond(seed, 3 * g + 1, 2) for g in range(G)])
+    S = np.stack([gen.gauge_log_uniform_cond(seed, 3 * g + 2, 2) for g in range(G)])
+    return P, Q, S
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0])); mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------ reference arm (CPU oracle)
+def oracle_sample(A64, B64, rows_per_block: int):
+    """Rows [0, rows_per_block) of every block row of A: the scheme acts position-wise on blocks, so
+    this is the same computation on a quarter (etc.) of the output rows."""
+    m = C2["grid"]
+    bm = C2["M"] // m
+    ridx = np.concatenate([i * bm + np.arange(rows_per_block) for i in range(m)])
+    return A64[ridx], B64
+
+
+def time_oracle(A64, B64, rows_per_block: int, steps: int, warmup: int):
+    import oracle
+    o2 = oracle.kron(oracle.strassen(), oracle.strassen())
+    As, Bs = oracle_sample(A64, B64, rows_per_block)
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.scheme_gemm(o2, As, Bs, pd="bf16", od="bf16")
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    t = float(np.mean(times))
+    flops = 2.0 * As.shape[0] * C2["K"] * C2["N"]
+    return flops / t / 1e12, t, oracle.num_threads(), As.shape[0]
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    _, _, A64, B64 = c2_inputs(0)
+    rpb = 256
+    val, t, cores, rows = time_oracle(A64, B64, rpb, args.steps, args.warmup)
+    sample = f"rows 0..{rpb - 1} of each of the 4 block rows of A ({rows} of {C2['M']} rows), full K and N, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "c2: two-level Strassen <4,4,4;49>, bf16, M=K=N=4096 (CPU oracle on a row sample)",
+                   "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ our arm
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(bf16=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"], hbm=p["hbm_gbs"], src="measured")
+    return dict(bf16=1590.0, bf16_sustained=1400.0, hbm=6650.0, src="fallback")
+
+
+def ncu_traffic_per_launch():
+    """DRAM bytes per launch of the block-product kernel at the bench workload, from the committed ncu
+    summary (profiles/traffic.json), or None when no capture has been recorded."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        return json.load(open(path))["block_products_c2_dram_bytes_per_launch"]
+    except Exception:
+        return None
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_39816_b200 as fmm
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- inputs: one independent problem per rank (weak scaling; the GEMM path does not shard)
+    At_h, Bt_h, A64, B64 = c2_inputs(rank)
+    A_h, B_h = At_h.pin_memory(), Bt_h.pin_memory()
+    A, B = A_h.to(dev), B_h.to(dev)
+    M, K, N = C2["M"], C2["K"], C2["N"]
+    s = fmm.scheme_builtin(C2["scheme"])
+    d = fmm.GemmDesc.make(M, K, N, "bf16", "bf16", "bf16", weight_layout=True)
+    ws = torch.empty(fmm.scheme_gemm_workspace(s, d), dtype=torch.uint8, device=dev)
+    C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    C_h = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    wsc = torch.empty(max(fmm.classical_gemm_workspace(d), 256), dtype=torch.uint8, device=dev)
+    Ccl = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            flush.zero_()
+            fn()
+        barrier()
+        evs = []
+        for _ in range(steps):
+            flush.zero_()                       # evict L2 (not timed)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            evs.append((e0, e1))
+        barrier()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    step = lambda: fmm.scheme_gemm(s, d, A, B, C, ws)  # noqa: E731
+
+    # ---- timed region: K steps of the whole path, inputs resident in HBM
+    sampler = ClockSampler(local)
+    timed(step, 0, args.warmup)
+    fmm.profile_enable(True)
+    fmm.profile_collect()
+    launches0 = fmm.launch_count()
+    sampler.start()
+    times = timed(step, args.steps, 0)
+    clocks = sampler.stop()
+    launches = fmm.launch_count() - launches0
+    phases = fmm.profile_collect()
+    fmm.profile_enable(False)
+    fmm.device_status(ws)
+    ms_step = max_over_ranks(float(np.mean(times)))
+    flops_eff = 2.0 * M * N * K
+    flops_r = 2.0 * C2["R"] * (M // 4) * (K // 4) * (N // 4)
+    value = world * flops_eff / (ms_step * 1e-3) / 1e12
+
+    # ---- same path with B's block sums cached (weights are static)
+    d_reuse = fmm.GemmDesc.make(M, K, N, "bf16", "bf16", "bf16", weight_layout=True, flags=fmm.FLAG_REUSE_BHAT)
+    t_reuse = float(np.mean(timed(lambda: fmm.scheme_gemm(s, d_reuse, A, B, C, ws), args.steps, 1)))
+
+    # ---- classical comparator built in the same library (same tcgen05 kernel, R = 1)
+    t_cl = float(np.mean(timed(lambda: fmm.classical_gemm(d, A, B, Ccl, wsc), args.steps, args.warmup)))
+
+    # ---- end to end: host buffers, copies inside the timed region
+    def e2e_step():
+        A.copy_(A_h, non_blocking=True)
+        B.copy_(B_h, non_blocking=True)
+        fmm.scheme_gemm(s, d, A, B, C, ws)
+        C_h.copy_(C, non_blocking=True)
+    t_e2e = max_over_ranks(float(np.mean(timed(e2e_step, args.steps, args.warmup))))
+    h2d = A_h.numel() * 2 + B_h.numel() * 2
+    d2h = C_h.numel() * 2
+
+    # ---- roofline of the dominant kernel (block products), timed live by the library's phase events
+    peaks = measured_peaks()
+    prod_ms, prod_n = phases["products"]
+    t_prod = prod_ms / max(prod_n, 1)
+    achieved = flops_r / (t_prod * 1e-3) / 1e12 if t_prod > 0 else 0.0
+    roofline = {"bound": "tensor", "kernel": "block_products_kernel<256,bf16>", "achieved": achieved,
+                "peak": peaks["bf16"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16"],
+                "peak_source": f"{peaks['src']} bf16 burst", "frac_of_sustained": achieved / peaks["bf16_sustained"],
+                "flops_per_launch": flops_r, "ms_per_launch": t_prod, "traffic": ncu_traffic_per_launch()}
+    bm, bk, bn = M // 4, K // 4, N // 4
+    pass_bytes = {  # algorithmic bytes of the streaming passes (read once + write once)
+        "encode_a": M * K * 2 + 49 * bm * bk * 2,
+        "encode_b": N * K * 2 + 49 * bn * bk * 2,
+        "decode": 49 * bm * bn * 4 + M * N * 2,
+    }
+    phase_out = {}
+    for name in ("encode_a", "encode_b", "products", "decode"):
+        ms, n = phases[name]
+        per = ms / max(n, 1)
+        phase_out[name] = {"ms": per}
+        if name in pass_bytes and per > 0:
+            gbs = pass_bytes[name] / (per * 1e-3) / 1e9
+            phase_out[name].update(gb_per_s=gbs, frac_of_hbm_peak=gbs / peaks["hbm"])
+
+    # ---- gauge sweep (c3), gauges sharded over ranks
+    sweep = None
+    if args.sweep_gauges > 0:
+        A3h, B3h = c3_inputs(0)
+        A3, B3 = A3h.to(dev), B3h.to(dev)
+        s1 = fmm.scheme_builtin(C3["scheme"])
+        d3 = fmm.GemmDesc.make(C3["M"], C3["K"], C3["N"], "bf16", "bf16", "bf16", weight_layout=True)
+        G = args.sweep_gauges * world
+        P, Q, S = sweep_gauges(G)
+        mine = shard_gauges(G, rank, world)
+        ws3 = torch.empty(fmm.error_sweep_workspace(s1, d3, len(mine)), dtype=torch.uint8, device=dev)
+        Cs = torch.empty((C3["M"], C3["N"]), dtype=torch.float64, device=dev)
+        fmm.exact_gemm_f64(d3, A3, B3, Cs)
+        fmm.error_sweep(s1, 0, P[mine][:2], Q[mine][:2], S[mine][:2], d3, A3, B3, ws3, Cstar=Cs)   # warm-up
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ratios, summ = fmm.error_sweep(s1, 0, P[mine], Q[mine], S[mine], d3, A3, B3, ws3, Cstar=Cs)
+        e1.record()
+        barrier()
+        t_sweep = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+        full = gather_ratios(torch.from_numpy(ratios), mine, G, rank, world, device=dev).cpu().numpy()
+        srt = np.sort(full)
+        sweep = {"workload": "c3: <2,2,2;7> one level, bf16, A 2048x4096, B 4096x4096, log-uniform-cond GL2 gauges",
+                 "gauges": G, "seconds": t_sweep, "gauges_per_s": G / t_sweep,
+                 "tensor_bound_gauges_per_s": peaks["bf16"] * 1e12 / (2.0 * 7 * 1024 * 2048 * 2048),
+                 "min": float(srt[0]), "median": float(srt[G // 2]), "max": float(srt[-1]),
+                 "count_gt2": int((full > 2).sum()), "e_classical_rel": summ["e_classical_rel"],
+                 "includes": "classical product + its error, reference norm, G x (encode A, encode B, 7 products, decode+error)"}
+        del ws3, Cs, A3, B3
+
+    # ---- CPU oracle timed beside it (rank 0, N=1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, t, cores, rows = time_oracle(A64, B64, C2["M"] // 4, 1, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": t,
+               "sample": f"the full c2 workload once ({rows} rows): encode, 49 fp64 block products, decode"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": "c2: two-level Strassen <4,4,4;49>, bf16 in / bf16 block sums / fp32 products / bf16 out, "
+                                   "M=K=N=4096, A~N(0,1) with 0.5% K-columns x100, B~N(0,0.02) stored [N,K]",
+                       "step": "encode A + encode B + 49 block products (tcgen05) + decode",
+                       "l2": f"flushed between steps by zeroing a {L2_FLUSH_BYTES >> 20} MiB buffer (untimed)",
+                       "parallelism": "replicas" if world > 1 else "single GPU"},
+            "clocks": clocks,
+            "e2e": {"value": world * flops_eff / (t_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": t_e2e,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches,
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "r_product_tflops": world * flops_r / (ms_step * 1e-3) / 1e12,
+            "r_product_frac_of_peak": flops_r / (ms_step * 1e-3) / 1e12 / peaks["bf16"],
+            "weights_cached": {"ms_per_step": t_reuse, "value": flops_eff / (t_reuse * 1e-3) / 1e12},
+            "classical_same_library": {"ms": t_cl, "tflops": flops_eff / (t_cl * 1e-3) / 1e12,
+                                       "scheme_time_over_classical": float(np.mean(times)) / t_cl},
+            "phases": phase_out,
+            "sweep": sweep,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep-gauges", type=int, default=32, help="gauges per rank in the c3 sweep (0 = skip)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -205,6 +205,15 @@ const char* fmm_status_string(fmm_status st);
 /* Number of kernels this library has launched in this process (for benchmarks' accounting). */
 int64_t fmm_launch_count(void);
 
+/* Phase timing.  While enabled, every device call brackets each step of the path with CUDA events on
+ * the caller's stream (events only; no synchronisation, no change to the kernels).  Phases:
+ *   0 encode A   1 encode B (incl. the transpose of a K x N operand)   2 block products (scheme)
+ *   3 decode (+ error reduction)   4 block products of classical_gemm   5 everything else.
+ * fmm_profile_collect synchronises the recorded events, adds their durations (milliseconds) to ms[8]
+ * and the number of bracketed regions to count[8] (HOST arrays, overwritten), and clears the record. */
+void fmm_profile_enable(int on);
+fmm_status fmm_profile_collect(double ms[8], int64_t count[8]);
+
 #ifdef __cplusplus
 }
 #endif

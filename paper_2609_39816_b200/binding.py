@@ -21,7 +21,8 @@ EXPORTED_SYMBOLS = [
     "scheme_load", "scheme_builtin", "scheme_kron", "gauge_apply", "scheme_info", "scheme_coefficients",
     "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius",
-    "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count",
+    "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
+    "fmm_profile_collect",
 ]
 
 
@@ -93,6 +94,9 @@ _lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(Gem
 _lib.fmm_status_string.argtypes = [C.c_int]
 _lib.fmm_status_string.restype = C.c_char_p
 _lib.fmm_launch_count.restype = C.c_int64
+_lib.fmm_profile_enable.argtypes = [C.c_int]
+_lib.fmm_profile_enable.restype = None
+_lib.fmm_profile_collect.argtypes = [_dp, C.POINTER(C.c_int64)]
 
 
 def lib_path() -> str:
@@ -242,3 +246,18 @@ def device_status(ws) -> None:
 
 def launch_count() -> int:
     return int(_lib.fmm_launch_count())
+
+
+PHASES = ["encode_a", "encode_b", "products", "decode", "classical_products", "other"]
+
+
+def profile_enable(on: bool) -> None:
+    _lib.fmm_profile_enable(int(on))
+
+
+def profile_collect() -> dict:
+    """{phase: (total milliseconds, number of bracketed regions)} since the last collect."""
+    ms = np.zeros(8)
+    cnt = (C.c_int64 * 8)()
+    _check(_lib.fmm_profile_collect(ms.ctypes.data_as(_dp), cnt), "fmm_profile_collect")
+    return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(PHASES)}

@@ -10,6 +10,26 @@
 
 #include "kernels_stream.cuh"
 
+// ---------------------------------------------------------------- phase timing
+namespace {
+struct ProfRec { int kind; cudaEvent_t a, b; };
+bool g_prof_on = false;
+std::vector<ProfRec> g_prof;
+}  // namespace
+
+ProfScope::ProfScope(int kind, cudaStream_t s) : slot(-1), st(s) {
+  if (!g_prof_on) return;
+  ProfRec r{kind, nullptr, nullptr};
+  if (cudaEventCreate(&r.a) != cudaSuccess) return;
+  if (cudaEventCreate(&r.b) != cudaSuccess) { cudaEventDestroy(r.a); return; }
+  cudaEventRecord(r.a, st);
+  g_prof.push_back(r);
+  slot = (int)g_prof.size() - 1;
+}
+ProfScope::~ProfScope() {
+  if (slot >= 0) cudaEventRecord(g_prof[slot].b, st);
+}
+
 namespace {
 
 inline size_t align_up(size_t x, size_t a = 1024) { return (x + a - 1) / a * a; }
@@ -99,10 +119,15 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
   float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
   float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
 
-  FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
-  if (!skip_b)
+  {
+    ProfScope ps(0, st);
+    FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
+  }
+  if (!skip_b) {
+    ProfScope ps(1, st);
     FMM_TRY(encode_operand(d, Bsrc_kmajor, ldb_kmajor, n, k, bn, bk, dB_tab, at<char>(ws, L.bhat),
                            at<unsigned>(ws, L.amaxB), sB, st));
+  }
   BlockProductArgs g{};
   g.product = d->product;
   g.A = at<char>(ws, L.ahat); g.lda = bk; g.a_batch = bm * bk;
@@ -110,7 +135,11 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
   g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = R;
   g.out = at<char>(ws, L.prod); g.ldo = bn; g.o_batch = bm * bn; g.out_mode = 0; g.output = FMM_F32;
   g.status = at<DeviceStatus>(ws, L.status);
-  FMM_TRY(launch_block_products(g, st));
+  {
+    ProfScope ps(2, st);
+    FMM_TRY(launch_block_products(g, st));
+  }
+  ProfScope ps(3, st);
   int np = 0;
   FMM_CUDA(launch_decode(d->output, at<float>(ws, L.prod), dW_tab, sA, sB, m, n, bm, bn, C, d->ldc, cstar32,
                          at<double>(ws, L.partials), &np, st));
@@ -123,6 +152,7 @@ fmm_status kmajor_b(const fmm_gemm_desc* d, const void* B, void* ws, size_t bt_o
                     bool skip, cudaStream_t st) {
   if (d->b_is_weight_layout) { *out = B; *ld = d->ldb; return FMM_OK; }
   void* bt = at<char>(ws, bt_off);
+  ProfScope ps(1, st);
   if (!skip) FMM_CUDA(launch_transpose(esize(d->storage), B, d->ldb, d->K, d->N, bt, st));
   *out = bt; *ld = d->K;
   return FMM_OK;
@@ -182,6 +212,7 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     const bool scaled = d->scale_mode == 1;
     float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
     float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
+    ProfScope pe(5, st);
     FMM_TRY(encode_operand(d, A, d->lda, 1, 1, d->M, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.ahat),
                            at<unsigned>(ws, L.amaxA), sA, st));
     FMM_TRY(encode_operand(d, bk_ptr, bk_ld, 1, 1, d->N, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.bhat),
@@ -190,6 +221,7 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
     g.sA = sA; g.sB = sB;
   }
+  ProfScope ps(4, st);
   return launch_block_products(g, st);
 }
 
@@ -220,6 +252,22 @@ SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
 extern "C" {
 
 int64_t fmm_launch_count(void) { return fmm_launch_counter(); }
+
+void fmm_profile_enable(int on) { g_prof_on = on != 0; }
+
+fmm_status fmm_profile_collect(double ms[8], int64_t count[8]) {
+  if (!ms || !count) return FMM_ERR_ARG;
+  for (int i = 0; i < 8; ++i) { ms[i] = 0.0; count[i] = 0; }
+  fmm_status rc = FMM_OK;
+  for (ProfRec& r : g_prof) {
+    float t = 0.f;
+    if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) rc = FMM_ERR_CUDA;
+    if (r.kind >= 0 && r.kind < 8) { ms[r.kind] += t; count[r.kind] += 1; }
+    cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+  }
+  g_prof.clear();
+  return rc;
+}
 
 size_t scheme_gemm_workspace(const fmm_scheme* s, const fmm_gemm_desc* d) {
   if (!s || check_desc(d, s->m, s->k, s->n) != FMM_OK) return 0;

@@ -63,3 +63,11 @@ struct BlockProductArgs {
   DeviceStatus* status;
 };
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
+
+// Phase timing (see fmm_profile_enable): RAII bracket of a region of the caller's stream.
+struct ProfScope {
+  ProfScope(int kind, cudaStream_t st);
+  ~ProfScope();
+  int slot;
+  cudaStream_t st;
+};

@@ -1,0 +1,144 @@
+"""Host-side checks of the C-ABI library that need no GPU: the shared object loads and exports every
+symbol the header declares; scheme handles, nesting, gauges and criteria agree with the oracle (the two
+share no code); argument validation returns the documented status codes."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from fmm_inputs import generators as gen
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import __graft_entry__
+    __graft_entry__.build()
+    import paper_2609_39816_b200 as fmm
+    return fmm
+
+
+def test_header_symbols_are_exported(lib):
+    header = open(os.path.join(ROOT, "include", "fmm_b200.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(\w+)\s*\([^;{]*\)\s*;", header))
+    declared -= {"defined"}
+    assert {"scheme_load", "gauge_apply", "scheme_gemm", "error_sweep"} <= declared
+    so = ctypes.CDLL(lib.lib_path())
+    for name in declared:
+        assert hasattr(so, name), f"{name} declared in the header but not exported"
+    assert declared == set(lib.EXPORTED_SYMBOLS)
+
+
+def test_builtin_schemes_match_oracle_tables(lib):
+    s1, s2 = oracle.strassen(), oracle.kron(oracle.strassen(), oracle.strassen())
+    for name, o in (("strassen222", s1), ("strassen444", s2), ("classical222", oracle.classical_scheme(2, 2, 2))):
+        s = lib.scheme_builtin(name)
+        U, V, W = s.coefficients()
+        assert s.dims == o.dims
+        assert np.array_equal(U, o.U) and np.array_equal(V, o.V) and np.array_equal(W, o.W)
+        info, crit = s.info, oracle.criteria(o)
+        assert info == crit
+    assert lib.scheme_builtin("strassen444").info["Phi"] == 1024.0
+
+
+def test_scheme_load_checks_brent(lib):
+    o = oracle.strassen()
+    s = lib.scheme_load(o.U, o.V, o.W)
+    assert s.dims == (2, 2, 2, 7)
+    W = o.W.copy()
+    W[3, 0, 0] = -W[3, 0, 0]                         # one flipped decoding coefficient must be rejected
+    with pytest.raises(lib.FmmError) as e:
+        lib.scheme_load(o.U, o.V, W)
+    assert e.value.code == 3
+    big = oracle.classical_scheme(3, 3, 3)
+    lib.scheme_load(big.U, big.V, big.W)
+    with pytest.raises(lib.FmmError) as e:           # R = 125 > table limit
+        c5 = oracle.classical_scheme(5, 5, 5)
+        lib.scheme_load(c5.U, c5.V, c5.W)
+    assert e.value.code == 9
+    with pytest.raises(lib.FmmError):
+        lib.scheme_builtin("no-such-scheme")
+
+
+def test_kron_and_gauges_match_oracle(lib):
+    o1 = oracle.strassen()
+    s1 = lib.scheme_builtin("strassen222")
+    s2 = lib.scheme_kron(s1, s1)
+    o2 = oracle.kron(o1, o1)
+    assert np.array_equal(s2.coefficients()[0], o2.U)
+    # sign variants: exact, equal to the printed formula
+    for d, e, f in oracle.sign_variants(4, 4, 4)[::73]:
+        g = lib.gauge_apply(s2, np.diag(d), np.diag(e), np.diag(f))
+        ov = oracle.sign_variant(o2, d, e, f)
+        U, V, W = g.coefficients()
+        assert np.array_equal(U, ov.U) and np.array_equal(V, ov.V) and np.array_equal(W, ov.W)
+        assert g.info == s2.info
+    # identity gauge is the base scheme bit for bit
+    g = lib.gauge_apply(s1, np.eye(2), np.eye(2), np.eye(2))
+    assert all(np.array_equal(a, b) for a, b in zip(g.coefficients(), s1.coefficients()))
+    # general gauges, flat and on the outer factor
+    for idx in range(4):
+        P, Q, S = (gen.gauge_log_uniform_cond(3, 3 * idx + i, 2) for i in range(3))
+        g = lib.gauge_apply(s1, P, Q, S)
+        og = oracle.gauge(o1, P, Q, S)
+        for a, b in zip(g.coefficients(), (og.U, og.V, og.W)):
+            assert np.allclose(a, b, rtol=1e-12, atol=1e-12 * np.abs(b).max())
+        g2 = lib.gauge_apply(s2, P, Q, S, level=1)
+        og2 = oracle.kron(og, o1)
+        for a, b in zip(g2.coefficients(), (og2.U, og2.V, og2.W)):
+            assert np.allclose(a, b, rtol=1e-12, atol=1e-12 * np.abs(b).max())
+        U2, V2, W2 = g2.coefficients()
+        scale = 49 * np.abs(U2).max() * np.abs(V2).max() * np.abs(W2).max()
+        assert oracle.brent_residual(oracle.Scheme(U2, V2, W2)) <= 1e-13 * scale
+    with pytest.raises(lib.FmmError) as e:
+        lib.gauge_apply(s1, np.zeros((2, 2)), np.eye(2), np.eye(2))
+    assert e.value.code == 4
+    with pytest.raises(lib.FmmError) as e:           # condition limit
+        lib.gauge_apply(s1, np.diag([1.0, 1e-3]), np.eye(2), np.eye(2), cond_limit=10.0)
+    assert e.value.code == 4
+    with pytest.raises(lib.FmmError):                # level 1 needs a nested handle
+        lib.gauge_apply(s1, np.eye(2), np.eye(2), np.eye(2), level=1)
+
+
+def test_descriptor_validation_without_gpu(lib):
+    s2 = lib.scheme_builtin("strassen444")
+    ok = lib.GemmDesc.make(4096, 4096, 4096, "bf16", "bf16", "bf16")
+    need = lib.scheme_gemm_workspace(s2, ok)
+    bm = 1024
+    assert need >= 49 * bm * bm * (2 + 2 + 4)
+    assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4098, 4096, 4096, "bf16", "bf16", "bf16")) == 0
+    assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4096, 4096 + 32, 4096, "bf16", "bf16", "bf16")) == 0
+    assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4096, 4096, 4096, "bf16", "bf16", "bf16", scale_mode=1)) == 0
+    assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4096, 4096, 4096, "bf16", "e4m3", "bf16", scale_mode=1)) > 0
+    assert lib.error_sweep_workspace(s2, ok, 4) > need
+    assert lib.classical_gemm_workspace(ok) > 0
+    lay = lib.scheme_gemm_workspace_layout(s2, ok)
+    assert lay["Ahat"] < lay["Bhat"] < lay["M"] < need and all(v % 256 == 0 for v in lay.values())
+
+
+def test_sweep_sharding_over_ranks_gloo():
+    """Gauges are independent units: rank r of W takes gauges r, r+W, ...; results are gathered on rank 0.
+    Run as two gloo ranks on CPU with a stand-in ratio function (the partitioning logic is what is tested)."""
+    import torch.multiprocessing as mp
+    from bench import shard_gauges  # noqa: F401  (import check)
+    port = 29500 + os.getpid() % 1000
+    mp.spawn(_shard_worker, args=(2, port), nprocs=2, join=True)
+
+
+def _shard_worker(rank, world, port):
+    import torch
+    import torch.distributed as dist
+    from bench import gather_ratios, shard_gauges
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    G = 13
+    mine = shard_gauges(G, rank, world)
+    local = torch.tensor([float(g) * 1.5 for g in mine], dtype=torch.float64)
+    full = gather_ratios(local, mine, G, rank, world, device="cpu")
+    if rank == 0:
+        assert full.tolist() == [g * 1.5 for g in range(G)]
+    dist.destroy_process_group()
