@@ -90,42 +90,49 @@ T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws)
 
 // Encode one operand: optional amax pass, then block sums -> product dtype.
 fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
-                          const CoefTable* d_tab, void* hat, unsigned* amax, float* scale, cudaStream_t st) {
+                          const CoefTable* d_tab, const CoefTable* h_tab, void* hat, unsigned* amax, float* scale, cudaStream_t st) {
   const bool scaled = d->scale_mode == 1;
   if (scaled) {
     FMM_CUDA(cudaMemsetAsync(amax, 0, FMM_MAX_R * 4, st));
-    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, hat, amax, scale, true, true, st));
+    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, amax, scale, true, true, st));
   }
-  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, hat, amax, scale, false, scaled, st));
+  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, amax, scale, false, scaled, st));
   return FMM_OK;
 }
 
 // The whole path for one scheme on one operand pair.  If C is null the result is not stored; if cstar32 is
-// given the squared error is reduced into err_out[0] (device).  `tables` are host tables to upload, or null
-// when the device tables at L.tab* are already in place.
+// given the squared error is reduced into err_out[0] (device).  hA/hB/hW are the host tables (always given:
+// their entry counts size the kernels' shared memory); they are uploaded into the workspace unless device
+// copies dA_tab/dB_tab/dW_tab are already in place.
 fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLayout& L, const CoefTable* hA,
                       const CoefTable* hB, const CoefTable* hW, const CoefTable* dA_tab, const CoefTable* dB_tab,
                       const CoefTable* dW_tab, const void* A, const void* Bsrc_kmajor, int64_t ldb_kmajor, void* C,
                       const float* cstar32, double* err_out, void* ws, bool skip_b, cudaStream_t st) {
   const int m = s->m, k = s->k, n = s->n, R = s->R;
   const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
-  if (hA) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabA), hA, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
-  if (hB && !skip_b) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabB), hB, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
-  if (hW) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabW), hW, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
-  if (!dA_tab) dA_tab = at<CoefTable>(ws, L.tabA);
-  if (!dB_tab) dB_tab = at<CoefTable>(ws, L.tabB);
-  if (!dW_tab) dW_tab = at<CoefTable>(ws, L.tabW);
+  if (!dA_tab) {
+    FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabA), hA, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    dA_tab = at<CoefTable>(ws, L.tabA);
+  }
+  if (!dB_tab) {
+    if (!skip_b) FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabB), hB, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    dB_tab = at<CoefTable>(ws, L.tabB);
+  }
+  if (!dW_tab) {
+    FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabW), hW, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    dW_tab = at<CoefTable>(ws, L.tabW);
+  }
   const bool scaled = d->scale_mode == 1;
   float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
   float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
 
   {
     ProfScope ps(0, st);
-    FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
+    FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, hA, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
   }
   if (!skip_b) {
     ProfScope ps(1, st);
-    FMM_TRY(encode_operand(d, Bsrc_kmajor, ldb_kmajor, n, k, bn, bk, dB_tab, at<char>(ws, L.bhat),
+    FMM_TRY(encode_operand(d, Bsrc_kmajor, ldb_kmajor, n, k, bn, bk, dB_tab, hB, at<char>(ws, L.bhat),
                            at<unsigned>(ws, L.amaxB), sB, st));
   }
   BlockProductArgs g{};
@@ -141,7 +148,7 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
   }
   ProfScope ps(3, st);
   int np = 0;
-  FMM_CUDA(launch_decode(d->output, at<float>(ws, L.prod), dW_tab, sA, sB, m, n, bm, bn, C, d->ldc, cstar32,
+  FMM_CUDA(launch_decode(d->output, at<float>(ws, L.prod), dW_tab, hW, R, sA, sB, m, n, bm, bn, C, d->ldc, cstar32,
                          at<double>(ws, L.partials), &np, st));
   if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(ws, L.partials), np, err_out, st));
   return FMM_OK;
@@ -213,9 +220,9 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
     float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
     ProfScope pe(5, st);
-    FMM_TRY(encode_operand(d, A, d->lda, 1, 1, d->M, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.ahat),
+    FMM_TRY(encode_operand(d, A, d->lda, 1, 1, d->M, d->K, at<CoefTable>(ws, L.tab), &t, at<char>(ws, L.ahat),
                            at<unsigned>(ws, L.amaxA), sA, st));
-    FMM_TRY(encode_operand(d, bk_ptr, bk_ld, 1, 1, d->N, d->K, at<CoefTable>(ws, L.tab), at<char>(ws, L.bhat),
+    FMM_TRY(encode_operand(d, bk_ptr, bk_ld, 1, 1, d->N, d->K, at<CoefTable>(ws, L.tab), &t, at<char>(ws, L.bhat),
                            at<unsigned>(ws, L.amaxB), sB, st));
     g.A = at<char>(ws, L.ahat); g.lda = d->K; g.a_batch = 0;
     g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
@@ -413,8 +420,8 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   const void* bk_ptr; int64_t bk_ld;
   FMM_TRY(kmajor_b(d, dB, gws, L.g.bt, &bk_ptr, &bk_ld, false, st));
   for (int g = 0; g < G; ++g) {
-    FMM_TRY(run_scheme(base, d, L.g, nullptr, nullptr, nullptr, d_tabs + 3 * g, d_tabs + 3 * g + 1, d_tabs + 3 * g + 2,
-                       dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
+    FMM_TRY(run_scheme(base, d, L.g, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2], d_tabs + 3 * g, d_tabs + 3 * g + 1,
+                       d_tabs + 3 * g + 2, dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
   }
 
   // 5. results to the host

@@ -29,7 +29,8 @@ struct CoefTable {
 
 // host helpers (scheme_host.cpp)
 // tA: cells of A's m x k grid; tB: cells of B^T's n x k grid (B is always read K-major), entries in
-// ascending (l,j) order of V; tW: cells of C's m x n grid.  Any pointer may be null.
+// ascending (l,j) order of V; tW: cell-major decode table (R field = m*n lists, `cell` = product index r,
+// ascending).  Any pointer may be null.
 void fmm_build_tables(const fmm_scheme& s, CoefTable* tA, CoefTable* tB, CoefTable* tW);
 fmm_status fmm_gauge_core(const fmm_scheme& in, int level, const double* P, const double* Q, const double* S,
                           double cond_limit, fmm_scheme** out);

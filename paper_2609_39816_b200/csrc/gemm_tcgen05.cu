@@ -17,7 +17,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
-#include <cstdio>
+#include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "kernels_stream.cuh"
@@ -148,6 +149,62 @@ __host__ __device__ constexpr uint32_t make_idesc(bool fp8, int n) {
          ((uint32_t)(BM >> 4) << 24);
 }
 
+// 32-byte store: one full L2 sector per thread (16-byte stores touch half a sector each and double the
+// sector writes L2 sees).
+__device__ __forceinline__ void st_global_256(void* p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t a4, uint32_t a5, uint32_t a6, uint32_t a7) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a0), "r"(a1), "r"(a2),
+               "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&b2);
+}
+
+// Store up to 32 consecutive columns of one accumulator row (fp32 products, or the scaled and rounded result).
+// `wide` = the destination row is 32-byte aligned.
+__device__ __forceinline__ void store_row_chunk(void* out, long long off, int ncols, const uint32_t (&v)[32],
+                                                int out_mode, int out_bf16, float alpha, bool wide) {
+  if (out_mode == 1 && out_bf16) {
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + off;
+    if (ncols == 32) {
+      uint32_t w[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]) * alpha, __uint_as_float(v[2 * j + 1]) * alpha);
+      if (wide) {
+        st_global_256(dst, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+        st_global_256(dst + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) *reinterpret_cast<uint4*>(dst + 2 * j) = make_uint4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < ncols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * alpha);
+    }
+    return;
+  }
+  float* dst = reinterpret_cast<float*>(out) + off;
+  const float a = out_mode == 1 ? alpha : 1.0f;   // fp32 products are stored unscaled (x * 1.0f is exact)
+  if (ncols == 32) {
+    uint32_t w[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) w[j] = __float_as_uint(__uint_as_float(v[j]) * a);
+    if (wide) {
+#pragma unroll
+      for (int j = 0; j < 32; j += 8) st_global_256(dst + j, w[j], w[j + 1], w[j + 2], w[j + 3], w[j + 4], w[j + 5], w[j + 6], w[j + 7]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) *reinterpret_cast<uint4*>(dst + j) = make_uint4(w[j], w[j + 1], w[j + 2], w[j + 3]);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < ncols) dst[j] = __uint_as_float(v[j]) * a;
+  }
+}
+
 template <int BN>
 struct SmemLayout {
   static constexpr int kStages = (BN == 256) ? 4 : 6;
@@ -167,6 +224,7 @@ struct TileParams {
   long long ldo, o_batch;   // output strides in elements
   int out_mode;             // 0: fp32 products; 1: scaled + rounded result
   int out_bf16;             // out_mode 1: 1 -> bf16, 0 -> fp32
+  int wide;                 // every output row starts on a 32-byte boundary
 };
 
 template <int BN, bool kFp8>
@@ -319,55 +377,8 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         tc_ld32(taddr, v);
         tc_wait_ld();
         const int col0 = tn * BN + c * 32;
-        if (row_ok && col0 < tp.rows_b) {
-          const int ncols = min(32, tp.rows_b - col0);
-          if (tp.out_mode == 0) {
-            float* dst = reinterpret_cast<float*>(out) + row_off + col0;
-            if (ncols == 32) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols) dst[j] = __uint_as_float(v[j]);
-            }
-          } else if (tp.out_bf16) {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(out) + row_off + col0;
-            if (ncols == 32) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 pk;
-                uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
-#pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                  __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2 * h]) * alpha,
-                                                            __uint_as_float(v[j + 2 * h + 1]) * alpha);
-                  pw[h] = *reinterpret_cast<uint32_t*>(&b2);
-                }
-                *reinterpret_cast<uint4*>(dst + j) = pk;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * alpha);
-            }
-          } else {
-            float* dst = reinterpret_cast<float*>(out) + row_off + col0;
-            if (ncols == 32) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) =
-                    make_float4(__uint_as_float(v[j]) * alpha, __uint_as_float(v[j + 1]) * alpha,
-                                __uint_as_float(v[j + 2]) * alpha, __uint_as_float(v[j + 3]) * alpha);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (j < ncols) dst[j] = __uint_as_float(v[j]) * alpha;
-            }
-          }
-        }
+        if (row_ok && col0 < tp.rows_b)
+          store_row_chunk(out, row_off + col0, min(32, tp.rows_b - col0), v, tp.out_mode, tp.out_bf16, alpha, tp.wide != 0);
       }
       tc_fence_before();
       __syncwarp();
@@ -381,6 +392,236 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- CTA-pair kernel (cta_group::2)
+// Two CTAs of a cluster (consecutive SMs) own one 256 x 256 output tile.  Each CTA loads its own 128 rows
+// of Ahat_r and HALF of the Bhat_r tile (128 of the 256 rows), so the pair moves 2/3 of the bytes two
+// independent 128 x 256 tiles would pull through L2.  The even CTA (leader) issues tcgen05.mma with
+// M = 256 for both; the accumulator rows [128*rank, 128*rank + 128) live in each CTA's own TMEM.
+//   - TMA loads of both CTAs complete on the LEADER's "full" barrier (cp.async.bulk.tensor ... .cta_group::2,
+//     barrier address with the CTA-rank bit cleared); the leader alone arms it with the pair's byte count;
+//   - tcgen05.commit.cta_group::2 with a two-CTA mask releases the ring stage in both CTAs and publishes the
+//     accumulator to both epilogues;
+//   - the epilogue warps of both CTAs hand the accumulator buffer back on the leader's barrier.
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address
+
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int c0,
+                                                 int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(leader_bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}"
+      ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+template <bool kFp8>
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  if (kFp8) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+struct PairLayout {
+  static constexpr int BN = 256;                 // columns of the pair's tile
+  static constexpr int kStages = 6;
+  static constexpr int kABytes = BM * BKB;       // this CTA's 128 rows of A
+  static constexpr int kBBytes = (BN / 2) * BKB; // this CTA's half of the B tile
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;
+};
+
+template <bool kFp8>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                           void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
+                           TileParams tp, DeviceStatus* status) {
+  using L = PairLayout;
+  constexpr int BN = L::BN;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - raw_addr);
+  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
+  const uint32_t bar_base = smem_u32(bar_mem);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                       // used in the leader only
+  auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };       // one per CTA
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };   // one per CTA
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };  // used in the leader only
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();   // 0 = leader
+  const bool leader = rank == 0;
+  constexpr uint32_t kTmemCols = 2 * BN;     // two accumulator buffers of 256 columns
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // both CTAs' barriers are initialised before anything signals across the pair
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_kb = (tp.kbytes + BKB - 1) / BKB;
+  const int tiles_m = (tp.rows_a + 2 * BM - 1) / (2 * BM);
+  const int tiles_n = (tp.rows_b + BN - 1) / BN;
+  const int tiles_per_batch = tiles_m * tiles_n;
+  const int total_tiles = tiles_per_batch * tp.batches;
+  const int kelems_per_stage = BKB / tp.elem_bytes;
+  const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
+        const int r = tile / tiles_per_batch;
+        const int rem = tile - r * tiles_per_batch;
+        const int tm = rem / tiles_n, tn = rem - tm * tiles_n;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status);
+          if (!ok) break;
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t sb = sa + L::kABytes;
+          const uint32_t lead_full = full_bar(stage) & kPeerBitMask;
+          if (leader) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)L::kStageBytes);
+          tma_load_3d_pair(sa, &map_a, lead_full, kb * kelems_per_stage, tm * 2 * BM + (int)rank * BM, r);
+          tma_load_3d_pair(sb, &map_b, lead_full, kb * kelems_per_stage, tn * BN + (int)rank * (BN / 2), r);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) __nanosleep(2000000);   // let copies already issued land before shared memory goes away
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      // M = 256 across the pair, N = 256
+      constexpr uint32_t idesc = (1u << 4) | ((kFp8 ? 0u : 1u) << 7) | ((kFp8 ? 0u : 1u) << 10) |
+                                 ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
+        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + L::kABytes);
+#pragma unroll
+          for (int k = 0; k < BKB / UMMA_KB; ++k)
+            tc_mma_pair<kFp8>(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc,
+                              (kb | k) != 0 ? 1u : 0u);
+          tc_commit_pair(empty_bar(stage));   // frees this stage in both CTAs
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar(acc));       // accumulator complete, visible to both epilogues
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) {
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(drain_bar)
+                     : "memory");
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0)) {
+          if (global_timer_ns() - t0 > 20000000ull) break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
+    const int quad = warp & 3;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    float alpha = 1.0f;
+    if (tp.out_mode == 1 && sA != nullptr && sB != nullptr) alpha = sA[0] * sB[0];
+    for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
+      const int r = tile / tiles_per_batch;
+      const int rem = tile - r * tiles_per_batch;
+      const int tm = rem / tiles_n, tn = rem - tm * tiles_n;
+      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = tm * 2 * BM + (int)rank * BM + quad * 32 + lane;
+      const bool row_ok = row < tp.rows_a;
+      const long long row_off = (long long)r * tp.o_batch + (long long)row * tp.ldo;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c * 32);
+        tc_ld32(taddr, v);
+        tc_wait_ld();
+        const int col0 = tn * BN + c * 32;
+        if (row_ok && col0 < tp.rows_b)
+          store_row_chunk(out, row_off + col0, min(32, tp.rows_b - col0), v, tp.out_mode, tp.out_bf16, alpha, tp.wide != 0);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tempty_bar(acc) & kPeerBitMask);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // neither CTA frees TMEM / leaves while its partner may still touch it
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -428,6 +669,12 @@ int sm_count() {
   return n;
 }
 
+// 1 when every output row (and batch) starts on a 32-byte boundary
+int rows_32b_aligned(const BlockProductArgs& a) {
+  const int es = (a.out_mode == 1 && a.output == FMM_BF16) ? 2 : 4;
+  return (reinterpret_cast<uintptr_t>(a.out) % 32 == 0) && ((a.ldo * es) % 32 == 0) && ((a.o_batch * es) % 32 == 0);
+}
+
 template <int BN, bool kFp8>
 fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   using L = SmemLayout<BN>;
@@ -443,6 +690,7 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   tp.tiles_n = (int)((a.rows_b + BN - 1) / BN);
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
   tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
+  tp.wide = rows_32b_aligned(a);
   const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
   if (total <= 0) return FMM_OK;
   const int sms = sm_count();
@@ -455,12 +703,56 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
+template <bool kFp8>
+fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
+  using L = PairLayout;
+  CUtensorMap ma, mb;
+  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, L::BN / 2)) return FMM_ERR_CUDA;
+  TileParams tp;
+  tp.rows_a = (int)a.rows_a; tp.rows_b = (int)a.rows_b;
+  tp.elem_bytes = kFp8 ? 1 : 2;
+  tp.kbytes = (int)a.kdim * tp.elem_bytes;
+  tp.batches = a.batches;
+  tp.tiles_m = (int)((a.rows_a + 2 * BM - 1) / (2 * BM));
+  tp.tiles_n = (int)((a.rows_b + L::BN - 1) / L::BN);
+  tp.ldo = a.ldo; tp.o_batch = a.o_batch;
+  tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
+  tp.wide = rows_32b_aligned(a);
+  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
+  if (total <= 0) return FMM_OK;
+  const int sms = sm_count();
+  if (sms < 2) return FMM_ERR_CUDA;
+  const long long pairs = std::min<long long>(total, sms / 2);
+  auto k = block_products_pair_kernel<kFp8>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
+    attr_done = true;
+  }
+  k<<<(unsigned)(2 * pairs), kNumThreads, L::kTotal, st>>>(ma, mb, a.out, a.sA, a.sB, tp, a.status);
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+bool pair_kernel_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char* e = std::getenv("FMM_B200_NO_PAIR");
+    on = (e && e[0] == '1') ? 0 : 1;
+  }
+  return on == 1;
+}
+
 }  // namespace
 
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
   if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim > 0x3fffffff) return FMM_ERR_SHAPE;
   const bool fp8 = (a.product == FMM_E4M3);
   if (!fp8 && a.product != FMM_BF16) return FMM_ERR_DTYPE;
+  // large problems: CTA pairs on 256 x 256 tiles (less L2 traffic per flop)
+  if (a.rows_a > 128 && a.rows_b > 128 && pair_kernel_enabled())
+    return fp8 ? launch_pair<true>(a, st) : launch_pair<false>(a, st);
   // narrow problems use the 128-column tile (less padding, more tiles in flight)
   const bool narrow = a.rows_b <= 128;
   if (fp8) return narrow ? launch_t<128, true>(a, st) : launch_t<256, true>(a, st);

@@ -1,6 +1,6 @@
 // Streaming kernels of the scheme GEMM: encode (block sums -> product dtype), transpose,
 // decode (+ error reduction), Frobenius error, fp64 reference.  All are HBM-bound passes;
-// each thread moves 16-byte (8-byte for bf16 sources) vectors and the grid covers the data once.
+// each thread moves 16-byte vectors and the grid covers the data once.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
@@ -15,22 +15,10 @@ int64_t& fmm_launch_counter() {
 
 namespace {
 
-constexpr int kThreads = 256;
 
 // ------------------------------------------------------------------------------------------
 // small device helpers
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
-__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
-  const uint2 raw = *reinterpret_cast<const uint2*>(p);
-  float4 v;
-  v.x = __uint_as_float(raw.x << 16);
-  v.y = __uint_as_float(raw.x & 0xFFFF0000u);
-  v.z = __uint_as_float(raw.y << 16);
-  v.w = __uint_as_float(raw.y & 0xFFFF0000u);
-  return v;
-}
-
 __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
   __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
@@ -40,13 +28,6 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
   *reinterpret_cast<uint2*>(p) = raw;
 }
 __device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
-// e4m3: round to nearest even, saturate to +-448 (NaN stays NaN)
-__device__ __forceinline__ void store4(__nv_fp8_storage_t* p, float4 v) {
-  const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v.x, v.y), __NV_SATFINITE, __NV_E4M3);
-  const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v.z, v.w), __NV_SATFINITE, __NV_E4M3);
-  *reinterpret_cast<uint32_t*>(p) = lo | (hi << 16);
-}
-
 __device__ __forceinline__ float round_out(float x, float*) { return x; }
 __device__ __forceinline__ float round_out(float x, __nv_bfloat16*) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
@@ -75,35 +56,89 @@ __device__ __forceinline__ double block_sum_double(double v, double* red /* >= 8
 
 // ------------------------------------------------------------------------------------------
 // encode: block sums of Eq. 1 (inner parentheses), scale, one rounding to the product dtype.
-// Each thread owns 4 consecutive inner-dimension elements of one block row; it stages the
-// 4-vectors of all grid cells at that position in shared memory (used as an indexable register
-// file, [cell][thread] so accesses are conflict free) and then walks the sparse coefficient list
-// of every product: an fp32 FMA chain in list order.
+// A block of 256 threads owns 64 "position vectors" (16 bytes = 8 bf16 or 4 fp32 consecutive
+// inner-dimension elements of one block row).  Four threads share each position vector:
+//   1. together they load the vectors of all grid cells at that position, convert them to fp32 once and
+//      park them in shared memory ([cell][half][position], conflict free; slab `ncell` holds zeros);
+//   2. thread g of the four then forms the products r = g, g+4, g+8, ...: it walks the coefficient list
+//      of r in chunks of kChunk entries (lists are padded to a multiple of kChunk with (zero slab, 0.0f)
+//      entries, which add exactly nothing), an fp32 FMA chain in list order, two lanes per instruction
+//      (packed fma.rn.f32x2: each lane is an ordinary IEEE fp32 FMA), and stores 16 / 8 bytes.
 // ------------------------------------------------------------------------------------------
-struct EncSmem {
-  CoefTable tab;
+constexpr int kEncThreads = 256;
+constexpr int kEncPos = 64;      // position vectors per block
+constexpr int kEncSplit = 4;     // threads per position vector
+constexpr int kChunk = 4;
+
+struct EncSmemHead {
+  int off[FMM_MAX_R + 1];   // in units of entries, multiples of kChunk
+  int pad[3];
   float scale[FMM_MAX_R];
   float inv_scale[FMM_MAX_R];
   int use_mul[FMM_MAX_R];
   unsigned amax[FMM_MAX_R];
+};  // followed by int2 ent[] {byte offset of the cell's slab, coefficient bits}, then the stage
+
+template <typename SrcT> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int kElems = 4;
+  static __device__ __forceinline__ void unpack(const uint4& raw, float4 (&v)[1]) {
+    v[0] = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
+  }
+};
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  static __device__ __forceinline__ void unpack(const uint4& raw, float4 (&v)[2]) {
+    v[0] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
+                       __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+    v[1] = make_float4(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xFFFF0000u),
+                       __uint_as_float(raw.w << 16), __uint_as_float(raw.w & 0xFFFF0000u));
+  }
 };
 
+template <int NP> __device__ __forceinline__ void store_vec(__nv_bfloat16* p, const float2 (&a)[NP]) {
+  uint32_t w[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(a[i].x, a[i].y);
+    w[i] = *reinterpret_cast<uint32_t*>(&b);
+  }
+  if (NP == 4) *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2 % NP], w[3 % NP]);
+  else *reinterpret_cast<uint2*>(p) = make_uint2(w[0], w[1]);
+}
+// e4m3: round to nearest even, saturate to +-448 (NaN stays NaN)
+template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* p, const float2 (&a)[NP]) {
+  uint32_t h[NP];
+#pragma unroll
+  for (int i = 0; i < NP; ++i) h[i] = __nv_cvt_float2_to_fp8x2(a[i], __NV_SATFINITE, __NV_E4M3);
+  if (NP == 4) *reinterpret_cast<uint2*>(p) = make_uint2(h[0] | (h[1] << 16), h[2 % NP] | (h[3 % NP] << 16));
+  else *reinterpret_cast<uint32_t*>(p) = h[0] | (h[1] << 16);
+}
+
 template <typename SrcT, typename DstT, bool kAmaxOnly>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
               const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
               float* __restrict__ scale_out, int use_scale) {
+  constexpr int VE = Vec16<SrcT>::kElems;
+  constexpr int NV = VE / 4;                     // float4 per staged vector
+  constexpr int NP = VE / 2;                     // float2 pairs per vector
+  constexpr int kHalf = kEncPos * 16;            // bytes of one float4 plane of a slab
+  constexpr int kSlab = NV * kHalf;              // bytes of one cell's slab
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  EncSmem& sm = *reinterpret_cast<EncSmem*>(smem_raw);
-  float4* stage = reinterpret_cast<float4*>(smem_raw + ((sizeof(EncSmem) + 15) / 16) * 16);
+  EncSmemHead& sm = *reinterpret_cast<EncSmemHead*>(smem_raw);
+  const int R = d_tab->R, ncell = d_tab->ncell;
+  int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(EncSmemHead));
 
-  {  // cooperative copy of the table
-    const int* src = reinterpret_cast<const int*>(d_tab);
-    int* dst = reinterpret_cast<int*>(&sm.tab);
-    for (int i = threadIdx.x; i < (int)(sizeof(CoefTable) / 4); i += kThreads) dst[i] = src[i];
+  // pad every list to a multiple of kChunk (lists are short; thread 0 lays out the offsets)
+  if (threadIdx.x == 0) {
+    int o = 0;
+    for (int r = 0; r < R; ++r) {
+      sm.off[r] = o;
+      o += (d_tab->off[r + 1] - d_tab->off[r] + kChunk - 1) / kChunk * kChunk;
+    }
+    sm.off[R] = o;
   }
-  __syncthreads();
-  const int R = sm.tab.R, ncell = sm.tab.ncell;
   if (threadIdx.x < R) {
     float s = 1.0f;
     if (!kAmaxOnly && use_scale) s = pow2_scale_448(__uint_as_float(amax_bits[threadIdx.x]));
@@ -115,36 +150,86 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     if (!kAmaxOnly && use_scale && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
   }
   __syncthreads();
+  const int total = sm.off[R];
+  for (int r = threadIdx.x; r < R; r += kEncThreads) {
+    const int s0 = d_tab->off[r], cnt = d_tab->off[r + 1] - s0, d0 = sm.off[r], padded = sm.off[r + 1] - d0;
+    for (int i = 0; i < padded; ++i)
+      ent[d0 + i] = i < cnt ? make_int2(d_tab->cell[s0 + i] * kSlab, __float_as_int(d_tab->coef[s0 + i]))
+                            : make_int2(ncell * kSlab, 0);
+  }
+  unsigned char* stage = smem_raw + ((sizeof(EncSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
 
-  const int64_t vec_per_row = bc >> 2;
-  const int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int g = threadIdx.x / kEncPos;           // which quarter of the cells / products this thread handles
+  const int pv = threadIdx.x - g * kEncPos;      // position vector inside the block
+  const int64_t vec_per_row = bc / VE;
+  const int64_t idx = (int64_t)blockIdx.x * kEncPos + pv;
   const bool live = idx < br * vec_per_row;
   const int64_t p = live ? idx / vec_per_row : 0;
-  const int64_t t = live ? (idx - p * vec_per_row) << 2 : 0;
+  const int64_t t = live ? (idx - p * vec_per_row) * VE : 0;
+  unsigned char* my_stage = stage + pv * 16;
 
-  if (live) {
-    for (int c = 0; c < ncell; ++c) {
+  for (int c0 = g; c0 < ncell; c0 += 4 * kEncSplit) {   // up to four independent 16-byte loads in flight
+    uint4 raw[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + u * kEncSplit;
       const int gi = c / gc, gj = c - gi * gc;
-      stage[c * kThreads + threadIdx.x] = load4(X + (gi * br + p) * ldx + gj * bc + t);
+      raw[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (live && c < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(X + (gi * br + p) * ldx + gj * bc + t));
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + u * kEncSplit;
+      if (c < ncell) {
+        float4 v[NV];
+        Vec16<SrcT>::unpack(raw[u], v);
+#pragma unroll
+        for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
+      }
     }
   }
-  // (each thread reads back only what it wrote: no barrier needed)
-  for (int r = 0; r < R; ++r) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (live) {
-      const int e0 = sm.tab.off[r], e1 = sm.tab.off[r + 1];
-      for (int e = e0; e < e1; ++e) {
-        const float c = sm.tab.coef[e];
-        const float4 v = stage[sm.tab.cell[e] * kThreads + threadIdx.x];
-        acc.x = __fmaf_rn(c, v.x, acc.x);
-        acc.y = __fmaf_rn(c, v.y, acc.y);
-        acc.z = __fmaf_rn(c, v.z, acc.z);
-        acc.w = __fmaf_rn(c, v.w, acc.w);
+  if (g == 0) {
+#pragma unroll
+    for (int h = 0; h < NV; ++h)
+      *reinterpret_cast<float4*>(my_stage + ncell * kSlab + h * kHalf) = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  __syncthreads();   // staged vectors and table entries are now visible to the four sharing threads
+
+  DstT* dst = out + p * bc + t;
+  const int64_t rstride = br * bc;
+  for (int r = g; r < R; r += kEncSplit) {
+    float2 acc[NP];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
+    const int e1 = sm.off[r + 1];
+    for (int e = sm.off[r]; e < e1; e += kChunk) {
+      int2 en[kChunk];
+      float4 v[kChunk][NV];
+#pragma unroll
+      for (int u = 0; u < kChunk; u += 2) {
+        const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
+        en[u] = make_int2(two.x, two.y);
+        en[u + 1] = make_int2(two.z, two.w);
+      }
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u)
+#pragma unroll
+        for (int h = 0; h < NV; ++h) v[u][h] = *reinterpret_cast<const float4*>(my_stage + en[u].x + h * kHalf);
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u) {
+        const float c = __int_as_float(en[u].y);
+        const float2 cc = make_float2(c, c);
+#pragma unroll
+        for (int h = 0; h < NV; ++h) {
+          acc[2 * h] = __ffma2_rn(cc, make_float2(v[u][h].x, v[u][h].y), acc[2 * h]);
+          acc[2 * h + 1] = __ffma2_rn(cc, make_float2(v[u][h].z, v[u][h].w), acc[2 * h + 1]);
+        }
       }
     }
     if (kAmaxOnly) {
-      float a = fmaxf(fmaxf(fabsf(acc.x), fabsf(acc.y)), fmaxf(fabsf(acc.z), fabsf(acc.w)));
-      if (!(a == a)) a = 0.0f;  // NaN does not set a scale
+      float a = 0.0f;
+#pragma unroll
+      for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
       if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
@@ -152,14 +237,15 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
       if (use_scale) {
         if (sm.use_mul[r]) {
           const float inv = sm.inv_scale[r];
-          acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { acc[i].x *= inv; acc[i].y *= inv; }
         } else {
           const float s = sm.scale[r];
-          acc.x = __fdiv_rn(acc.x, s); acc.y = __fdiv_rn(acc.y, s);
-          acc.z = __fdiv_rn(acc.z, s); acc.w = __fdiv_rn(acc.w, s);
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, s); acc[i].y = __fdiv_rn(acc[i].y, s); }
         }
       }
-      store4(out + ((int64_t)r * br + p) * bc + t, acc);
+      store_vec<NP>(dst + r * rstride, acc);
     }
   }
   if (kAmaxOnly) {
@@ -168,25 +254,40 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   }
 }
 
+// entries after padding every list of `t` to a multiple of kChunk
+static int padded_entries(const CoefTable& t) {
+  int o = 0;
+  for (int r = 0; r < t.R; ++r) o += (t.off[r + 1] - t.off[r] + kChunk - 1) / kChunk * kChunk;
+  return o;
+}
+
 template <typename SrcT, typename DstT>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
-                            const CoefTable* d_tab, void* out, unsigned* amax_bits, float* scale, bool amax_only,
-                            bool use_scale, cudaStream_t st) {
-  const size_t smem = ((sizeof(EncSmem) + 15) / 16) * 16 + (size_t)gr * gc * kThreads * sizeof(float4);
-  const int64_t vecs = br * (bc >> 2);
-  const int grid = (int)((vecs + kThreads - 1) / kThreads);
+                            const CoefTable* d_tab, int padded, void* out, unsigned* amax_bits, float* scale,
+                            bool amax_only, bool use_scale, cudaStream_t st) {
+  constexpr int VE = Vec16<SrcT>::kElems;
+  const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
+                      (size_t)(gr * gc + 1) * (VE / 4) * kEncPos * 16;
+  const int64_t vecs = br * (bc / VE);
+  const int grid = (int)((vecs + kEncPos - 1) / kEncPos);
   if (grid == 0) return cudaSuccess;
-  cudaError_t e;
+  static bool attr_done[2] = {false, false};
   if (amax_only) {
     auto k = encode_kernel<SrcT, DstT, true>;
-    e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k<<<grid, kThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
+    if (!attr_done[0]) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done[0] = true;
+    }
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
   } else {
     auto k = encode_kernel<SrcT, DstT, false>;
-    e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k<<<grid, kThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
+    if (!attr_done[1]) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      if (e != cudaSuccess) return e;
+      attr_done[1] = true;
+    }
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
   }
   ++fmm_launch_counter();
   return cudaGetLastError();
@@ -213,65 +314,111 @@ __global__ void __launch_bounds__(256) transpose_kernel(const T* __restrict__ B,
 }
 
 // ------------------------------------------------------------------------------------------
-// decode: C_ij = rnd_O( sum_r w_{r,ij} sA_r sB_r M_r ), ascending r, fp32 FMA chain; optional
-// error reduction sum (rnd_O(c) - C*)^2 per block (fp32 per thread -> fp64 shuffle tree -> one fp64
-// partial per block).  Accumulators of the m*n output cells live in shared memory [cell][thread].
+// decode: C_ij = rnd_O( sum_r w_{r,ij} sA_r sB_r M_r ), ascending r, fp32 FMA chain; optional error
+// reduction sum (rnd_O(c) - C*)^2 per block (fp32 per thread -> fp64 shuffle tree -> one fp64 partial
+// per block).  A block of 256 threads owns 64 "position quads" (4 consecutive columns of one block
+// position).  Four threads share each quad:
+//   1. together they copy the R product vectors of that position straight into shared memory with
+//      cp.async ([r][position], slab R holds zeros) — thread g copies r = g, g+4, ...;
+//   2. thread g then forms the output cells c = g, g+4, ...: it walks the cell's (r, w) list (cell-major
+//      table, ascending r, padded to a multiple of 4 with (zero slab, 0.0f) entries) in registers, two
+//      lanes per packed fma.rn.f32x2, rounds, stores, and accumulates its share of the error.
 // ------------------------------------------------------------------------------------------
-struct DecSmem {
-  CoefTable tab;
-  double red[kThreads / 32];
-};
+constexpr int kDecThreads = 256;
+constexpr int kDecPos = 64;
+constexpr int kDecSplit = 4;
+
+struct DecSmemHead {
+  int off[kMaxCells + 1];   // entries, multiples of kChunk
+  int pad[3];
+  double red[kDecThreads / 32];
+};  // followed by int2 ent[] {byte offset of product r's slab, scaled coefficient bits}, then the stage
 
 template <typename OutT, bool kStore, bool kErr>
-__global__ void __launch_bounds__(kThreads)
-decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, const float* __restrict__ sA,
-              const float* __restrict__ sB, int n, int64_t bm, int64_t bn, OutT* __restrict__ C, int64_t ldc,
-              const float* __restrict__ cstar32, int64_t ldcs, double* __restrict__ partials) {
+__global__ void __launch_bounds__(kDecThreads)
+decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
+              const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
+              OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
+              double* __restrict__ partials) {
+  constexpr int kSlab = kDecPos * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  DecSmem& sm = *reinterpret_cast<DecSmem*>(smem_raw);
-  float4* acc = reinterpret_cast<float4*>(smem_raw + ((sizeof(DecSmem) + 15) / 16) * 16);
-  {
-    const int* src = reinterpret_cast<const int*>(d_tab);
-    int* dst = reinterpret_cast<int*>(&sm.tab);
-    for (int i = threadIdx.x; i < (int)(sizeof(CoefTable) / 4); i += kThreads) dst[i] = src[i];
-  }
-  __syncthreads();
-  const int R = sm.tab.R, ncell = sm.tab.ncell;
-  if (sA != nullptr) {  // fold the (power-of-two) scales into the coefficients: w * (sA_r * sB_r)
-    for (int r = threadIdx.x; r < R; r += kThreads) {
-      const float s = sA[r] * sB[r];
-      for (int e = sm.tab.off[r]; e < sm.tab.off[r + 1]; ++e) sm.tab.coef[e] *= s;
-    }
-    __syncthreads();
-  }
+  DecSmemHead& sm = *reinterpret_cast<DecSmemHead*>(smem_raw);
+  const int ncell = d_tab->R;   // number of lists = number of C blocks
+  int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(DecSmemHead));
+  int total = 0;                // padded entry count (every thread computes it: lists are few)
+  for (int c = 0; c < ncell; ++c) total += (d_tab->off[c + 1] - d_tab->off[c] + kChunk - 1) / kChunk * kChunk;
+  unsigned char* stage = smem_raw + ((sizeof(DecSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
+
+  const int g = threadIdx.x / kDecPos;
+  const int pq = threadIdx.x - g * kDecPos;
   const int64_t vec_per_row = bn >> 2;
-  const int64_t idx = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  const int64_t idx = (int64_t)blockIdx.x * kDecPos + pq;
   const bool live = idx < bm * vec_per_row;
   const int64_t p = live ? idx / vec_per_row : 0;
   const int64_t q = live ? (idx - p * vec_per_row) << 2 : 0;
-
-  float err = 0.0f;
-  if (live) {
-    for (int c = 0; c < ncell; ++c) acc[c * kThreads + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+  unsigned char* my_stage = stage + pq * 16;
+  {  // start the copies first so they overlap the table set-up
     const float* src = prod + p * bn + q;
     const int64_t rstride = bm * bn;
-    for (int r = 0; r < R; ++r) {
-      const float4 v = __ldcs(reinterpret_cast<const float4*>(src + r * rstride));
-      const int e0 = sm.tab.off[r], e1 = sm.tab.off[r + 1];
-      for (int e = e0; e < e1; ++e) {
-        const float w = sm.tab.coef[e];
-        float4* a = &acc[sm.tab.cell[e] * kThreads + threadIdx.x];
-        float4 x = *a;
-        x.x = __fmaf_rn(w, v.x, x.x);
-        x.y = __fmaf_rn(w, v.y, x.y);
-        x.z = __fmaf_rn(w, v.z, x.z);
-        x.w = __fmaf_rn(w, v.w, x.w);
-        *a = x;
+    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
+    const int nbytes = live ? 16 : 0;   // 0 source bytes -> the 16 destination bytes are zero-filled
+    for (int r = g; r < R; r += kDecSplit)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
+                   "r"(nbytes) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (g == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (threadIdx.x == 0) {
+    int o = 0;
+    for (int c = 0; c < ncell; ++c) {
+      sm.off[c] = o;
+      o += (d_tab->off[c + 1] - d_tab->off[c] + kChunk - 1) / kChunk * kChunk;
+    }
+    sm.off[ncell] = o;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < ncell; c += kDecThreads) {
+    const int s0 = d_tab->off[c], cnt = d_tab->off[c + 1] - s0, d0 = sm.off[c], padded = sm.off[c + 1] - d0;
+    for (int i = 0; i < padded; ++i) {
+      if (i < cnt) {
+        const int r = d_tab->cell[s0 + i];
+        float w = d_tab->coef[s0 + i];
+        if (sA != nullptr) w *= sA[r] * sB[r];   // power-of-two scales fold exactly into the coefficient
+        ent[d0 + i] = make_int2(r * kSlab, __float_as_int(w));
+      } else {
+        ent[d0 + i] = make_int2(R * kSlab, 0);
       }
     }
-    for (int c = 0; c < ncell; ++c) {
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  float err = 0.0f;
+  for (int c = g; c < ncell; c += kDecSplit) {
+    float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+    const int e1 = sm.off[c + 1];
+    for (int e = sm.off[c]; e < e1; e += kChunk) {
+      int2 en[kChunk];
+      float4 v[kChunk];
+#pragma unroll
+      for (int u = 0; u < kChunk; u += 2) {
+        const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
+        en[u] = make_int2(two.x, two.y);
+        en[u + 1] = make_int2(two.z, two.w);
+      }
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u) v[u] = *reinterpret_cast<const float4*>(my_stage + en[u].x);
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u) {
+        const float w = __int_as_float(en[u].y);
+        const float2 ww = make_float2(w, w);
+        x0 = __ffma2_rn(ww, make_float2(v[u].x, v[u].y), x0);
+        x1 = __ffma2_rn(ww, make_float2(v[u].z, v[u].w), x1);
+      }
+    }
+    if (live) {
+      const float4 x = make_float4(x0.x, x0.y, x1.x, x1.y);
       const int i = c / n, j = c - i * n;
-      float4 x = acc[c * kThreads + threadIdx.x];
       const int64_t row = i * bm + p, col = j * bn + q;
       if (kStore) store4(C + row * ldc + col, x);
       if (kErr) {
@@ -392,16 +539,17 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 // launch wrappers
 // ------------------------------------------------------------------------------------------
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
-                          int64_t bc, const CoefTable* d_tab, void* out, unsigned* amax_bits, float* scale,
-                          bool amax_only, bool use_scale, cudaStream_t st) {
+                          int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, unsigned* amax_bits,
+                          float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+  const int nnz = padded_entries(*h_tab);
   if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_encode_t<float, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_encode_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_encode_t<float, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
   return cudaErrorInvalidValue;
 }
 
@@ -418,37 +566,43 @@ cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t
   return cudaGetLastError();
 }
 
-int decode_grid(int64_t bm, int64_t bn) { return (int)((bm * (bn >> 2) + kThreads - 1) / kThreads); }
+int decode_grid(int64_t bm, int64_t bn) { return (int)((bm * (bn >> 2) + kDecPos - 1) / kDecPos); }
 
 template <typename OutT>
-static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, const float* sA, const float* sB, int m,
-                                   int n, int64_t bm, int64_t bn, void* C, int64_t ldc, const float* cstar32,
-                                   double* partials, cudaStream_t st) {
-  const size_t smem = ((sizeof(DecSmem) + 15) / 16) * 16 + (size_t)m * n * kThreads * sizeof(float4);
+static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, int R, int nnz, const float* sA,
+                                   const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
+                                   const float* cstar32, double* partials, cudaStream_t st) {
+  const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 16;
   const int grid = decode_grid(bm, bn);
   const int64_t ldcs = (int64_t)n * bn;
-#define FMM_DECODE_LAUNCH(STORE, ERR)                                                                         \
-  {                                                                                                           \
-    auto k = decode_kernel<OutT, STORE, ERR>;                                                                 \
-    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);          \
-    if (e != cudaSuccess) return e;                                                                           \
-    k<<<grid, kThreads, smem, st>>>(prod, d_tab, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials);  \
+  static bool attr_done[3] = {false, false, false};
+#define FMM_DECODE_LAUNCH(STORE, ERR, SLOT)                                                                      \
+  {                                                                                                              \
+    auto k = decode_kernel<OutT, STORE, ERR>;                                                                    \
+    if (!attr_done[SLOT]) {                                                                                      \
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);          \
+      if (e != cudaSuccess) return e;                                                                            \
+      attr_done[SLOT] = true;                                                                                    \
+    }                                                                                                            \
+    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials); \
   }
-  if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true)
-  else if (C != nullptr) FMM_DECODE_LAUNCH(true, false)
-  else FMM_DECODE_LAUNCH(false, true)
+  if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true, 0)
+  else if (C != nullptr) FMM_DECODE_LAUNCH(true, false, 1)
+  else FMM_DECODE_LAUNCH(false, true, 2)
 #undef FMM_DECODE_LAUNCH
+  (void)m;
   ++fmm_launch_counter();
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode(int output, const float* prod, const CoefTable* d_tab, const float* sA, const float* sB,
-                          int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc, const float* cstar32,
-                          double* partials, int* n_partials, cudaStream_t st) {
+cudaError_t launch_decode(int output, const float* prod, const CoefTable* d_tab, const CoefTable* h_tab, int R,
+                          const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
+                          int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
+  const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   if (n_partials) *n_partials = decode_grid(bm, bn);
-  if (output == FMM_F32) return launch_decode_t<float>(prod, d_tab, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
-  if (output == FMM_BF16) return launch_decode_t<__nv_bfloat16>(prod, d_tab, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
+  if (output == FMM_F32) return launch_decode_t<float>(prod, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
+  if (output == FMM_BF16) return launch_decode_t<__nv_bfloat16>(prod, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
   return cudaErrorInvalidValue;
 }
 

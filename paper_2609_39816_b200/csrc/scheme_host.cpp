@@ -211,15 +211,15 @@ void fmm_build_tables(const fmm_scheme& s, CoefTable* tA, CoefTable* tB, CoefTab
       tB->off[r + 1] = c;
     }
   }
-  if (tW) {
-    begin(tW, m * n);
+  if (tW) {  // cell-major: list x = i*n+j holds the (r, w_{r,ij}) pairs feeding C block (i,j), ascending r
+    tW->R = m * n; tW->ncell = s.R; tW->off[0] = 0;
     int c = 0;
-    for (int r = 0; r < s.R; ++r) {
-      for (int i = 0; i < m; ++i) for (int j = 0; j < n; ++j) {
+    for (int i = 0; i < m; ++i) for (int j = 0; j < n; ++j) {
+      for (int r = 0; r < s.R; ++r) {
         const float f = (float)at3(s.W, r, i, j, m, n);
-        if (f != 0.0f) { tW->cell[c] = i * n + j; tW->coef[c] = f; ++c; }
+        if (f != 0.0f) { tW->cell[c] = r; tW->coef[c] = f; ++c; }
       }
-      tW->off[r + 1] = c;
+      tW->off[i * n + j + 1] = c;
     }
   }
 }
