@@ -7,7 +7,8 @@
 #include "fmm_b200.h"
 
 constexpr int kMaxCells = FMM_MAX_GRID * FMM_MAX_GRID;  // blocks in one operand grid
-constexpr int kMaxNnz = FMM_MAX_R * kMaxCells;          // nonzero coefficients in one table
+constexpr int kMaxNnz = FMM_MAX_R * kMaxCells;          // entries in one table (padding included)
+constexpr int kTablePad = 4;                            // every list is padded to a multiple of this
 
 struct fmm_scheme {
   int m = 0, k = 0, n = 0, R = 0;
@@ -15,13 +16,14 @@ struct fmm_scheme {
   std::unique_ptr<fmm_scheme> outer, inner;    // factors, when built by scheme_kron
 };
 
-// Sparse coefficient table as the kernels read it: for each product r the nonzero
-// (cell, coefficient) pairs, in the order in which they are to be accumulated.
-// For the encode tables `cell` is the flat index of a block in the SOURCE matrix's
-// grid as stored in memory; for the decode table it is the flat index i*n+j of a C block.
+// Sparse coefficient table as the kernels read it: R lists of (slab, coefficient) pairs in the order in
+// which they are to be accumulated, each list padded to a multiple of kTablePad with (ncell, 0.0f).
+// Encode tables: one list per product, slab = flat index of a block in the SOURCE matrix's grid as stored
+// in memory, ncell = number of blocks.  Decode table: one list per C block (cell-major), slab = product
+// index r (ascending), ncell = number of products.
 struct CoefTable {
-  int32_t R;
-  int32_t ncell;
+  int32_t R;       // number of lists
+  int32_t ncell;   // number of data slabs; index ncell is the all-zero padding slab
   int32_t off[FMM_MAX_R + 1];
   int32_t cell[kMaxNnz];
   float coef[kMaxNnz];

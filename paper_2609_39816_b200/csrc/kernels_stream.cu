@@ -68,7 +68,7 @@ __device__ __forceinline__ double block_sum_double(double v, double* red /* >= 8
 constexpr int kEncThreads = 256;
 constexpr int kEncPos = 64;      // position vectors per block
 constexpr int kEncSplit = 4;     // threads per position vector
-constexpr int kChunk = 4;
+constexpr int kChunk = kTablePad;   // lists arrive padded to this multiple
 
 struct EncSmemHead {
   int off[FMM_MAX_R + 1];   // in units of entries, multiples of kChunk
@@ -119,7 +119,7 @@ template <typename SrcT, typename DstT, bool kAmaxOnly>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
               const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
-              float* __restrict__ scale_out, int use_scale) {
+              float* __restrict__ scale_out, int use_scale, int tiles_per_block) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int NV = VE / 4;                     // float4 per staged vector
   constexpr int NP = VE / 2;                     // float2 pairs per vector
@@ -128,17 +128,13 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   extern __shared__ __align__(16) unsigned char smem_raw[];
   EncSmemHead& sm = *reinterpret_cast<EncSmemHead*>(smem_raw);
   const int R = d_tab->R, ncell = d_tab->ncell;
+  const int total = d_tab->off[R];               // lists arrive padded to multiples of kChunk
   int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(EncSmemHead));
+  unsigned char* stage = smem_raw + ((sizeof(EncSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
 
-  // pad every list to a multiple of kChunk (lists are short; thread 0 lays out the offsets)
-  if (threadIdx.x == 0) {
-    int o = 0;
-    for (int r = 0; r < R; ++r) {
-      sm.off[r] = o;
-      o += (d_tab->off[r + 1] - d_tab->off[r] + kChunk - 1) / kChunk * kChunk;
-    }
-    sm.off[R] = o;
-  }
+  for (int i = threadIdx.x; i <= R; i += kEncThreads) sm.off[i] = d_tab->off[i];
+  for (int i = threadIdx.x; i < total; i += kEncThreads)
+    ent[i] = make_int2(d_tab->cell[i] * kSlab, __float_as_int(d_tab->coef[i]));
   if (threadIdx.x < R) {
     float s = 1.0f;
     if (!kAmaxOnly && use_scale) s = pow2_scale_448(__uint_as_float(amax_bits[threadIdx.x]));
@@ -149,103 +145,105 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     sm.amax[threadIdx.x] = 0u;
     if (!kAmaxOnly && use_scale && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
   }
-  __syncthreads();
-  const int total = sm.off[R];
-  for (int r = threadIdx.x; r < R; r += kEncThreads) {
-    const int s0 = d_tab->off[r], cnt = d_tab->off[r + 1] - s0, d0 = sm.off[r], padded = sm.off[r + 1] - d0;
-    for (int i = 0; i < padded; ++i)
-      ent[d0 + i] = i < cnt ? make_int2(d_tab->cell[s0 + i] * kSlab, __float_as_int(d_tab->coef[s0 + i]))
-                            : make_int2(ncell * kSlab, 0);
-  }
-  unsigned char* stage = smem_raw + ((sizeof(EncSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
 
   const int g = threadIdx.x / kEncPos;           // which quarter of the cells / products this thread handles
-  const int pv = threadIdx.x - g * kEncPos;      // position vector inside the block
-  const int64_t vec_per_row = bc / VE;
-  const int64_t idx = (int64_t)blockIdx.x * kEncPos + pv;
-  const bool live = idx < br * vec_per_row;
-  const int64_t p = live ? idx / vec_per_row : 0;
-  const int64_t t = live ? (idx - p * vec_per_row) * VE : 0;
+  const int pv = threadIdx.x - g * kEncPos;      // position vector inside the tile
+  const int vec_per_row = (int)(bc / VE);        // 32-bit index arithmetic: br * bc / VE < 2^31 (checked by the host)
+  const int nvec = (int)br * vec_per_row;
+  const int64_t rstride = br * bc;
   unsigned char* my_stage = stage + pv * 16;
-
-  for (int c0 = g; c0 < ncell; c0 += 4 * kEncSplit) {   // up to four independent 16-byte loads in flight
-    uint4 raw[4];
+  // element offset of each grid cell this thread stages (cells g, g+4, ...), computed once
+  int64_t cell_base[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int c = c0 + u * kEncSplit;
-      const int gi = c / gc, gj = c - gi * gc;
-      raw[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (live && c < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(X + (gi * br + p) * ldx + gj * bc + t));
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int c = c0 + u * kEncSplit;
-      if (c < ncell) {
-        float4 v[NV];
-        Vec16<SrcT>::unpack(raw[u], v);
-#pragma unroll
-        for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
-      }
-    }
+  for (int u = 0; u < 4; ++u) {
+    const int c = g + u * kEncSplit;
+    const int gi = c / gc, gj = c - gi * gc;
+    cell_base[u] = (int64_t)gi * br * ldx + (int64_t)gj * bc;
   }
   if (g == 0) {
 #pragma unroll
     for (int h = 0; h < NV; ++h)
       *reinterpret_cast<float4*>(my_stage + ncell * kSlab + h * kHalf) = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  __syncthreads();   // staged vectors and table entries are now visible to the four sharing threads
 
-  DstT* dst = out + p * bc + t;
-  const int64_t rstride = br * bc;
-  for (int r = g; r < R; r += kEncSplit) {
-    float2 acc[NP];
+  for (int it = 0; it < tiles_per_block; ++it) {
+    const int idx = (blockIdx.x * tiles_per_block + it) * kEncPos + pv;
+    const bool live = idx < nvec;
+    const int p = live ? idx / vec_per_row : 0;
+    const int t = live ? (idx - p * vec_per_row) * VE : 0;
+    if (it > 0) __syncthreads();                 // previous tile's readers are done with the stage
+    {                                            // up to four independent 16-byte loads in flight (ncell <= 16)
+      const SrcT* src = X + (int64_t)p * ldx + t;
+      uint4 raw[4];
 #pragma unroll
-    for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
-    const int e1 = sm.off[r + 1];
-    for (int e = sm.off[r]; e < e1; e += kChunk) {
-      int2 en[kChunk];
-      float4 v[kChunk][NV];
-#pragma unroll
-      for (int u = 0; u < kChunk; u += 2) {
-        const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
-        en[u] = make_int2(two.x, two.y);
-        en[u + 1] = make_int2(two.z, two.w);
+      for (int u = 0; u < 4; ++u) {
+        raw[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (live && g + u * kEncSplit < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(src + cell_base[u]));
       }
 #pragma unroll
-      for (int u = 0; u < kChunk; ++u)
+      for (int u = 0; u < 4; ++u) {
+        const int c = g + u * kEncSplit;
+        if (c < ncell) {
+          float4 v[NV];
+          Vec16<SrcT>::unpack(raw[u], v);
 #pragma unroll
-        for (int h = 0; h < NV; ++h) v[u][h] = *reinterpret_cast<const float4*>(my_stage + en[u].x + h * kHalf);
-#pragma unroll
-      for (int u = 0; u < kChunk; ++u) {
-        const float c = __int_as_float(en[u].y);
-        const float2 cc = make_float2(c, c);
-#pragma unroll
-        for (int h = 0; h < NV; ++h) {
-          acc[2 * h] = __ffma2_rn(cc, make_float2(v[u][h].x, v[u][h].y), acc[2 * h]);
-          acc[2 * h + 1] = __ffma2_rn(cc, make_float2(v[u][h].z, v[u][h].w), acc[2 * h + 1]);
+          for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
         }
       }
     }
-    if (kAmaxOnly) {
-      float a = 0.0f;
+    __syncthreads();   // staged vectors (and, first time, the table) are visible to the four sharing threads
+
+    DstT* dst = out + (int64_t)p * bc + t;
+    for (int r = g; r < R; r += kEncSplit) {
+      float2 acc[NP];
 #pragma unroll
-      for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
+      for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
+      const int e1 = sm.off[r + 1];
+      for (int e = sm.off[r]; e < e1; e += kChunk) {
+        int2 en[kChunk];
+        float4 v[kChunk][NV];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-      if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
-    } else if (live) {
-      if (use_scale) {
-        if (sm.use_mul[r]) {
-          const float inv = sm.inv_scale[r];
+        for (int u = 0; u < kChunk; u += 2) {
+          const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
+          en[u] = make_int2(two.x, two.y);
+          en[u + 1] = make_int2(two.z, two.w);
+        }
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { acc[i].x *= inv; acc[i].y *= inv; }
-        } else {
-          const float s = sm.scale[r];
+        for (int u = 0; u < kChunk; ++u)
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, s); acc[i].y = __fdiv_rn(acc[i].y, s); }
+          for (int h = 0; h < NV; ++h) v[u][h] = *reinterpret_cast<const float4*>(my_stage + en[u].x + h * kHalf);
+#pragma unroll
+        for (int u = 0; u < kChunk; ++u) {
+          const float c = __int_as_float(en[u].y);
+          const float2 cc = make_float2(c, c);
+#pragma unroll
+          for (int h = 0; h < NV; ++h) {
+            acc[2 * h] = __ffma2_rn(cc, make_float2(v[u][h].x, v[u][h].y), acc[2 * h]);
+            acc[2 * h + 1] = __ffma2_rn(cc, make_float2(v[u][h].z, v[u][h].w), acc[2 * h + 1]);
+          }
         }
       }
-      store_vec<NP>(dst + r * rstride, acc);
+      if (kAmaxOnly) {
+        float a = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+        if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
+      } else if (live) {
+        if (use_scale) {
+          if (sm.use_mul[r]) {
+            const float inv = sm.inv_scale[r];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { acc[i].x *= inv; acc[i].y *= inv; }
+          } else {
+            const float s = sm.scale[r];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, s); acc[i].y = __fdiv_rn(acc[i].y, s); }
+          }
+        }
+        store_vec<NP>(dst + r * rstride, acc);
+      }
     }
   }
   if (kAmaxOnly) {
@@ -254,12 +252,16 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   }
 }
 
-// entries after padding every list of `t` to a multiple of kChunk
-static int padded_entries(const CoefTable& t) {
-  int o = 0;
-  for (int r = 0; r < t.R; ++r) o += (t.off[r + 1] - t.off[r] + kChunk - 1) / kChunk * kChunk;
-  return o;
+// Blocks of a streaming pass: enough to fill the machine about four times over, each block walking a
+// contiguous run of tiles so that its table set-up is paid once.
+static void split_tiles(int64_t tiles, int* grid, int* tiles_per_block) {
+  const int64_t target = 148 * 4;
+  const int64_t tpb = (tiles + target - 1) / target;
+  *tiles_per_block = (int)(tpb < 1 ? 1 : tpb);
+  *grid = (int)((tiles + *tiles_per_block - 1) / *tiles_per_block);
 }
+
+static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists arrive padded from the host
 
 template <typename SrcT, typename DstT>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
@@ -269,8 +271,10 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
   const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
                       (size_t)(gr * gc + 1) * (VE / 4) * kEncPos * 16;
   const int64_t vecs = br * (bc / VE);
-  const int grid = (int)((vecs + kEncPos - 1) / kEncPos);
-  if (grid == 0) return cudaSuccess;
+  if (vecs == 0) return cudaSuccess;
+  if (vecs + kEncPos * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // kernels index positions in 32 bits
+  int grid, tpb;
+  split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
   static bool attr_done[2] = {false, false};
   if (amax_only) {
     auto k = encode_kernel<SrcT, DstT, true>;
@@ -279,7 +283,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[0] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb);
   } else {
     auto k = encode_kernel<SrcT, DstT, false>;
     if (!attr_done[1]) {
@@ -287,7 +291,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[1] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb);
   }
   ++fmm_launch_counter();
   return cudaGetLastError();
@@ -339,94 +343,95 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
               const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
               OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
-              double* __restrict__ partials) {
+              double* __restrict__ partials, int tiles_per_block) {
   constexpr int kSlab = kDecPos * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DecSmemHead& sm = *reinterpret_cast<DecSmemHead*>(smem_raw);
-  const int ncell = d_tab->R;   // number of lists = number of C blocks
+  const int ncell = d_tab->R;                  // number of lists = number of C blocks
+  const int total = d_tab->off[ncell];         // lists arrive padded to multiples of kChunk
   int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(DecSmemHead));
-  int total = 0;                // padded entry count (every thread computes it: lists are few)
-  for (int c = 0; c < ncell; ++c) total += (d_tab->off[c + 1] - d_tab->off[c] + kChunk - 1) / kChunk * kChunk;
   unsigned char* stage = smem_raw + ((sizeof(DecSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
 
   const int g = threadIdx.x / kDecPos;
   const int pq = threadIdx.x - g * kDecPos;
-  const int64_t vec_per_row = bn >> 2;
-  const int64_t idx = (int64_t)blockIdx.x * kDecPos + pq;
-  const bool live = idx < bm * vec_per_row;
-  const int64_t p = live ? idx / vec_per_row : 0;
-  const int64_t q = live ? (idx - p * vec_per_row) << 2 : 0;
+  const int vec_per_row = (int)(bn >> 2);      // 32-bit index arithmetic: bm * bn / 4 < 2^31 (checked by the host)
+  const int nvec = (int)bm * vec_per_row;
+  const int64_t rstride = bm * bn;
   unsigned char* my_stage = stage + pq * 16;
-  {  // start the copies first so they overlap the table set-up
-    const float* src = prod + p * bn + q;
-    const int64_t rstride = bm * bn;
-    const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
-    const int nbytes = live ? 16 : 0;   // 0 source bytes -> the 16 destination bytes are zero-filled
-    for (int r = g; r < R; r += kDecSplit)
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
-                   "r"(nbytes) : "memory");
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    if (g == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
+  const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
+  // element offsets of the output cells this thread forms (cells g, g+4, ...), computed once
+  int64_t out_base[4], cs_base[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int c = g + u * kDecSplit;
+    const int i = c / n, j = c - i * n;
+    out_base[u] = (int64_t)i * bm * ldc + (int64_t)j * bn;
+    cs_base[u] = (int64_t)i * bm * ldcs + (int64_t)j * bn;
   }
-  if (threadIdx.x == 0) {
-    int o = 0;
-    for (int c = 0; c < ncell; ++c) {
-      sm.off[c] = o;
-      o += (d_tab->off[c + 1] - d_tab->off[c] + kChunk - 1) / kChunk * kChunk;
-    }
-    sm.off[ncell] = o;
-  }
-  __syncthreads();
-  for (int c = threadIdx.x; c < ncell; c += kDecThreads) {
-    const int s0 = d_tab->off[c], cnt = d_tab->off[c + 1] - s0, d0 = sm.off[c], padded = sm.off[c + 1] - d0;
-    for (int i = 0; i < padded; ++i) {
-      if (i < cnt) {
-        const int r = d_tab->cell[s0 + i];
-        float w = d_tab->coef[s0 + i];
-        if (sA != nullptr) w *= sA[r] * sB[r];   // power-of-two scales fold exactly into the coefficient
-        ent[d0 + i] = make_int2(r * kSlab, __float_as_int(w));
-      } else {
-        ent[d0 + i] = make_int2(R * kSlab, 0);
-      }
-    }
-  }
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  __syncthreads();
 
   float err = 0.0f;
-  for (int c = g; c < ncell; c += kDecSplit) {
-    float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
-    const int e1 = sm.off[c + 1];
-    for (int e = sm.off[c]; e < e1; e += kChunk) {
-      int2 en[kChunk];
-      float4 v[kChunk];
-#pragma unroll
-      for (int u = 0; u < kChunk; u += 2) {
-        const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
-        en[u] = make_int2(two.x, two.y);
-        en[u + 1] = make_int2(two.z, two.w);
-      }
-#pragma unroll
-      for (int u = 0; u < kChunk; ++u) v[u] = *reinterpret_cast<const float4*>(my_stage + en[u].x);
-#pragma unroll
-      for (int u = 0; u < kChunk; ++u) {
-        const float w = __int_as_float(en[u].y);
-        const float2 ww = make_float2(w, w);
-        x0 = __ffma2_rn(ww, make_float2(v[u].x, v[u].y), x0);
-        x1 = __ffma2_rn(ww, make_float2(v[u].z, v[u].w), x1);
+  for (int it = 0; it < tiles_per_block; ++it) {
+    const int idx = (blockIdx.x * tiles_per_block + it) * kDecPos + pq;
+    const bool live = idx < nvec;
+    const int p = live ? idx / vec_per_row : 0;
+    const int q = live ? (idx - p * vec_per_row) << 2 : 0;
+    if (it > 0) __syncthreads();               // previous tile's readers are done with the stage
+    {
+      const float* src = prod + (int64_t)p * bn + q;
+      const int nbytes = live ? 16 : 0;        // 0 source bytes -> the 16 destination bytes are zero-filled
+      for (int r = g; r < R; r += kDecSplit)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
+                     "r"(nbytes) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    if (it == 0) {                             // table set-up overlaps the first tile's copies
+      if (g == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = threadIdx.x; i <= ncell; i += kDecThreads) sm.off[i] = d_tab->off[i];
+      for (int i = threadIdx.x; i < total; i += kDecThreads) {
+        const int r = d_tab->cell[i];
+        float w = d_tab->coef[i];
+        if (sA != nullptr && r < R) w *= sA[r] * sB[r];   // power-of-two scales fold exactly into the coefficient
+        ent[i] = make_int2(r * kSlab, __float_as_int(w));
       }
     }
-    if (live) {
-      const float4 x = make_float4(x0.x, x0.y, x1.x, x1.y);
-      const int i = c / n, j = c - i * n;
-      const int64_t row = i * bm + p, col = j * bn + q;
-      if (kStore) store4(C + row * ldc + col, x);
-      if (kErr) {
-        const float4 cs = __ldcs(reinterpret_cast<const float4*>(cstar32 + row * ldcs + col));
-        const float d0 = round_out(x.x, (OutT*)nullptr) - cs.x, d1 = round_out(x.y, (OutT*)nullptr) - cs.y;
-        const float d2 = round_out(x.z, (OutT*)nullptr) - cs.z, d3 = round_out(x.w, (OutT*)nullptr) - cs.w;
-        err = __fmaf_rn(d0, d0, err); err = __fmaf_rn(d1, d1, err);
-        err = __fmaf_rn(d2, d2, err); err = __fmaf_rn(d3, d3, err);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+#pragma unroll
+    for (int u4 = 0; u4 < 4; ++u4) {           // ncell <= 16: at most four cells per thread
+      const int c = g + u4 * kDecSplit;
+      if (c >= ncell) break;
+      float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+      const int e1 = sm.off[c + 1];
+      for (int e = sm.off[c]; e < e1; e += kChunk) {
+        int2 en[kChunk];
+        float4 v[kChunk];
+#pragma unroll
+        for (int u = 0; u < kChunk; u += 2) {
+          const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
+          en[u] = make_int2(two.x, two.y);
+          en[u + 1] = make_int2(two.z, two.w);
+        }
+#pragma unroll
+        for (int u = 0; u < kChunk; ++u) v[u] = *reinterpret_cast<const float4*>(my_stage + en[u].x);
+#pragma unroll
+        for (int u = 0; u < kChunk; ++u) {
+          const float w = __int_as_float(en[u].y);
+          const float2 ww = make_float2(w, w);
+          x0 = __ffma2_rn(ww, make_float2(v[u].x, v[u].y), x0);
+          x1 = __ffma2_rn(ww, make_float2(v[u].z, v[u].w), x1);
+        }
+      }
+      if (live) {
+        const float4 x = make_float4(x0.x, x0.y, x1.x, x1.y);
+        if (kStore) store4(C + out_base[u4] + (int64_t)p * ldc + q, x);
+        if (kErr) {
+          const float4 cs = __ldcs(reinterpret_cast<const float4*>(cstar32 + cs_base[u4] + (int64_t)p * ldcs + q));
+          const float d0 = round_out(x.x, (OutT*)nullptr) - cs.x, d1 = round_out(x.y, (OutT*)nullptr) - cs.y;
+          const float d2 = round_out(x.z, (OutT*)nullptr) - cs.z, d3 = round_out(x.w, (OutT*)nullptr) - cs.w;
+          err = __fmaf_rn(d0, d0, err); err = __fmaf_rn(d1, d1, err);
+          err = __fmaf_rn(d2, d2, err); err = __fmaf_rn(d3, d3, err);
+        }
       }
     }
   }
@@ -566,14 +571,20 @@ cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t
   return cudaGetLastError();
 }
 
-int decode_grid(int64_t bm, int64_t bn) { return (int)((bm * (bn >> 2) + kDecPos - 1) / kDecPos); }
+int decode_grid(int64_t bm, int64_t bn) {
+  int grid, tpb;
+  split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
+  return grid;
+}
 
 template <typename OutT>
 static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, int R, int nnz, const float* sA,
                                    const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
                                    const float* cstar32, double* partials, cudaStream_t st) {
   const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 16;
-  const int grid = decode_grid(bm, bn);
+  if (bm * (bn >> 2) + kDecPos * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
+  int grid, tpb;
+  split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
   const int64_t ldcs = (int64_t)n * bn;
   static bool attr_done[3] = {false, false, false};
 #define FMM_DECODE_LAUNCH(STORE, ERR, SLOT)                                                                      \
@@ -584,7 +595,7 @@ static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, in
       if (e != cudaSuccess) return e;                                                                            \
       attr_done[SLOT] = true;                                                                                    \
     }                                                                                                            \
-    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials); \
+    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials, tpb); \
   }
   if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true, 0)
   else if (C != nullptr) FMM_DECODE_LAUNCH(true, false, 1)

@@ -186,40 +186,42 @@ void fill_classical(fmm_scheme* s, int m, int k, int n) {
 
 }  // namespace
 
+// Lists are padded to a multiple of kTablePad entries with (pad slab, 0.0f): the kernels walk them in
+// fixed chunks, and a padding entry multiplies a slab of zeros by zero, which adds exactly nothing.
+namespace {
+struct ListBuilder {
+  CoefTable* t;
+  int c = 0, lists = 0;
+  ListBuilder(CoefTable* tab, int nlists, int nslabs) : t(tab) { t->R = nlists; t->ncell = nslabs; t->off[0] = 0; }
+  void add(int slab, float f) { if (f != 0.0f) { t->cell[c] = slab; t->coef[c] = f; ++c; } }
+  void close() {
+    while (c % kTablePad) { t->cell[c] = t->ncell; t->coef[c] = 0.0f; ++c; }
+    t->off[++lists] = c;
+  }
+};
+}  // namespace
+
 void fmm_build_tables(const fmm_scheme& s, CoefTable* tA, CoefTable* tB, CoefTable* tW) {
   const int m = s.m, k = s.k, n = s.n;
-  auto begin = [&](CoefTable* t, int ncell) { t->R = s.R; t->ncell = ncell; t->off[0] = 0; };
   if (tA) {
-    begin(tA, m * k);
-    int c = 0;
+    ListBuilder b(tA, s.R, m * k);
     for (int r = 0; r < s.R; ++r) {
-      for (int i = 0; i < m; ++i) for (int l = 0; l < k; ++l) {
-        const float f = (float)at3(s.U, r, i, l, m, k);
-        if (f != 0.0f) { tA->cell[c] = i * k + l; tA->coef[c] = f; ++c; }
-      }
-      tA->off[r + 1] = c;
+      for (int i = 0; i < m; ++i) for (int l = 0; l < k; ++l) b.add(i * k + l, (float)at3(s.U, r, i, l, m, k));
+      b.close();
     }
   }
   if (tB) {  // source is B^T stored [N x K]: block (l,j) of B is cell j*k + l; order ascending (l,j)
-    begin(tB, n * k);
-    int c = 0;
+    ListBuilder b(tB, s.R, n * k);
     for (int r = 0; r < s.R; ++r) {
-      for (int l = 0; l < k; ++l) for (int j = 0; j < n; ++j) {
-        const float f = (float)at3(s.V, r, l, j, k, n);
-        if (f != 0.0f) { tB->cell[c] = j * k + l; tB->coef[c] = f; ++c; }
-      }
-      tB->off[r + 1] = c;
+      for (int l = 0; l < k; ++l) for (int j = 0; j < n; ++j) b.add(j * k + l, (float)at3(s.V, r, l, j, k, n));
+      b.close();
     }
   }
   if (tW) {  // cell-major: list x = i*n+j holds the (r, w_{r,ij}) pairs feeding C block (i,j), ascending r
-    tW->R = m * n; tW->ncell = s.R; tW->off[0] = 0;
-    int c = 0;
+    ListBuilder b(tW, m * n, s.R);
     for (int i = 0; i < m; ++i) for (int j = 0; j < n; ++j) {
-      for (int r = 0; r < s.R; ++r) {
-        const float f = (float)at3(s.W, r, i, j, m, n);
-        if (f != 0.0f) { tW->cell[c] = r; tW->coef[c] = f; ++c; }
-      }
-      tW->off[i * n + j + 1] = c;
+      for (int r = 0; r < s.R; ++r) b.add(r, (float)at3(s.W, r, i, j, m, n));
+      b.close();
     }
   }
 }
