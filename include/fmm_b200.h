@@ -183,6 +183,29 @@ size_t error_frobenius_workspace(void);
 fmm_status error_frobenius(const fmm_gemm_desc* d, const void* dC, const double* dCstar, double* d_out,
                            void* d_ws, size_t ws_bytes, void* cuda_stream);
 
+/* error_frobenius without any allocation or caller-supplied workspace.  (The paper has no counterpart: this
+ * entry point exists for callers, not for the method.)
+ *
+ * Some callers may not allocate device memory at the point where they need the error: they are inside a
+ * CUDA-graph capture or another no-allocation region, their memory pool is fully committed, or their host
+ * application forbids libraries from growing their device footprint after start-up.  error_frobenius asks
+ * such a caller for a workspace; this variant instead keeps its per-block partial sums in a fixed 32 KiB
+ * array that is part of the library itself, so every GPU that loads the library carries that array until
+ * the process exits.
+ *
+ * Same arguments and result as error_frobenius (d_out[0] = sum (C - C*)^2, d_out[1] = sum C*^2; DEVICE), minus
+ * the workspace.  It calls no cudaMalloc / cudaFree and no routine that allocates.
+ *   - Size limit: M * N <= error_frobenius_noalloc_max_elements() (67,108,864); larger problems return
+ *     FMM_ERR_LIMIT and nothing is launched.
+ *   - First call on a device: looks up the array's device address (once per device, with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it needs clearing between calls (each block
+ *     overwrites its own slot), but two calls whose kernels overlap on the GPU — different streams without an
+ *     ordering between them — race on it: order such calls yourself.                                        */
+fmm_status error_frobenius_noalloc(const fmm_gemm_desc* d, const void* dC, const double* dCstar, double* d_out,
+                                   void* cuda_stream);
+int64_t error_frobenius_noalloc_max_elements(void);
+
 size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int G);
 
 /* Sweep over G gauge-equivalent copies of one scheme (Section 3.3 / Table 3, model-free form of

@@ -20,7 +20,8 @@ _DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
 EXPORTED_SYMBOLS = [
     "scheme_load", "scheme_builtin", "scheme_kron", "gauge_apply", "scheme_info", "scheme_coefficients",
     "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status", "classical_gemm_workspace",
-    "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius",
+    "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
+    "error_frobenius_noalloc_max_elements",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
 ]
@@ -87,6 +88,8 @@ _lib.exact_gemm_f64.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp]
 _lib.error_frobenius_workspace.argtypes = []
 _lib.error_frobenius_workspace.restype = _sz
 _lib.error_frobenius.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.error_frobenius_noalloc.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp]
+_lib.error_frobenius_noalloc_max_elements.restype = C.c_int64
 _lib.error_sweep_workspace.argtypes = [_vp, C.POINTER(GemmDesc), C.c_int]
 _lib.error_sweep_workspace.restype = _sz
 _lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(GemmDesc), _vp, _vp, _vp, _dp,
@@ -226,6 +229,18 @@ def exact_gemm_f64(d: GemmDesc, A, B, Cstar) -> None:
 def error_frobenius(d: GemmDesc, Cmat, Cstar, out2, ws) -> None:
     _check(_lib.error_frobenius(C.byref(d), _ptr(Cmat), _ptr(Cstar), _ptr(out2), _ptr(ws),
                                 ws.numel() * ws.element_size(), _stream()), "error_frobenius")
+
+
+def error_frobenius_noalloc(d: GemmDesc, Cmat, Cstar, out2) -> None:
+    """error_frobenius for callers that may not allocate: no workspace argument; the partial sums live in
+    a fixed array inside the library.  Raises FmmError (FMM_ERR_LIMIT) above
+    error_frobenius_noalloc_max_elements() elements.  Calls that overlap on the GPU race on that array."""
+    _check(_lib.error_frobenius_noalloc(C.byref(d), _ptr(Cmat), _ptr(Cstar), _ptr(out2), _stream()),
+           "error_frobenius_noalloc")
+
+
+def error_frobenius_noalloc_max_elements() -> int:
+    return int(_lib.error_frobenius_noalloc_max_elements())
 
 
 def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=None):

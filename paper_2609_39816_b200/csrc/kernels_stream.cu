@@ -653,6 +653,19 @@ cudaError_t launch_frob_err(int output, const void* C, int64_t ldc, const double
   return cudaGetLastError();
 }
 
+cudaError_t launch_frob_err_fixed_grid(int output, const void* C, int64_t ldc, const double* cstar, int64_t M,
+                                       int64_t N, double* part_err, double* part_ref, int grid, cudaStream_t st) {
+  if (grid < 1) return cudaErrorInvalidValue;
+  if (output == FMM_F32)
+    frob_err_kernel<float><<<grid, 256, 0, st>>>((const float*)C, ldc, cstar, M, N, part_err, part_ref);
+  else if (output == FMM_BF16)
+    frob_err_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)C, ldc, cstar, M, N, part_err, part_ref);
+  else
+    return cudaErrorInvalidValue;
+  ++fmm_launch_counter();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_exact_f64(int storage, const void* A, int64_t lda, const void* B, int64_t ldb,
                              int b_weight_layout, int64_t M, int64_t K, int64_t N, double* C, cudaStream_t st) {
   dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));

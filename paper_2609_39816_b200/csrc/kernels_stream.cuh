@@ -47,6 +47,9 @@ cudaError_t launch_cstar_prepare(const double* cstar, int64_t count, float* csta
 cudaError_t launch_frob_err(int output, const void* C, int64_t ldc, const double* cstar, int64_t M, int64_t N,
                             double* part_err, double* part_ref, int* n_partials, cudaStream_t st);
 int stream_grid(int64_t count);
+// same kernel, caller-chosen number of blocks (= number of partial sums written to each array)
+cudaError_t launch_frob_err_fixed_grid(int output, const void* C, int64_t ldc, const double* cstar, int64_t M,
+                                       int64_t N, double* part_err, double* part_ref, int grid, cudaStream_t st);
 
 cudaError_t launch_exact_f64(int storage, const void* A, int64_t lda, const void* B, int64_t ldb,
                              int b_weight_layout, int64_t M, int64_t K, int64_t N, double* C, cudaStream_t st);
