@@ -193,12 +193,15 @@ def measured_peaks():
 
 def ncu_traffic_per_launch():
     """DRAM bytes per launch of the block-product kernel at the bench workload, from the committed ncu
-    summary (profiles/traffic.json), or None when no capture has been recorded."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    summary (profiles/traffic_block_products_c2.txt), or None when no capture has been recorded."""
+    path = os.path.join(ROOT, "profiles", "traffic_block_products_c2.txt")
     try:
-        return json.load(open(path))["block_products_c2_dram_bytes_per_launch"]
+        for line in open(path):
+            if line.startswith("dram_bytes_per_launch"):
+                return int(line.split()[1])
     except Exception:
-        return None
+        pass
+    return None
 
 
 def run_ours(args):
@@ -296,13 +299,15 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel (block products), timed live by the library's phase events
     peaks = measured_peaks()
+    bm_, bk_, bn_ = M // 4, K // 4, N // 4
     prod_ms, prod_n = phases["products"]
     t_prod = prod_ms / max(prod_n, 1)
     achieved = flops_r / (t_prod * 1e-3) / 1e12 if t_prod > 0 else 0.0
-    roofline = {"bound": "tensor", "kernel": "block_products_kernel<256,bf16>", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "block_products_pair_kernel<bf16>", "achieved": achieved,
                 "peak": peaks["bf16"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16"],
                 "peak_source": f"{peaks['src']} bf16 burst", "frac_of_sustained": achieved / peaks["bf16_sustained"],
-                "flops_per_launch": flops_r, "ms_per_launch": t_prod, "traffic": ncu_traffic_per_launch()}
+                "flops_per_launch": flops_r, "ms_per_launch": t_prod, "traffic": ncu_traffic_per_launch(),
+                "algorithmic_bytes_per_launch": 2 * 49 * (bm_ * bk_ * 2) + 49 * bm_ * bn_ * 4}
     bm, bk, bn = M // 4, K // 4, N // 4
     pass_bytes = {  # algorithmic bytes of the streaming passes (read once + write once)
         "encode_a": M * K * 2 + 49 * bm * bk * 2,
