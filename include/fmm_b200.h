@@ -142,12 +142,14 @@ void scheme_free(fmm_scheme* s);
 /* Bytes of DEVICE workspace scheme_gemm needs for this scheme and problem (0 on bad args). */
 size_t scheme_gemm_workspace(const fmm_scheme* s, const fmm_gemm_desc* d);
 
-/* Where scheme_gemm leaves its intermediates inside the workspace (byte offsets from d_ws), so that a
- * caller (or a test) can inspect each step of Eq. 1 after the call:
- *   off[0] Ahat  [R][M/m][K/k]  product dtype      off[1] Bhat [R][N/n][K/k] product dtype (K-major)
- *   off[2] M_r   [R][M/m][N/n]  fp32               off[3] sA[R] fp32    off[4] sB[R] fp32
- * (sA, sB are written only in scale_mode 1).                                                   */
-fmm_status scheme_gemm_workspace_layout(const fmm_scheme* s, const fmm_gemm_desc* d, size_t off[5]);
+/* Where scheme_gemm leaves its intermediates inside the workspace, so that a caller (or a test) can inspect
+ * each step of Eq. 1 after the call.  Byte offsets from d_ws:
+ *   off[0] Ahat_r  R blocks [M/m][K/k], product dtype      off[1] Bhat_r  R blocks [N/n][K/k], product dtype (K-major)
+ *   off[2] M_r     R blocks [M/m][N/n], fp32               off[3] sA[R] fp32    off[4] sB[R] fp32 (scale_mode 1 only)
+ * and the distance, in ELEMENTS, between consecutive blocks r and r+1 of each array (block size plus a small
+ * padding that keeps the R streams off the same memory channels):
+ *   off[5] Ahat    off[6] Bhat    off[7] M                                                                  */
+fmm_status scheme_gemm_workspace_layout(const fmm_scheme* s, const fmm_gemm_desc* d, size_t off[8]);
 
 /* C = scheme(A, B) as defined at the top of this file (Eq. 1 with rounded block sums).
  * dA, dB, dC: DEVICE.  d_ws: DEVICE, >= scheme_gemm_workspace bytes, 256-byte aligned; its

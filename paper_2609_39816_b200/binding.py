@@ -199,9 +199,9 @@ def scheme_gemm_workspace(s: Scheme, d: GemmDesc) -> int:
 
 
 def scheme_gemm_workspace_layout(s: Scheme, d: GemmDesc) -> dict:
-    off = (_sz * 5)()
+    off = (_sz * 8)()
     _check(_lib.scheme_gemm_workspace_layout(s.handle, C.byref(d), off), "scheme_gemm_workspace_layout")
-    return dict(zip(["Ahat", "Bhat", "M", "sA", "sB"], [int(x) for x in off]))
+    return dict(zip(["Ahat", "Bhat", "M", "sA", "sB", "stride_Ahat", "stride_Bhat", "stride_M"], [int(x) for x in off]))
 
 
 def classical_gemm_workspace(d: GemmDesc) -> int:

@@ -119,7 +119,7 @@ template <typename SrcT, typename DstT, bool kAmaxOnly>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
               const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
-              float* __restrict__ scale_out, int use_scale, int tiles_per_block) {
+              float* __restrict__ scale_out, int use_scale, int tiles_per_block, int64_t rstride) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int NV = VE / 4;                     // float4 per staged vector
   constexpr int NP = VE / 2;                     // float2 pairs per vector
@@ -150,7 +150,6 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   const int pv = threadIdx.x - g * kEncPos;      // position vector inside the tile
   const int vec_per_row = (int)(bc / VE);        // 32-bit index arithmetic: br * bc / VE < 2^31 (checked by the host)
   const int nvec = (int)br * vec_per_row;
-  const int64_t rstride = br * bc;
   unsigned char* my_stage = stage + pv * 16;
   // element offset of each grid cell this thread stages (cells g, g+4, ...), computed once
   int64_t cell_base[4];
@@ -265,8 +264,8 @@ static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists 
 
 template <typename SrcT, typename DstT>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
-                            const CoefTable* d_tab, int padded, void* out, unsigned* amax_bits, float* scale,
-                            bool amax_only, bool use_scale, cudaStream_t st) {
+                            const CoefTable* d_tab, int padded, void* out, int64_t out_stride, unsigned* amax_bits,
+                            float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   constexpr int VE = Vec16<SrcT>::kElems;
   const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
                       (size_t)(gr * gc + 1) * (VE / 4) * kEncPos * 16;
@@ -283,7 +282,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[0] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride);
   } else {
     auto k = encode_kernel<SrcT, DstT, false>;
     if (!attr_done[1]) {
@@ -291,7 +290,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[1] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride);
   }
   ++fmm_launch_counter();
   return cudaGetLastError();
@@ -343,7 +342,7 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
               const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
               OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
-              double* __restrict__ partials, int tiles_per_block) {
+              double* __restrict__ partials, int tiles_per_block, int64_t rstride) {
   constexpr int kSlab = kDecPos * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DecSmemHead& sm = *reinterpret_cast<DecSmemHead*>(smem_raw);
@@ -356,7 +355,6 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
   const int pq = threadIdx.x - g * kDecPos;
   const int vec_per_row = (int)(bn >> 2);      // 32-bit index arithmetic: bm * bn / 4 < 2^31 (checked by the host)
   const int nvec = (int)bm * vec_per_row;
-  const int64_t rstride = bm * bn;
   unsigned char* my_stage = stage + pq * 16;
   const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
   // element offsets of the output cells this thread forms (cells g, g+4, ...), computed once
@@ -544,17 +542,17 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 // launch wrappers
 // ------------------------------------------------------------------------------------------
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
-                          int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, unsigned* amax_bits,
-                          float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+                          int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
+                          unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_encode_t<float, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_encode_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_encode_t<float, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   return cudaErrorInvalidValue;
 }
 
@@ -578,7 +576,7 @@ int decode_grid(int64_t bm, int64_t bn) {
 }
 
 template <typename OutT>
-static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, int R, int nnz, const float* sA,
+static cudaError_t launch_decode_t(const float* prod, int64_t prod_stride, const CoefTable* d_tab, int R, int nnz, const float* sA,
                                    const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
                                    const float* cstar32, double* partials, cudaStream_t st) {
   const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 16;
@@ -595,7 +593,7 @@ static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, in
       if (e != cudaSuccess) return e;                                                                            \
       attr_done[SLOT] = true;                                                                                    \
     }                                                                                                            \
-    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials, tpb); \
+    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials, tpb, prod_stride); \
   }
   if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true, 0)
   else if (C != nullptr) FMM_DECODE_LAUNCH(true, false, 1)
@@ -606,14 +604,14 @@ static cudaError_t launch_decode_t(const float* prod, const CoefTable* d_tab, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode(int output, const float* prod, const CoefTable* d_tab, const CoefTable* h_tab, int R,
+cudaError_t launch_decode(int output, const float* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
                           const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
                           int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   if (n_partials) *n_partials = decode_grid(bm, bn);
-  if (output == FMM_F32) return launch_decode_t<float>(prod, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
-  if (output == FMM_BF16) return launch_decode_t<__nv_bfloat16>(prod, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
+  if (output == FMM_F32) return launch_decode_t<float>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
+  if (output == FMM_BF16) return launch_decode_t<__nv_bfloat16>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
   return cudaErrorInvalidValue;
 }
 

@@ -14,25 +14,25 @@ struct DeviceStatus {
 int64_t& fmm_launch_counter();
 
 // X: source matrix (storage dtype), rows x cols with leading dimension ldx, split into a gr x gc grid of
-// br x bc blocks.  out[R][br][bc] in the product dtype.  With amax_only the kernel only accumulates
+// br x bc blocks.  out: R blocks [br][bc] in the product dtype, out_stride elements apart.  With amax_only the kernel only accumulates
 // max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).
 // With use_scale, scale[r] is derived from amax_bits[r] (2^ceil(log2(amax/448)), 1 if amax==0),
 // written to scale[R] and divided out before rounding.
 // h_tab = host copy of the same table (its list lengths size the kernel's shared memory).
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
-                          int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, unsigned* amax_bits,
-                          float* scale, bool amax_only, bool use_scale, cudaStream_t st);
+                          int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
+                          unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st);
 
 // Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
                              cudaStream_t st);
 
-// Decode (+ optional error reduction).  prod[R][bm][bn] fp32.  If C != nullptr the rounded result is stored
+// Decode (+ optional error reduction).  prod: R blocks [bm][bn] fp32, prod_stride elements apart.  If C != nullptr the rounded result is stored
 // (dtype `output`, leading dimension ldc).  If cstar32 != nullptr the per-block partial sums of
 // (rnd_O(c) - C*)^2 are written to partials[gridDim.x] and *n_partials receives gridDim.x.
 // d_tab is the CELL-MAJOR decode table (list c = the (r, w) pairs feeding C block c, ascending r); R is the
 // number of products; h_tab is the host copy of d_tab (its list lengths size the shared memory).
-cudaError_t launch_decode(int output, const float* prod, const CoefTable* d_tab, const CoefTable* h_tab, int R,
+cudaError_t launch_decode(int output, const float* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
                           const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
                           int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st);
 int decode_grid(int64_t bm, int64_t bn);

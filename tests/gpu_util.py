@@ -49,19 +49,21 @@ def run_scheme_gemm(s, A_t, B_t, S, Pd, O, weight_layout=False, scale_mode=0, fl
     m, k, n, R = s.dims
     bm, bk, bn = M // m, K // k, N // n
 
-    def grab(o, count, dt):
+    def grab(o, stride, rows, cols, dt):
+        """R blocks [rows, cols] of dtype dt, `stride` elements apart, starting at byte offset o."""
         es = torch.empty((), dtype=dt).element_size()
-        return ws[o:o + count * es].view(dt)
+        flat = ws[o:o + R * stride * es].view(dt).view(R, stride)[:, :rows * cols]
+        return flat.to(torch.float64).cpu().numpy().reshape(R, rows, cols)
 
     pdt = torch.bfloat16 if Pd == "bf16" else torch.float8_e4m3fn
     p = dict(
-        Ahat=grab(off["Ahat"], R * bm * bk, pdt).to(torch.float64).cpu().numpy().reshape(R, bm, bk),
-        BhatT=grab(off["Bhat"], R * bn * bk, pdt).to(torch.float64).cpu().numpy().reshape(R, bn, bk),
-        M=grab(off["M"], R * bm * bn, torch.float32).to(torch.float64).cpu().numpy().reshape(R, bm, bn),
+        Ahat=grab(off["Ahat"], off["stride_Ahat"], bm, bk, pdt),
+        BhatT=grab(off["Bhat"], off["stride_Bhat"], bn, bk, pdt),
+        M=grab(off["M"], off["stride_M"], bm, bn, torch.float32),
     )
     if scale_mode == 1:
-        p["sA"] = grab(off["sA"], R, torch.float32).to(torch.float64).cpu().numpy()
-        p["sB"] = grab(off["sB"], R, torch.float32).to(torch.float64).cpu().numpy()
+        p["sA"] = ws[off["sA"]:off["sA"] + 4 * R].view(torch.float32).to(torch.float64).cpu().numpy()
+        p["sB"] = ws[off["sB"]:off["sB"] + 4 * R].view(torch.float32).to(torch.float64).cpu().numpy()
     return out, p, ws
 
 

@@ -118,7 +118,9 @@ def test_descriptor_validation_without_gpu(lib):
     assert lib.error_sweep_workspace(s2, ok, 4) > need
     assert lib.classical_gemm_workspace(ok) > 0
     lay = lib.scheme_gemm_workspace_layout(s2, ok)
-    assert lay["Ahat"] < lay["Bhat"] < lay["M"] < need and all(v % 256 == 0 for v in lay.values())
+    assert lay["Ahat"] < lay["Bhat"] < lay["M"] < need
+    assert all(lay[key] % 256 == 0 for key in ("Ahat", "Bhat", "M", "sA", "sB"))
+    assert lay["stride_Ahat"] >= bm * bm and lay["stride_M"] >= bm * bm
 
 
 def test_sweep_sharding_over_ranks_gloo():
