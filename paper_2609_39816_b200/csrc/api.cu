@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -29,6 +30,55 @@ ProfScope::ProfScope(int kind, cudaStream_t s) : slot(-1), st(s) {
 ProfScope::~ProfScope() {
   if (slot >= 0) cudaEventRecord(g_prof[slot].b, st);
 }
+
+// ---------------------------------------------------------------- side stream for concurrent passes
+// The streaming passes leave most of the machine idle (they are latency-bound), so independent ones run side
+// by side: work is forked from the caller's stream onto one library-owned stream and joined back with events.
+// Nothing here synchronises the host.  One side stream and a ring of events per device, created on first use
+// (device calls of this library are therefore not safe to issue from several host threads at once).
+namespace {
+constexpr int kMaxDev = 64, kEventRing = 64;
+struct SideStream {
+  cudaStream_t stream = nullptr;    // general side stream (encode B beside encode A)
+  cudaStream_t stream2 = nullptr;   // second side stream (decode stage of a pipelined sweep)
+  cudaEvent_t ev[kEventRing] = {};
+  int next = 0;
+};
+SideStream g_side[kMaxDev];
+
+SideStream* side_stream() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+  SideStream& s = g_side[dev];
+  if (s.stream == nullptr) {
+    if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&s.stream2, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    for (int i = 0; i < kEventRing; ++i)
+      if (cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  }
+  return &s;
+}
+// record a fresh event of the ring on `from` (an event handed out stays untouched for kEventRing - 1 more records)
+cudaEvent_t record_event(SideStream* s, cudaStream_t from) {
+  cudaEvent_t e = s->ev[s->next];
+  s->next = (s->next + 1) % kEventRing;
+  return cudaEventRecord(e, from) == cudaSuccess ? e : nullptr;
+}
+// `to` waits for everything enqueued on `from` so far
+bool stream_wait(SideStream* s, cudaStream_t from, cudaStream_t to) {
+  cudaEvent_t e = s->ev[s->next];
+  s->next = (s->next + 1) % kEventRing;
+  return cudaEventRecord(e, from) == cudaSuccess && cudaStreamWaitEvent(to, e, 0) == cudaSuccess;
+}
+bool concurrency_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char* e = std::getenv("FMM_B200_NO_OVERLAP");
+    on = (e && e[0] == '1') ? 0 : 1;
+  }
+  return on == 1;
+}
+}  // namespace
 
 namespace {
 
@@ -109,16 +159,60 @@ fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, in
   return FMM_OK;
 }
 
-// The whole path for one scheme on one operand pair.  If C is null the result is not stored; if cstar32 is
-// given the squared error is reduced into err_out[0] (device).  hA/hB/hW are the host tables (always given:
-// their entry counts size the kernels' shared memory); they are uploaded into the workspace unless device
-// copies dA_tab/dB_tab/dW_tab are already in place.
+// One scheme applied to one operand pair inside one workspace: the pieces every stage needs.
+struct SchemeRun {
+  const fmm_scheme* s;
+  const fmm_gemm_desc* d;
+  GemmLayout L;
+  void* ws;
+  const CoefTable *hA, *hB, *hW;   // host tables (list lengths size the kernels' shared memory)
+  const CoefTable *dA, *dB, *dW;   // device copies
+  float* sA() const { return d->scale_mode == 1 ? at<float>(ws, L.sA) : nullptr; }
+  float* sB() const { return d->scale_mode == 1 ? at<float>(ws, L.sB) : nullptr; }
+};
+
+fmm_status stage_encode_a(const SchemeRun& r, const void* A, cudaStream_t st) {
+  const fmm_scheme* s = r.s;
+  ProfScope ps(0, st);
+  return encode_operand(r.d, A, r.d->lda, s->m, s->k, r.d->M / s->m, r.d->K / s->k, r.dA, r.hA, at<char>(r.ws, r.L.ahat),
+                        r.L.sAhat, at<unsigned>(r.ws, r.L.amaxA), r.sA(), st);
+}
+fmm_status stage_encode_b(const SchemeRun& r, const void* Bk, int64_t ldbk, cudaStream_t st) {
+  const fmm_scheme* s = r.s;
+  ProfScope ps(1, st);
+  return encode_operand(r.d, Bk, ldbk, s->n, s->k, r.d->N / s->n, r.d->K / s->k, r.dB, r.hB, at<char>(r.ws, r.L.bhat),
+                        r.L.sBhat, at<unsigned>(r.ws, r.L.amaxB), r.sB(), st);
+}
+fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
+  const fmm_scheme* s = r.s;
+  const int64_t bm = r.d->M / s->m, bk = r.d->K / s->k, bn = r.d->N / s->n;
+  BlockProductArgs g{};
+  g.product = r.d->product;
+  g.A = at<char>(r.ws, r.L.ahat); g.lda = bk; g.a_batch = r.L.sAhat;
+  g.B = at<char>(r.ws, r.L.bhat); g.ldb = bk; g.b_batch = r.L.sBhat;
+  g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = s->R;
+  g.out = at<char>(r.ws, r.L.prod); g.ldo = bn; g.o_batch = r.L.sProd; g.out_mode = 0; g.output = FMM_F32;
+  g.status = at<DeviceStatus>(r.ws, r.L.status);
+  ProfScope ps(2, st);
+  return launch_block_products(g, st);
+}
+// If C is null the result is not stored; if cstar32 is given the squared error is reduced into err_out[0].
+fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, double* err_out, cudaStream_t st) {
+  const fmm_scheme* s = r.s;
+  ProfScope ps(3, st);
+  int np = 0;
+  FMM_CUDA(launch_decode(r.d->output, at<float>(r.ws, r.L.prod), r.L.sProd, r.dW, r.hW, s->R, r.sA(), r.sB(), s->m, s->n,
+                         r.d->M / s->m, r.d->N / s->n, C, r.d->ldc, cstar32, at<double>(r.ws, r.L.partials), &np, st));
+  if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(r.ws, r.L.partials), np, err_out, st));
+  return FMM_OK;
+}
+
+// The whole path on the caller's stream (encode B runs beside encode A on the side stream).  Host tables are
+// uploaded into the workspace unless device copies are passed in.
 fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLayout& L, const CoefTable* hA,
                       const CoefTable* hB, const CoefTable* hW, const CoefTable* dA_tab, const CoefTable* dB_tab,
                       const CoefTable* dW_tab, const void* A, const void* Bsrc_kmajor, int64_t ldb_kmajor, void* C,
                       const float* cstar32, double* err_out, void* ws, bool skip_b, cudaStream_t st) {
-  const int m = s->m, k = s->k, n = s->n, R = s->R;
-  const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
   if (!dA_tab) {
     FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabA), hA, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
     dA_tab = at<CoefTable>(ws, L.tabA);
@@ -131,36 +225,19 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
     FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tabW), hW, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
     dW_tab = at<CoefTable>(ws, L.tabW);
   }
-  const bool scaled = d->scale_mode == 1;
-  float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
-  float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
-
-  {
-    ProfScope ps(0, st);
-    FMM_TRY(encode_operand(d, A, d->lda, m, k, bm, bk, dA_tab, hA, at<char>(ws, L.ahat), L.sAhat, at<unsigned>(ws, L.amaxA), sA, st));
+  const SchemeRun r{s, d, L, ws, hA, hB, hW, dA_tab, dB_tab, dW_tab};
+  // encode A on the caller's stream and encode B beside it on the side stream (they share nothing)
+  SideStream* side = (!skip_b && concurrency_enabled()) ? side_stream() : nullptr;
+  cudaStream_t stB = st;
+  if (side) {
+    if (!stream_wait(side, st, side->stream)) return FMM_ERR_CUDA;
+    stB = side->stream;
   }
-  if (!skip_b) {
-    ProfScope ps(1, st);
-    FMM_TRY(encode_operand(d, Bsrc_kmajor, ldb_kmajor, n, k, bn, bk, dB_tab, hB, at<char>(ws, L.bhat),
-                           L.sBhat, at<unsigned>(ws, L.amaxB), sB, st));
-  }
-  BlockProductArgs g{};
-  g.product = d->product;
-  g.A = at<char>(ws, L.ahat); g.lda = bk; g.a_batch = L.sAhat;
-  g.B = at<char>(ws, L.bhat); g.ldb = bk; g.b_batch = L.sBhat;
-  g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = R;
-  g.out = at<char>(ws, L.prod); g.ldo = bn; g.o_batch = L.sProd; g.out_mode = 0; g.output = FMM_F32;
-  g.status = at<DeviceStatus>(ws, L.status);
-  {
-    ProfScope ps(2, st);
-    FMM_TRY(launch_block_products(g, st));
-  }
-  ProfScope ps(3, st);
-  int np = 0;
-  FMM_CUDA(launch_decode(d->output, at<float>(ws, L.prod), L.sProd, dW_tab, hW, R, sA, sB, m, n, bm, bn, C, d->ldc, cstar32,
-                         at<double>(ws, L.partials), &np, st));
-  if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(ws, L.partials), np, err_out, st));
-  return FMM_OK;
+  if (!skip_b) FMM_TRY(stage_encode_b(r, Bsrc_kmajor, ldb_kmajor, stB));
+  FMM_TRY(stage_encode_a(r, A, st));
+  if (side && !stream_wait(side, side->stream, st)) return FMM_ERR_CUDA;
+  FMM_TRY(stage_products(r, st));
+  return stage_decode(r, C, cstar32, err_out, st);
 }
 
 // B as a K-major matrix [N x K]: in place for the weight layout, else transposed into the workspace.
@@ -244,7 +321,7 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
 // Workspace of a sweep: the GEMM layout plus reference copies, classical result, tables and sums.
 struct SweepLayout {
   GemmLayout g; ClassicalLayout c;
-  size_t gemm, classical, cstar, cstar32, ccl, tables, sums, total;
+  size_t gemm, gemm2, classical, cstar, cstar32, ccl, tables, sums, total;   // two GEMM workspaces: gauges are pipelined
 };
 
 SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
@@ -253,6 +330,7 @@ SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
   L.c = classical_layout(d);
   size_t o = 0;
   L.gemm = o; o += align_up(L.g.total);
+  L.gemm2 = o; o += align_up(L.g.total);
   L.classical = o; o += align_up(L.c.total);
   L.cstar = o; o += align_up((size_t)d->M * d->N * 8);
   L.cstar32 = o; o += align_up((size_t)d->M * d->N * 4);
@@ -426,22 +504,57 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   FMM_CUDA(launch_frob_err(d->output, ccl, d->N, cstar, d->M, d->N, part, nullptr, &np, st));
   FMM_CUDA(launch_sum_partials(part, np, sums + 1, st));
 
-  // 4. the sweep: per gauge encode A, encode B, R products, decode + error reduction
+  // 4. the sweep: per gauge encode A, encode B, R products, decode + error reduction.
+  // The three stages stress different parts of the machine (memory system, tensor cores + L2, memory system),
+  // so consecutive gauges are software-pipelined over three streams with two workspaces:
+  //   encode(g+1)  ||  products(g)  ||  decode(g-1).
   const void* bk_ptr; int64_t bk_ld;
   FMM_TRY(kmajor_b(d, dB, gws, L.g.bt, &bk_ptr, &bk_ld, false, st));
-  for (int g = 0; g < G; ++g) {
-    FMM_TRY(run_scheme(base, d, L.g, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2], d_tabs + 3 * g, d_tabs + 3 * g + 1,
-                       d_tabs + 3 * g + 2, dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
+  void* gws2 = ws + L.gemm2;
+  FMM_CUDA(cudaMemsetAsync(at<char>(gws2, L.g.status), 0, sizeof(DeviceStatus), st));
+  SideStream* side = concurrency_enabled() ? side_stream() : nullptr;
+  if (side == nullptr) {
+    for (int g = 0; g < G; ++g) {
+      FMM_TRY(run_scheme(base, d, L.g, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2], d_tabs + 3 * g, d_tabs + 3 * g + 1,
+                         d_tabs + 3 * g + 2, dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
+    }
+  } else {
+    cudaStream_t sE = side->stream, sG = st, sD = side->stream2;
+    if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;
+    cudaEvent_t evG[2] = {nullptr, nullptr}, evD[2] = {nullptr, nullptr};
+    for (int g = 0; g < G; ++g) {
+      const int b = g & 1;
+      const SchemeRun r{base, d, L.g, b ? gws2 : gws, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2],
+                        d_tabs + 3 * g, d_tabs + 3 * g + 1, d_tabs + 3 * g + 2};
+      // encode: the products of gauge g-2 must have finished reading this buffer's Ahat / Bhat
+      if (evG[b] && cudaStreamWaitEvent(sE, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
+      FMM_TRY(stage_encode_b(r, bk_ptr, bk_ld, sE));
+      FMM_TRY(stage_encode_a(r, dA, sE));
+      cudaEvent_t evE = record_event(side, sE);
+      // products: need this gauge's encode, and the decode of gauge g-2 must be done with this product buffer
+      if (!evE || cudaStreamWaitEvent(sG, evE, 0) != cudaSuccess) return FMM_ERR_CUDA;
+      if (evD[b] && cudaStreamWaitEvent(sG, evD[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
+      FMM_TRY(stage_products(r, sG));
+      evG[b] = record_event(side, sG);
+      // decode + error reduction
+      if (!evG[b] || cudaStreamWaitEvent(sD, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
+      FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + g, sD));
+      evD[b] = record_event(side, sD);
+      if (!evD[b]) return FMM_ERR_CUDA;
+    }
+    // join: the caller's stream continues after the last decode (the encode stream is ahead of it by construction)
+    if (!stream_wait(side, sD, st) || !stream_wait(side, sE, st)) return FMM_ERR_CUDA;
   }
 
   // 5. results to the host
   std::vector<double> h((size_t)G + 8);
-  DeviceStatus hs_g, hs_c;
+  DeviceStatus hs_g, hs_g2, hs_c;
   FMM_CUDA(cudaMemcpyAsync(h.data(), sums, h.size() * 8, cudaMemcpyDeviceToHost, st));
   FMM_CUDA(cudaMemcpyAsync(&hs_g, at<char>(gws, L.g.status), sizeof(DeviceStatus), cudaMemcpyDeviceToHost, st));
+  FMM_CUDA(cudaMemcpyAsync(&hs_g2, at<char>(ws + L.gemm2, L.g.status), sizeof(DeviceStatus), cudaMemcpyDeviceToHost, st));
   FMM_CUDA(cudaMemcpyAsync(&hs_c, at<char>(cws, L.c.status), sizeof(DeviceStatus), cudaMemcpyDeviceToHost, st));
   FMM_CUDA(cudaStreamSynchronize(st));
-  if (hs_g.code != 0 || hs_c.code != 0) return FMM_ERR_TIMEOUT;
+  if (hs_g.code != 0 || hs_g2.code != 0 || hs_c.code != 0) return FMM_ERR_TIMEOUT;
 
   const double nref = h[0], ecl = h[1];
   std::vector<double> rho(G);

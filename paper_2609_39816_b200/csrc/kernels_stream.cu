@@ -66,8 +66,9 @@ __device__ __forceinline__ double block_sum_double(double v, double* red /* >= 8
 //      (packed fma.rn.f32x2: each lane is an ordinary IEEE fp32 FMA), and stores 16 / 8 bytes.
 // ------------------------------------------------------------------------------------------
 constexpr int kEncThreads = 256;
-constexpr int kEncPos = 64;      // position vectors per block
-constexpr int kEncSplit = 4;     // threads per position vector
+// kEncSplit threads share one position vector (4 for the 4 x 4 grids / 49 products; 1 when the scheme is small,
+// where splitting would leave each thread almost nothing to do between barriers); kEncPos position vectors
+// per block.
 constexpr int kChunk = kTablePad;   // lists arrive padded to this multiple
 
 struct EncSmemHead {
@@ -115,12 +116,14 @@ template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* 
   else *reinterpret_cast<uint32_t*>(p) = h[0] | (h[1] << 16);
 }
 
-template <typename SrcT, typename DstT, bool kAmaxOnly>
+template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
               const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
               float* __restrict__ scale_out, int use_scale, int tiles_per_block, int64_t rstride) {
   constexpr int VE = Vec16<SrcT>::kElems;
+  constexpr int kEncPos = kEncThreads / kEncSplit;
+  constexpr int kCellsPerThread = 16 / kEncSplit; // grids have at most 16 cells
   constexpr int NV = VE / 4;                     // float4 per staged vector
   constexpr int NP = VE / 2;                     // float2 pairs per vector
   constexpr int kHalf = kEncPos * 16;            // bytes of one float4 plane of a slab
@@ -151,10 +154,10 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   const int vec_per_row = (int)(bc / VE);        // 32-bit index arithmetic: br * bc / VE < 2^31 (checked by the host)
   const int nvec = (int)br * vec_per_row;
   unsigned char* my_stage = stage + pv * 16;
-  // element offset of each grid cell this thread stages (cells g, g+4, ...), computed once
-  int64_t cell_base[4];
+  // element offset of each grid cell this thread stages (cells g, g+kEncSplit, ...), computed once
+  int64_t cell_base[kCellsPerThread];
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
+  for (int u = 0; u < kCellsPerThread; ++u) {
     const int c = g + u * kEncSplit;
     const int gi = c / gc, gj = c - gi * gc;
     cell_base[u] = (int64_t)gi * br * ldx + (int64_t)gj * bc;
@@ -171,26 +174,30 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     const int p = live ? idx / vec_per_row : 0;
     const int t = live ? (idx - p * vec_per_row) * VE : 0;
     if (it > 0) __syncthreads();                 // previous tile's readers are done with the stage
-    {                                            // up to four independent 16-byte loads in flight (ncell <= 16)
+    {                                            // four independent 16-byte loads in flight at a time
       const SrcT* src = X + (int64_t)p * ldx + t;
-      uint4 raw[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        raw[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (live && g + u * kEncSplit < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(src + cell_base[u]));
-      }
+      for (int u0 = 0; u0 < kCellsPerThread; u0 += 4) {
+        if (g + u0 * kEncSplit >= ncell) break;
+        uint4 raw[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int c = g + u * kEncSplit;
-        if (c < ncell) {
-          float4 v[NV];
-          Vec16<SrcT>::unpack(raw[u], v);
+        for (int u = 0; u < 4; ++u) {
+          raw[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (live && g + (u0 + u) * kEncSplit < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(src + cell_base[u0 + u]));
+        }
 #pragma unroll
-          for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
+        for (int u = 0; u < 4; ++u) {
+          const int c = g + (u0 + u) * kEncSplit;
+          if (c < ncell) {
+            float4 v[NV];
+            Vec16<SrcT>::unpack(raw[u], v);
+#pragma unroll
+            for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
+          }
         }
       }
     }
-    __syncthreads();   // staged vectors (and, first time, the table) are visible to the four sharing threads
+    __syncthreads();   // staged vectors (and, first time, the table) are visible to the sharing threads
 
     DstT* dst = out + (int64_t)p * bc + t;
     for (int r = g; r < R; r += kEncSplit) {
@@ -262,21 +269,22 @@ static void split_tiles(int64_t tiles, int* grid, int* tiles_per_block) {
 
 static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists arrive padded from the host
 
-template <typename SrcT, typename DstT>
+template <typename SrcT, typename DstT, int kSplit>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
                             const CoefTable* d_tab, int padded, void* out, int64_t out_stride, unsigned* amax_bits,
                             float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   constexpr int VE = Vec16<SrcT>::kElems;
+  constexpr int kEncPos = kEncThreads / kSplit;
   const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
                       (size_t)(gr * gc + 1) * (VE / 4) * kEncPos * 16;
   const int64_t vecs = br * (bc / VE);
   if (vecs == 0) return cudaSuccess;
-  if (vecs + kEncPos * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // kernels index positions in 32 bits
+  if (vecs + kEncThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // kernels index positions in 32 bits
   int grid, tpb;
   split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
   static bool attr_done[2] = {false, false};
   if (amax_only) {
-    auto k = encode_kernel<SrcT, DstT, true>;
+    auto k = encode_kernel<SrcT, DstT, true, kSplit>;
     if (!attr_done[0]) {
       cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
@@ -284,7 +292,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
     }
     k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride);
   } else {
-    auto k = encode_kernel<SrcT, DstT, false>;
+    auto k = encode_kernel<SrcT, DstT, false, kSplit>;
     if (!attr_done[1]) {
       cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
@@ -327,9 +335,7 @@ __global__ void __launch_bounds__(256) transpose_kernel(const T* __restrict__ B,
 //      table, ascending r, padded to a multiple of 4 with (zero slab, 0.0f) entries) in registers, two
 //      lanes per packed fma.rn.f32x2, rounds, stores, and accumulates its share of the error.
 // ------------------------------------------------------------------------------------------
-constexpr int kDecThreads = 256;
-constexpr int kDecPos = 64;
-constexpr int kDecSplit = 4;
+constexpr int kDecThreads = 256;   // kDecSplit threads share one position quad (4, or 1 for small schemes)
 
 struct DecSmemHead {
   int off[kMaxCells + 1];   // entries, multiples of kChunk
@@ -337,12 +343,14 @@ struct DecSmemHead {
   double red[kDecThreads / 32];
 };  // followed by int2 ent[] {byte offset of product r's slab, scaled coefficient bits}, then the stage
 
-template <typename OutT, bool kStore, bool kErr>
+template <typename OutT, bool kStore, bool kErr, int kDecSplit>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
               const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
               OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
               double* __restrict__ partials, int tiles_per_block, int64_t rstride) {
+  constexpr int kDecPos = kDecThreads / kDecSplit;
+  constexpr int kCellsPerThread = 16 / kDecSplit;
   constexpr int kSlab = kDecPos * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DecSmemHead& sm = *reinterpret_cast<DecSmemHead*>(smem_raw);
@@ -358,9 +366,9 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
   unsigned char* my_stage = stage + pq * 16;
   const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
   // element offsets of the output cells this thread forms (cells g, g+4, ...), computed once
-  int64_t out_base[4], cs_base[4];
+  int64_t out_base[kCellsPerThread], cs_base[kCellsPerThread];
 #pragma unroll
-  for (int u = 0; u < 4; ++u) {
+  for (int u = 0; u < kCellsPerThread; ++u) {
     const int c = g + u * kDecSplit;
     const int i = c / n, j = c - i * n;
     out_base[u] = (int64_t)i * bm * ldc + (int64_t)j * bn;
@@ -396,7 +404,7 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
     __syncthreads();
 
 #pragma unroll
-    for (int u4 = 0; u4 < 4; ++u4) {           // ncell <= 16: at most four cells per thread
+    for (int u4 = 0; u4 < kCellsPerThread; ++u4) {   // ncell <= 16
       const int c = g + u4 * kDecSplit;
       if (c >= ncell) break;
       float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
@@ -541,19 +549,29 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 // ------------------------------------------------------------------------------------------
 // launch wrappers
 // ------------------------------------------------------------------------------------------
+template <int kSplit>
+static cudaError_t launch_encode_split(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
+                                       int64_t bc, const CoefTable* d_tab, int nnz, void* out, int64_t out_stride,
+                                       unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+  if (storage == FMM_F32 && product == FMM_BF16)
+    return launch_encode_t<float, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  if (storage == FMM_BF16 && product == FMM_BF16)
+    return launch_encode_t<__nv_bfloat16, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  if (storage == FMM_F32 && product == FMM_E4M3)
+    return launch_encode_t<float, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  if (storage == FMM_BF16 && product == FMM_E4M3)
+    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  return cudaErrorInvalidValue;
+}
+
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
                           unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
-  if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_encode_t<float, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_encode_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_encode_t<float, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  return cudaErrorInvalidValue;
+  // small schemes (at most 4 cells): one thread per position vector; otherwise four threads share one
+  if (gr * gc <= 4)
+    return launch_encode_split<1>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  return launch_encode_split<4>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
 }
 
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
@@ -569,25 +587,28 @@ cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t
   return cudaGetLastError();
 }
 
+// upper bound of the number of decode blocks (= partial sums) over both thread splits
 int decode_grid(int64_t bm, int64_t bn) {
   int grid, tpb;
-  split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
+  split_tiles((bm * (bn >> 2) + 63) / 64, &grid, &tpb);
   return grid;
 }
 
-template <typename OutT>
+template <typename OutT, int kSplit>
 static cudaError_t launch_decode_t(const float* prod, int64_t prod_stride, const CoefTable* d_tab, int R, int nnz, const float* sA,
                                    const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
-                                   const float* cstar32, double* partials, cudaStream_t st) {
+                                   const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
+  constexpr int kDecPos = kDecThreads / kSplit;
   const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 16;
-  if (bm * (bn >> 2) + kDecPos * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
+  if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
   int grid, tpb;
   split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
+  if (n_partials) *n_partials = grid;
   const int64_t ldcs = (int64_t)n * bn;
   static bool attr_done[3] = {false, false, false};
 #define FMM_DECODE_LAUNCH(STORE, ERR, SLOT)                                                                      \
   {                                                                                                              \
-    auto k = decode_kernel<OutT, STORE, ERR>;                                                                    \
+    auto k = decode_kernel<OutT, STORE, ERR, kSplit>;                                                            \
     if (!attr_done[SLOT]) {                                                                                      \
       cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);          \
       if (e != cudaSuccess) return e;                                                                            \
@@ -609,9 +630,14 @@ cudaError_t launch_decode(int output, const float* prod, int64_t prod_stride, co
                           int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
-  if (n_partials) *n_partials = decode_grid(bm, bn);
-  if (output == FMM_F32) return launch_decode_t<float>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
-  if (output == FMM_BF16) return launch_decode_t<__nv_bfloat16>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, st);
+  // small schemes (at most 8 products, 4 output cells): one thread per position quad; otherwise four share one
+  const bool small = R <= 8 && m * n <= 4;
+  if (output == FMM_F32)
+    return small ? launch_decode_t<float, 1>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
+                 : launch_decode_t<float, 4>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
+  if (output == FMM_BF16)
+    return small ? launch_decode_t<__nv_bfloat16, 1>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
+                 : launch_decode_t<__nv_bfloat16, 4>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
   return cudaErrorInvalidValue;
 }
 
