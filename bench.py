@@ -96,7 +96,7 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -390,6 +390,79 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------ other configurations (not the default line)
+def run_workload(args):
+    """Throughput of the other benchmark configurations on one GPU; prints one JSON line for --workload."""
+    import torch
+
+    import paper_2609_39816_b200 as fmm
+    from fmm_inputs import generators as gen
+
+    torch.cuda.set_device(0)
+    peaks = measured_peaks()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, steps=10, warmup=3):
+        for _ in range(warmup):
+            flush.zero_(); fn()
+        torch.cuda.synchronize()
+        evs = []
+        for _ in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return float(np.median([a.elapsed_time(b) for a, b in evs]))
+
+    def one_gemm(scheme, T, K, N, S, Pd, O, scale, dist):
+        A = gen.activations_outlier(0, 1, T, K, dist=dist, frac=0.001 if dist == "t3" else 0.005,
+                                    factor=300.0 if dist == "t3" else 100.0, at_least=1 if dist == "t3" else 0)
+        if S == "f32":
+            A = gen.normal(0, 1, (T, K))
+        W = gen.normal(0, 2, (N, K), std=1.0 if S == "f32" else 0.02)          # weight layout [N, K]
+        At = gen.to_storage(A, S)[0].cuda()
+        Wt = gen.to_storage(W, S)[0].cuda()
+        s = fmm.scheme_builtin(scheme)
+        m, k, n, R = s.dims
+        d = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale)
+        ws = torch.empty(fmm.scheme_gemm_workspace(s, d), dtype=torch.uint8, device="cuda")
+        C = torch.empty((T, N), dtype=torch.float32 if O == "f32" else torch.bfloat16, device="cuda")
+        t = timed(lambda: fmm.scheme_gemm(s, d, At, Wt, C, ws))
+        fmm.device_status(ws)
+        dr = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale, flags=fmm.FLAG_REUSE_BHAT)
+        t_cached = timed(lambda: fmm.scheme_gemm(s, dr, At, Wt, C, ws))
+        wsc = torch.empty(max(fmm.classical_gemm_workspace(d), 256), dtype=torch.uint8, device="cuda")
+        t_cl = timed(lambda: fmm.classical_gemm(d, At, Wt, C, wsc))
+        eff = 2.0 * T * K * N
+        rfl = 2.0 * R * (T // m) * (K // k) * (N // n)
+        return {"shape": [T, K, N], "product": Pd, "ms": t, "eff_tflops": eff / t / 1e9, "r_tflops": rfl / t / 1e9,
+                "ms_weights_cached": t_cached, "eff_tflops_weights_cached": eff / t_cached / 1e9,
+                "classical_ms": t_cl, "classical_tflops": eff / t_cl / 1e9, "scheme_over_classical": t / t_cl}
+
+    wl = args.workload
+    out = {"workload": wl, "n_gpus": 1, "data": "synthetic", "unit": UNIT, "peaks": peaks,
+           "protocol": "median of 10 CUDA-event timings, 3 warm-ups, 256 MiB L2 flush before each"}
+    if wl == "c1":
+        out["gemms"] = [one_gemm("strassen222", 256, 256, 256, "f32", "bf16", "f32", 0, "normal")]
+        out["note"] = "one tile position: a latency case (four launches), not a throughput case"
+    elif wl == "c4":
+        shapes = [(4096, 12288), (4096, 4096), (4096, 22016), (11008, 4096)]
+        out["gemms"] = [one_gemm("strassen444", 2048, K, N, "bf16", "e4m3", "bf16", 1, "t3") for K, N in shapes]
+    elif wl == "c5":
+        shapes = [(5120, 15360), (5120, 27648), (13824, 5120)]
+        out["gemms"] = [one_gemm("strassen444", 8192, K, N, "bf16", pd, "bf16", 1 if pd == "e4m3" else 0, "t3")
+                        for pd in ("bf16", "e4m3") for K, N in shapes]
+    else:
+        raise SystemExit(f"unknown workload {wl}")
+    tot_t = sum(g["ms"] for g in out["gemms"])
+    tot_f = sum(2.0 * g["shape"][0] * g["shape"][1] * g["shape"][2] for g in out["gemms"])
+    out["metric"] = METRIC
+    out["value"] = tot_f / tot_t / 1e9
+    out["ms_total"] = tot_t
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -398,11 +471,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=32, help="gauges per rank in the c3 sweep (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c5")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "c2":
+        run_workload(args)
     else:
         run_ours(args)
 

@@ -53,6 +53,7 @@ def _inputs(seed, M, K, N, S, kind="normal", bound=None):
     ("strassen444", 512, 1024, 512, "bf16", "e4m3", "bf16", "t3", 1),       # fp8 with per-tensor scales
     ("strassen222", 256, 2240, 272, "bf16", "e4m3", "f32", "llm", 1),       # fp8, K tail inside a stage
     ("strassen444", 64, 64, 32, "f32", "bf16", "f32", "normal", 0),         # smallest legal blocks
+    ("strassen444", 256, 11008, 512, "bf16", "e4m3", "bf16", "t3", 1),      # config-4 down-projection K: K/4 = 2752 = 21.5 stages
 ])
 def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     At, Bt, A64, B64 = _inputs(3, M, K, N, S, kind)
