@@ -5,6 +5,7 @@
 #include <cuda_fp8.h>
 
 #include <cmath>
+#include <cstdlib>
 
 #include "kernels_stream.cuh"
 
@@ -83,57 +84,69 @@ struct EncSmemHead {
 template <typename SrcT> struct Vec16;
 template <> struct Vec16<float> {
   static constexpr int kElems = 4;
-  static __device__ __forceinline__ void unpack(const uint4& raw, float4 (&v)[1]) {
-    v[0] = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
+  static __device__ __forceinline__ void unpack(const uint4& raw, float2 (&v)[2]) {
+    v[0] = make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y));
+    v[1] = make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
   }
 };
 template <> struct Vec16<__nv_bfloat16> {
   static constexpr int kElems = 8;
-  static __device__ __forceinline__ void unpack(const uint4& raw, float4 (&v)[2]) {
-    v[0] = make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u),
-                       __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
-    v[1] = make_float4(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xFFFF0000u),
-                       __uint_as_float(raw.w << 16), __uint_as_float(raw.w & 0xFFFF0000u));
+  static __device__ __forceinline__ void unpack(const uint4& raw, float2 (&v)[4]) {
+    v[0] = make_float2(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xFFFF0000u));
+    v[1] = make_float2(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xFFFF0000u));
+    v[2] = make_float2(__uint_as_float(raw.z << 16), __uint_as_float(raw.z & 0xFFFF0000u));
+    v[3] = make_float2(__uint_as_float(raw.w << 16), __uint_as_float(raw.w & 0xFFFF0000u));
   }
 };
 
-template <int NP> __device__ __forceinline__ void store_vec(__nv_bfloat16* p, const float2 (&a)[NP]) {
+// `stream`: the outputs will have left L2 before they are read again, so store them evict-first (st.global.cs)
+template <int NP> __device__ __forceinline__ void store_vec(__nv_bfloat16* p, const float2 (&a)[NP], bool stream) {
   uint32_t w[NP];
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
     __nv_bfloat162 b = __floats2bfloat162_rn(a[i].x, a[i].y);
     w[i] = *reinterpret_cast<uint32_t*>(&b);
   }
-  if (NP == 4) *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2 % NP], w[3 % NP]);
-  else *reinterpret_cast<uint2*>(p) = make_uint2(w[0], w[1]);
+  if (NP == 4) {
+    const uint4 v = make_uint4(w[0], w[1], w[2 % NP], w[3 % NP]);
+    if (stream) __stcs(reinterpret_cast<uint4*>(p), v); else *reinterpret_cast<uint4*>(p) = v;
+  } else {
+    const uint2 v = make_uint2(w[0], w[1]);
+    if (stream) __stcs(reinterpret_cast<uint2*>(p), v); else *reinterpret_cast<uint2*>(p) = v;
+  }
 }
 // e4m3: round to nearest even, saturate to +-448 (NaN stays NaN)
-template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* p, const float2 (&a)[NP]) {
+template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* p, const float2 (&a)[NP], bool stream) {
   uint32_t h[NP];
 #pragma unroll
   for (int i = 0; i < NP; ++i) h[i] = __nv_cvt_float2_to_fp8x2(a[i], __NV_SATFINITE, __NV_E4M3);
-  if (NP == 4) *reinterpret_cast<uint2*>(p) = make_uint2(h[0] | (h[1] << 16), h[2 % NP] | (h[3 % NP] << 16));
-  else *reinterpret_cast<uint32_t*>(p) = h[0] | (h[1] << 16);
+  if (NP == 4) {
+    const uint2 v = make_uint2(h[0] | (h[1] << 16), h[2 % NP] | (h[3 % NP] << 16));
+    if (stream) __stcs(reinterpret_cast<uint2*>(p), v); else *reinterpret_cast<uint2*>(p) = v;
+  } else {
+    const unsigned v = h[0] | (h[1] << 16);
+    if (stream) __stcs(reinterpret_cast<unsigned*>(p), v); else *reinterpret_cast<unsigned*>(p) = v;
+  }
 }
 
 template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
               const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
-              float* __restrict__ scale_out, int use_scale, int tiles_per_block, int64_t rstride) {
+              float* __restrict__ scale_out, int use_scale, int tiles_per_block, int64_t rstride, int stream_out) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kEncSplit;
   constexpr int kCellsPerThread = 16 / kEncSplit; // grids have at most 16 cells
-  constexpr int NV = VE / 4;                     // float4 per staged vector
   constexpr int NP = VE / 2;                     // float2 pairs per vector
-  constexpr int kHalf = kEncPos * 16;            // bytes of one float4 plane of a slab
-  constexpr int kSlab = NV * kHalf;              // bytes of one cell's slab
+  constexpr int kSlab = kEncPos * 16;            // bytes of one cell's slab: the raw 16-byte vectors of a tile
   extern __shared__ __align__(16) unsigned char smem_raw[];
   EncSmemHead& sm = *reinterpret_cast<EncSmemHead*>(smem_raw);
   const int R = d_tab->R, ncell = d_tab->ncell;
   const int total = d_tab->off[R];               // lists arrive padded to multiples of kChunk
   int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(EncSmemHead));
+  // two stages of (ncell + 1) slabs: the copies of tile it+1 land in one while tile it is read from the other
   unsigned char* stage = smem_raw + ((sizeof(EncSmemHead) + (size_t)total * 8 + 15) / 16) * 16;
+  const int kStageBytes = (ncell + 1) * kSlab;
 
   for (int i = threadIdx.x; i <= R; i += kEncThreads) sm.off[i] = d_tab->off[i];
   for (int i = threadIdx.x; i < total; i += kEncThreads)
@@ -149,11 +162,10 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     if (!kAmaxOnly && use_scale && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
   }
 
-  const int g = threadIdx.x / kEncPos;           // which quarter of the cells / products this thread handles
+  const int g = threadIdx.x / kEncPos;           // which share of the cells / products this thread handles
   const int pv = threadIdx.x - g * kEncPos;      // position vector inside the tile
   const int vec_per_row = (int)(bc / VE);        // 32-bit index arithmetic: br * bc / VE < 2^31 (checked by the host)
   const int nvec = (int)br * vec_per_row;
-  unsigned char* my_stage = stage + pv * 16;
   // element offset of each grid cell this thread stages (cells g, g+kEncSplit, ...), computed once
   int64_t cell_base[kCellsPerThread];
 #pragma unroll
@@ -162,93 +174,115 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     const int gi = c / gc, gj = c - gi * gc;
     cell_base[u] = (int64_t)gi * br * ldx + (int64_t)gj * bc;
   }
-  if (g == 0) {
-#pragma unroll
-    for (int h = 0; h < NV; ++h)
-      *reinterpret_cast<float4*>(my_stage + ncell * kSlab + h * kHalf) = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (g == 0) {   // the all-zero slab behind the data slabs, in both stages
+    *reinterpret_cast<uint4*>(stage + ncell * kSlab + pv * 16) = make_uint4(0u, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(stage + kStageBytes + ncell * kSlab + pv * 16) = make_uint4(0u, 0u, 0u, 0u);
   }
+  const uint32_t stage_u32 = (uint32_t)__cvta_generic_to_shared(stage) + pv * 16;
+
+  // asynchronous copies of this thread's cells of tile `it` into stage `it & 1` (16 bytes each, L2 only)
+  auto issue_copies = [&](int it) {
+    if (it < tiles_per_block) {
+      const int idx = (blockIdx.x * tiles_per_block + it) * kEncPos + pv;
+      const bool live = idx < nvec;
+      const int p = live ? idx / vec_per_row : 0;
+      const int t = live ? (idx - p * vec_per_row) * VE : 0;
+      const SrcT* src = X + (int64_t)p * ldx + t;
+      const uint32_t dst = stage_u32 + (it & 1) * kStageBytes;
+      const int nbytes = live ? 16 : 0;          // 0 source bytes: the destination is zero-filled
+#pragma unroll
+      for (int u = 0; u < kCellsPerThread; ++u) {
+        const int c = g + u * kEncSplit;
+        if (c < ncell)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + c * kSlab), "l"(src + cell_base[u]),
+                       "r"(nbytes) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  issue_copies(0);
 
   for (int it = 0; it < tiles_per_block; ++it) {
     const int idx = (blockIdx.x * tiles_per_block + it) * kEncPos + pv;
     const bool live = idx < nvec;
     const int p = live ? idx / vec_per_row : 0;
     const int t = live ? (idx - p * vec_per_row) * VE : 0;
-    if (it > 0) __syncthreads();                 // previous tile's readers are done with the stage
-    {                                            // four independent 16-byte loads in flight at a time
-      const SrcT* src = X + (int64_t)p * ldx + t;
-#pragma unroll
-      for (int u0 = 0; u0 < kCellsPerThread; u0 += 4) {
-        if (g + u0 * kEncSplit >= ncell) break;
-        uint4 raw[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          raw[u] = make_uint4(0u, 0u, 0u, 0u);
-          if (live && g + (u0 + u) * kEncSplit < ncell) raw[u] = __ldg(reinterpret_cast<const uint4*>(src + cell_base[u0 + u]));
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int c = g + (u0 + u) * kEncSplit;
-          if (c < ncell) {
-            float4 v[NV];
-            Vec16<SrcT>::unpack(raw[u], v);
-#pragma unroll
-            for (int h = 0; h < NV; ++h) *reinterpret_cast<float4*>(my_stage + c * kSlab + h * kHalf) = v[h];
-          }
-        }
-      }
-    }
-    __syncthreads();   // staged vectors (and, first time, the table) are visible to the sharing threads
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();        // tile it has landed for every thread, and everyone is done reading tile it-1's stage
+    issue_copies(it + 1);   // overlaps the arithmetic and the stores below
+    const unsigned char* my_stage = stage + (it & 1) * kStageBytes + pv * 16;
 
     DstT* dst = out + (int64_t)p * bc + t;
-    for (int r = g; r < R; r += kEncSplit) {
-      float2 acc[NP];
+    // two products per iteration (r and r + kEncSplit): their loads are issued together so that the two
+    // FMA chains overlap each other's shared-memory latency
+    for (int r0 = g; r0 < R; r0 += 2 * kEncSplit) {
+      const int r1 = r0 + kEncSplit;
+      const bool two = r1 < R;
+      float2 acc[2][NP];
 #pragma unroll
-      for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
-      const int e1 = sm.off[r + 1];
-      for (int e = sm.off[r]; e < e1; e += kChunk) {
-        int2 en[kChunk];
-        float4 v[kChunk][NV];
+      for (int j = 0; j < 2; ++j)
 #pragma unroll
-        for (int u = 0; u < kChunk; u += 2) {
-          const int4 two = *reinterpret_cast<const int4*>(&ent[e + u]);
-          en[u] = make_int2(two.x, two.y);
-          en[u + 1] = make_int2(two.z, two.w);
+        for (int i = 0; i < NP; ++i) acc[j][i] = make_float2(0.0f, 0.0f);
+      int e[2] = {sm.off[r0], two ? sm.off[r1] : 0};
+      const int eend[2] = {sm.off[r0 + 1], two ? sm.off[r1 + 1] : 0};
+      while (e[0] < eend[0] || e[1] < eend[1]) {
+        int2 en[2][kChunk];
+        uint4 raw[2][kChunk];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const bool on = e[j] < eend[j];
+#pragma unroll
+          for (int u = 0; u < kChunk; u += 2) {
+            // an exhausted list reads the padding pattern (zero slab, 0.0f): adds exactly nothing
+            const int4 pair = on ? *reinterpret_cast<const int4*>(&ent[e[j] + u])
+                                 : make_int4(ncell * kSlab, 0, ncell * kSlab, 0);
+            en[j][u] = make_int2(pair.x, pair.y);
+            en[j][u + 1] = make_int2(pair.z, pair.w);
+          }
         }
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+          for (int u = 0; u < kChunk; ++u) raw[j][u] = *reinterpret_cast<const uint4*>(my_stage + en[j][u].x);
 #pragma unroll
         for (int u = 0; u < kChunk; ++u)
 #pragma unroll
-          for (int h = 0; h < NV; ++h) v[u][h] = *reinterpret_cast<const float4*>(my_stage + en[u].x + h * kHalf);
+          for (int j = 0; j < 2; ++j) {
+            const float c = __int_as_float(en[j][u].y);
+            const float2 cc = make_float2(c, c);
+            float2 v[NP];
+            Vec16<SrcT>::unpack(raw[j][u], v);
 #pragma unroll
-        for (int u = 0; u < kChunk; ++u) {
-          const float c = __int_as_float(en[u].y);
-          const float2 cc = make_float2(c, c);
-#pragma unroll
-          for (int h = 0; h < NV; ++h) {
-            acc[2 * h] = __ffma2_rn(cc, make_float2(v[u][h].x, v[u][h].y), acc[2 * h]);
-            acc[2 * h + 1] = __ffma2_rn(cc, make_float2(v[u][h].z, v[u][h].w), acc[2 * h + 1]);
+            for (int i = 0; i < NP; ++i) acc[j][i] = __ffma2_rn(cc, v[i], acc[j][i]);
           }
-        }
+        e[0] += kChunk;
+        e[1] += kChunk;
       }
-      if (kAmaxOnly) {
-        float a = 0.0f;
 #pragma unroll
-        for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
+      for (int j = 0; j < 2; ++j) {
+        const int r = j == 0 ? r0 : r1;
+        if (j == 1 && !two) break;
+        if (kAmaxOnly) {
+          float a = 0.0f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-        if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
-      } else if (live) {
-        if (use_scale) {
-          if (sm.use_mul[r]) {
-            const float inv = sm.inv_scale[r];
+          for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[j][i].x), fabsf(acc[j][i].y)));   // fmaxf drops NaN
 #pragma unroll
-            for (int i = 0; i < NP; ++i) { acc[i].x *= inv; acc[i].y *= inv; }
-          } else {
-            const float s = sm.scale[r];
+          for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+          if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
+        } else if (live) {
+          if (use_scale) {
+            if (sm.use_mul[r]) {
+              const float inv = sm.inv_scale[r];
 #pragma unroll
-            for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, s); acc[i].y = __fdiv_rn(acc[i].y, s); }
+              for (int i = 0; i < NP; ++i) { acc[j][i].x *= inv; acc[j][i].y *= inv; }
+            } else {
+              const float sc = sm.scale[r];
+#pragma unroll
+              for (int i = 0; i < NP; ++i) { acc[j][i].x = __fdiv_rn(acc[j][i].x, sc); acc[j][i].y = __fdiv_rn(acc[j][i].y, sc); }
+            }
           }
+          store_vec<NP>(dst + r * rstride, acc[j], stream_out != 0);
         }
-        store_vec<NP>(dst + r * rstride, acc);
       }
     }
   }
@@ -271,17 +305,20 @@ static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists 
 
 template <typename SrcT, typename DstT, int kSplit>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
-                            const CoefTable* d_tab, int padded, void* out, int64_t out_stride, unsigned* amax_bits,
-                            float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+                            const CoefTable* d_tab, int padded, int lists, void* out, int64_t out_stride,
+                            unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kSplit;
   const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
-                      (size_t)(gr * gc + 1) * (VE / 4) * kEncPos * 16;
+                      2 * (size_t)(gr * gc + 1) * kEncPos * 16;
   const int64_t vecs = br * (bc / VE);
   if (vecs == 0) return cudaSuccess;
   if (vecs + kEncThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // kernels index positions in 32 bits
   int grid, tpb;
   split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
+  // outputs larger than the part of L2 that keeps shared data (~60 MB) will have left it before they are read
+  int stream_out = (int64_t)lists * out_stride * (int64_t)sizeof(DstT) > ((int64_t)48 << 20) ? 1 : 0;
+  if (const char* e = std::getenv("FMM_B200_ENC_STREAM")) stream_out = std::atoi(e);
   static bool attr_done[2] = {false, false};
   if (amax_only) {
     auto k = encode_kernel<SrcT, DstT, true, kSplit>;
@@ -290,7 +327,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[0] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride, stream_out);
   } else {
     auto k = encode_kernel<SrcT, DstT, false, kSplit>;
     if (!attr_done[1]) {
@@ -298,7 +335,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[1] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride);
+    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride, stream_out);
   }
   ++fmm_launch_counter();
   return cudaGetLastError();
@@ -551,16 +588,16 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 // ------------------------------------------------------------------------------------------
 template <int kSplit>
 static cudaError_t launch_encode_split(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
-                                       int64_t bc, const CoefTable* d_tab, int nnz, void* out, int64_t out_stride,
+                                       int64_t bc, const CoefTable* d_tab, int nnz, int lists, void* out, int64_t out_stride,
                                        unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
   if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_encode_t<float, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_encode_t<__nv_bfloat16, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_encode_t<float, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   return cudaErrorInvalidValue;
 }
 
@@ -570,8 +607,8 @@ cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, 
   const int nnz = padded_entries(*h_tab);
   // small schemes (at most 4 cells): one thread per position vector; otherwise four threads share one
   if (gr * gc <= 4)
-    return launch_encode_split<1>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  return launch_encode_split<4>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_split<1>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, h_tab->R, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  return launch_encode_split<4>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, h_tab->R, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
 }
 
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
