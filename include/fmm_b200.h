@@ -163,6 +163,14 @@ fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* 
  * on this workspace left: FMM_OK or FMM_ERR_TIMEOUT.                                        */
 fmm_status fmm_device_status(const void* d_ws, void* cuda_stream);
 
+/* Self-test of device-side failure reporting.  Launches ONE block of the block-product kernel on a 128 x 128 x 64
+ * tile held in the workspace, with its copy-issuing warp switched off and every wait bounded by wait_ms
+ * (1..2000 ms) instead of the default 2 s: the consumer's wait can never be satisfied, so it must expire, the
+ * block must record FMM_ERR_TIMEOUT in the status word, release its resources and return normally.  The call only
+ * enqueues; fmm_device_status(d_ws, stream) then reports FMM_ERR_TIMEOUT and the context stays usable.
+ * d_ws: DEVICE, >= 128 KiB, 256-byte aligned.  Nothing in this test faults, traps or spins without bound.      */
+fmm_status fmm_selftest_timeout(void* d_ws, size_t ws_bytes, unsigned wait_ms, void* cuda_stream);
+
 size_t classical_gemm_workspace(const fmm_gemm_desc* d);
 
 /* The classical product at the same dtypes (the paper's control, Section 3.1):

@@ -7,6 +7,6 @@ every step of the path runs in the library's CUDA kernels).  There is no CPU fal
 from .binding import (  # noqa: F401
     FmmError, Scheme, GemmDesc, SweepSummary, scheme_load, scheme_builtin, scheme_kron, gauge_apply,
     scheme_gemm, scheme_gemm_workspace, scheme_gemm_workspace_layout, classical_gemm, classical_gemm_workspace, exact_gemm_f64,
-    error_frobenius, error_frobenius_noalloc, error_frobenius_noalloc_max_elements, error_sweep, error_sweep_workspace, device_status, launch_count, lib_path,
+    error_frobenius, error_frobenius_noalloc, error_frobenius_noalloc_max_elements, error_sweep, error_sweep_workspace, device_status, selftest_timeout, launch_count, lib_path,
     F32, BF16, E4M3, FLAG_REUSE_BHAT, EXPORTED_SYMBOLS, profile_enable, profile_collect, PHASES,
 )

@@ -19,7 +19,8 @@ _DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
 
 EXPORTED_SYMBOLS = [
     "scheme_load", "scheme_builtin", "scheme_kron", "gauge_apply", "scheme_info", "scheme_coefficients",
-    "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status", "classical_gemm_workspace",
+    "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status",
+    "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
@@ -81,6 +82,7 @@ _lib.scheme_gemm_workspace.restype = _sz
 _lib.scheme_gemm_workspace_layout.argtypes = [_vp, C.POINTER(GemmDesc), C.POINTER(_sz)]
 _lib.scheme_gemm.argtypes = [_vp, C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.fmm_device_status.argtypes = [_vp, _vp]
+_lib.fmm_selftest_timeout.argtypes = [_vp, _sz, C.c_uint, _vp]
 _lib.classical_gemm_workspace.argtypes = [C.POINTER(GemmDesc)]
 _lib.classical_gemm_workspace.restype = _sz
 _lib.classical_gemm.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
@@ -257,6 +259,13 @@ def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=
 
 def device_status(ws) -> None:
     _check(_lib.fmm_device_status(_ptr(ws), _stream()), "fmm_device_status")
+
+
+def selftest_timeout(ws, wait_ms: int = 50) -> None:
+    """Enqueue the failure-reporting self-test (one block whose wait must expire); follow with device_status(ws),
+    which then raises FmmError with code 8 (FMM_ERR_TIMEOUT)."""
+    _check(_lib.fmm_selftest_timeout(_ptr(ws), ws.numel() * ws.element_size(), wait_ms, _stream()),
+           "fmm_selftest_timeout")
 
 
 def launch_count() -> int:

@@ -429,6 +429,25 @@ fmm_status exact_gemm_f64(const fmm_gemm_desc* d, const void* dA, const void* dB
   return FMM_OK;
 }
 
+fmm_status fmm_selftest_timeout(void* d_ws, size_t ws_bytes, unsigned wait_ms, void* cuda_stream) {
+  // one 128 x 128 x 64 bf16 tile, one block; operands and output live in the workspace
+  const size_t need = 1024 + 2 * (128 * 64 * 2) + 128 * 128 * 4;
+  FMM_TRY(check_ws(d_ws, ws_bytes, need));
+  if (wait_ms == 0 || wait_ms > 2000) return FMM_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  FMM_CUDA(cudaMemsetAsync(d_ws, 0, need, st));
+  BlockProductArgs g{};
+  g.product = FMM_BF16;
+  g.A = at<char>(d_ws, 1024); g.lda = 64; g.a_batch = 0;
+  g.B = at<char>(d_ws, 1024 + 128 * 64 * 2); g.ldb = 64; g.b_batch = 0;
+  g.rows_a = 128; g.rows_b = 128; g.kdim = 64; g.batches = 1;
+  g.out = at<char>(d_ws, 1024 + 2 * 128 * 64 * 2); g.ldo = 128; g.o_batch = 0; g.out_mode = 0; g.output = FMM_F32;
+  g.status = at<DeviceStatus>(d_ws, 0);
+  g.selftest_no_producer = 1;
+  g.wait_limit_ns = (unsigned long long)wait_ms * 1000000ull;
+  return launch_block_products(g, st);
+}
+
 size_t error_frobenius_workspace(void) { return align_up((size_t)kMaxStreamPartials * 8 * 2); }
 
 fmm_status error_frobenius(const fmm_gemm_desc* d, const void* dC, const double* dCstar, double* d_out, void* d_ws,

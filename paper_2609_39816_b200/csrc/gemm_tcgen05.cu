@@ -29,7 +29,7 @@ constexpr int BM = 128;             // rows of A per tile = UMMA M
 constexpr int BKB = 128;            // bytes of the inner dimension per ring stage (one swizzle span)
 constexpr int UMMA_KB = 32;         // bytes of the inner dimension per tcgen05.mma
 constexpr int kNumThreads = 192;    // 6 warps
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // 2 s
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -62,14 +62,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where,
-                                          DeviceStatus* status) {
+                                          DeviceStatus* status, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         if (status != nullptr) {
           atomicExch(&status->code, (int)FMM_ERR_TIMEOUT);
@@ -225,6 +225,8 @@ struct TileParams {
   int out_mode;             // 0: fp32 products; 1: scaled + rounded result
   int out_bf16;             // out_mode 1: 1 -> bf16, 0 -> fp32
   int wide;                 // every output row starts on a 32-byte boundary
+  int selftest_no_producer; // failure-reporting self-test: the TMA producer issues nothing
+  unsigned long long wait_limit_ns;   // bound of every mbarrier wait
 };
 
 template <int BN, bool kFp8>
@@ -278,7 +280,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && !tp.selftest_no_producer) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -287,7 +289,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const int rem = tile - r * tiles_per_batch;
         const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status);
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status, tp.wait_limit_ns);
           if (!ok) break;
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
@@ -319,12 +321,12 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status);
+        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status, tp.wait_limit_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status);
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status, tp.wait_limit_ns);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
@@ -363,7 +365,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       const int r = tile / tiles_per_batch;
       const int rem = tile - r * tiles_per_batch;
       const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
-      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status);
+      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status, tp.wait_limit_ns);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -524,7 +526,7 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         const int rem = tile - r * tiles_per_batch;
         const int tm = rem / tiles_n, tn = rem - tm * tiles_n;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status);
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status, tp.wait_limit_ns);
           if (!ok) break;
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
@@ -549,12 +551,12 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
-        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status);
+        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status, tp.wait_limit_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status);
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status, tp.wait_limit_ns);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
@@ -592,7 +594,7 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       const int r = tile / tiles_per_batch;
       const int rem = tile - r * tiles_per_batch;
       const int tm = rem / tiles_n, tn = rem - tm * tiles_n;
-      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status);
+      ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status, tp.wait_limit_ns);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -691,6 +693,8 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
   tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
   tp.wide = rows_32b_aligned(a);
+  tp.selftest_no_producer = a.selftest_no_producer;
+  tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
   const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
   if (total <= 0) return FMM_OK;
   const int sms = sm_count();
@@ -719,6 +723,8 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
   tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
   tp.wide = rows_32b_aligned(a);
+  tp.selftest_no_producer = a.selftest_no_producer;
+  tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
   const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
   if (total <= 0) return FMM_OK;
   const int sms = sm_count();
@@ -751,7 +757,7 @@ fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
   const bool fp8 = (a.product == FMM_E4M3);
   if (!fp8 && a.product != FMM_BF16) return FMM_ERR_DTYPE;
   // large problems: CTA pairs on 256 x 256 tiles (less L2 traffic per flop)
-  if (a.rows_a > 128 && a.rows_b > 128 && pair_kernel_enabled())
+  if (a.rows_a > 128 && a.rows_b > 128 && pair_kernel_enabled() && !a.selftest_no_producer)
     return fp8 ? launch_pair<true>(a, st) : launch_pair<false>(a, st);
   // narrow problems use the 128-column tile (less padding, more tiles in flight)
   const bool narrow = a.rows_b <= 128;

@@ -67,6 +67,8 @@ struct BlockProductArgs {
   void* out; int64_t ldo; int64_t o_batch; int out_mode; int output;
   const float* sA; const float* sB;
   DeviceStatus* status;
+  int selftest_no_producer;            // 1: the producer issues no copies (failure-reporting self-test)
+  unsigned long long wait_limit_ns;    // 0: default (2 s)
 };
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
 

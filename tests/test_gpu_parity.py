@@ -274,3 +274,18 @@ def test_config2_full_size_sampled_outputs(lib):
     # and the whole result is close to the exact product at the level the rounding allows
     Cs = gu.run_exact(At, Bt, "bf16").cpu().numpy()
     assert gu.rel_fro(C, Cs) < 0.05
+
+
+# ---------------------------------------------------------------------------- failure reporting
+def test_bounded_wait_expires_reports_timeout_and_context_survives(lib):
+    """A wait that nothing will ever satisfy (the copy-issuing warp of one block is switched off) must run out,
+    leave FMM_ERR_TIMEOUT in the status word and return; the next ordinary call must work."""
+    ws = gu.workspace(256 * 1024)
+    lib.selftest_timeout(ws, wait_ms=50)
+    with pytest.raises(lib.FmmError) as err:
+        lib.device_status(ws)
+    assert err.value.code == 8
+    torch.cuda.synchronize()
+    At, Bt, A64, B64 = _inputs(13, 256, 256, 256, "bf16", "int", 3)
+    C = gu.run_scheme_gemm(lib.scheme_builtin("strassen222"), At, Bt, "bf16", "bf16", "f32")
+    assert np.array_equal(C, A64 @ B64)
