@@ -30,6 +30,10 @@
  * Pins (see tests): printed Strassen example values, Brent equations on integer
  * matrices, identity/sign gauges, printed constants (L_A=L_B=4, L_W=16, Phi=1024,
  * nnz=432), the same-offset row leak pattern, brute-force triple loops.
+ * The certified int8 realisation (Section 4.2, Proposition 1, Appendix D) is pinned by
+ * the printed constants (b = 31, L_A b = 124, inner length 8729), bit-identity with the
+ * classical int8 operator over all 512 sign variants, brute-force integer products on
+ * 200 random tiles, and the 0-of-496 row-pair count.
  * Parity unpinned: the error-amplification ratios at the benchmark workloads (the
  * paper prints none for synthetic inputs of these shapes).
  *
@@ -428,4 +432,148 @@ void orc_fro_err(const double* C, const double* Cs, int64_t n, double* out) {
   double e = 0.0, s = 0.0;
   for (int64_t i = 0; i < n; ++i) { double d = C[i] - Cs[i]; e += d * d; s += Cs[i] * Cs[i]; }
   out[0] = e; out[1] = s;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Certified realisation on bounded integer codes (Section 4.2, Proposition 1; */
+/* quantisation specification of Appendix D).                                  */
+/* ------------------------------------------------------------------------- */
+
+/* Quantiser.  X is rows x K (fp32 values held in doubles), groups of g consecutive entries along
+ * the inner dimension share a scale per row: d = max|x| / b computed in fp32 (d = 1 for an all-zero
+ * group), codes = x / d in fp32, rounded to nearest with ties to even, no clipping.  K % g == 0 (the
+ * caller pads with zeros).  codes: rows x K integers as doubles; scales: rows x (K/g) fp32 values.   */
+void orc_quantize_rows(const double* X, int64_t rows, int64_t K, int g, int b, double* codes, double* scales) {
+  const int64_t G = K / g;
+  for (int64_t t = 0; t < rows; ++t)
+    for (int64_t q = 0; q < G; ++q) {
+      float amax = 0.0f;
+      for (int x = 0; x < g; ++x) { float a = fabsf((float)X[t * K + q * g + x]); if (a > amax) amax = a; }
+      float d = amax == 0.0f ? 1.0f : amax / (float)b;
+      scales[t * G + q] = (double)d;
+      for (int x = 0; x < g; ++x) codes[t * K + q * g + x] = (double)rintf((float)X[t * K + q * g + x] / d);
+    }
+}
+
+/* Rescale and accumulate as the specification fixes it: for each group in ascending order the exact
+ * integer P is converted to fp32, multiplied by d_A, then by d_B (two separate fp32 multiplications) and
+ * added to a zero-initialised fp32 output; after the last group the output is cast to `od`.
+ * P is [G][M][N] integers (as doubles), dA [M][G], dB [N][G].                                        */
+static void int8_rescale(const double* P, const double* dA, const double* dB, int64_t M, int64_t N, int64_t G,
+                         int od, double* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < M; ++t)
+    for (int64_t j = 0; j < N; ++j) {
+      float acc = 0.0f;
+      for (int64_t q = 0; q < G; ++q) {
+        float p = (float)P[(q * M + t) * N + j];
+        float x = p * (float)dA[t * G + q];
+        x = x * (float)dB[j * G + q];
+        acc = acc + x;
+      }
+      out[t * N + j] = orc_round((double)acc, od);
+    }
+}
+
+/* Classical int8 operator at the specification: exact integer product of the codes of each group.
+ * cA [M][K], cB [N][K] (weight layout: one row per output column).  Also returns the group products
+ * Pout [G][M][N] if not NULL.                                                                       */
+void orc_int8_classical(const double* cA, const double* dA, const double* cB, const double* dB, int64_t M,
+                        int64_t K, int64_t N, int g, int od, double* out, double* Pout) {
+  const int64_t G = K / g;
+  double* P = Pout ? Pout : (double*)malloc(sizeof(double) * G * M * N);
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < M; ++t)
+    for (int64_t j = 0; j < N; ++j)
+      for (int64_t q = 0; q < G; ++q) {
+        int64_t s = 0;
+        for (int x = 0; x < g; ++x) s += (int64_t)cA[t * K + q * g + x] * (int64_t)cB[j * K + q * g + x];
+        P[(q * M + t) * N + j] = (double)s;
+      }
+  int8_rescale(P, dA, dB, M, N, G, od, out);
+  if (!Pout) free(P);
+}
+
+/* The same operator with every group's integer product computed by an algorithm <m,k,n;R> with integer
+ * coefficients, one call per group: rows split into m contiguous blocks, columns into n, the group's g
+ * inner indices into k blocks of length h = g/k (condition (iii): a call lies within one group).
+ * All arithmetic in 64-bit integers, so the result is what an overflow-free machine computes; `maxabs`
+ * reports what Proposition 1 bounds: maxabs[0] = largest |block sum of A codes|, [1] = of B codes (must be
+ * <= 127 for int8 multipliers, condition (i)), [2] = largest |product or partial sum| formed in the calls
+ * (must be < 2^31 for int32, < 2^24 for fp32, condition (ii)).  Returns 1 if a dimension does not divide
+ * or a coefficient is not an integer.                                                                  */
+int orc_int8_certified(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                       const double* cA, const double* dA, const double* cB, const double* dB, int64_t M,
+                       int64_t K, int64_t N, int g, int od, double* out, double* Pout, double* maxabs) {
+  if (M % m || N % n || g % k || K % g) return 1;
+  for (int x = 0; x < R * m * k; ++x) if (U[x] != rint(U[x])) return 1;
+  for (int x = 0; x < R * k * n; ++x) if (V[x] != rint(V[x])) return 1;
+  for (int x = 0; x < R * m * n; ++x) if (W[x] != rint(W[x])) return 1;
+  const int64_t G = K / g, bm = M / m, bn = N / n;
+  const int h = g / k;
+  double* P = Pout ? Pout : (double*)malloc(sizeof(double) * G * M * N);
+  int64_t* Ah = (int64_t*)malloc(sizeof(int64_t) * bm * h);
+  int64_t* Bh = (int64_t*)malloc(sizeof(int64_t) * bn * h);
+  int64_t* acc = (int64_t*)malloc(sizeof(int64_t) * M * N);
+  int64_t mxA = 0, mxB = 0, mxP = 0;
+  for (int64_t q = 0; q < G; ++q) {
+    for (int64_t x = 0; x < M * N; ++x) acc[x] = 0;
+    for (int r = 0; r < R; ++r) {
+      for (int64_t p = 0; p < bm; ++p)
+        for (int t = 0; t < h; ++t) {
+          int64_t s = 0;
+          for (int i = 0; i < m; ++i)
+            for (int l = 0; l < k; ++l)
+              s += (int64_t)U[(r * m + i) * k + l] * (int64_t)cA[(i * bm + p) * K + q * g + l * h + t];
+          Ah[p * h + t] = s;
+          if (llabs(s) > mxA) mxA = llabs(s);
+        }
+      for (int64_t c = 0; c < bn; ++c)
+        for (int t = 0; t < h; ++t) {
+          int64_t s = 0;
+          for (int l = 0; l < k; ++l)
+            for (int j = 0; j < n; ++j)
+              s += (int64_t)V[(r * k + l) * n + j] * (int64_t)cB[(j * bn + c) * K + q * g + l * h + t];
+          Bh[c * h + t] = s;
+          if (llabs(s) > mxB) mxB = llabs(s);
+        }
+      for (int64_t p = 0; p < bm; ++p)
+        for (int64_t c = 0; c < bn; ++c) {
+          int64_t s = 0;
+          for (int t = 0; t < h; ++t) {
+            s += Ah[p * h + t] * Bh[c * h + t];
+            if (llabs(s) > mxP) mxP = llabs(s);
+          }
+          for (int i = 0; i < m; ++i)
+            for (int j = 0; j < n; ++j) {
+              int64_t w = (int64_t)W[(r * m + i) * n + j];
+              if (w == 0) continue;
+              int64_t* dst = &acc[(i * bm + p) * N + j * bn + c];
+              *dst += w * s;
+              if (llabs(*dst) > mxP) mxP = llabs(*dst);
+            }
+        }
+    }
+    for (int64_t x = 0; x < M * N; ++x) P[q * M * N + x] = (double)acc[x];
+  }
+  int8_rescale(P, dA, dB, M, N, G, od, out);
+  if (maxabs) { maxabs[0] = (double)mxA; maxabs[1] = (double)mxB; maxabs[2] = (double)mxP; }
+  free(Ah); free(Bh); free(acc);
+  if (!Pout) free(P);
+  return 0;
+}
+
+/* Proposition 1, checked from the coefficients, the tiling and the specification alone:
+ * cert[0] = L_A b_A, cert[1] = L_B b_B (condition (i): both <= 127), cert[2] = max{L_W h (L_A b_A)(L_B b_B),
+ * g b_A b_B} (condition (ii): < 2^acc_bits), cert[3] = 1 if a call (k blocks of length h) spans exactly one
+ * group (condition (iii)).  Returns 1 if all three hold.                                               */
+int orc_certificate(int m, int k, int n, int R, const double* U, const double* V, const double* W, int bA, int bB,
+                    int h, int g, int acc_bits, double* cert) {
+  double meta[8];
+  orc_criteria(m, k, n, R, U, V, W, meta);
+  const double a = meta[0] * bA, b = meta[1] * bB;
+  const double big = fmax(meta[2] * h * a * b, (double)g * bA * bB);
+  const int one_group = (k * h == g);
+  if (cert) { cert[0] = a; cert[1] = b; cert[2] = big; cert[3] = one_group; }
+  return a <= 127.0 && b <= 127.0 && big < ldexp(1.0, acc_bits) && one_group;
 }

@@ -28,7 +28,7 @@ __all__ = [
     "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "round_to", "strassen",
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
-    "error_ratio", "summary",
+    "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "certificate",
 ]
 
 
@@ -67,6 +67,12 @@ def _L():
         lib.orc_classical_gemm.argtypes = [i64] * 3 + [dp] * 2 + [C.c_int] * 3 + [dp]
         lib.orc_exact_gemm.argtypes = [i64] * 3 + [dp] * 3
         lib.orc_fro_err.argtypes = [dp, dp, i64, dp]
+        lib.orc_quantize_rows.argtypes = [dp, i64, i64, C.c_int, C.c_int, dp, dp]
+        lib.orc_int8_classical.argtypes = [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 2
+        lib.orc_int8_certified.restype = C.c_int
+        lib.orc_int8_certified.argtypes = ([C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 3)
+        lib.orc_certificate.restype = C.c_int
+        lib.orc_certificate.argtypes = [C.c_int] * 4 + [dp] * 3 + [C.c_int] * 5 + [dp]
         _lib = lib
     return _lib
 
@@ -280,3 +286,51 @@ def summary(ratios) -> dict:
     return dict(min=float(r[0]), median=float(r[G // 2]), max=float(r[-1]),
                 spread=float(r[-1] / r[0]) if r[0] > 0 else math.inf,
                 count_gt2=int(np.sum(r > 2.0)), G=int(G))
+
+
+# ---------------------------------------------------------------- certified int8 realisation (Section 4.2)
+def quantize_rows(X, b: int, g: int = 128):
+    """Appendix D quantiser: per row and per group of g inner indices, d = max|x|/b in fp32 (1 if all zero),
+    codes = x/d rounded to nearest even, no clipping.  Returns (codes, scales[rows, K/g])."""
+    X = _d(X)
+    rows, K = X.shape
+    assert K % g == 0
+    codes = np.empty((rows, K)); scales = np.empty((rows, K // g))
+    _L().orc_quantize_rows(_p(X), rows, K, g, b, _p(codes), _p(scales))
+    return codes, scales
+
+
+def int8_classical(cA, dA, cB, dB, g: int = 128, od="bf16", products: bool = False):
+    """Classical int8 operator: exact group products, (P*dA)*dB in fp32, ascending groups, one cast to `od`.
+    cA [M,K], cB [N,K] (one row per output column)."""
+    cA = _d(cA); cB = _d(cB); dA = _d(dA); dB = _d(dB)
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = np.empty((M, N))
+    P = np.empty((K // g, M, N)) if products else None
+    _L().orc_int8_classical(_p(cA), _p(dA), _p(cB), _p(dB), M, K, N, g, _fmt(od), _p(out), _p(P))
+    return (out, P) if products else out
+
+
+def int8_certified(s: "Scheme", cA, dA, cB, dB, g: int = 128, od="bf16", products: bool = False):
+    """The same operator with each group's integer product computed by the algorithm `s` (one call per group).
+    Returns (out, maxabs[3]) or (out, maxabs, P)."""
+    m, k, n, R = s.dims
+    cA = _d(cA); cB = _d(cB); dA = _d(dA); dB = _d(dB)
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = np.empty((M, N)); mx = np.zeros(3)
+    P = np.empty((K // g, M, N)) if products else None
+    rc = _L().orc_int8_certified(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), _p(cA), _p(dA), _p(cB), _p(dB),
+                                 M, K, N, g, _fmt(od), _p(out), _p(P), _p(mx))
+    if rc:
+        raise ValueError("shape does not divide, or coefficients are not integers")
+    return (out, mx, P) if products else (out, mx)
+
+
+def certificate(s: "Scheme", bA: int, bB: int, h: int, g: int, acc_bits: int = 31):
+    """Proposition 1 from coefficients, tiling and specification.  Returns (holds, dict)."""
+    m, k, n, R = s.dims
+    c = np.zeros(4)
+    ok = _L().orc_certificate(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), bA, bB, h, g, acc_bits, _p(c))
+    return bool(ok), dict(LAbA=c[0], LBbB=c[1], largest=c[2], one_group=bool(c[3]))

@@ -1,0 +1,104 @@
+"""Pins of the oracle's certified int8 realisation (Section 4.2, Proposition 1, Appendix D) — no GPU."""
+import numpy as np
+import pytest
+
+import oracle
+from fmm_inputs import generators as gen
+
+S1 = oracle.strassen()
+S2 = oracle.kron(S1, S1)
+
+
+def _quantised(seed, M, K, N, b):
+    A = gen.to_storage(gen.normal(seed, 1, (M, K)), "f32")[1]
+    Bt = gen.to_storage(gen.normal(seed, 2, (N, K)) * 0.02, "f32")[1]
+    cA, dA = oracle.quantize_rows(A, b)
+    cB, dB = oracle.quantize_rows(Bt, b)
+    return A, Bt, cA, dA, cB, dB
+
+
+def test_quantiser_rules():
+    X = np.zeros((2, 256))
+    X[0, :128] = np.linspace(-3.0, 3.0, 128)
+    X[1, 128:] = 1e-3 * np.arange(128)
+    c, d = oracle.quantize_rows(X, 31)
+    assert d.shape == (2, 2) and d[0, 1] == 1.0 and d[1, 0] == 1.0          # all-zero group: d = 1
+    assert np.float32(d[0, 0]) == np.float32(3.0) / np.float32(31)          # d = max|x| / b in fp32
+    assert np.abs(c).max() == 31 and np.all(c == np.rint(c))                # no clipping needed: |code| <= b
+    assert c[0, 0] == -31 and c[0, 127] == 31 and np.all(c[0, 128:] == 0)
+    # ties to even: x/d = 0.5 -> 0, 1.5 -> 2, 2.5 -> 2   (d = 1 when max|x| = b)
+    Y = np.zeros((1, 128)); Y[0, :4] = [31.0, 0.5, 1.5, 2.5]
+    c2, d2 = oracle.quantize_rows(Y, 31)
+    assert d2[0, 0] == 1.0 and c2[0, :4].tolist() == [31.0, 0.0, 2.0, 2.0]
+
+
+def test_certificate_constants_of_two_level_strassen():
+    """Section 4.2: L_A = L_B = 4 admit b = 31; with L_W = 16, g = 128 and h = 32 the certificate holds for
+    int32 and for exact integers in fp32; inner length 8729 is the int32 limit; b = 32 breaks condition (i);
+    a call spanning more than one group breaks condition (iii)."""
+    ok, c = oracle.certificate(S2, 31, 31, 32, 128, 31)
+    assert ok and c["LAbA"] == 124 and c["LBbB"] == 124 and c["largest"] == 16 * 32 * 124 * 124
+    assert oracle.certificate(S2, 31, 31, 32, 128, 24)[0]                    # 7.87e6 < 2^24: fp32 emulation is exact
+    assert not oracle.certificate(S2, 32, 31, 32, 128, 31)[0]                # 4 * 32 = 128 > 127
+    assert oracle.certificate(S2, 31, 31, 8729, 4 * 8729, 31)[0]
+    assert not oracle.certificate(S2, 31, 31, 8730, 4 * 8730, 31)[0]
+    assert not oracle.certificate(S2, 31, 31, 64, 128, 31)[0]                # call of 256 over groups of 128
+    ok1, c1 = oracle.certificate(S1, 63, 63, 64, 128, 31)                    # one level: L = 2 admits b = 63
+    assert ok1 and c1["LAbA"] == 126
+
+
+def test_certified_equals_classical_bit_for_bit_all_sign_variants():
+    """All 512 sign variants compute one integer product and one output, the classical int8 operator's."""
+    A, Bt, cA, dA, cB, dB = _quantised(3, 32, 256, 16, 31)
+    ref, Pref = oracle.int8_classical(cA, dA, cB, dB, products=True)
+    outs, prods = set(), set()
+    for d, e, f in oracle.sign_variants(4, 4, 4):
+        out, mx, P = oracle.int8_certified(oracle.sign_variant(S2, d, e, f), cA, dA, cB, dB, products=True)
+        outs.add(out.tobytes()); prods.add(P.tobytes())
+        assert mx[0] <= 124 and mx[1] <= 124 and mx[2] <= 16 * 32 * 124 * 124
+    assert outs == {ref.tobytes()} and prods == {Pref.tobytes()}
+    # the operator is close to the fp64 product at the accuracy 31 codes allow
+    assert oracle.rel_error(ref, A @ Bt.T) < 0.05
+
+
+def test_200_random_tiles_exact():
+    for trial in range(200):
+        cA = gen.integer_matrix(100 + trial, 1, (8, 128), 31)
+        cB = gen.integer_matrix(100 + trial, 2, (8, 128), 31)
+        one = np.ones((8, 1))
+        _, mx, P = oracle.int8_certified(S2, cA, one, cB, one, products=True, od="f32")
+        assert np.array_equal(P[0], cA @ cB.T)
+
+
+def test_row_locality_zero_of_496_pairs_move():
+    """Section 4.2: 32 token rows in four blocks, one row changed at a time: no earlier output row moves."""
+    A, Bt, cA, dA, cB, dB = _quantised(5, 32, 128, 32, 31)
+    base, _ = oracle.int8_certified(S2, cA, dA, cB, dB)
+    moved = pairs = 0
+    for later in range(32):
+        A2 = A.copy()
+        A2[later] = gen.to_storage(gen.normal(5, 300 + later, (128,)), "f32")[1]
+        c2, d2 = oracle.quantize_rows(A2, 31)
+        out, _ = oracle.int8_certified(S2, c2, d2, cB, dB)
+        for earlier in range(later):
+            pairs += 1
+            moved += int(np.any(out[earlier] != base[earlier]))
+        assert np.any(out[later] != base[later])
+    assert pairs == 496 and moved == 0
+
+
+def test_bound_is_sharp_and_violations_are_reported():
+    """Codes whose signs follow the coefficients reach L_A * b (Appendix D: the bound is sharp); at b = 32 a
+    block sum leaves the int8 range."""
+    for b, limit in ((31, 124), (32, 128)):
+        cA = np.zeros((4, 128)); cB = gen.integer_matrix(9, 2, (4, 128), b)
+        r = int(np.argmax(np.abs(S2.U).sum(axis=(1, 2))))                  # a product with four nonzero u
+        for i in range(4):
+            for l in range(4):
+                cA[i, 32 * l:32 * l + 32] = b * np.sign(S2.U[r, i, l])
+        one = np.ones((4, 1))
+        _, mx = oracle.int8_certified(S2, cA, one, cB, one, od="f32")
+        assert mx[0] == limit
+    with pytest.raises(ValueError):
+        P = gen.gauge_cond_limited(1, 0, 2)
+        oracle.int8_certified(oracle.gauge(S1, P, P, P), cA[:2], one[:2], cB[:2], one[:2])
