@@ -55,7 +55,8 @@ typedef enum {
   FMM_ERR_WORKSPACE = 6, /* workspace null, misaligned or too small */
   FMM_ERR_CUDA = 7,      /* a CUDA runtime/driver call failed (incl. no device) */
   FMM_ERR_TIMEOUT = 8,   /* a bounded device-side wait expired; results are invalid */
-  FMM_ERR_LIMIT = 9      /* scheme larger than the library's table limits */
+  FMM_ERR_LIMIT = 9,     /* scheme larger than the library's table limits */
+  FMM_ERR_CERTIFICATE = 10 /* Proposition 1 does not hold for this algorithm, code bound and tiling */
 } fmm_status;
 
 typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
@@ -232,6 +233,46 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
                        const double* S, const fmm_gemm_desc* d, const void* dA, const void* dB,
                        const double* dCstar, double* h_ratios, fmm_sweep_summary* out, void* d_ws,
                        size_t ws_bytes, void* cuda_stream);
+
+/* ---- Certified realisation on bounded integer codes (Section 4.2, Proposition 1; Appendix D) ------------
+ *
+ * The int8 operator of the quantisation specification: inputs in fp32 (or bf16), one fp32 scale per row and
+ * per group of 128 consecutive inner indices, d = max|x| / b (d = 1 for an all-zero group), codes = x / d
+ * rounded to nearest even, no clipping; per group in ascending order the exact integer product P of the codes is
+ * converted to fp32, multiplied by the row's scale, then by the column's scale (two fp32 multiplications) and
+ * added to a zero-initialised fp32 output, which is cast once to the output dtype.  K must be a multiple of
+ * 128 (the caller pads with zeros, as the specification says).                                              */
+
+/* Proposition 1 from the coefficients, the code bounds, the block inner length h, the group size g and the
+ * accumulator width alone.  cert[4] (HOST, may be NULL) = {L_A*bA, L_B*bB, max{L_W*h*(L_A*bA)*(L_B*bB),
+ * g*bA*bB}, 1 if a call (k blocks of length h) spans exactly one group}.  Returns 1 when the coefficients are
+ * integers, (i) both block-sum bounds are <= 127, (ii) the largest bound is < 2^acc_bits and (iii) holds;
+ * 0 otherwise.  s == NULL means the classical algorithm <1,1,1;1>.  Host only.                              */
+int scheme_certificate(const fmm_scheme* s, int bA, int bB, int h, int g, int acc_bits, double cert[4]);
+
+/* Quantiser.  d_X: DEVICE, rows x K of `storage` (FMM_F32 or FMM_BF16), leading dimension ldx (elements,
+ * multiple of 4, pointer aligned to 4 elements).  d_codes: DEVICE int8 [rows][K]; d_scales: DEVICE fp32
+ * [rows][K/128].  For B pass the weight layout [N][K] (one row per output column).  1 <= code_bound <= 127.
+ * Asynchronous on the stream.                                                                                */
+fmm_status int8_quantize(const void* d_X, int storage, int64_t rows, int64_t K, int64_t ldx, int code_bound,
+                         int8_t* d_codes, float* d_scales, void* cuda_stream);
+
+size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N);
+
+/* The int8 operator on quantised operands: d_cA int8 [M][K] with scales d_dA [M][K/128], d_cB int8 [N][K]
+ * with d_dB [N][K/128] (all DEVICE, code pointers 8-byte aligned); d_C: DEVICE [M][ldc] of `output` (FMM_F32
+ * or FMM_BF16, 16-byte aligned rows).  s == NULL computes every group's integer product classically; otherwise
+ * each group's product is computed by one call of s on the group's 128 inner indices split into k blocks of
+ * length 128/k (which must be 32, 64 or 128), rows into m and columns into n contiguous blocks.  Codes, block
+ * sums and all partial sums are integers held exactly (bf16 operands <= 127, fp32 accumulators < 2^24), so
+ * when the certificate holds the output is bit-identical to the classical operator's for every such s.
+ * Returns FMM_ERR_CERTIFICATE, launching nothing, if scheme_certificate(s, code_bound, code_bound, 128/k, 128,
+ * 24) fails; the caller vouches that |code| <= code_bound.  Requires M % m == 0, N % n == 0, (N/n) % 8 == 0,
+ * K % 128 == 0.  d_ws: DEVICE, >= int8_gemm_workspace bytes, 256-byte aligned; it holds a status word that
+ * fmm_device_status reads.  Asynchronous on the stream.                                                      */
+fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, const float* d_dA,
+                     const int8_t* d_cB, const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C,
+                     int64_t ldc, void* d_ws, size_t ws_bytes, void* cuda_stream);
 
 const char* fmm_status_string(fmm_status st);
 

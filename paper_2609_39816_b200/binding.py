@@ -22,7 +22,7 @@ EXPORTED_SYMBOLS = [
     "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status",
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
-    "error_frobenius_noalloc_max_elements",
+    "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
 ]
@@ -92,6 +92,13 @@ _lib.error_frobenius_workspace.restype = _sz
 _lib.error_frobenius.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
 _lib.error_frobenius_noalloc.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp]
 _lib.error_frobenius_noalloc_max_elements.restype = C.c_int64
+_lib.scheme_certificate.argtypes = [_vp] + [C.c_int] * 5 + [_dp]
+_lib.scheme_certificate.restype = C.c_int
+_lib.int8_quantize.argtypes = [_vp, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, _vp]
+_lib.int8_gemm_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
+_lib.int8_gemm_workspace.restype = _sz
+_lib.int8_gemm.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
+                           _vp, _sz, _vp]
 _lib.error_sweep_workspace.argtypes = [_vp, C.POINTER(GemmDesc), C.c_int]
 _lib.error_sweep_workspace.restype = _sz
 _lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(GemmDesc), _vp, _vp, _vp, _dp,
@@ -243,6 +250,37 @@ def error_frobenius_noalloc(d: GemmDesc, Cmat, Cstar, out2) -> None:
 
 def error_frobenius_noalloc_max_elements() -> int:
     return int(_lib.error_frobenius_noalloc_max_elements())
+
+
+def scheme_certificate(s, bA: int, bB: int, h: int, g: int = 128, acc_bits: int = 31):
+    """Proposition 1 for scheme `s` (None: classical).  Returns (holds, dict of the bounded quantities)."""
+    c = np.zeros(4)
+    ok = _lib.scheme_certificate(s.handle if s is not None else None, bA, bB, h, g, acc_bits, c.ctypes.data_as(_dp))
+    return bool(ok), dict(LAbA=c[0], LBbB=c[1], largest=c[2], one_group=bool(c[3]))
+
+
+def int8_quantize(X, code_bound: int, codes, scales) -> None:
+    """X [rows, K] fp32/bf16 (K % 128 == 0) -> codes int8 [rows, K], scales fp32 [rows, K/128]."""
+    import torch
+    rows, K = X.shape
+    st = F32 if X.dtype == torch.float32 else BF16
+    _check(_lib.int8_quantize(_ptr(X), st, rows, K, X.stride(0), code_bound, _ptr(codes), _ptr(scales), _stream()),
+           "int8_quantize")
+
+
+def int8_gemm_workspace(s, M: int, K: int, N: int) -> int:
+    return int(_lib.int8_gemm_workspace(s.handle if s is not None else None, M, K, N))
+
+
+def int8_gemm(s, code_bound: int, cA, dA, cB, dB, Cmat, ws) -> None:
+    """The group-scaled int8 operator; s None -> classical integer products, else one call of s per group."""
+    import torch
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = F32 if Cmat.dtype == torch.float32 else BF16
+    _check(_lib.int8_gemm(s.handle if s is not None else None, code_bound, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB), M, K, N,
+                          out, _ptr(Cmat), Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "int8_gemm")
 
 
 def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=None):

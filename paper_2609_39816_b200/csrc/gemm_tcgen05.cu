@@ -220,6 +220,7 @@ struct TileParams {
   int kbytes;               // inner extent in bytes
   int elem_bytes;           // 2 (bf16) or 1 (e4m3)
   int batches;
+  int groups;               // row groups per batch entry: product (r, g) pairs rows [g*rows_a, +rows_a) with [g*rows_b, +rows_b)
   int tiles_m, tiles_n;
   long long ldo, o_batch;   // output strides in elements
   int out_mode;             // 0: fp32 products; 1: scaled + rounded result
@@ -275,7 +276,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
   const int num_kb = (tp.kbytes + BKB - 1) / BKB;
   const int tiles_per_batch = tp.tiles_m * tp.tiles_n;
-  const int total_tiles = tiles_per_batch * tp.batches;
+  const int total_tiles = tiles_per_batch * tp.batches * tp.groups;
   const int kelems_per_stage = BKB / tp.elem_bytes;
 
   if (warp == 0) {
@@ -285,8 +286,9 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int r = tile / tiles_per_batch;
-        const int rem = tile - r * tiles_per_batch;
+        const int bb = tile / tiles_per_batch;
+        const int rem = tile - bb * tiles_per_batch;
+        const int r = bb / tp.groups, g = bb - r * tp.groups;
         const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status, tp.wait_limit_ns);
@@ -294,8 +296,8 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint32_t sb = sa + L::kABytes;
           mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::kStageBytes);
-          tma_load_3d(sa, &map_a, full_bar(stage), kb * kelems_per_stage, tm * BM, r);
-          tma_load_3d(sb, &map_b, full_bar(stage), kb * kelems_per_stage, tn * BN, r);
+          tma_load_3d(sa, &map_a, full_bar(stage), kb * kelems_per_stage, g * tp.rows_a + tm * BM, r);
+          tma_load_3d(sb, &map_b, full_bar(stage), kb * kelems_per_stage, g * tp.rows_b + tn * BN, r);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -362,7 +364,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     float alpha = 1.0f;
     if (tp.out_mode == 1 && sA != nullptr && sB != nullptr) alpha = sA[0] * sB[0];
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int r = tile / tiles_per_batch;
+      const int r = tile / tiles_per_batch;     // index of the (batch, group) product
       const int rem = tile - r * tiles_per_batch;
       const int tm = rem / tp.tiles_n, tn = rem - tm * tp.tiles_n;
       ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x23, status, tp.wait_limit_ns);
@@ -511,7 +513,7 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   const int tiles_m = (tp.rows_a + 2 * BM - 1) / (2 * BM);
   const int tiles_n = (tp.rows_b + BN - 1) / BN;
   const int tiles_per_batch = tiles_m * tiles_n;
-  const int total_tiles = tiles_per_batch * tp.batches;
+  const int total_tiles = tiles_per_batch * tp.batches * tp.groups;
   const int kelems_per_stage = BKB / tp.elem_bytes;
   const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
@@ -522,8 +524,9 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
-        const int r = tile / tiles_per_batch;
-        const int rem = tile - r * tiles_per_batch;
+        const int bb = tile / tiles_per_batch;
+        const int rem = tile - bb * tiles_per_batch;
+        const int r = bb / tp.groups, g = bb - r * tp.groups;
         const int tm = rem / tiles_n, tn = rem - tm * tiles_n;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x01, status, tp.wait_limit_ns);
@@ -532,8 +535,8 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
           const uint32_t sb = sa + L::kABytes;
           const uint32_t lead_full = full_bar(stage) & kPeerBitMask;
           if (leader) mbar_arrive_expect_tx(full_bar(stage), 2u * (uint32_t)L::kStageBytes);
-          tma_load_3d_pair(sa, &map_a, lead_full, kb * kelems_per_stage, tm * 2 * BM + (int)rank * BM, r);
-          tma_load_3d_pair(sb, &map_b, lead_full, kb * kelems_per_stage, tn * BN + (int)rank * (BN / 2), r);
+          tma_load_3d_pair(sa, &map_a, lead_full, kb * kelems_per_stage, g * tp.rows_a + tm * 2 * BM + (int)rank * BM, r);
+          tma_load_3d_pair(sb, &map_b, lead_full, kb * kelems_per_stage, g * tp.rows_b + tn * BN + (int)rank * (BN / 2), r);
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -681,13 +684,15 @@ template <int BN, bool kFp8>
 fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   using L = SmemLayout<BN>;
   CUtensorMap ma, mb;
-  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
-  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, BN)) return FMM_ERR_CUDA;
+  const int groups = a.groups > 1 ? a.groups : 1;
+  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a * groups, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b * groups, a.kdim, a.ldb, a.b_batch, a.batches, BN)) return FMM_ERR_CUDA;
   TileParams tp;
   tp.rows_a = (int)a.rows_a; tp.rows_b = (int)a.rows_b;
   tp.elem_bytes = kFp8 ? 1 : 2;
   tp.kbytes = (int)a.kdim * tp.elem_bytes;
   tp.batches = a.batches;
+  tp.groups = groups;
   tp.tiles_m = (int)((a.rows_a + BM - 1) / BM);
   tp.tiles_n = (int)((a.rows_b + BN - 1) / BN);
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
@@ -695,7 +700,7 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   tp.wide = rows_32b_aligned(a);
   tp.selftest_no_producer = a.selftest_no_producer;
   tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
-  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
+  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches * tp.groups;
   if (total <= 0) return FMM_OK;
   const int sms = sm_count();
   if (sms <= 0) return FMM_ERR_CUDA;
@@ -711,13 +716,15 @@ template <bool kFp8>
 fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   using L = PairLayout;
   CUtensorMap ma, mb;
-  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
-  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, L::BN / 2)) return FMM_ERR_CUDA;
+  const int groups = a.groups > 1 ? a.groups : 1;
+  if (!make_operand_map(&ma, kFp8, a.A, a.rows_a * groups, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, kFp8, a.B, a.rows_b * groups, a.kdim, a.ldb, a.b_batch, a.batches, L::BN / 2)) return FMM_ERR_CUDA;
   TileParams tp;
   tp.rows_a = (int)a.rows_a; tp.rows_b = (int)a.rows_b;
   tp.elem_bytes = kFp8 ? 1 : 2;
   tp.kbytes = (int)a.kdim * tp.elem_bytes;
   tp.batches = a.batches;
+  tp.groups = groups;
   tp.tiles_m = (int)((a.rows_a + 2 * BM - 1) / (2 * BM));
   tp.tiles_n = (int)((a.rows_b + L::BN - 1) / L::BN);
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
@@ -725,7 +732,7 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   tp.wide = rows_32b_aligned(a);
   tp.selftest_no_producer = a.selftest_no_producer;
   tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
-  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches;
+  const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches * tp.groups;
   if (total <= 0) return FMM_OK;
   const int sms = sm_count();
   if (sms < 2) return FMM_ERR_CUDA;

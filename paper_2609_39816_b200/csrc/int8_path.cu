@@ -1,0 +1,422 @@
+// Certified realisation on bounded integer codes (Section 4.2, Proposition 1; quantisation specification of
+// Appendix D): quantiser, the group-scaled int8 operator computed classically or by an algorithm <m,k,n;R> with
+// integer coefficients called once per group of 128 inner indices, and the certificate check.
+//
+// Arithmetic: codes and block sums are integers of magnitude <= 127, exact in bf16; every product and every
+// partial sum formed in a call is an integer below 2^24, exact in the fp32 accumulators of the tensor cores and
+// of the decode.  The integer product of a group is therefore the exact one whatever the algorithm, and the
+// rescale (P * d_A) * d_B, accumulated over ascending groups in fp32, gives the classical operator's bits.
+//
+// Data flow per call (all groups at once):
+//   pack     int8 codes [rows][K]            -> bf16 cell matrix [(i, group, p)][(l, t)], t padded to 64
+//   encode   block sums over the m x k grid  -> Ahat_r [group][bm][w]           (existing encode kernel)
+//   products (r, group): Ahat_r[group] Bhat_r[group]^T -> fp32 [R][G][bm][bn]   (existing tcgen05 kernels)
+//   decode   per group: P = sum_r w M_r, x = (P * d_A) * d_B, C += x; one cast at the end
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
+#include "fmm_internal.h"
+#include "kernels_stream.cuh"
+
+namespace {
+
+constexpr int kGroup = 128;           // inner indices that share a scale (Appendix D)
+constexpr int kQuantThreads = 256;
+constexpr int kDecThreads = 256;
+constexpr size_t kAlign = 256;
+constexpr int kSlabPadBytes = 256;    // spacing pad between consecutive slabs (avoids power-of-two strides)
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+#define FMM_CUDA(x) do { if ((x) != cudaSuccess) return FMM_ERR_CUDA; } while (0)
+#define FMM_TRY(x) do { fmm_status _s = (x); if (_s != FMM_OK) return _s; } while (0)
+
+// ------------------------------------------------------------------------------------------
+// Quantiser: one warp per (row, group).  d = max|x| / b in fp32 (1 for an all-zero group), code = x / d rounded
+// to nearest even; IEEE division on both (the decision that fixes an integer is taken in fp32, as specified).
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void load4(const float* p, float v[4]) {
+  const float4 x = *reinterpret_cast<const float4*>(p);
+  v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float v[4]) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  v[0] = __low2float(lo); v[1] = __high2float(lo); v[2] = __low2float(hi); v[3] = __high2float(hi);
+}
+
+template <typename SrcT>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int G, float b, int8_t* __restrict__ codes,
+                float* __restrict__ scales) {
+  const int lane = threadIdx.x & 31;
+  const int64_t total = rows * G;
+  for (int64_t id = (int64_t)blockIdx.x * (kQuantThreads / 32) + (threadIdx.x >> 5); id < total;
+       id += (int64_t)gridDim.x * (kQuantThreads / 32)) {
+    const int64_t row = id / G;
+    const int g = (int)(id - row * G);
+    float v[4];
+    load4(X + row * ldx + (int64_t)g * kGroup + lane * 4, v);
+    float amax = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float d = amax == 0.0f ? 1.0f : __fdiv_rn(amax, b);
+    uint32_t packed = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int c = __float2int_rn(__fdiv_rn(v[e], d));
+      packed |= ((uint32_t)c & 0xffu) << (8 * e);
+    }
+    *reinterpret_cast<uint32_t*>(codes + (row * G + g) * kGroup + lane * 4) = packed;
+    if (lane == 0) scales[row * G + g] = d;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Pack: int8 codes [gr*br][K] -> bf16 matrix with rows (i, group, p) and columns (l, t), t in [0, w), zero for
+// t >= h.  Block (i, l) of that matrix is the stack over groups of the [br x h] code blocks, so one encode pass
+// and one grouped product launch serve every group.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+pack_kernel(const int8_t* __restrict__ codes, int64_t K, int64_t br, int G, int kk, int h, int w, int64_t nvec,
+            __nv_bfloat16* __restrict__ Xq) {
+  const int vpr = kk * w / 8;   // 16-byte vectors per packed row
+  for (int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x; idx < nvec; idx += (int64_t)gridDim.x * 256) {
+    const int64_t rowp = idx / vpr;
+    const int col = (int)(idx - rowp * vpr) * 8;
+    const int l = col / w, t = col - l * w;
+    const int64_t i = rowp / (G * br);
+    const int64_t rem = rowp - i * (G * br);
+    const int64_t g = rem / br, p = rem - g * br;
+    uint4 out = make_uint4(0u, 0u, 0u, 0u);
+    if (t < h) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(codes + (i * br + p) * K + g * kGroup + l * h + t);
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t word = e < 2 ? raw.x : raw.y;
+        const int c0 = (int)(int8_t)((word >> (16 * (e & 1))) & 0xffu);
+        const int c1 = (int)(int8_t)((word >> (16 * (e & 1) + 8)) & 0xffu);
+        const __nv_bfloat162 two = __floats2bfloat162_rn((float)c0, (float)c1);
+        o[e] = *reinterpret_cast<const uint32_t*>(&two);
+      }
+      out = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    *reinterpret_cast<uint4*>(Xq + idx * 8) = out;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Grouped decode and rescale.  A block owns kPos position quads (4 consecutive columns of one row position of
+// every C block); kSplit threads share a position and split the C blocks between them.  For every group in
+// ascending order the R product vectors of the position are staged in shared memory, each thread forms its
+// blocks' integer sums (exact in fp32), multiplies by d_A and then by d_B (two roundings, no fused
+// multiply-add), and adds to its fp32 accumulators; one rounding to the output dtype after the last group.
+// ------------------------------------------------------------------------------------------
+struct GDecHead {
+  int off[FMM_MAX_GRID * FMM_MAX_GRID + 1];
+  int pad[3];
+};
+
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 raw;
+  raw.x = *reinterpret_cast<const uint32_t*>(&lo);
+  raw.y = *reinterpret_cast<const uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = raw;
+}
+__device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+
+template <typename OutT, int kSplit>
+__global__ void __launch_bounds__(kDecThreads)
+decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, const CoefTable* __restrict__ d_tab,
+                    int R, const float* __restrict__ dA, const float* __restrict__ dB, int n, int64_t bm,
+                    int64_t bn, OutT* __restrict__ C, int64_t ldc) {
+  constexpr int kPos = kDecThreads / kSplit;
+  constexpr int kCells = 16 / kSplit;
+  constexpr int kSlab = kPos * 16;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  GDecHead& sm = *reinterpret_cast<GDecHead*>(smem_raw);
+  const int ncell = d_tab->R;
+  const int total = d_tab->off[ncell];
+  int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(GDecHead));
+  unsigned char* stage = smem_raw + ((sizeof(GDecHead) + (size_t)total * 8 + 15) / 16) * 16;
+
+  const int tg = threadIdx.x / kPos;
+  const int pq = threadIdx.x - tg * kPos;
+  const int vec_per_row = (int)(bn >> 2);
+  const int nvec = (int)bm * vec_per_row;
+  const int idx = blockIdx.x * kPos + pq;
+  const bool live = idx < nvec;
+  const int p = live ? idx / vec_per_row : 0;
+  const int q = live ? (idx - p * vec_per_row) << 2 : 0;
+  unsigned char* my_stage = stage + pq * 16;
+  const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
+
+  for (int i = threadIdx.x; i <= ncell; i += kDecThreads) sm.off[i] = d_tab->off[i];
+  for (int i = threadIdx.x; i < total; i += kDecThreads)
+    ent[i] = make_int2(d_tab->cell[i] * kSlab, __float_as_int(d_tab->coef[i]));
+  if (tg == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);   // padding slab
+
+  float4 acc[kCells];
+#pragma unroll
+  for (int u = 0; u < kCells; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  const float* src = prod + (int64_t)p * bn + q;
+  for (int g = 0; g < G; ++g) {
+    __syncthreads();   // table ready (first pass); previous group's readers are done with the stage
+    {
+      const int nbytes = live ? 16 : 0;
+      for (int r = tg; r < R; r += kSplit)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab),
+                     "l"(src + ((int64_t)r * G + g) * pstride), "r"(nbytes) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u4 = 0; u4 < kCells; ++u4) {
+      const int c = tg + u4 * kSplit;
+      if (c >= ncell) break;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int e1 = sm.off[c + 1];
+      for (int e = sm.off[c]; e < e1; ++e) {
+        const int2 en = ent[e];
+        const float w = __int_as_float(en.y);
+        const float4 v = *reinterpret_cast<const float4*>(my_stage + en.x);
+        x.x = __fmaf_rn(w, v.x, x.x); x.y = __fmaf_rn(w, v.y, x.y);   // integers below 2^24: exact
+        x.z = __fmaf_rn(w, v.z, x.z); x.w = __fmaf_rn(w, v.w, x.w);
+      }
+      if (live) {
+        const int i = c / n, j = c - i * n;
+        const float da = dA[((int64_t)i * bm + p) * G + g];
+        const int64_t col = (int64_t)j * bn + q;
+        const float b0 = dB[(col + 0) * G + g], b1 = dB[(col + 1) * G + g];
+        const float b2 = dB[(col + 2) * G + g], b3 = dB[(col + 3) * G + g];
+        acc[u4].x = __fadd_rn(acc[u4].x, __fmul_rn(__fmul_rn(x.x, da), b0));
+        acc[u4].y = __fadd_rn(acc[u4].y, __fmul_rn(__fmul_rn(x.y, da), b1));
+        acc[u4].z = __fadd_rn(acc[u4].z, __fmul_rn(__fmul_rn(x.z, da), b2));
+        acc[u4].w = __fadd_rn(acc[u4].w, __fmul_rn(__fmul_rn(x.w, da), b3));
+      }
+    }
+  }
+  if (live) {
+#pragma unroll
+    for (int u4 = 0; u4 < kCells; ++u4) {
+      const int c = tg + u4 * kSplit;
+      if (c >= ncell) break;
+      const int i = c / n, j = c - i * n;
+      store4(C + ((int64_t)i * bm + p) * ldc + (int64_t)j * bn + q, acc[u4]);
+    }
+  }
+}
+
+int padded_total(const CoefTable& t) { return t.off[t.R]; }
+
+template <typename OutT, int kSplit>
+cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
+                                  const CoefTable* h_tab, int R, const float* dA, const float* dB, int n, int64_t bm,
+                                  int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+  constexpr int kPos = kDecThreads / kSplit;
+  const size_t smem = ((sizeof(GDecHead) + (size_t)padded_total(*h_tab) * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kPos * 16;
+  const int64_t nvec = bm * (bn >> 2);
+  if (nvec + kDecThreads >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+  auto k = decode_group_kernel<OutT, kSplit>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e != cudaSuccess) return e;
+  const unsigned grid = (unsigned)((nvec + kPos - 1) / kPos);
+  k<<<grid, kDecThreads, smem, st>>>(prod, pstride, G, d_tab, R, dA, dB, n, bm, bn, (OutT*)C, ldc);
+  ++fmm_launch_counter();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_group(int output, const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
+                                const CoefTable* h_tab, int R, const float* dA, const float* dB, int m, int n,
+                                int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+  const bool small = m * n <= 4;
+  if (output == FMM_F32)
+    return small ? launch_decode_group_t<float, 1>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st)
+                 : launch_decode_group_t<float, 4>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st);
+  if (output == FMM_BF16)
+    return small ? launch_decode_group_t<__nv_bfloat16, 1>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st)
+                 : launch_decode_group_t<__nv_bfloat16, 4>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st);
+  return cudaErrorInvalidValue;
+}
+
+int stream_blocks(int64_t items, int per_block) {
+  int64_t g = (items + per_block - 1) / per_block;
+  return (int)std::min<int64_t>(std::max<int64_t>(g, 1), 148 * 16);
+}
+
+// Workspace of one int8 product.
+struct Int8Layout {
+  size_t status, tabA, tabB, tabW, xqa, xqb, ahat, bhat, prod, total;
+  int64_t sAhat, sBhat, sProd;   // element strides between products (Ahat/Bhat) and between (r, group) entries (prod)
+  int G, h, w;
+  bool trivial;
+};
+
+fmm_scheme trivial_scheme() {
+  fmm_scheme c;
+  c.m = c.k = c.n = c.R = 1;
+  c.U = {1.0}; c.V = {1.0}; c.W = {1.0};
+  return c;
+}
+
+fmm_status int8_shape_ok(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
+  if (M <= 0 || K <= 0 || N <= 0 || K % kGroup) return FMM_ERR_SHAPE;
+  if (M % s.m || N % s.n || kGroup % s.k) return FMM_ERR_SHAPE;
+  const int h = kGroup / s.k;
+  if (h != 32 && h != 64 && h != 128) return FMM_ERR_SHAPE;
+  if ((N / s.n) % 8) return FMM_ERR_SHAPE;
+  if (M * (K / kGroup) > 0x7fffffffLL / 2 || N * (K / kGroup) > 0x7fffffffLL / 2) return FMM_ERR_SHAPE;
+  return FMM_OK;
+}
+
+Int8Layout int8_layout(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
+  Int8Layout L;
+  L.G = (int)(K / kGroup);
+  L.h = kGroup / s.k;
+  L.w = std::max(L.h, 64);
+  L.trivial = s.m == 1 && s.k == 1 && s.n == 1 && s.R == 1;
+  const int64_t bm = M / s.m, bn = N / s.n;
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.tabA = o; o += align_up(sizeof(CoefTable));
+  L.tabB = o; o += align_up(sizeof(CoefTable));
+  L.tabW = o; o += align_up(sizeof(CoefTable));
+  L.xqa = o; o += align_up((size_t)M * L.G * s.k * L.w * 2);
+  L.xqb = o; o += align_up((size_t)N * L.G * s.k * L.w * 2);
+  L.sAhat = (int64_t)L.G * bm * L.w + kSlabPadBytes / 2;
+  L.sBhat = (int64_t)L.G * bn * L.w + kSlabPadBytes / 2;
+  L.sProd = bm * bn + kSlabPadBytes / 4;
+  L.ahat = o; o += L.trivial ? 0 : align_up((size_t)s.R * L.sAhat * 2);
+  L.bhat = o; o += L.trivial ? 0 : align_up((size_t)s.R * L.sBhat * 2);
+  L.prod = o; o += align_up((size_t)s.R * L.G * L.sProd * 4);
+  L.total = o;
+  return L;
+}
+
+bool integer_coefficients(const fmm_scheme& s) {
+  for (const std::vector<double>* v : {&s.U, &s.V, &s.W})
+    for (double c : *v)
+      if (c != std::rint(c)) return false;
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int scheme_certificate(const fmm_scheme* s, int bA, int bB, int h, int g, int acc_bits, double cert[4]) {
+  fmm_scheme one = trivial_scheme();
+  const fmm_scheme& sc = s ? *s : one;
+  double meta[8];
+  if (scheme_info(&sc, nullptr, meta) != FMM_OK) return 0;
+  const double a = meta[0] * bA, b = meta[1] * bB;
+  const double big = std::max(meta[2] * h * a * b, (double)g * bA * bB);
+  const bool one_group = (int64_t)sc.k * h == g;
+  if (cert) { cert[0] = a; cert[1] = b; cert[2] = big; cert[3] = one_group ? 1.0 : 0.0; }
+  return integer_coefficients(sc) && a <= 127.0 && b <= 127.0 && big < std::ldexp(1.0, acc_bits) && one_group;
+}
+
+fmm_status int8_quantize(const void* d_X, int storage, int64_t rows, int64_t K, int64_t ldx, int code_bound,
+                         int8_t* d_codes, float* d_scales, void* stream) {
+  if (!d_X || !d_codes || !d_scales) return FMM_ERR_ARG;
+  if (rows <= 0 || K <= 0 || K % kGroup || ldx < K) return FMM_ERR_SHAPE;
+  if (code_bound < 1 || code_bound > 127) return FMM_ERR_ARG;
+  if (storage != FMM_F32 && storage != FMM_BF16) return FMM_ERR_DTYPE;
+  const int es = storage == FMM_F32 ? 4 : 2;
+  if ((ldx * es) % (4 * es) || (reinterpret_cast<uintptr_t>(d_X) % (4 * es)) || (reinterpret_cast<uintptr_t>(d_codes) % 4))
+    return FMM_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int G = (int)(K / kGroup);
+  const int grid = stream_blocks(rows * G, kQuantThreads / 32);
+  if (storage == FMM_F32)
+    quantize_kernel<float><<<grid, kQuantThreads, 0, st>>>((const float*)d_X, ldx, rows, G, (float)code_bound, d_codes, d_scales);
+  else
+    quantize_kernel<__nv_bfloat16><<<grid, kQuantThreads, 0, st>>>((const __nv_bfloat16*)d_X, ldx, rows, G, (float)code_bound, d_codes, d_scales);
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N) {
+  fmm_scheme one = trivial_scheme();
+  const fmm_scheme& sc = s ? *s : one;
+  if (int8_shape_ok(sc, M, K, N) != FMM_OK) return 0;
+  return int8_layout(sc, M, K, N).total;
+}
+
+fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
+                     const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc, void* d_ws,
+                     size_t ws_bytes, void* stream) {
+  if (!d_cA || !d_dA || !d_cB || !d_dB || !d_C) return FMM_ERR_ARG;
+  if (output != FMM_F32 && output != FMM_BF16) return FMM_ERR_DTYPE;
+  if (code_bound < 1 || code_bound > 127) return FMM_ERR_ARG;
+  fmm_scheme one = trivial_scheme();
+  const fmm_scheme& sc = s ? *s : one;
+  FMM_TRY(int8_shape_ok(sc, M, K, N));
+  const int eo = output == FMM_F32 ? 4 : 2;
+  if (ldc < N || (ldc * eo) % 16 || (reinterpret_cast<uintptr_t>(d_C) % 16)) return FMM_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(d_cA) % 8) || (reinterpret_cast<uintptr_t>(d_cB) % 8)) return FMM_ERR_SHAPE;
+  // Proposition 1 for this realisation: int8 block sums, integers exact in the fp32 accumulators (24 bits)
+  if (!scheme_certificate(&sc, code_bound, code_bound, kGroup / sc.k, kGroup, 24, nullptr)) return FMM_ERR_CERTIFICATE;
+  const Int8Layout L = int8_layout(sc, M, K, N);
+  if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t bm = M / sc.m, bn = N / sc.n;
+  const int kw = sc.k * L.w;
+
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  CoefTable *hA = new CoefTable, *hB = new CoefTable, *hW = new CoefTable;
+  std::unique_ptr<CoefTable> ga(hA), gb(hB), gw(hW);
+  std::memset(hA, 0, sizeof(CoefTable)); std::memset(hB, 0, sizeof(CoefTable)); std::memset(hW, 0, sizeof(CoefTable));
+  fmm_build_tables(sc, hA, hB, hW);
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabW), hW, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  if (!L.trivial) {
+    FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabA), hA, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabB), hB, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  }
+  {
+    ProfScope ps(0, st);
+    const int64_t nva = M * L.G * (kw / 8), nvb = N * L.G * (kw / 8);
+    pack_kernel<<<stream_blocks(nva, 256 * 4), 256, 0, st>>>(d_cA, K, bm, L.G, sc.k, L.h, L.w, nva, at<__nv_bfloat16>(d_ws, L.xqa));
+    ++fmm_launch_counter();
+    pack_kernel<<<stream_blocks(nvb, 256 * 4), 256, 0, st>>>(d_cB, K, bn, L.G, sc.k, L.h, L.w, nvb, at<__nv_bfloat16>(d_ws, L.xqb));
+    ++fmm_launch_counter();
+    FMM_CUDA(cudaGetLastError());
+    if (!L.trivial) {
+      FMM_CUDA(launch_encode(FMM_BF16, FMM_BF16, at<char>(d_ws, L.xqa), kw, sc.m, sc.k, (int64_t)L.G * bm, L.w,
+                             at<CoefTable>(d_ws, L.tabA), hA, at<char>(d_ws, L.ahat), L.sAhat, nullptr, nullptr, false, false, st));
+      FMM_CUDA(launch_encode(FMM_BF16, FMM_BF16, at<char>(d_ws, L.xqb), kw, sc.n, sc.k, (int64_t)L.G * bn, L.w,
+                             at<CoefTable>(d_ws, L.tabB), hB, at<char>(d_ws, L.bhat), L.sBhat, nullptr, nullptr, false, false, st));
+    }
+  }
+  {
+    BlockProductArgs g{};
+    g.product = FMM_BF16;
+    g.A = L.trivial ? at<char>(d_ws, L.xqa) : at<char>(d_ws, L.ahat); g.lda = L.w; g.a_batch = L.trivial ? 0 : L.sAhat;
+    g.B = L.trivial ? at<char>(d_ws, L.xqb) : at<char>(d_ws, L.bhat); g.ldb = L.w; g.b_batch = L.trivial ? 0 : L.sBhat;
+    g.rows_a = bm; g.rows_b = bn; g.kdim = L.w; g.batches = sc.R; g.groups = L.G;
+    g.out = at<char>(d_ws, L.prod); g.ldo = bn; g.o_batch = L.sProd; g.out_mode = 0; g.output = FMM_F32;
+    g.status = at<DeviceStatus>(d_ws, L.status);
+    ProfScope ps(2, st);
+    FMM_TRY(launch_block_products(g, st));
+  }
+  {
+    ProfScope ps(3, st);
+    FMM_CUDA(launch_decode_group(output, at<float>(d_ws, L.prod), L.sProd, L.G, at<CoefTable>(d_ws, L.tabW), hW, sc.R, d_dA,
+                                 d_dB, sc.m, sc.n, bm, bn, d_C, ldc, st));
+  }
+  // the tables were copied from pageable host memory: the copies are complete when cudaMemcpyAsync returns
+  return FMM_OK;
+}
+
+}  // extern "C"

@@ -64,6 +64,8 @@ struct BlockProductArgs {
   const void* A; int64_t lda; int64_t a_batch;   // elements
   const void* B; int64_t ldb; int64_t b_batch;
   int64_t rows_a, rows_b, kdim; int batches;
+  int groups;                // > 1: each batch entry holds `groups` row groups of rows_a (rows_b) rows; product (r, g)
+                             // multiplies group g of A_r with group g of B_r and lands at out + (r*groups + g)*o_batch
   void* out; int64_t ldo; int64_t o_batch; int out_mode; int output;
   const float* sA; const float* sB;
   DeviceStatus* status;

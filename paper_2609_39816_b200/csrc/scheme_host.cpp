@@ -364,6 +364,7 @@ const char* fmm_status_string(fmm_status st) {
     case FMM_ERR_CUDA: return "CUDA call failed";
     case FMM_ERR_TIMEOUT: return "device-side wait timed out";
     case FMM_ERR_LIMIT: return "scheme exceeds table limits";
+    case FMM_ERR_CERTIFICATE: return "exactness certificate does not hold";
   }
   return "unknown status";
 }

@@ -1,0 +1,148 @@
+"""GPU parity of the certified int8 realisation (Section 4.2, Proposition 1, Appendix D) against the oracle:
+integer work, so every comparison is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from fmm_inputs import generators as gen
+from gpu_util import fmm, workspace
+
+pytestmark = pytest.mark.gpu
+
+S1 = oracle.strassen()
+S2 = oracle.kron(S1, S1)
+
+
+def _lib_scheme(lib, o):
+    return lib.scheme_load(o.U, o.V, o.W)
+
+
+def _inputs(seed, M, K, N, dtype="f32"):
+    At, A = gen.to_storage(gen.activations_outlier(seed, 1, M, K), dtype)
+    Bt, B = gen.to_storage(gen.weights(seed, 2, N, K), dtype)
+    return At.cuda(), A, Bt.cuda(), B
+
+
+def _quantize(lib, X, b):
+    rows, K = X.shape
+    codes = torch.empty((rows, K), dtype=torch.int8, device="cuda")
+    scales = torch.empty((rows, K // 128), dtype=torch.float32, device="cuda")
+    lib.int8_quantize(X, b, codes, scales)
+    torch.cuda.synchronize()
+    return codes, scales
+
+
+def _gemm(lib, s, b, cA, dA, cB, dB, out_dtype=torch.bfloat16):
+    M, K = cA.shape
+    N = cB.shape[0]
+    ws = workspace(lib.int8_gemm_workspace(s, M, K, N))
+    C = torch.empty((M, N), dtype=out_dtype, device="cuda")
+    lib.int8_gemm(s, b, cA, dA, cB, dB, C, ws)
+    lib.device_status(ws)
+    return C.to(torch.float64).cpu().numpy()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("b", [31, 63, 127])
+def test_quantiser_bit_exact(dtype, b):
+    lib = fmm()
+    At, A, _, _ = _inputs(11, 200, 512, 8, dtype)
+    A[3, 128:256] = 0.0                      # an all-zero group: d = 1
+    At[3, 128:256] = 0
+    codes, scales = _quantize(lib, At, b)
+    oc, od = oracle.quantize_rows(A, b)
+    assert np.array_equal(scales.cpu().numpy().astype(np.float64), od)
+    assert np.array_equal(codes.cpu().numpy().astype(np.float64), oc)
+    assert np.abs(oc).max() == b and od[3, 1] == 1.0
+
+
+@pytest.mark.parametrize("M,K,N", [(32, 128, 32), (512, 1024, 544), (200, 384, 96)])
+def test_classical_and_certified_match_oracle_and_each_other(M, K, N):
+    """Same bits from the classical int8 operator, the certified two-level realisation and the oracle."""
+    lib = fmm()
+    At, A, Bt, B = _inputs(21, M, K, N)
+    cA, dA = _quantize(lib, At, 31)
+    cB, dB = _quantize(lib, Bt, 31)
+    oA, odA = oracle.quantize_rows(A, 31)
+    oB, odB = oracle.quantize_rows(B, 31)
+    want = oracle.int8_classical(oA, odA, oB, odB)
+    got_cl = _gemm(lib, None, 31, cA, dA, cB, dB)
+    assert np.array_equal(got_cl, want)
+    s2 = _lib_scheme(lib, S2)
+    got = _gemm(lib, s2, 31, cA, dA, cB, dB)
+    assert np.array_equal(got, want)
+    want_cert, mx = oracle.int8_certified(S2, oA, odA, oB, odB)
+    assert np.array_equal(want_cert, want) and mx[0] <= 124 and mx[1] <= 124
+    # fp32 output: the accumulated value itself, before the cast
+    got32 = _gemm(lib, s2, 31, cA, dA, cB, dB, torch.float32)
+    assert np.array_equal(got32, oracle.int8_classical(oA, odA, oB, odB, od="f32"))
+    assert oracle.rel_error(got32, A @ B.T) < 0.2
+
+
+def test_sign_variants_and_one_level_are_bit_identical():
+    lib = fmm()
+    M, K, N = 128, 256, 64
+    At, A, Bt, B = _inputs(31, M, K, N)
+    outs = set()
+    variants = list(oracle.sign_variants(4, 4, 4))
+    for b, base, picks in ((31, S2, variants[::37] + [variants[-1]]), (63, S1, list(oracle.sign_variants(2, 2, 2)))):
+        cA, dA = _quantize(lib, At, b)
+        cB, dB = _quantize(lib, Bt, b)
+        ref = _gemm(lib, None, b, cA, dA, cB, dB, torch.float32)
+        for d, e, f in picks:
+            s = _lib_scheme(lib, oracle.sign_variant(base, d, e, f))
+            got = _gemm(lib, s, b, cA, dA, cB, dB, torch.float32)
+            assert np.array_equal(got, ref)
+        oA, odA = oracle.quantize_rows(A, b)
+        oB, odB = oracle.quantize_rows(B, b)
+        assert np.array_equal(ref, oracle.int8_classical(oA, odA, oB, odB, od="f32"))
+        outs.add(ref.tobytes())
+    assert len(outs) == 2                     # b = 31 and b = 63 are different operators
+
+
+def test_certificate_is_enforced():
+    lib = fmm()
+    M, K, N = 32, 128, 32
+    At, A, Bt, B = _inputs(41, M, K, N)
+    cA, dA = _quantize(lib, At, 32)
+    cB, dB = _quantize(lib, Bt, 32)
+    s2 = _lib_scheme(lib, S2)
+    ws = workspace(lib.int8_gemm_workspace(s2, M, K, N))
+    C = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.FmmError) as ei:
+        lib.int8_gemm(s2, 32, cA, dA, cB, dB, C, ws)        # L_A * 32 = 128 > 127
+    assert ei.value.code == 10
+    # a gauged scheme has non-integer coefficients: no certificate at any code bound
+    P = gen.gauge_cond_limited(7, 0, 4)
+    with pytest.raises(lib.FmmError) as ei:
+        lib.int8_gemm(lib.gauge_apply(s2, P, P, P), 1, cA, dA, cB, dB, C, ws)
+    assert ei.value.code == 10
+    # one level of Strassen has L_A = 2 and admits the same codes
+    s1 = _lib_scheme(lib, S1)
+    ws1 = workspace(lib.int8_gemm_workspace(s1, M, K, N))
+    lib.int8_gemm(s1, 32, cA, dA, cB, dB, C, ws1)
+    lib.device_status(ws1)
+    oA, odA = oracle.quantize_rows(A, 32)
+    oB, odB = oracle.quantize_rows(B, 32)
+    assert np.array_equal(C.to(torch.float64).cpu().numpy(), oracle.int8_classical(oA, odA, oB, odB))
+
+
+def test_row_locality_on_device():
+    """Section 4.2: changing a later token row leaves every earlier output row's bits alone (32 rows, 4 blocks)."""
+    lib = fmm()
+    M, K, N = 32, 256, 64
+    At, A, Bt, B = _inputs(51, M, K, N)
+    s2 = _lib_scheme(lib, S2)
+    cB, dB = _quantize(lib, Bt, 31)
+    cA, dA = _quantize(lib, At, 31)
+    base = _gemm(lib, s2, 31, cA, dA, cB, dB)
+    moved = 0
+    for later in (1, 9, 17, 31):
+        A2 = At.clone()
+        A2[later] = gen.to_storage(gen.normal(51, 700 + later, (K,)), "f32")[0].cuda()
+        c2, d2 = _quantize(lib, A2, 31)
+        out = _gemm(lib, s2, 31, c2, d2, cB, dB)
+        moved += sum(int(np.any(out[e] != base[e])) for e in range(later))
+        assert np.any(out[later] != base[later])
+    assert moved == 0

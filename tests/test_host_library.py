@@ -144,3 +144,26 @@ def _shard_worker(rank, world, port):
     if rank == 0:
         assert full.tolist() == [g * 1.5 for g in range(G)]
     dist.destroy_process_group()
+
+
+def test_certificate_on_host_matches_oracle(lib):
+    """Proposition 1 evaluated by the library agrees with the oracle's and with the printed constants."""
+    s1 = lib.scheme_builtin("strassen222")
+    s2 = lib.scheme_builtin("strassen444")
+    o2 = oracle.kron(oracle.strassen(), oracle.strassen())
+    for args in ((31, 31, 32, 128, 31), (31, 31, 32, 128, 24), (32, 31, 32, 128, 31), (31, 31, 8729, 4 * 8729, 31),
+                 (31, 31, 8730, 4 * 8730, 31), (31, 31, 64, 128, 31)):
+        got = lib.scheme_certificate(s2, *args)
+        want = oracle.certificate(o2, *args)
+        assert got[0] == want[0] and got[1] == want[1], args
+    assert lib.scheme_certificate(s2, 31, 31, 32)[1]["LAbA"] == 124
+    assert lib.scheme_certificate(s1, 63, 63, 64)[0] and not lib.scheme_certificate(s1, 64, 63, 64)[0]
+    assert lib.scheme_certificate(None, 127, 127, 128)[0]
+    # a gauged (non-integer) scheme never certifies
+    P = gen.gauge_cond_limited(3, 0, 2)
+    g = lib.gauge_apply(s1, P, P, P)
+    assert not lib.scheme_certificate(g, 1, 1, 64)[0]
+    # workspace query rejects what the path cannot tile
+    assert lib.int8_gemm_workspace(s2, 64, 100, 64) == 0          # K not a multiple of 128
+    assert lib.int8_gemm_workspace(s2, 66, 128, 64) == 0          # M not divisible by m
+    assert lib.int8_gemm_workspace(s2, 64, 128, 64) > 0
