@@ -134,13 +134,12 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
 }
 __device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 
-template <typename OutT, int kSplit>
+template <typename OutT, int kSplit, int kStages, int kCells>
 __global__ void __launch_bounds__(kDecThreads)
 decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, const CoefTable* __restrict__ d_tab,
-                    int R, const float* __restrict__ dA, const float* __restrict__ dB, int n, int64_t bm,
-                    int64_t bn, OutT* __restrict__ C, int64_t ldc) {
-  constexpr int kPos = kDecThreads / kSplit;
-  constexpr int kCells = 16 / kSplit;
+                    int R, const float* __restrict__ dAt, const float* __restrict__ dBt, int64_t Mtot, int64_t Ntot,
+                    int n, int64_t bm, int64_t bn, OutT* __restrict__ C, int64_t ldc) {
+  constexpr int kPos = kDecThreads / kSplit;   // kSplit * kCells >= number of C blocks
   constexpr int kSlab = kPos * 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   GDecHead& sm = *reinterpret_cast<GDecHead*>(smem_raw);
@@ -148,6 +147,7 @@ decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, cons
   const int total = d_tab->off[ncell];
   int2* ent = reinterpret_cast<int2*>(smem_raw + sizeof(GDecHead));
   unsigned char* stage = smem_raw + ((sizeof(GDecHead) + (size_t)total * 8 + 15) / 16) * 16;
+  const int stage_bytes = (R + 1) * kSlab;   // R product slabs and the all-zero padding slab
 
   const int tg = threadIdx.x / kPos;
   const int pq = threadIdx.x - tg * kPos;
@@ -159,51 +159,63 @@ decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, cons
   const int q = live ? (idx - p * vec_per_row) << 2 : 0;
   unsigned char* my_stage = stage + pq * 16;
   const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
+  const float* src = prod + (int64_t)p * bn + q;
+  const int nbytes = live ? 16 : 0;   // 0 source bytes: the destination is zero-filled
+
+  // the copies of group g land in ring slot g % kStages; kStages - 1 groups are in flight ahead of the reader
+  auto issue = [&](int g) {
+    if (g < G) {
+      const uint32_t dst = dst0 + (uint32_t)((g % kStages) * stage_bytes);
+      for (int r = tg; r < R; r += kSplit)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + r * kSlab),
+                     "l"(src + ((int64_t)r * G + g) * pstride), "r"(nbytes) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");   // one (possibly empty) commit per step keeps the count uniform
+  };
+#pragma unroll
+  for (int g = 0; g < kStages - 1; ++g) issue(g);
 
   for (int i = threadIdx.x; i <= ncell; i += kDecThreads) sm.off[i] = d_tab->off[i];
   for (int i = threadIdx.x; i < total; i += kDecThreads)
     ent[i] = make_int2(d_tab->cell[i] * kSlab, __float_as_int(d_tab->coef[i]));
-  if (tg == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);   // padding slab
+  if (tg == 0)
+#pragma unroll
+    for (int b = 0; b < kStages; ++b)
+      *reinterpret_cast<float4*>(my_stage + b * stage_bytes + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
 
   float4 acc[kCells];
 #pragma unroll
   for (int u = 0; u < kCells; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  const float* src = prod + (int64_t)p * bn + q;
   for (int g = 0; g < G; ++g) {
-    __syncthreads();   // table ready (first pass); previous group's readers are done with the stage
-    {
-      const int nbytes = live ? 16 : 0;
-      for (int r = tg; r < R; r += kSplit)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab),
-                     "l"(src + ((int64_t)r * G + g) * pstride), "r"(nbytes) : "memory");
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-    }
-    __syncthreads();
+    asm volatile("cp.async.wait_group %0;" ::"n"(kStages - 2) : "memory");   // this thread's copies of group g are done
+    __syncthreads();            // everyone's are; and the slot read in the previous step is free again
+    issue(g + kStages - 1);
+    const unsigned char* cur = my_stage + (g % kStages) * stage_bytes;
 #pragma unroll
     for (int u4 = 0; u4 < kCells; ++u4) {
       const int c = tg + u4 * kSplit;
       if (c >= ncell) break;
       float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
       const int e1 = sm.off[c + 1];
-      for (int e = sm.off[c]; e < e1; ++e) {
-        const int2 en = ent[e];
-        const float w = __int_as_float(en.y);
-        const float4 v = *reinterpret_cast<const float4*>(my_stage + en.x);
-        x.x = __fmaf_rn(w, v.x, x.x); x.y = __fmaf_rn(w, v.y, x.y);   // integers below 2^24: exact
-        x.z = __fmaf_rn(w, v.z, x.z); x.w = __fmaf_rn(w, v.w, x.w);
+      for (int e = sm.off[c]; e < e1; e += 2) {   // lists are padded to a multiple of four entries
+        const int4 two = *reinterpret_cast<const int4*>(&ent[e]);
+        const float4 v0 = *reinterpret_cast<const float4*>(cur + two.x);
+        const float4 v1 = *reinterpret_cast<const float4*>(cur + two.z);
+        const float w0 = __int_as_float(two.y), w1 = __int_as_float(two.w);
+        x.x = __fmaf_rn(w0, v0.x, x.x); x.y = __fmaf_rn(w0, v0.y, x.y);   // integers below 2^24: exact
+        x.z = __fmaf_rn(w0, v0.z, x.z); x.w = __fmaf_rn(w0, v0.w, x.w);
+        x.x = __fmaf_rn(w1, v1.x, x.x); x.y = __fmaf_rn(w1, v1.y, x.y);
+        x.z = __fmaf_rn(w1, v1.z, x.z); x.w = __fmaf_rn(w1, v1.w, x.w);
       }
       if (live) {
         const int i = c / n, j = c - i * n;
-        const float da = dA[((int64_t)i * bm + p) * G + g];
-        const int64_t col = (int64_t)j * bn + q;
-        const float b0 = dB[(col + 0) * G + g], b1 = dB[(col + 1) * G + g];
-        const float b2 = dB[(col + 2) * G + g], b3 = dB[(col + 3) * G + g];
-        acc[u4].x = __fadd_rn(acc[u4].x, __fmul_rn(__fmul_rn(x.x, da), b0));
-        acc[u4].y = __fadd_rn(acc[u4].y, __fmul_rn(__fmul_rn(x.y, da), b1));
-        acc[u4].z = __fadd_rn(acc[u4].z, __fmul_rn(__fmul_rn(x.z, da), b2));
-        acc[u4].w = __fadd_rn(acc[u4].w, __fmul_rn(__fmul_rn(x.w, da), b3));
+        const float da = dAt[(int64_t)g * Mtot + (int64_t)i * bm + p];
+        const float4 db = *reinterpret_cast<const float4*>(dBt + (int64_t)g * Ntot + (int64_t)j * bn + q);
+        acc[u4].x = __fadd_rn(acc[u4].x, __fmul_rn(__fmul_rn(x.x, da), db.x));
+        acc[u4].y = __fadd_rn(acc[u4].y, __fmul_rn(__fmul_rn(x.y, da), db.y));
+        acc[u4].z = __fadd_rn(acc[u4].z, __fmul_rn(__fmul_rn(x.z, da), db.z));
+        acc[u4].w = __fadd_rn(acc[u4].w, __fmul_rn(__fmul_rn(x.w, da), db.w));
       }
     }
   }
@@ -218,35 +230,101 @@ decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, cons
   }
 }
 
+// The classical operator needs no decode: one product per group.  A thread owns four consecutive outputs and walks
+// the groups in ascending order, eight independent 16-byte loads in flight per step.
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+rescale_groups_kernel(const float* __restrict__ prod, int64_t pstride, int G, const float* __restrict__ dAt,
+                      const float* __restrict__ dBt, int64_t M, int64_t N, OutT* __restrict__ C, int64_t ldc) {
+  const int vec_per_row = (int)(N >> 2);
+  const int64_t nvec = M * vec_per_row;
+  const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= nvec) return;
+  const int64_t p = idx / vec_per_row;
+  const int64_t q = (idx - p * vec_per_row) << 2;
+  const float* src = prod + p * N + q;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int kU = 8;
+  for (int g0 = 0; g0 < G; g0 += kU) {
+    float4 v[kU], db[kU];
+    float da[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int g = min(g0 + u, G - 1);   // the tail re-reads the last group; its result is not used
+      v[u] = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)g * pstride));
+      db[u] = *reinterpret_cast<const float4*>(dBt + (int64_t)g * N + q);
+      da[u] = dAt[(int64_t)g * M + p];
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      if (g0 + u < G) {
+        acc.x = __fadd_rn(acc.x, __fmul_rn(__fmul_rn(v[u].x, da[u]), db[u].x));
+        acc.y = __fadd_rn(acc.y, __fmul_rn(__fmul_rn(v[u].y, da[u]), db[u].y));
+        acc.z = __fadd_rn(acc.z, __fmul_rn(__fmul_rn(v[u].z, da[u]), db[u].z));
+        acc.w = __fadd_rn(acc.w, __fmul_rn(__fmul_rn(v[u].w, da[u]), db[u].w));
+      }
+    }
+  }
+  store4(C + p * ldc + q, acc);
+}
+
+// scales [rows][G] -> [G][rows] (a few hundred KB: the decode reads one contiguous vector per group)
+__global__ void __launch_bounds__(256) transpose_scales_kernel(const float* __restrict__ d, int64_t rows, int G,
+                                                               float* __restrict__ dt) {
+  const int64_t total = rows * G;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (int64_t)gridDim.x * 256) {
+    const int64_t g = i / rows, r = i - g * rows;
+    dt[i] = d[r * G + g];
+  }
+}
+
 int padded_total(const CoefTable& t) { return t.off[t.R]; }
 
-template <typename OutT, int kSplit>
+template <typename OutT, int kSplit, int kStages, int kCells>
 cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
-                                  const CoefTable* h_tab, int R, const float* dA, const float* dB, int n, int64_t bm,
-                                  int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+                                  const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
+                                  int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
   constexpr int kPos = kDecThreads / kSplit;
-  const size_t smem = ((sizeof(GDecHead) + (size_t)padded_total(*h_tab) * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kPos * 16;
+  const size_t smem = ((sizeof(GDecHead) + (size_t)padded_total(*h_tab) * 8 + 15) / 16) * 16 +
+                      (size_t)kStages * (R + 1) * kPos * 16;
   const int64_t nvec = bm * (bn >> 2);
-  if (nvec + kDecThreads >= (int64_t)1 << 31) return cudaErrorInvalidValue;
-  auto k = decode_group_kernel<OutT, kSplit>;
+  if (nvec + kDecThreads >= (int64_t)1 << 31 || smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (m * n > kSplit * kCells) return cudaErrorInvalidValue;
+  auto k = decode_group_kernel<OutT, kSplit, kStages, kCells>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
   const unsigned grid = (unsigned)((nvec + kPos - 1) / kPos);
-  k<<<grid, kDecThreads, smem, st>>>(prod, pstride, G, d_tab, R, dA, dB, n, bm, bn, (OutT*)C, ldc);
+  k<<<grid, kDecThreads, smem, st>>>(prod, pstride, G, d_tab, R, dAt, dBt, (int64_t)m * bm, (int64_t)n * bn, n, bm, bn,
+                                     (OutT*)C, ldc);
   ++fmm_launch_counter();
   return cudaGetLastError();
 }
 
+// One C block and one product (the classical operator): the plain rescale kernel.  At most four C blocks and
+// eight products: four threads share a position, four groups in flight; otherwise eight threads share a
+// position (two C blocks each), two groups in flight.
+template <typename OutT>
+cudaError_t launch_decode_group_o(const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
+                                  const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
+                                  int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+  if (m * n == 1 && R == 1) {
+    const int64_t nvec = bm * (bn >> 2);
+    rescale_groups_kernel<OutT><<<(unsigned)((nvec + 255) / 256), 256, 0, st>>>(prod, pstride, G, dAt, dBt, bm, bn, (OutT*)C, ldc);
+    ++fmm_launch_counter();
+    return cudaGetLastError();
+  }
+  if (m * n <= 4 && R <= 8)
+    return launch_decode_group_t<OutT, 4, 4, 1>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+  return launch_decode_group_t<OutT, 8, 2, 2>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+}
+
 cudaError_t launch_decode_group(int output, const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
-                                const CoefTable* h_tab, int R, const float* dA, const float* dB, int m, int n,
+                                const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
                                 int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
-  const bool small = m * n <= 4;
   if (output == FMM_F32)
-    return small ? launch_decode_group_t<float, 1>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st)
-                 : launch_decode_group_t<float, 4>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st);
+    return launch_decode_group_o<float>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
   if (output == FMM_BF16)
-    return small ? launch_decode_group_t<__nv_bfloat16, 1>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st)
-                 : launch_decode_group_t<__nv_bfloat16, 4>(prod, pstride, G, d_tab, h_tab, R, dA, dB, n, bm, bn, C, ldc, st);
+    return launch_decode_group_o<__nv_bfloat16>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
   return cudaErrorInvalidValue;
 }
 
@@ -257,7 +335,7 @@ int stream_blocks(int64_t items, int per_block) {
 
 // Workspace of one int8 product.
 struct Int8Layout {
-  size_t status, tabA, tabB, tabW, xqa, xqb, ahat, bhat, prod, total;
+  size_t status, tabA, tabB, tabW, dAt, dBt, xqa, xqb, ahat, bhat, prod, total;
   int64_t sAhat, sBhat, sProd;   // element strides between products (Ahat/Bhat) and between (r, group) entries (prod)
   int G, h, w;
   bool trivial;
@@ -292,6 +370,8 @@ Int8Layout int8_layout(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
   L.tabA = o; o += align_up(sizeof(CoefTable));
   L.tabB = o; o += align_up(sizeof(CoefTable));
   L.tabW = o; o += align_up(sizeof(CoefTable));
+  L.dAt = o; o += align_up((size_t)M * L.G * 4);
+  L.dBt = o; o += align_up((size_t)N * L.G * 4);
   L.xqa = o; o += align_up((size_t)M * L.G * s.k * L.w * 2);
   L.xqb = o; o += align_up((size_t)N * L.G * s.k * L.w * 2);
   L.sAhat = (int64_t)L.G * bm * L.w + kSlabPadBytes / 2;
@@ -412,8 +492,13 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
   }
   {
     ProfScope ps(3, st);
-    FMM_CUDA(launch_decode_group(output, at<float>(d_ws, L.prod), L.sProd, L.G, at<CoefTable>(d_ws, L.tabW), hW, sc.R, d_dA,
-                                 d_dB, sc.m, sc.n, bm, bn, d_C, ldc, st));
+    transpose_scales_kernel<<<stream_blocks(M * L.G, 256), 256, 0, st>>>(d_dA, M, L.G, at<float>(d_ws, L.dAt));
+    ++fmm_launch_counter();
+    transpose_scales_kernel<<<stream_blocks(N * L.G, 256), 256, 0, st>>>(d_dB, N, L.G, at<float>(d_ws, L.dBt));
+    ++fmm_launch_counter();
+    FMM_CUDA(cudaGetLastError());
+    FMM_CUDA(launch_decode_group(output, at<float>(d_ws, L.prod), L.sProd, L.G, at<CoefTable>(d_ws, L.tabW), hW, sc.R,
+                                 at<float>(d_ws, L.dAt), at<float>(d_ws, L.dBt), sc.m, sc.n, bm, bn, d_C, ldc, st));
   }
   // the tables were copied from pageable host memory: the copies are complete when cudaMemcpyAsync returns
   return FMM_OK;
