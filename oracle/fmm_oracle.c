@@ -34,8 +34,12 @@
  * the printed constants (b = 31, L_A b = 124, inner length 8729), bit-identity with the
  * classical int8 operator over all 512 sign variants, brute-force integer products on
  * 200 random tiles, and the 0-of-496 row-pair count.
- * Parity unpinned: the error-amplification ratios at the benchmark workloads (the
- * paper prints none for synthetic inputs of these shapes).
+ * The error statistic (relative Frobenius error of a realisation, compared across sign
+ * variants) is pinned softly by the ensemble of Appendix B.1 on 128 x 128 operands: spread
+ * 2.59 / split-half correlation 0.9997 on U[0,1], 1.005 / 0.121 on U[-1,1], reproduced within
+ * sampling noise at 24 pairs (scale_mode 2).
+ * Parity unpinned: the error-amplification ratios at the benchmark workloads themselves
+ * (the paper prints none for synthetic inputs of these shapes).
  *
  * All matrices are dense row-major arrays of double.
  */
@@ -50,6 +54,15 @@
 #endif
 
 enum { ORC_F32 = 0, ORC_BF16 = 1, ORC_E4M3 = 2, ORC_F64 = 3 };
+
+/* Thread count of the OpenMP loops (tiny problems run faster on one thread; the arithmetic is the same). */
+void orc_set_num_threads(int n) {
+#ifdef _OPENMP
+  omp_set_num_threads(n < 1 ? 1 : n);
+#else
+  (void)n;
+#endif
+}
 
 int orc_num_threads(void) {
 #ifdef _OPENMP
@@ -348,9 +361,14 @@ static void matmul_f64(const double* A, const double* B, double* C, int64_t M, i
 
 /* Apply an algorithm <m,k,n;R> to A (M x K) and B (K x N); C is M x N.
  * pd = product dtype the block sums are rounded to, od = output dtype,
- * scale_mode 0: no scales; 1: per-encoded-tensor power-of-two scale (e4m3).
+ * scale_mode 0: no scales; 1: per-encoded-tensor power-of-two scale (e4m3); 2: the
+ * simplified synthetic schedule of Appendix B.1, one scale per row of each block sum of A
+ * and per column of each block sum of B, scale = max|x| / 448 in fp32 (1 for an all-zero
+ * row), code = x / scale in fp32, then rounded to e4m3 (a reading: the paper states who
+ * owns a scale, not its rule; max|x| / b is the rule of its int8 specification).
  * Optional outputs (may be NULL): Ahat [R][bm][bk], Bhat [R][bk][bn] (the rounded,
- * scaled block sums), sA[R], sB[R], Mout [R][bm][bn] (the fp64 products).
+ * scaled block sums), sA[R], sB[R] (mode 2: sA[R][bm], sB[R][bn]), Mout [R][bm][bn]
+ * (the fp64 products of the codes; mode 2: times the row and column scales).
  * Returns 0, or 1 if a dimension does not divide.                                 */
 int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V, const double* W,
                     int64_t M, int64_t K, int64_t N, const double* A, const double* B,
@@ -366,6 +384,8 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
   double* acc = (double*)calloc((size_t)M * N, sizeof(double));
   double* cu = (double*)malloc(sizeof(double) * m * k);
   double* cv = (double*)malloc(sizeof(double) * k * n);
+  double* rs = (double*)malloc(sizeof(double) * bm);   /* mode 2: row scales of the A block sum */
+  double* cs = (double*)malloc(sizeof(double) * bn);   /* mode 2: column scales of the B block sum */
   for (int r = 0; r < R; ++r) {
     /* coefficients as the kernel sees them: fp32 values (exact mode keeps fp64) */
     for (int x = 0; x < m * k; ++x) cu[x] = quant ? (double)(float)U[r * m * k + x] : U[r * m * k + x];
@@ -375,16 +395,38 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
     block_sum(B, N, k, n, bk, bn, cv, quant, Bh);
     double sa = 1.0, sb = 1.0;
     if (scale_mode == 1) { sa = pow2_scale_448(Ah, bm * bk); sb = pow2_scale_448(Bh, bk * bn); }
-    if (quant) {
-      for (int64_t x = 0; x < bm * bk; ++x) Ah[x] = orc_round(Ah[x] / sa, pd);
-      for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x] / sb, pd);
+    if (scale_mode == 2) {
+      for (int64_t p = 0; p < bm; ++p) {
+        float amax = 0.0f;
+        for (int64_t t = 0; t < bk; ++t) { float a = fabsf((float)Ah[p * bk + t]); if (a > amax) amax = a; }
+        float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+        rs[p] = (double)d;
+        for (int64_t t = 0; t < bk; ++t) Ah[p * bk + t] = orc_round((double)((float)Ah[p * bk + t] / d), pd);
+      }
+      for (int64_t c = 0; c < bn; ++c) {
+        float amax = 0.0f;
+        for (int64_t t = 0; t < bk; ++t) { float a = fabsf((float)Bh[t * bn + c]); if (a > amax) amax = a; }
+        float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+        cs[c] = (double)d;
+        for (int64_t t = 0; t < bk; ++t) Bh[t * bn + c] = orc_round((double)((float)Bh[t * bn + c] / d), pd);
+      }
+      if (sA_out) memcpy(sA_out + (size_t)r * bm, rs, sizeof(double) * bm);
+      if (sB_out) memcpy(sB_out + (size_t)r * bn, cs, sizeof(double) * bn);
+    } else {
+      if (quant) {
+        for (int64_t x = 0; x < bm * bk; ++x) Ah[x] = orc_round(Ah[x] / sa, pd);
+        for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x] / sb, pd);
+      }
+      if (sA_out) sA_out[r] = sa;
+      if (sB_out) sB_out[r] = sb;
     }
     if (Ahat_out) memcpy(Ahat_out + (size_t)r * bm * bk, Ah, sizeof(double) * bm * bk);
     if (Bhat_out) memcpy(Bhat_out + (size_t)r * bk * bn, Bh, sizeof(double) * bk * bn);
-    if (sA_out) sA_out[r] = sa;
-    if (sB_out) sB_out[r] = sb;
     /* product */
     matmul_f64(Ah, Bh, Mr, bm, bk, bn);
+    if (scale_mode == 2)
+      for (int64_t p = 0; p < bm; ++p)
+        for (int64_t q = 0; q < bn; ++q) Mr[p * bn + q] = (Mr[p * bn + q] * rs[p]) * cs[q];
     if (M_out) memcpy(M_out + (size_t)r * bm * bn, Mr, sizeof(double) * bm * bn);
     /* decode, ascending r: C_ij += w_{r,ij} * (sA_r sB_r) * M_r */
     for (int i = 0; i < m; ++i)
@@ -399,19 +441,42 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
       }
   }
   for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x], od);
-  free(Ah); free(Bh); free(Mr); free(acc); free(cu); free(cv);
+  free(Ah); free(Bh); free(Mr); free(acc); free(cu); free(cv); free(rs); free(cs);
   return 0;
 }
 
 /* Classical product at the same dtypes (the control): operands rounded to the product
- * dtype (after a per-tensor power-of-two scale in scale_mode 1), fp64 accumulation,
- * one rounding to the output dtype.                                                */
+ * dtype (after a per-tensor power-of-two scale in scale_mode 1, or per-row / per-column
+ * scales max|x| / 448 in scale_mode 2), fp64 accumulation, one rounding to the output dtype. */
 int orc_classical_gemm(int64_t M, int64_t K, int64_t N, const double* A, const double* B,
                        int pd, int od, int scale_mode, double* C) {
   double* Ah = (double*)malloc(sizeof(double) * M * K);
   double* Bh = (double*)malloc(sizeof(double) * K * N);
   double* acc = (double*)malloc(sizeof(double) * M * N);
   double sa = 1.0, sb = 1.0;
+  if (scale_mode == 2) {
+    double* rs = (double*)malloc(sizeof(double) * M);
+    double* cs = (double*)malloc(sizeof(double) * N);
+    for (int64_t p = 0; p < M; ++p) {
+      float amax = 0.0f;
+      for (int64_t t = 0; t < K; ++t) { float a = fabsf((float)A[p * K + t]); if (a > amax) amax = a; }
+      float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+      rs[p] = (double)d;
+      for (int64_t t = 0; t < K; ++t) Ah[p * K + t] = orc_round((double)((float)A[p * K + t] / d), pd);
+    }
+    for (int64_t c = 0; c < N; ++c) {
+      float amax = 0.0f;
+      for (int64_t t = 0; t < K; ++t) { float a = fabsf((float)B[t * N + c]); if (a > amax) amax = a; }
+      float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+      cs[c] = (double)d;
+      for (int64_t t = 0; t < K; ++t) Bh[t * N + c] = orc_round((double)((float)B[t * N + c] / d), pd);
+    }
+    matmul_f64(Ah, Bh, acc, M, K, N);
+    for (int64_t p = 0; p < M; ++p)
+      for (int64_t q = 0; q < N; ++q) C[p * N + q] = orc_round((acc[p * N + q] * rs[p]) * cs[q], od);
+    free(rs); free(cs); free(Ah); free(Bh); free(acc);
+    return 0;
+  }
   if (scale_mode == 1) { sa = pow2_scale_448(A, M * K); sb = pow2_scale_448(B, K * N); }
   for (int64_t x = 0; x < M * K; ++x) Ah[x] = orc_round(A[x] / sa, pd);
   for (int64_t x = 0; x < K * N; ++x) Bh[x] = orc_round(B[x] / sb, pd);

@@ -25,7 +25,7 @@ F32, BF16, E4M3, F64 = 0, 1, 2, 3
 _FMT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3, "f64": F64, "fp64": F64}
 
 __all__ = [
-    "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "round_to", "strassen",
+    "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "set_num_threads", "round_to", "strassen",
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
     "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "certificate",
@@ -51,6 +51,7 @@ def _L():
         dp = C.POINTER(C.c_double)
         i64 = C.c_int64
         lib.orc_num_threads.restype = C.c_int
+        lib.orc_set_num_threads.argtypes = [C.c_int]
         lib.orc_round.restype = C.c_double
         lib.orc_round.argtypes = [C.c_double, C.c_int]
         lib.orc_round_array.argtypes = [dp, dp, i64, C.c_int]
@@ -91,6 +92,11 @@ def _fmt(f):
 
 def num_threads() -> int:
     return int(_L().orc_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    """Threads of the oracle's OpenMP loops (results do not depend on it)."""
+    _L().orc_set_num_threads(int(n))
 
 
 def round_to(x, fmt):
@@ -227,7 +233,7 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
     if parts:
         bm, bk, bn = M // m, K // k, N // n
         Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
-        sA = np.empty(R); sB = np.empty(R)
+        sA = np.empty((R, bm) if scale_mode == 2 else R); sB = np.empty((R, bn) if scale_mode == 2 else R)
     rc = _L().orc_scheme_gemm(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
                               _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
                               _p(sB), _p(Mr))
