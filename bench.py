@@ -453,6 +453,10 @@ def run_workload(args):
         shapes = [(5120, 15360), (5120, 27648), (13824, 5120)]
         out["gemms"] = [one_gemm("strassen444", 8192, K, N, "bf16", pd, "bf16", 1 if pd == "e4m3" else 0, "t3")
                         for pd in ("bf16", "e4m3") for K, N in shapes]
+    elif wl == "ensemble":
+        out.update(ensemble_workload(fmm, gen, torch))
+        print(json.dumps(out))
+        return
     elif wl == "int8":
         out.update(int8_workload(fmm, gen, torch, timed, peaks))
         print(json.dumps(out))
@@ -465,6 +469,44 @@ def run_workload(args):
     out["value"] = tot_f / tot_t / 1e9
     out["ms_total"] = tot_t
     print(json.dumps(out))
+
+
+def ensemble_workload(fmm, gen, torch, pairs: int = 200):
+    """The paper's synthetic sign-variant ensemble (Appendix B.1) through error_sweep: 512 sign variants of
+    two-level Strassen, 128 x 128 operands, e4m3 block sums with per-row / per-column scales, `pairs` operand pairs
+    from each of U[0,1] and U[-1,1]; spread of the variants' average errors and split-half correlation."""
+    import itertools
+    signs = [np.array((1.0,) + t) for t in itertools.product((1.0, -1.0), repeat=3)]   # d_1 = e_1 = f_1 = 1 (Section 2.1)
+    var = [(dd, ee, ff) for dd in signs for ee in signs for ff in signs]
+    P = np.stack([np.diag(v[0]) for v in var]); Q = np.stack([np.diag(v[1]) for v in var]); S = np.stack([np.diag(v[2]) for v in var])
+    s1 = fmm.scheme_builtin("strassen222")
+    s2 = fmm.scheme_kron(s1, s1)
+    d = fmm.GemmDesc.make(128, 128, 128, "f32", "e4m3", "f32", scale_mode=2)
+    ws = torch.empty(fmm.error_sweep_workspace(s2, d, len(var)), dtype=torch.uint8, device="cuda")
+    res = {}
+    t_total = 0.0
+    for name, lo, seed in (("uniform_01", 0.0, 71), ("uniform_pm1", -1.0, 72)):
+        errs = np.empty((len(var), pairs))
+        ops = []
+        for p in range(pairs):
+            A = gen.to_storage(gen.uniform(seed + 100 * p, 1, (128, 128), lo, 1.0), "f32")[0].cuda()
+            B = gen.to_storage(gen.uniform(seed + 100 * p, 2, (128, 128), lo, 1.0), "f32")[0].cuda()
+            ops.append((A, B))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for p, (A, B) in enumerate(ops):
+            ratios, summ = fmm.error_sweep(s2, 0, P, Q, S, d, A, B, ws)
+            errs[:, p] = ratios * summ["e_classical_rel"]
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        t_total += dt
+        avg = errs.mean(axis=1)
+        res[name] = {"spread": float(avg.max() / avg.min()),
+                     "split_half_correlation": float(np.corrcoef(errs[:, 0::2].mean(axis=1), errs[:, 1::2].mean(axis=1))[0, 1]),
+                     "mean_rel_error": float(avg.mean()), "seconds": dt, "realisations_per_s": len(var) * pairs / dt}
+    return {"metric": "realisations_per_s", "unit": "1/s", "value": 2 * len(var) * pairs / t_total, "pairs": pairs,
+            "variants": len(var), "ensemble": res, "paper": {"uniform_01": [2.59, 0.9997], "uniform_pm1": [1.005, 0.121]},
+            "note": "host wall clock around error_sweep calls (each synchronises once); a latency-bound workload of 128^3 problems"}
 
 
 def int8_workload(fmm, gen, torch, timed, peaks):
@@ -519,7 +561,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=32, help="gauges per rank in the c3 sweep (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c5 | int8")
+    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c5 | int8 | ensemble")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

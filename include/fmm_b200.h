@@ -84,7 +84,12 @@ typedef struct {
                                  (K contiguous, the nn.Linear weight layout) */
   int32_t scale_mode;    /* 0: no scales.  1 (e4m3 only): one power-of-two scale per encoded
                             tensor, s = 2^ceil(log2(amax/448)), s = 1 for an all-zero tensor;
-                            classical_gemm uses one such scale per operand */
+                            classical_gemm uses one such scale per operand.
+                            2 (e4m3 only): the simplified synthetic schedule of Appendix B.1, one
+                            scale per row of each block sum of A and per column of each block sum of
+                            B, s = amax / 448 in fp32 (1 for an all-zero row), code = x / s in fp32,
+                            then rounded; each product is stored as (M_r * s_row) * s_col.  In the
+                            workspace the scales are then [R][M/m] and [R][N/n] arrays */
   int32_t flags;         /* FMM_FLAG_* */
 } fmm_gemm_desc;
 

@@ -101,7 +101,7 @@ fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
   if (d->storage != FMM_F32 && d->storage != FMM_BF16) return FMM_ERR_DTYPE;
   if (d->product != FMM_BF16 && d->product != FMM_E4M3) return FMM_ERR_DTYPE;
   if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
-  if (d->scale_mode != 0 && !(d->scale_mode == 1 && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
+  if (d->scale_mode != 0 && !((d->scale_mode == 1 || d->scale_mode == 2) && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
   if (d->M % m || d->K % k || d->N % n) return FMM_ERR_SHAPE;
   if ((d->K / k) % 16 || (d->N / n) % 8) return FMM_ERR_SHAPE;
   const int es = esize(d->storage), eo = esize(d->output);
@@ -120,10 +120,12 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.tabA = o; o += align_up(sizeof(CoefTable));
   L.tabB = o; o += align_up(sizeof(CoefTable));
   L.tabW = o; o += align_up(sizeof(CoefTable));
-  L.amaxA = o; o += align_up(FMM_MAX_R * 4);
-  L.amaxB = o; o += align_up(FMM_MAX_R * 4);
-  L.sA = o; o += align_up(FMM_MAX_R * 4);
-  L.sB = o; o += align_up(FMM_MAX_R * 4);
+  // scale_mode 2 keeps one amax / scale per row of every block sum: [R][bm] and [R][bn]
+  const size_t nsa = d->scale_mode == 2 ? (size_t)R * bm : FMM_MAX_R, nsb = d->scale_mode == 2 ? (size_t)R * bn : FMM_MAX_R;
+  L.amaxA = o; o += align_up(nsa * 4);
+  L.amaxB = o; o += align_up(nsb * 4);
+  L.sA = o; o += align_up(nsa * 4);
+  L.sB = o; o += align_up(nsb * 4);
   L.n_partials = std::max(decode_grid(bm, bn), kMaxStreamPartials);
   L.partials = o; o += align_up((size_t)L.n_partials * 8 * 2);
   L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
@@ -150,12 +152,13 @@ T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws)
 fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
                           const CoefTable* d_tab, const CoefTable* h_tab, void* hat, int64_t hat_stride, unsigned* amax,
                           float* scale, cudaStream_t st) {
-  const bool scaled = d->scale_mode == 1;
-  if (scaled) {
-    FMM_CUDA(cudaMemsetAsync(amax, 0, FMM_MAX_R * 4, st));
-    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, true, true, st));
+  const int mode = d->scale_mode;   // 0 none, 1 one power-of-two scale per encoded tensor, 2 one scale per row of it
+  if (mode != 0) {
+    const size_t n_amax = mode == 2 ? (size_t)h_tab->R * br : FMM_MAX_R;
+    FMM_CUDA(cudaMemsetAsync(amax, 0, n_amax * 4, st));
+    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, true, mode, st));
   }
-  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, false, scaled, st));
+  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, false, mode, st));
   return FMM_OK;
 }
 
@@ -167,8 +170,8 @@ struct SchemeRun {
   void* ws;
   const CoefTable *hA, *hB, *hW;   // host tables (list lengths size the kernels' shared memory)
   const CoefTable *dA, *dB, *dW;   // device copies
-  float* sA() const { return d->scale_mode == 1 ? at<float>(ws, L.sA) : nullptr; }
-  float* sB() const { return d->scale_mode == 1 ? at<float>(ws, L.sB) : nullptr; }
+  float* sA() const { return d->scale_mode != 0 ? at<float>(ws, L.sA) : nullptr; }
+  float* sB() const { return d->scale_mode != 0 ? at<float>(ws, L.sB) : nullptr; }
 };
 
 fmm_status stage_encode_a(const SchemeRun& r, const void* A, cudaStream_t st) {
@@ -192,6 +195,10 @@ fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   g.B = at<char>(r.ws, r.L.bhat); g.ldb = bk; g.b_batch = r.L.sBhat;
   g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = s->R;
   g.out = at<char>(r.ws, r.L.prod); g.ldo = bn; g.o_batch = r.L.sProd; g.out_mode = 0; g.output = FMM_F32;
+  if (r.d->scale_mode == 2) {   // row / column scales are folded into the stored products
+    g.row_scale = r.sA(); g.rs_batch = bm;
+    g.col_scale = r.sB(); g.cs_batch = bn;
+  }
   g.status = at<DeviceStatus>(r.ws, r.L.status);
   ProfScope ps(2, st);
   return launch_block_products(g, st);
@@ -201,7 +208,9 @@ fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, doubl
   const fmm_scheme* s = r.s;
   ProfScope ps(3, st);
   int np = 0;
-  FMM_CUDA(launch_decode(r.d->output, at<float>(r.ws, r.L.prod), r.L.sProd, r.dW, r.hW, s->R, r.sA(), r.sB(), s->m, s->n,
+  const bool per_product = r.d->scale_mode == 1;   // mode 2: the products already carry their scales
+  FMM_CUDA(launch_decode(r.d->output, at<float>(r.ws, r.L.prod), r.L.sProd, r.dW, r.hW, s->R, per_product ? r.sA() : nullptr,
+                         per_product ? r.sB() : nullptr, s->m, s->n,
                          r.d->M / s->m, r.d->N / s->n, C, r.d->ldc, cstar32, at<double>(r.ws, r.L.partials), &np, st));
   if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(r.ws, r.L.partials), np, err_out, st));
   return FMM_OK;
@@ -273,10 +282,11 @@ ClassicalLayout classical_layout(const fmm_gemm_desc* d) {
   size_t o = 0;
   L.status = o; o += align_up(sizeof(DeviceStatus));
   L.tab = o; o += align_up(sizeof(CoefTable));
-  L.amaxA = o; o += align_up(FMM_MAX_R * 4);
-  L.amaxB = o; o += align_up(FMM_MAX_R * 4);
-  L.sA = o; o += align_up(FMM_MAX_R * 4);
-  L.sB = o; o += align_up(FMM_MAX_R * 4);
+  const size_t nsa = d->scale_mode == 2 ? (size_t)d->M : FMM_MAX_R, nsb = d->scale_mode == 2 ? (size_t)d->N : FMM_MAX_R;
+  L.amaxA = o; o += align_up(nsa * 4);
+  L.amaxB = o; o += align_up(nsb * 4);
+  L.sA = o; o += align_up(nsa * 4);
+  L.sB = o; o += align_up(nsb * 4);
   L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
   L.ahat = o; o += L.direct ? 0 : align_up((size_t)d->M * d->K * ep);
   L.bhat = o; o += L.direct ? 0 : align_up((size_t)d->N * d->K * ep);
@@ -302,7 +312,7 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     std::memset(&t, 0, sizeof(t));
     fmm_build_tables(one, &t, nullptr, nullptr);
     FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tab), &t, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
-    const bool scaled = d->scale_mode == 1;
+    const bool scaled = d->scale_mode != 0;
     float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
     float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
     ProfScope pe(5, st);
@@ -312,7 +322,8 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
                            d->N * d->K, at<unsigned>(ws, L.amaxB), sB, st));
     g.A = at<char>(ws, L.ahat); g.lda = d->K; g.a_batch = 0;
     g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
-    g.sA = sA; g.sB = sB;
+    if (d->scale_mode == 2) { g.row_scale = sA; g.col_scale = sB; g.rs_batch = 0; g.cs_batch = 0; }
+    else { g.sA = sA; g.sB = sB; }
   }
   ProfScope ps(4, st);
   return launch_block_products(g, st);

@@ -215,6 +215,20 @@ struct SmemLayout {
   static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;  // + alignment slack
 };
 
+// acc -> (acc * row factor) * column factor for the 32 columns starting at col0 (columns come in multiples of 4)
+__device__ __forceinline__ void apply_row_col_scale(uint32_t (&v)[32], float rs, const float* __restrict__ cs, int ncols) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    if (4 * q < ncols) {
+      const float4 c = *reinterpret_cast<const float4*>(cs + 4 * q);
+      v[4 * q + 0] = __float_as_uint(__fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 0]), rs), c.x));
+      v[4 * q + 1] = __float_as_uint(__fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 1]), rs), c.y));
+      v[4 * q + 2] = __float_as_uint(__fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), rs), c.z));
+      v[4 * q + 3] = __float_as_uint(__fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), rs), c.w));
+    }
+  }
+}
+
 struct TileParams {
   int rows_a, rows_b;       // extents of one batch entry
   int kbytes;               // inner extent in bytes
@@ -226,6 +240,9 @@ struct TileParams {
   int out_mode;             // 0: fp32 products; 1: scaled + rounded result
   int out_bf16;             // out_mode 1: 1 -> bf16, 0 -> fp32
   int wide;                 // every output row starts on a 32-byte boundary
+  const float* row_scale;   // optional factors of the accumulator: per output row and per output column
+  const float* col_scale;
+  long long rs_batch, cs_batch;
   int selftest_no_producer; // failure-reporting self-test: the TMA producer issues nothing
   unsigned long long wait_limit_ns;   // bound of every mbarrier wait
 };
@@ -381,8 +398,12 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         tc_ld32(taddr, v);
         tc_wait_ld();
         const int col0 = tn * BN + c * 32;
-        if (row_ok && col0 < tp.rows_b)
+        if (row_ok && col0 < tp.rows_b) {
+          if (tp.row_scale != nullptr)
+            apply_row_col_scale(v, tp.row_scale[(long long)r * tp.rs_batch + row],
+                                tp.col_scale + (long long)r * tp.cs_batch + col0, min(32, tp.rows_b - col0));
           store_row_chunk(out, row_off + col0, min(32, tp.rows_b - col0), v, tp.out_mode, tp.out_bf16, alpha, tp.wide != 0);
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -611,8 +632,12 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
         tc_ld32(taddr, v);
         tc_wait_ld();
         const int col0 = tn * BN + c * 32;
-        if (row_ok && col0 < tp.rows_b)
+        if (row_ok && col0 < tp.rows_b) {
+          if (tp.row_scale != nullptr)
+            apply_row_col_scale(v, tp.row_scale[(long long)r * tp.rs_batch + row],
+                                tp.col_scale + (long long)r * tp.cs_batch + col0, min(32, tp.rows_b - col0));
           store_row_chunk(out, row_off + col0, min(32, tp.rows_b - col0), v, tp.out_mode, tp.out_bf16, alpha, tp.wide != 0);
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -698,6 +723,7 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
   tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
   tp.wide = rows_32b_aligned(a);
+  tp.row_scale = a.row_scale; tp.col_scale = a.col_scale; tp.rs_batch = a.rs_batch; tp.cs_batch = a.cs_batch;
   tp.selftest_no_producer = a.selftest_no_producer;
   tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
   const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches * tp.groups;
@@ -730,6 +756,7 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   tp.ldo = a.ldo; tp.o_batch = a.o_batch;
   tp.out_mode = a.out_mode; tp.out_bf16 = (a.output == FMM_BF16);
   tp.wide = rows_32b_aligned(a);
+  tp.row_scale = a.row_scale; tp.col_scale = a.col_scale; tp.rs_batch = a.rs_batch; tp.cs_batch = a.cs_batch;
   tp.selftest_no_producer = a.selftest_no_producer;
   tp.wait_limit_ns = a.wait_limit_ns ? a.wait_limit_ns : kDefaultWaitLimitNs;
   const long long total = (long long)tp.tiles_m * tp.tiles_n * tp.batches * tp.groups;

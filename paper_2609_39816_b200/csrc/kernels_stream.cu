@@ -153,13 +153,13 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     ent[i] = make_int2(d_tab->cell[i] * kSlab, __float_as_int(d_tab->coef[i]));
   if (threadIdx.x < R) {
     float s = 1.0f;
-    if (!kAmaxOnly && use_scale) s = pow2_scale_448(__uint_as_float(amax_bits[threadIdx.x]));
+    if (!kAmaxOnly && use_scale == 1) s = pow2_scale_448(__uint_as_float(amax_bits[threadIdx.x]));
     sm.scale[threadIdx.x] = s;
     const float inv = 1.0f / s;
     sm.use_mul[threadIdx.x] = (isfinite(inv) && inv * s == 1.0f && fabsf(inv) >= 1.17549435e-38f);
     sm.inv_scale[threadIdx.x] = inv;
     sm.amax[threadIdx.x] = 0u;
-    if (!kAmaxOnly && use_scale && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
+    if (!kAmaxOnly && use_scale == 1 && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
   }
 
   const int g = threadIdx.x / kEncPos;           // which share of the cells / products this thread handles
@@ -266,11 +266,29 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
           float a = 0.0f;
 #pragma unroll
           for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[j][i].x), fabsf(acc[j][i].y)));   // fmaxf drops NaN
+          if (use_scale == 2) {
+            // one scale per row of the block sum: largest magnitude of row p of product r
+            if ((vec_per_row & 31) == 0) {       // a warp's 32 consecutive vectors lie in one row
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+              if ((threadIdx.x & 31) == 0 && live && a > 0.0f) atomicMax(&amax_bits[(int64_t)r * br + p], __float_as_uint(a));
+            } else if (live && a > 0.0f) {
+              atomicMax(&amax_bits[(int64_t)r * br + p], __float_as_uint(a));
+            }
+            continue;
+          }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
           if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
         } else if (live) {
-          if (use_scale) {
+          if (use_scale == 2) {
+            // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
+            const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
+            const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { acc[j][i].x = __fdiv_rn(acc[j][i].x, sc); acc[j][i].y = __fdiv_rn(acc[j][i].y, sc); }
+            if (t == 0 && scale_out) scale_out[(int64_t)r * br + p] = sc;
+          } else if (use_scale) {
             if (sm.use_mul[r]) {
               const float inv = sm.inv_scale[r];
 #pragma unroll
@@ -286,7 +304,7 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
       }
     }
   }
-  if (kAmaxOnly) {
+  if (kAmaxOnly && use_scale != 2) {
     __syncthreads();
     if (threadIdx.x < R && sm.amax[threadIdx.x] != 0u) atomicMax(&amax_bits[threadIdx.x], sm.amax[threadIdx.x]);
   }
@@ -306,7 +324,7 @@ static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists 
 template <typename SrcT, typename DstT, int kSplit>
 cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
                             const CoefTable* d_tab, int padded, int lists, void* out, int64_t out_stride,
-                            unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+                            unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kSplit;
   const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
@@ -589,7 +607,7 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 template <int kSplit>
 static cudaError_t launch_encode_split(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                                        int64_t bc, const CoefTable* d_tab, int nnz, int lists, void* out, int64_t out_stride,
-                                       unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+                                       unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
   if (storage == FMM_F32 && product == FMM_BF16)
     return launch_encode_t<float, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
@@ -603,7 +621,7 @@ static cudaError_t launch_encode_split(int storage, int product, const void* X, 
 
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
-                          unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st) {
+                          unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   // small schemes (at most 4 cells): one thread per position vector; otherwise four threads share one
   if (gr * gc <= 4)

@@ -16,12 +16,13 @@ int64_t& fmm_launch_counter();
 // X: source matrix (storage dtype), rows x cols with leading dimension ldx, split into a gr x gc grid of
 // br x bc blocks.  out: R blocks [br][bc] in the product dtype, out_stride elements apart.  With amax_only the kernel only accumulates
 // max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).
-// With use_scale, scale[r] is derived from amax_bits[r] (2^ceil(log2(amax/448)), 1 if amax==0),
-// written to scale[R] and divided out before rounding.
+// With use_scale == 1, scale[r] is derived from amax_bits[r] (2^ceil(log2(amax/448)), 1 if amax==0),
+// written to scale[R] and divided out before rounding.  With use_scale == 2 there is one scale per row of every
+// block sum: amax_bits and scale are [R][br]; scale = amax / 448 in fp32 (1 for an all-zero row).
 // h_tab = host copy of the same table (its list lengths size the kernel's shared memory).
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
-                          unsigned* amax_bits, float* scale, bool amax_only, bool use_scale, cudaStream_t st);
+                          unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st);
 
 // Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
@@ -68,6 +69,9 @@ struct BlockProductArgs {
                              // multiplies group g of A_r with group g of B_r and lands at out + (r*groups + g)*o_batch
   void* out; int64_t ldo; int64_t o_batch; int out_mode; int output;
   const float* sA; const float* sB;
+  // optional per-row / per-column factors applied to the fp32 accumulator before it is stored:
+  // out[r][row][col] = (acc * row_scale[r*rs_batch + row]) * col_scale[r*cs_batch + col]   (null: none)
+  const float* row_scale; const float* col_scale; int64_t rs_batch, cs_batch;
   DeviceStatus* status;
   int selftest_no_producer;            // 1: the producer issues no copies (failure-reporting self-test)
   unsigned long long wait_limit_ns;    // 0: default (2 s)

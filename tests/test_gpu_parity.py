@@ -34,6 +34,9 @@ def _inputs(seed, M, K, N, S, kind="normal", bound=None):
         A, B = gen.integer_matrix(seed, 1, (M, K), bound), gen.integer_matrix(seed, 2, (K, N), bound)
     elif kind == "llm":
         A, B = gen.activations_outlier(seed, 1, M, K, frac=0.01, factor=100.0), gen.weights(seed, 2, K, N)
+    elif kind in ("u01", "upm1"):
+        lo = 0.0 if kind == "u01" else -1.0
+        A, B = gen.uniform(seed, 1, (M, K), lo, 1.0), gen.uniform(seed, 2, (K, N), lo, 1.0)
     elif kind == "t3":
         A = gen.activations_outlier(seed, 1, M, K, dist="t3", frac=0.001, factor=300.0, at_least=1)
         B = gen.weights(seed, 2, K, N)
@@ -54,6 +57,9 @@ def _inputs(seed, M, K, N, S, kind="normal", bound=None):
     ("strassen222", 256, 2240, 272, "bf16", "e4m3", "f32", "llm", 1),       # fp8, K tail inside a stage
     ("strassen444", 64, 64, 32, "f32", "bf16", "f32", "normal", 0),         # smallest legal blocks
     ("strassen444", 256, 11008, 512, "bf16", "e4m3", "bf16", "t3", 1),      # config-4 down-projection K: K/4 = 2752 = 21.5 stages
+    ("strassen444", 128, 128, 128, "f32", "e4m3", "f32", "u01", 2),         # the ensemble's shape: row / column scales
+    ("strassen444", 512, 1024, 544, "bf16", "e4m3", "bf16", "t3", 2),       # row / column scales, several tiles, CTA pairs
+    ("strassen222", 200, 2240, 272, "bf16", "e4m3", "f32", "llm", 2),       # rows of 280 vectors: per-thread amax path
 ])
 def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     At, Bt, A64, B64 = _inputs(3, M, K, N, S, kind)
@@ -156,6 +162,8 @@ def test_row_leak_pattern_on_gpu(lib):
     (512, 1024, 768, "bf16", "bf16", "bf16", 0, True),     # direct path, weight layout
     (256, 256, 256, "f32", "bf16", "f32", 0, False),       # conversion pass fp32 -> bf16
     (384, 2240, 264, "bf16", "e4m3", "bf16", 1, False),    # fp8 with per-tensor scales
+    (384, 2240, 264, "bf16", "e4m3", "f32", 2, False),     # fp8 with per-row / per-column scales
+    (128, 128, 128, "f32", "e4m3", "f32", 2, True),
 ])
 def test_classical_and_exact_match_oracle(lib, M, K, N, S, Pd, O, scale, wl):
     At, Bt, A64, B64 = _inputs(9, M, K, N, S, "llm")
@@ -289,3 +297,33 @@ def test_bounded_wait_expires_reports_timeout_and_context_survives(lib):
     At, Bt, A64, B64 = _inputs(13, 256, 256, 256, "bf16", "int", 3)
     C = gu.run_scheme_gemm(lib.scheme_builtin("strassen222"), At, Bt, "bf16", "bf16", "f32")
     assert np.array_equal(C, A64 @ B64)
+
+
+def test_sign_variant_ensemble_on_the_device(lib):
+    """Appendix B.1: all 512 sign variants of two-level Strassen on synthetic 128 x 128 operands, e4m3 block sums
+    with one scale per row / column, through error_sweep.  Per-variant errors agree with the oracle on a sample;
+    the ensemble statistics land where the paper prints them (2.59 / 0.9997 on U[0,1], 1.005 / 0.121 on U[-1,1])."""
+    var = oracle.sign_variants(4, 4, 4)
+    P = np.stack([np.diag(v[0]) for v in var]); Q = np.stack([np.diag(v[1]) for v in var]); S = np.stack([np.diag(v[2]) for v in var])
+    s2, o2 = lib.scheme_builtin("strassen444"), gu.oracle_scheme("strassen444")
+    d = lib.GemmDesc.make(128, 128, 128, "f32", "e4m3", "f32", scale_mode=2)
+    ws = gu.workspace(lib.error_sweep_workspace(s2, d, len(var)))
+    pairs = 24
+    stats = {}
+    for kind, seed in (("u01", 71), ("upm1", 72)):
+        errs = np.empty((len(var), pairs))
+        for p in range(pairs):
+            At, Bt, A64, B64 = _inputs(seed + 100 * p, 128, 128, 128, "f32", kind)
+            ratios, summ = lib.error_sweep(s2, 0, P, Q, S, d, At, Bt, ws)
+            errs[:, p] = ratios * summ["e_classical_rel"]
+            if p == 0:       # parity of a sample of variants against the oracle
+                Cs = A64 @ B64
+                Ecl = oracle.rel_error(oracle.classical_gemm(A64, B64, "e4m3", "f32", 2), Cs)
+                assert math.isclose(summ["e_classical_rel"], Ecl, rel_tol=TOL_RATIO)
+                for vi in range(0, len(var), 57):
+                    E = oracle.rel_error(oracle.scheme_gemm(oracle.sign_variant(o2, *var[vi]), A64, B64, "e4m3", "f32", 2), Cs)
+                    assert abs(errs[vi, 0] - E) <= TOL_RATIO * E
+        avg = errs.mean(axis=1)
+        stats[kind] = (avg.max() / avg.min(), float(np.corrcoef(errs[:, 0::2].mean(axis=1), errs[:, 1::2].mean(axis=1))[0, 1]))
+    assert abs(stats["u01"][0] - 2.59) < 0.12 * 2.59 and stats["u01"][1] > 0.99, stats
+    assert 1.0 <= stats["upm1"][0] < 1.03 and abs(stats["upm1"][1]) < 0.6, stats
