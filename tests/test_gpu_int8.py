@@ -146,3 +146,29 @@ def test_row_locality_on_device():
         moved += sum(int(np.any(out[e] != base[e])) for e in range(later))
         assert np.any(out[later] != base[later])
     assert moved == 0
+
+
+def test_fp8_schedule_moves_the_48_same_offset_pairs_on_device():
+    """The FP8 counterpart (Section 4.2): block sums rounded before multiplying move exactly the 48 of 496 row pairs
+    that share an offset in their blocks, with or without row-owned scales; the classical product moves none."""
+    import gpu_util as gu
+    lib = fmm()
+    s2 = lib.scheme_builtin("strassen444")
+    At, A = gen.to_storage(gen.normal(6, 1, (32, 128)), "f32")
+    Bt, B = gen.to_storage(gen.normal(6, 2, (128, 32)), "f32")
+    At, Bt = At.cuda(), Bt.cuda()
+    want = {(e, l) for l in range(32) for e in range(l) if e % 8 == l % 8}
+
+    def moved(run):
+        base = run(At)
+        out_set = set()
+        for later in range(32):
+            A2 = At.clone()
+            A2[later] = gen.to_storage(gen.normal(77, 900 + later, (128,)), "f32")[0].cuda()
+            out = run(A2)
+            out_set |= {(e, later) for e in range(later) if np.any(out[e] != base[e])}
+        return out_set
+
+    for mode in (0, 2):
+        assert moved(lambda X: gu.run_scheme_gemm(s2, X, Bt, "f32", "e4m3", "f32", scale_mode=mode)) == want
+    assert moved(lambda X: gu.run_classical(X, Bt, "f32", "e4m3", "f32", scale_mode=2)) == set()

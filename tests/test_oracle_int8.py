@@ -102,3 +102,48 @@ def test_bound_is_sharp_and_violations_are_reported():
     with pytest.raises(ValueError):
         P = gen.gauge_cond_limited(1, 0, 2)
         oracle.int8_certified(oracle.gauge(S1, P, P, P), cA[:2], one[:2], cB[:2], one[:2])
+
+
+def _pairs_moved(run, A, rows=32):
+    base = run(A)
+    moved = set()
+    for later in range(rows):
+        A2 = A.copy()
+        A2[later] = gen.to_storage(gen.normal(77, 900 + later, (A.shape[1],)), "f32")[1]
+        out = run(A2)
+        for earlier in range(later):
+            if np.any(out[earlier] != base[earlier]):
+                moved.add((earlier, later))
+    return moved
+
+
+def test_fp8_schedule_moves_exactly_the_48_same_offset_pairs():
+    """Section 4.2: the same coefficients under an FP8 schedule that rounds the block sums before multiplying move
+    48 of the 496 (earlier, later) row pairs — exactly those whose rows share an offset in their blocks (32 rows in
+    four blocks of 8: 8 offsets x C(4,2) pairs).  Row-owned scales (one per row of each block sum) keep it at 48;
+    the classical product at the same dtype moves none."""
+    A = gen.to_storage(gen.normal(6, 1, (32, 128)), "f32")[1]
+    B = gen.to_storage(gen.normal(6, 2, (128, 32)), "f32")[1]
+    want = {(e, l) for l in range(32) for e in range(l) if e % 8 == l % 8}
+    assert len(want) == 48
+    for mode in (0, 2):
+        moved = _pairs_moved(lambda X: oracle.scheme_gemm(S2, X, B, "e4m3", "f32", scale_mode=mode), A)
+        assert moved == want, (mode, len(moved))
+    assert _pairs_moved(lambda X: oracle.classical_gemm(X, B, "e4m3", "f32", 2), A) == set()
+
+
+def test_fp8_block_sums_leave_no_sign_variant_exact_on_integer_codes():
+    """Section 4.2: on a tile of integer codes every sign variant gives the one exact integer product, but with the
+    block sums rounded to e4m3 (4 significant bits: sums up to 124 are not representable) none of the 512 does,
+    and their largest errors differ severalfold (the paper's tile: 3.17x)."""
+    cA = gen.integer_matrix(8, 1, (32, 128), 31)
+    cB = gen.integer_matrix(8, 2, (128, 32), 31)
+    exact = cA @ cB
+    worst = []
+    for d, e, f in oracle.sign_variants(4, 4, 4):
+        sv = oracle.sign_variant(S2, d, e, f)
+        worst.append(np.abs(oracle.scheme_gemm(sv, cA, cB, "e4m3", "f32") - exact).max())
+    worst = np.array(worst)
+    assert np.all(worst > 0)
+    assert 1.5 < worst.max() / worst.min() < 8.0
+    assert np.array_equal(oracle.scheme_gemm(S2, cA, cB, "f64", "f64"), exact)
