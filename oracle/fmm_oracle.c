@@ -642,3 +642,97 @@ int orc_certificate(int m, int k, int n, int R, const double* U, const double* V
   if (cert) { cert[0] = a; cert[1] = b; cert[2] = big; cert[3] = one_group; }
   return a <= 127.0 && b <= 127.0 && big < ldexp(1.0, acc_bits) && one_group;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Full-range codes with an overflow correction (Section 4.3, Eq. 2; certificate in */
+/* Appendix D).                                                                   */
+/* ------------------------------------------------------------------------- */
+
+/* floor((x + 128) / 256) for any sign of x */
+static int64_t split_high(int64_t x) {
+  int64_t y = x + 128;
+  return y >= 0 ? y / 256 : -((-y + 255) / 256);
+}
+
+/* As orc_int8_certified, but every block sum of codes is split exactly, Ahat = A0 + 256 R_A with
+ * R_A = floor((Ahat + 128) / 256) and A0 in [-128, 127], likewise Bhat, and each block product is rebuilt from
+ * the four products of Eq. 2: A0 B0 + 256 (R_A B0 + A0 R_B) + 256^2 R_A R_B.  Arithmetic in 64-bit integers;
+ * maxabs reports what the certificate bounds: [0] max|A0|-like excess (largest value outside [-128,127] seen in
+ * A0 or B0, 0 if none), [1] max |R_A|, |R_B| (must be <= 2), [2] largest |partial sum| of the weighted terms
+ * inside one reconstructed product (bound h (128 + 512)^2), [3] largest |partial sum| of the combination (must be
+ * < 2^31), [4] largest |block sum| (L_A * 127 = 508 for two-level Strassen).                                   */
+int orc_int8_corrected(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                       const double* cA, const double* dA, const double* cB, const double* dB, int64_t M,
+                       int64_t K, int64_t N, int g, int od, double* out, double* Pout, double* maxabs) {
+  if (M % m || N % n || g % k || K % g) return 1;
+  for (int x = 0; x < R * m * k; ++x) if (U[x] != rint(U[x])) return 1;
+  for (int x = 0; x < R * k * n; ++x) if (V[x] != rint(V[x])) return 1;
+  for (int x = 0; x < R * m * n; ++x) if (W[x] != rint(W[x])) return 1;
+  const int64_t G = K / g, bm = M / m, bn = N / n;
+  const int h = g / k;
+  double* P = Pout ? Pout : (double*)malloc(sizeof(double) * G * M * N);
+  int64_t* A0 = (int64_t*)malloc(sizeof(int64_t) * bm * h);
+  int64_t* RA = (int64_t*)malloc(sizeof(int64_t) * bm * h);
+  int64_t* B0 = (int64_t*)malloc(sizeof(int64_t) * bn * h);
+  int64_t* RB = (int64_t*)malloc(sizeof(int64_t) * bn * h);
+  int64_t* acc = (int64_t*)malloc(sizeof(int64_t) * M * N);
+  int64_t out_of_range = 0, mxR = 0, mxTerm = 0, mxComb = 0, mxSum = 0;
+  for (int64_t q = 0; q < G; ++q) {
+    for (int64_t x = 0; x < M * N; ++x) acc[x] = 0;
+    for (int r = 0; r < R; ++r) {
+      for (int64_t p = 0; p < bm; ++p)
+        for (int t = 0; t < h; ++t) {
+          int64_t s = 0;
+          for (int i = 0; i < m; ++i)
+            for (int l = 0; l < k; ++l)
+              s += (int64_t)U[(r * m + i) * k + l] * (int64_t)cA[(i * bm + p) * K + q * g + l * h + t];
+          if (llabs(s) > mxSum) mxSum = llabs(s);
+          int64_t hi = split_high(s), lo = s - 256 * hi;
+          A0[p * h + t] = lo; RA[p * h + t] = hi;
+          if (lo < -128 || lo > 127) out_of_range = llabs(lo);
+          if (llabs(hi) > mxR) mxR = llabs(hi);
+        }
+      for (int64_t c = 0; c < bn; ++c)
+        for (int t = 0; t < h; ++t) {
+          int64_t s = 0;
+          for (int l = 0; l < k; ++l)
+            for (int j = 0; j < n; ++j)
+              s += (int64_t)V[(r * k + l) * n + j] * (int64_t)cB[(j * bn + c) * K + q * g + l * h + t];
+          if (llabs(s) > mxSum) mxSum = llabs(s);
+          int64_t hi = split_high(s), lo = s - 256 * hi;
+          B0[c * h + t] = lo; RB[c * h + t] = hi;
+          if (lo < -128 || lo > 127) out_of_range = llabs(lo);
+          if (llabs(hi) > mxR) mxR = llabs(hi);
+        }
+      for (int64_t p = 0; p < bm; ++p)
+        for (int64_t c = 0; c < bn; ++c) {
+          /* the four products of Eq. 2, each on int8 multiplicands, then the weighted recombination */
+          int64_t p00 = 0, p10 = 0, p01 = 0, p11 = 0, absum = 0;
+          for (int t = 0; t < h; ++t) {
+            int64_t a0 = A0[p * h + t], ra = RA[p * h + t], b0 = B0[c * h + t], rb = RB[c * h + t];
+            p00 += a0 * b0; p10 += ra * b0; p01 += a0 * rb; p11 += ra * rb;
+            absum += llabs(a0 * b0) + 256 * (llabs(ra * b0) + llabs(a0 * rb)) + 65536 * llabs(ra * rb);
+          }
+          if (absum > mxTerm) mxTerm = absum;
+          int64_t s = p00 + 256 * (p10 + p01) + 65536 * p11;
+          for (int i = 0; i < m; ++i)
+            for (int j = 0; j < n; ++j) {
+              int64_t w = (int64_t)W[(r * m + i) * n + j];
+              if (w == 0) continue;
+              int64_t* dst = &acc[(i * bm + p) * N + j * bn + c];
+              *dst += w * s;
+              if (llabs(*dst) > mxComb) mxComb = llabs(*dst);
+            }
+        }
+    }
+    for (int64_t x = 0; x < M * N; ++x) P[q * M * N + x] = (double)acc[x];
+  }
+  int8_rescale(P, dA, dB, M, N, G, od, out);
+  if (maxabs) {
+    maxabs[0] = (double)out_of_range; maxabs[1] = (double)mxR; maxabs[2] = (double)mxTerm;
+    maxabs[3] = (double)mxComb; maxabs[4] = (double)mxSum;
+  }
+  free(A0); free(RA); free(B0); free(RB); free(acc);
+  if (!Pout) free(P);
+  return 0;
+}

@@ -28,7 +28,7 @@ __all__ = [
     "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "set_num_threads", "round_to", "strassen",
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
-    "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "certificate",
+    "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "certificate",
 ]
 
 
@@ -72,6 +72,8 @@ def _L():
         lib.orc_int8_classical.argtypes = [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 2
         lib.orc_int8_certified.restype = C.c_int
         lib.orc_int8_certified.argtypes = ([C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 3)
+        lib.orc_int8_corrected.restype = C.c_int
+        lib.orc_int8_corrected.argtypes = ([C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 3)
         lib.orc_certificate.restype = C.c_int
         lib.orc_certificate.argtypes = [C.c_int] * 4 + [dp] * 3 + [C.c_int] * 5 + [dp]
         _lib = lib
@@ -340,3 +342,21 @@ def certificate(s: "Scheme", bA: int, bB: int, h: int, g: int, acc_bits: int = 3
     c = np.zeros(4)
     ok = _L().orc_certificate(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), bA, bB, h, g, acc_bits, _p(c))
     return bool(ok), dict(LAbA=c[0], LBbB=c[1], largest=c[2], one_group=bool(c[3]))
+
+
+def int8_corrected(s: "Scheme", cA, dA, cB, dB, g: int = 128, od="bf16", products: bool = False):
+    """Section 4.3: the algorithm `s` per group with every block sum split as X0 + 256 R (X0 in int8) and each block
+    product rebuilt from the four products of Eq. 2.  Returns (out, maxabs[5]) or (out, maxabs, P); maxabs =
+    [excess of X0 over the int8 range, max |R|, largest sum of |terms| inside a rebuilt product, largest partial sum
+    of the combination, largest |block sum|]."""
+    m, k, n, R = s.dims
+    cA = _d(cA); cB = _d(cB); dA = _d(dA); dB = _d(dB)
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = np.empty((M, N)); mx = np.zeros(5)
+    P = np.empty((K // g, M, N)) if products else None
+    rc = _L().orc_int8_corrected(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), _p(cA), _p(dA), _p(cB), _p(dB),
+                                 M, K, N, g, _fmt(od), _p(out), _p(P), _p(mx))
+    if rc:
+        raise ValueError("shape does not divide, or coefficients are not integers")
+    return (out, mx, P) if products else (out, mx)

@@ -147,3 +147,34 @@ def test_fp8_block_sums_leave_no_sign_variant_exact_on_integer_codes():
     assert np.all(worst > 0)
     assert 1.5 < worst.max() / worst.min() < 8.0
     assert np.array_equal(oracle.scheme_gemm(S2, cA, cB, "f64", "f64"), exact)
+
+
+def test_overflow_correction_full_range_codes():
+    """Section 4.3 and its certificate: at code bound 127 the block sums reach L_A * 127 = 508, the split keeps
+    every multiplicand in int8 with |R| <= 2, the terms of a rebuilt product stay within h (128 + 512)^2 =
+    13,107,200, the combination within 16 times that (< 2^31), and the output is classical int8's bit for bit."""
+    A, Bt, cA, dA, cB, dB = _quantised(13, 32, 256, 32, 127)
+    ref, Pref = oracle.int8_classical(cA, dA, cB, dB, products=True)
+    for v in oracle.sign_variants(4, 4, 4)[::57]:
+        out, mx, P = oracle.int8_corrected(oracle.sign_variant(S2, *v), cA, dA, cB, dB, products=True)
+        assert np.array_equal(P, Pref) and np.array_equal(out, ref)
+        assert mx[0] == 0 and mx[1] <= 2 and mx[2] <= 32 * (128 + 512) ** 2 == 13107200
+        assert mx[3] <= 16 * 13107200 < 2 ** 31 and 127 < mx[4] <= 508
+    assert np.abs(Pref).max() <= 128 * 127 ** 2 == 2064512 < 2 ** 24
+    # the uncorrected call at this code bound has no certificate: block sums leave the int8 range
+    assert not oracle.certificate(S2, 127, 127, 32, 128, 31)[0]
+    _, mx_plain = oracle.int8_certified(S2, cA, dA, cB, dB)
+    assert mx_plain[0] > 127
+    # sign-aligned codes reach the bound 508 and the largest correction |R| = 2
+    cA2 = np.zeros((4, 128)); r = int(np.argmax(np.abs(S2.U).sum(axis=(1, 2))))
+    for i in range(4):
+        for l in range(4):
+            cA2[i, 32 * l:32 * l + 32] = 127 * np.sign(S2.U[r, i, l])
+    one = np.ones((4, 1))
+    cB2 = gen.integer_matrix(9, 2, (4, 128), 127)
+    outc, mx2, P2 = oracle.int8_corrected(S2, cA2, one, cB2, one, od="f32", products=True)
+    assert mx2[4] == 508 and mx2[1] == 2 and np.array_equal(P2[0], cA2 @ cB2.T)
+    # split identity on every residue: floor((x + 128) / 256), remainder in [-128, 127]
+    for x in range(-508, 509):
+        hi = (x + 128) // 256
+        assert -128 <= x - 256 * hi <= 127 and abs(hi) <= 2
