@@ -279,6 +279,26 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
                      const int8_t* d_cB, const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C,
                      int64_t ldc, void* d_ws, size_t ws_bytes, void* cuda_stream);
 
+/* ---- Full-range codes with an overflow correction (Section 4.3, Eq. 2; certificate in Appendix D) --------
+ *
+ * At code bound 127 the block sums of codes reach L_A * 127 (508 for two-level Strassen) and no longer fit the
+ * multiplier's range.  Each is split exactly, X = X0 + 256 R with R = floor((X + 128) / 256) and X0 in
+ * [-128, 127], and every block product is rebuilt from the four products of Eq. 2,
+ *     Ahat Bhat = A0 B0 + 256 (R_A B0 + A0 R_B) + 256^2 R_A R_B,
+ * here as one contraction over rows [A0 | 256 R_A | A0 | 256 R_A] and [B0 | B0 | 256 R_B | 256 R_B] (all entries
+ * exact in bf16).  Same operands, layouts, requirements and output as int8_gemm at code bound 127; the result is
+ * bit-identical to int8_gemm(NULL, 127, ...).  s must not be NULL.
+ *
+ * scheme_certificate_corrected: cert[4] (HOST, may be NULL) = {largest block sum L*127, largest |R|, bound
+ * h (128 + 256 |R|max)^2 on the summed magnitudes inside one rebuilt product, L_W times that}.  Returns 1 when
+ * the coefficients are integers, the third value is below 2^24 (fp32 accumulators), the fourth below 2^31 (int32
+ * combination) and k * h == 128; int8_gemm_corrected returns FMM_ERR_CERTIFICATE otherwise.               */
+int scheme_certificate_corrected(const fmm_scheme* s, int h, double cert[4]);
+size_t int8_gemm_corrected_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N);
+fmm_status int8_gemm_corrected(const fmm_scheme* s, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
+                               const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc,
+                               void* d_ws, size_t ws_bytes, void* cuda_stream);
+
 const char* fmm_status_string(fmm_status st);
 
 /* Number of kernels this library has launched in this process (for benchmarks' accounting). */

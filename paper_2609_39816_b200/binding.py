@@ -23,6 +23,7 @@ EXPORTED_SYMBOLS = [
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
+    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
 ]
@@ -99,6 +100,12 @@ _lib.int8_gemm_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
 _lib.int8_gemm_workspace.restype = _sz
 _lib.int8_gemm.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
                            _vp, _sz, _vp]
+_lib.scheme_certificate_corrected.argtypes = [_vp, C.c_int, _dp]
+_lib.scheme_certificate_corrected.restype = C.c_int
+_lib.int8_gemm_corrected_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
+_lib.int8_gemm_corrected_workspace.restype = _sz
+_lib.int8_gemm_corrected.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
+                                     _vp, _sz, _vp]
 _lib.error_sweep_workspace.argtypes = [_vp, C.POINTER(GemmDesc), C.c_int]
 _lib.error_sweep_workspace.restype = _sz
 _lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(GemmDesc), _vp, _vp, _vp, _dp,
@@ -281,6 +288,28 @@ def int8_gemm(s, code_bound: int, cA, dA, cB, dB, Cmat, ws) -> None:
     _check(_lib.int8_gemm(s.handle if s is not None else None, code_bound, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB), M, K, N,
                           out, _ptr(Cmat), Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "int8_gemm")
+
+
+def scheme_certificate_corrected(s, h: int):
+    """Certificate of the overflow-corrected computation (Section 4.3).  Returns (holds, dict)."""
+    c = np.zeros(4)
+    ok = _lib.scheme_certificate_corrected(s.handle, h, c.ctypes.data_as(_dp))
+    return bool(ok), dict(block_sum_max=c[0], r_max=c[1], product_terms=c[2], combination=c[3])
+
+
+def int8_gemm_corrected_workspace(s, M: int, K: int, N: int) -> int:
+    return int(_lib.int8_gemm_corrected_workspace(s.handle, M, K, N))
+
+
+def int8_gemm_corrected(s, cA, dA, cB, dB, Cmat, ws) -> None:
+    """The int8 operator at code bound 127 computed by `s` per group with the overflow correction of Eq. 2."""
+    import torch
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = F32 if Cmat.dtype == torch.float32 else BF16
+    _check(_lib.int8_gemm_corrected(s.handle, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB), M, K, N, out, _ptr(Cmat),
+                                    Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "int8_gemm_corrected")
 
 
 def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=None):

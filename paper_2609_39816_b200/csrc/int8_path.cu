@@ -134,7 +134,7 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
 }
 __device__ __forceinline__ void store4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
 
-template <typename OutT, int kSplit, int kStages, int kCells>
+template <typename OutT, int kSplit, int kStages, int kCells, bool kIntAcc>
 __global__ void __launch_bounds__(kDecThreads)
 decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, const CoefTable* __restrict__ d_tab,
                     int R, const float* __restrict__ dAt, const float* __restrict__ dBt, int64_t Mtot, int64_t Ntot,
@@ -198,15 +198,28 @@ decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, cons
       if (c >= ncell) break;
       float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
       const int e1 = sm.off[c + 1];
-      for (int e = sm.off[c]; e < e1; e += 2) {   // lists are padded to a multiple of four entries
-        const int4 two = *reinterpret_cast<const int4*>(&ent[e]);
-        const float4 v0 = *reinterpret_cast<const float4*>(cur + two.x);
-        const float4 v1 = *reinterpret_cast<const float4*>(cur + two.z);
-        const float w0 = __int_as_float(two.y), w1 = __int_as_float(two.w);
-        x.x = __fmaf_rn(w0, v0.x, x.x); x.y = __fmaf_rn(w0, v0.y, x.y);   // integers below 2^24: exact
-        x.z = __fmaf_rn(w0, v0.z, x.z); x.w = __fmaf_rn(w0, v0.w, x.w);
-        x.x = __fmaf_rn(w1, v1.x, x.x); x.y = __fmaf_rn(w1, v1.y, x.y);
-        x.z = __fmaf_rn(w1, v1.z, x.z); x.w = __fmaf_rn(w1, v1.w, x.w);
+      if (kIntAcc) {
+        // partial sums may pass 2^24 (each product is below it, the result is below it): add in int32
+        int4 xi = make_int4(0, 0, 0, 0);
+        for (int e = sm.off[c]; e < e1; ++e) {
+          const int2 en = ent[e];
+          const float4 v = *reinterpret_cast<const float4*>(cur + en.x);
+          const int w = __float2int_rn(__int_as_float(en.y));
+          xi.x += w * __float2int_rn(v.x); xi.y += w * __float2int_rn(v.y);
+          xi.z += w * __float2int_rn(v.z); xi.w += w * __float2int_rn(v.w);
+        }
+        x = make_float4((float)xi.x, (float)xi.y, (float)xi.z, (float)xi.w);
+      } else {
+        for (int e = sm.off[c]; e < e1; e += 2) {   // lists are padded to a multiple of four entries
+          const int4 two = *reinterpret_cast<const int4*>(&ent[e]);
+          const float4 v0 = *reinterpret_cast<const float4*>(cur + two.x);
+          const float4 v1 = *reinterpret_cast<const float4*>(cur + two.z);
+          const float w0 = __int_as_float(two.y), w1 = __int_as_float(two.w);
+          x.x = __fmaf_rn(w0, v0.x, x.x); x.y = __fmaf_rn(w0, v0.y, x.y);   // integers below 2^24: exact
+          x.z = __fmaf_rn(w0, v0.z, x.z); x.w = __fmaf_rn(w0, v0.w, x.w);
+          x.x = __fmaf_rn(w1, v1.x, x.x); x.y = __fmaf_rn(w1, v1.y, x.y);
+          x.z = __fmaf_rn(w1, v1.z, x.z); x.w = __fmaf_rn(w1, v1.w, x.w);
+        }
       }
       if (live) {
         const int i = c / n, j = c - i * n;
@@ -278,9 +291,89 @@ __global__ void __launch_bounds__(256) transpose_scales_kernel(const float* __re
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Block sums of int8 codes with the overflow split of Section 4.3: X = X0 + 256 R, R = floor((X + 128) / 256),
+// X0 in [-128, 127].  One thread forms, for one (group, row position) and four consecutive inner indices t, the
+// block sums of every product and writes them as bf16 (all values exact: |X0| <= 128, 256 |R| <= 512) into rows
+// of 4h elements laid out so that ONE contraction over the row gives all four products of Eq. 2:
+//   A side: [ A0 | 256 R_A | A0 | 256 R_A ]      B side: [ B0 | B0 | 256 R_B | 256 R_B ]
+//   sum = A0 B0 + 256 R_A B0 + 256 A0 R_B + 256^2 R_A R_B = Ahat Bhat.
+// The thread's codes are staged in shared memory ([cell][thread] words) so that the coefficient lists can index them.
+// ------------------------------------------------------------------------------------------
+constexpr int kSplitThreads = 128;
+
+__global__ void __launch_bounds__(kSplitThreads)
+encode_split_kernel(const int8_t* __restrict__ codes, int64_t K, int gc, int64_t br, int G, int h, int b_side,
+                    const CoefTable* __restrict__ d_tab, __nv_bfloat16* __restrict__ out, int64_t rstride, int64_t nquad) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R = d_tab->R, ncell = d_tab->ncell;
+  const int total = d_tab->off[R];
+  int* off = reinterpret_cast<int*>(smem_raw);                       // R + 1 list offsets
+  int2* ent = reinterpret_cast<int2*>(smem_raw + ((size_t)(R + 1) * 4 + 15) / 16 * 16);
+  uint32_t* stage = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(ent) + (size_t)total * 8);
+  for (int i = threadIdx.x; i <= R; i += kSplitThreads) off[i] = d_tab->off[i];
+  for (int i = threadIdx.x; i < total; i += kSplitThreads)
+    ent[i] = make_int2(d_tab->cell[i], __float2int_rn(d_tab->coef[i]));
+  stage[ncell * kSplitThreads + threadIdx.x] = 0u;                    // the padding cell
+  const int64_t idx = (int64_t)blockIdx.x * kSplitThreads + threadIdx.x;
+  const bool live = idx < nquad;
+  const int qpr = h / 4;                                              // quads per (group, row position)
+  const int64_t rowp = live ? idx / qpr : 0;                          // (group, p)
+  const int t = live ? (int)(idx - rowp * qpr) * 4 : 0;
+  const int64_t g = rowp / br, p = rowp - g * br;
+  for (int c = 0; c < ncell; ++c) {
+    const int gi = c / gc, gj = c - gi * gc;
+    stage[c * kSplitThreads + threadIdx.x] =
+        live ? *reinterpret_cast<const uint32_t*>(codes + ((int64_t)gi * br + p) * K + g * kGroup + gj * h + t) : 0u;
+  }
+  __syncthreads();
+  if (!live) return;
+  __nv_bfloat16* row = out + rowp * (4 * h) + t;
+  for (int r = 0; r < R; ++r) {
+    int s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    for (int e = off[r]; e < off[r + 1]; ++e) {
+      const int2 en = ent[e];
+      const uint32_t wv = stage[en.x * kSplitThreads + threadIdx.x];
+      s0 += en.y * (int)(int8_t)(wv & 0xffu);
+      s1 += en.y * (int)(int8_t)((wv >> 8) & 0xffu);
+      s2 += en.y * (int)(int8_t)((wv >> 16) & 0xffu);
+      s3 += en.y * (int)(int8_t)(wv >> 24);
+    }
+    // arithmetic shift = floor division by 256 for either sign
+    const int h0 = (s0 + 128) >> 8, h1 = (s1 + 128) >> 8, h2 = (s2 + 128) >> 8, h3 = (s3 + 128) >> 8;
+    const __nv_bfloat162 lo01 = __floats2bfloat162_rn((float)(s0 - 256 * h0), (float)(s1 - 256 * h1));
+    const __nv_bfloat162 lo23 = __floats2bfloat162_rn((float)(s2 - 256 * h2), (float)(s3 - 256 * h3));
+    const __nv_bfloat162 hi01 = __floats2bfloat162_rn((float)(256 * h0), (float)(256 * h1));
+    const __nv_bfloat162 hi23 = __floats2bfloat162_rn((float)(256 * h2), (float)(256 * h3));
+    const uint2 lo = make_uint2(*reinterpret_cast<const uint32_t*>(&lo01), *reinterpret_cast<const uint32_t*>(&lo23));
+    const uint2 hi = make_uint2(*reinterpret_cast<const uint32_t*>(&hi01), *reinterpret_cast<const uint32_t*>(&hi23));
+    __nv_bfloat16* dst = row + (int64_t)r * rstride;
+    *reinterpret_cast<uint2*>(dst) = lo;
+    *reinterpret_cast<uint2*>(dst + h) = b_side ? lo : hi;
+    *reinterpret_cast<uint2*>(dst + 2 * h) = b_side ? hi : lo;
+    *reinterpret_cast<uint2*>(dst + 3 * h) = hi;
+  }
+}
+
+cudaError_t launch_encode_split(const int8_t* codes, int64_t K, int gr, int gc, int64_t br, int G, int h, bool b_side,
+                                const CoefTable* d_tab, const CoefTable* h_tab, __nv_bfloat16* out, int64_t rstride,
+                                cudaStream_t st) {
+  const int64_t nquad = (int64_t)G * br * (h / 4);
+  const size_t smem = ((size_t)(h_tab->R + 1) * 4 + 15) / 16 * 16 + (size_t)h_tab->off[h_tab->R] * 8 +
+                      (size_t)(gr * gc + 1) * kSplitThreads * 4;
+  if (smem > 96 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(encode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  if (e != cudaSuccess) return e;
+  const int64_t grid = (nquad + kSplitThreads - 1) / kSplitThreads;
+  if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
+  encode_split_kernel<<<(unsigned)grid, kSplitThreads, smem, st>>>(codes, K, gc, br, G, h, b_side ? 1 : 0, d_tab, out, rstride, nquad);
+  ++fmm_launch_counter();
+  return cudaGetLastError();
+}
+
 int padded_total(const CoefTable& t) { return t.off[t.R]; }
 
-template <typename OutT, int kSplit, int kStages, int kCells>
+template <typename OutT, int kSplit, int kStages, int kCells, bool kIntAcc = false>
 cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
                                   const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
                                   int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
@@ -290,7 +383,7 @@ cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, con
   const int64_t nvec = bm * (bn >> 2);
   if (nvec + kDecThreads >= (int64_t)1 << 31 || smem > 200 * 1024) return cudaErrorInvalidValue;
   if (m * n > kSplit * kCells) return cudaErrorInvalidValue;
-  auto k = decode_group_kernel<OutT, kSplit, kStages, kCells>;
+  auto k = decode_group_kernel<OutT, kSplit, kStages, kCells, kIntAcc>;
   cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   if (e != cudaSuccess) return e;
   const unsigned grid = (unsigned)((nvec + kPos - 1) / kPos);
@@ -306,7 +399,12 @@ cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, con
 template <typename OutT>
 cudaError_t launch_decode_group_o(const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
                                   const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
-                                  int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+                                  int64_t bm, int64_t bn, void* C, int64_t ldc, bool int_acc, cudaStream_t st) {
+  if (int_acc) {
+    if (m * n <= 4 && R <= 8)
+      return launch_decode_group_t<OutT, 4, 4, 1, true>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+    return launch_decode_group_t<OutT, 8, 2, 2, true>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+  }
   if (m * n == 1 && R == 1) {
     const int64_t nvec = bm * (bn >> 2);
     rescale_groups_kernel<OutT><<<(unsigned)((nvec + 255) / 256), 256, 0, st>>>(prod, pstride, G, dAt, dBt, bm, bn, (OutT*)C, ldc);
@@ -320,11 +418,11 @@ cudaError_t launch_decode_group_o(const float* prod, int64_t pstride, int G, con
 
 cudaError_t launch_decode_group(int output, const float* prod, int64_t pstride, int G, const CoefTable* d_tab,
                                 const CoefTable* h_tab, int R, const float* dAt, const float* dBt, int m, int n,
-                                int64_t bm, int64_t bn, void* C, int64_t ldc, cudaStream_t st) {
+                                int64_t bm, int64_t bn, void* C, int64_t ldc, bool int_acc, cudaStream_t st) {
   if (output == FMM_F32)
-    return launch_decode_group_o<float>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+    return launch_decode_group_o<float>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, int_acc, st);
   if (output == FMM_BF16)
-    return launch_decode_group_o<__nv_bfloat16>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, st);
+    return launch_decode_group_o<__nv_bfloat16>(prod, pstride, G, d_tab, h_tab, R, dAt, dBt, m, n, bm, bn, C, ldc, int_acc, st);
   return cudaErrorInvalidValue;
 }
 
@@ -389,6 +487,52 @@ bool integer_coefficients(const fmm_scheme& s) {
     for (double c : *v)
       if (c != std::rint(c)) return false;
   return true;
+}
+
+// Workspace of the corrected product: split block sums in rows of 4h, products, transposed scales.
+struct CorrLayout {
+  size_t status, tabA, tabB, tabW, dAt, dBt, ahat, bhat, prod, total;
+  int64_t sAhat, sBhat, sProd;
+  int G, h;
+};
+
+CorrLayout corr_layout(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
+  CorrLayout L;
+  L.G = (int)(K / kGroup);
+  L.h = kGroup / s.k;
+  const int64_t bm = M / s.m, bn = N / s.n;
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.tabA = o; o += align_up(sizeof(CoefTable));
+  L.tabB = o; o += align_up(sizeof(CoefTable));
+  L.tabW = o; o += align_up(sizeof(CoefTable));
+  L.dAt = o; o += align_up((size_t)M * L.G * 4);
+  L.dBt = o; o += align_up((size_t)N * L.G * 4);
+  L.sAhat = (int64_t)L.G * bm * 4 * L.h + kSlabPadBytes / 2;
+  L.sBhat = (int64_t)L.G * bn * 4 * L.h + kSlabPadBytes / 2;
+  L.sProd = bm * bn + kSlabPadBytes / 4;
+  L.ahat = o; o += align_up((size_t)s.R * L.sAhat * 2);
+  L.bhat = o; o += align_up((size_t)s.R * L.sBhat * 2);
+  L.prod = o; o += align_up((size_t)s.R * L.G * L.sProd * 4);
+  L.total = o;
+  return L;
+}
+
+// The corrected computation's certificate (Appendix D) for this realisation: integer coefficients; block sums
+// |X| <= L * 127 split as X0 + 256 R with |R| <= rmax; inside one rebuilt product the absolute values of all weighted
+// terms add up to at most h (128 + 256 rmax)^2, which must stay below 2^24 (fp32 accumulators of the tensor cores);
+// the combination adds at most L_W such products and must stay below 2^31 (int32 in the decode); the group's result
+// is the classical product, at most 128 * 127^2 < 2^24, so its conversion to fp32 is exact.
+bool corrected_certificate(const fmm_scheme& s, int h, double cert[4]) {
+  double meta[8];
+  if (scheme_info(&s, nullptr, meta) != FMM_OK) return false;
+  const double sum_max = std::max(meta[0], meta[1]) * 127.0;
+  const double rmax = std::floor((sum_max + 128.0) / 256.0);
+  const double terms = (double)h * (128.0 + 256.0 * rmax) * (128.0 + 256.0 * rmax);
+  const double comb = meta[2] * terms;
+  if (cert) { cert[0] = sum_max; cert[1] = rmax; cert[2] = terms; cert[3] = comb; }
+  return integer_coefficients(s) && terms < std::ldexp(1.0, 24) && comb < std::ldexp(1.0, 31) &&
+         (int64_t)s.k * h == kGroup;
 }
 
 }  // namespace
@@ -498,9 +642,73 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
     ++fmm_launch_counter();
     FMM_CUDA(cudaGetLastError());
     FMM_CUDA(launch_decode_group(output, at<float>(d_ws, L.prod), L.sProd, L.G, at<CoefTable>(d_ws, L.tabW), hW, sc.R,
-                                 at<float>(d_ws, L.dAt), at<float>(d_ws, L.dBt), sc.m, sc.n, bm, bn, d_C, ldc, st));
+                                 at<float>(d_ws, L.dAt), at<float>(d_ws, L.dBt), sc.m, sc.n, bm, bn, d_C, ldc, false, st));
   }
   // the tables were copied from pageable host memory: the copies are complete when cudaMemcpyAsync returns
+  return FMM_OK;
+}
+
+int scheme_certificate_corrected(const fmm_scheme* s, int h, double cert[4]) {
+  if (!s) return 0;
+  return corrected_certificate(*s, h, cert) ? 1 : 0;
+}
+
+size_t int8_gemm_corrected_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N) {
+  if (!s || int8_shape_ok(*s, M, K, N) != FMM_OK) return 0;
+  return corr_layout(*s, M, K, N).total;
+}
+
+fmm_status int8_gemm_corrected(const fmm_scheme* s, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
+                               const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc,
+                               void* d_ws, size_t ws_bytes, void* stream) {
+  if (!s || !d_cA || !d_dA || !d_cB || !d_dB || !d_C) return FMM_ERR_ARG;
+  if (output != FMM_F32 && output != FMM_BF16) return FMM_ERR_DTYPE;
+  const fmm_scheme& sc = *s;
+  FMM_TRY(int8_shape_ok(sc, M, K, N));
+  const int eo = output == FMM_F32 ? 4 : 2;
+  if (ldc < N || (ldc * eo) % 16 || (reinterpret_cast<uintptr_t>(d_C) % 16)) return FMM_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(d_cA) % 8) || (reinterpret_cast<uintptr_t>(d_cB) % 8)) return FMM_ERR_SHAPE;
+  const CorrLayout L = corr_layout(sc, M, K, N);
+  if (!corrected_certificate(sc, L.h, nullptr)) return FMM_ERR_CERTIFICATE;
+  if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t bm = M / sc.m, bn = N / sc.n;
+
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  std::unique_ptr<CoefTable> hA(new CoefTable), hB(new CoefTable), hW(new CoefTable);
+  std::memset(hA.get(), 0, sizeof(CoefTable)); std::memset(hB.get(), 0, sizeof(CoefTable)); std::memset(hW.get(), 0, sizeof(CoefTable));
+  fmm_build_tables(sc, hA.get(), hB.get(), hW.get());
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabA), hA.get(), sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabB), hB.get(), sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabW), hW.get(), sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  {
+    ProfScope ps(0, st);
+    FMM_CUDA(launch_encode_split(d_cA, K, sc.m, sc.k, bm, L.G, L.h, false, at<CoefTable>(d_ws, L.tabA), hA.get(),
+                                 at<__nv_bfloat16>(d_ws, L.ahat), L.sAhat, st));
+    FMM_CUDA(launch_encode_split(d_cB, K, sc.n, sc.k, bn, L.G, L.h, true, at<CoefTable>(d_ws, L.tabB), hB.get(),
+                                 at<__nv_bfloat16>(d_ws, L.bhat), L.sBhat, st));
+  }
+  {
+    BlockProductArgs g{};
+    g.product = FMM_BF16;
+    g.A = at<char>(d_ws, L.ahat); g.lda = 4 * L.h; g.a_batch = L.sAhat;
+    g.B = at<char>(d_ws, L.bhat); g.ldb = 4 * L.h; g.b_batch = L.sBhat;
+    g.rows_a = bm; g.rows_b = bn; g.kdim = 4 * L.h; g.batches = sc.R; g.groups = L.G;
+    g.out = at<char>(d_ws, L.prod); g.ldo = bn; g.o_batch = L.sProd; g.out_mode = 0; g.output = FMM_F32;
+    g.status = at<DeviceStatus>(d_ws, L.status);
+    ProfScope ps(2, st);
+    FMM_TRY(launch_block_products(g, st));
+  }
+  {
+    ProfScope ps(3, st);
+    transpose_scales_kernel<<<stream_blocks(M * L.G, 256), 256, 0, st>>>(d_dA, M, L.G, at<float>(d_ws, L.dAt));
+    ++fmm_launch_counter();
+    transpose_scales_kernel<<<stream_blocks(N * L.G, 256), 256, 0, st>>>(d_dB, N, L.G, at<float>(d_ws, L.dBt));
+    ++fmm_launch_counter();
+    FMM_CUDA(cudaGetLastError());
+    FMM_CUDA(launch_decode_group(output, at<float>(d_ws, L.prod), L.sProd, L.G, at<CoefTable>(d_ws, L.tabW), hW.get(), sc.R,
+                                 at<float>(d_ws, L.dAt), at<float>(d_ws, L.dBt), sc.m, sc.n, bm, bn, d_C, ldc, true, st));
+  }
   return FMM_OK;
 }
 

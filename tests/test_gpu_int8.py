@@ -172,3 +172,38 @@ def test_fp8_schedule_moves_the_48_same_offset_pairs_on_device():
     for mode in (0, 2):
         assert moved(lambda X: gu.run_scheme_gemm(s2, X, Bt, "f32", "e4m3", "f32", scale_mode=mode)) == want
     assert moved(lambda X: gu.run_classical(X, Bt, "f32", "e4m3", "f32", scale_mode=2)) == set()
+
+
+@pytest.mark.parametrize("M,K,N", [(32, 128, 32), (512, 1024, 544), (200, 384, 96)])
+def test_overflow_corrected_full_range_codes(M, K, N):
+    """Section 4.3: two-level Strassen at code bound 127 with the split X = X0 + 256 R gives classical int8's bits."""
+    lib = fmm()
+    At, A, Bt, B = _inputs(61, M, K, N)
+    cA, dA = _quantize(lib, At, 127)
+    cB, dB = _quantize(lib, Bt, 127)
+    oA, odA = oracle.quantize_rows(A, 127)
+    oB, odB = oracle.quantize_rows(B, 127)
+    want = oracle.int8_classical(oA, odA, oB, odB)
+    assert np.array_equal(_gemm(lib, None, 127, cA, dA, cB, dB), want)
+    variants = list(oracle.sign_variants(4, 4, 4))
+    for v in (variants[0], variants[203], variants[-1]):
+        s = _lib_scheme(lib, oracle.sign_variant(S2, *v))
+        ws = workspace(lib.int8_gemm_corrected_workspace(s, M, K, N))
+        C = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        lib.int8_gemm_corrected(s, cA, dA, cB, dB, C, ws)
+        lib.device_status(ws)
+        assert np.array_equal(C.to(torch.float64).cpu().numpy(), want)
+    want_corr, mx = oracle.int8_corrected(S2, oA, odA, oB, odB)
+    assert np.array_equal(want_corr, want) and mx[0] == 0 and mx[1] <= 2
+    # one level of Strassen (h = 64, |R| <= 1), fp32 output
+    s1 = _lib_scheme(lib, S1)
+    ws = workspace(lib.int8_gemm_corrected_workspace(s1, M, K, N))
+    C32 = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    lib.int8_gemm_corrected(s1, cA, dA, cB, dB, C32, ws)
+    lib.device_status(ws)
+    assert np.array_equal(C32.to(torch.float64).cpu().numpy(), oracle.int8_classical(oA, odA, oB, odB, od="f32"))
+    # the uncorrected call has no certificate at this code bound
+    s2 = _lib_scheme(lib, S2)
+    with pytest.raises(lib.FmmError) as ei:
+        _gemm(lib, s2, 127, cA, dA, cB, dB)
+    assert ei.value.code == 10

@@ -167,3 +167,19 @@ def test_certificate_on_host_matches_oracle(lib):
     assert lib.int8_gemm_workspace(s2, 64, 100, 64) == 0          # K not a multiple of 128
     assert lib.int8_gemm_workspace(s2, 66, 128, 64) == 0          # M not divisible by m
     assert lib.int8_gemm_workspace(s2, 64, 128, 64) > 0
+
+
+def test_corrected_certificate_constants(lib):
+    """Appendix D, certificate of the corrected computation: block sums up to 4 * 127 = 508, |R| <= 2, the terms
+    of one rebuilt product within h (128 + 256 * 2)^2 = 13,107,200, sixteen of them below 2^31."""
+    s1 = lib.scheme_builtin("strassen222")
+    s2 = lib.scheme_kron(s1, s1)
+    ok, c = lib.scheme_certificate_corrected(s2, 32)
+    assert ok and c == dict(block_sum_max=508.0, r_max=2.0, product_terms=13107200.0, combination=16 * 13107200.0)
+    ok1, c1 = lib.scheme_certificate_corrected(s1, 64)
+    assert ok1 and c1["block_sum_max"] == 254 and c1["r_max"] == 1
+    assert not lib.scheme_certificate_corrected(s2, 64)[0]          # a call of 256 indices over groups of 128
+    P = gen.gauge_cond_limited(3, 0, 2)
+    assert not lib.scheme_certificate_corrected(lib.gauge_apply(s1, P, P, P), 64)[0]
+    assert lib.int8_gemm_corrected_workspace(s2, 64, 128, 64) > 0
+    assert lib.int8_gemm_corrected_workspace(s2, 64, 100, 64) == 0
