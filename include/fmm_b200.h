@@ -31,6 +31,10 @@
  *   - M % m, K % k, N % n must be 0, K/k must be a multiple of 16 and N/n a multiple
  *     of 8 (FMM_ERR_SHAPE otherwise): zero padding is the caller's job, as in the paper
  *     (Appendix B.2 pads 40 rows to 48);
+ *   - maximum sizes: one block may hold fewer than 2^31 - 4096 sixteen-byte vectors of the source
+ *     ((M/m) * (K/k) * storage bytes / 16, likewise for B) and fewer than that many quads of products
+ *     ((M/m) * (N/n) / 4); M/m, N/n < 2^31 - 4096 and K/k < 2^30.  Larger shapes, empty shapes
+ *     (M, K or N <= 0) included, return FMM_ERR_SHAPE (the workspace queries return 0) and launch nothing;
  *   - NaN/Inf in operands propagate; e4m3 conversion saturates at +-448.
  */
 #ifndef FMM_B200_H

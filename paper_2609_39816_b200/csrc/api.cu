@@ -108,6 +108,12 @@ fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
   const int64_t min_ldb = d->b_is_weight_layout ? d->K : d->N;
   if (d->lda < d->K || d->ldb < min_ldb || d->ldc < d->N) return FMM_ERR_SHAPE;
   if ((d->lda * es) % 16 || (d->ldb * es) % 16 || (d->ldc * eo) % 16) return FMM_ERR_SHAPE;
+  // the streaming kernels index the positions of one block in 32 bits (16-byte vectors of the source / of fp32
+  // products), and the tensor maps take 32-bit extents: reject anything beyond, before any launch
+  const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
+  const int64_t limit = ((int64_t)1 << 31) - 4096;
+  if (bm * (bk / (16 / es)) >= limit || bn * (bk / (16 / es)) >= limit || bm * (bn / 4) >= limit) return FMM_ERR_SHAPE;
+  if (bm >= limit || bn >= limit || bk >= ((int64_t)1 << 30)) return FMM_ERR_SHAPE;
   return FMM_OK;
 }
 

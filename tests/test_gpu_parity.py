@@ -284,6 +284,25 @@ def test_config2_full_size_sampled_outputs(lib):
     assert gu.rel_fro(C, Cs) < 0.05
 
 
+@pytest.mark.parametrize("Pd,scale", [("bf16", 0), ("e4m3", 2)])
+def test_largest_benchmark_shape_sampled_outputs(lib, Pd, scale):
+    """The largest GEMM of the benchmark configurations (8192 tokens, K = 5120, N = 27648; 2.8 GB of products),
+    weight layout: sampled rows / columns against the oracle.  With row / column scales the sub-problem keeps the
+    whole inner dimension, so its scales are the full problem's."""
+    M, K, N = 8192, 5120, 27648
+    A = gen.activations_outlier(2, 1, M, K, dist="t3", frac=0.001, factor=300.0, at_least=1)
+    B = gen.weights(2, 2, K, N)
+    At, A64 = gu.storage_pair(A, "bf16")
+    Bt, B64 = gu.storage_pair(B, "bf16")
+    s = lib.scheme_builtin("strassen444")
+    C = gu.run_scheme_gemm(s, At, Bt.t().contiguous(), "bf16", Pd, "bf16", weight_layout=True, scale_mode=scale)
+    rows = [0, 129, 1023, 1024, 2047]
+    cols = [0, 7, 255, 256, 4095, 4096, 6911]
+    As, Bs, ridx, cidx = gu.subsample_problem(A64, B64, 4, 4, 4, rows, cols)
+    Co = oracle.scheme_gemm(gu.oracle_scheme("strassen444"), As, Bs, Pd, "bf16", scale_mode=scale)
+    assert gu.rel_fro(C[np.ix_(ridx, cidx)], Co) <= TOL_FRO
+
+
 # ---------------------------------------------------------------------------- failure reporting
 def test_bounded_wait_expires_reports_timeout_and_context_survives(lib):
     """A wait that nothing will ever satisfy (the copy-issuing warp of one block is switched off) must run out,

@@ -183,3 +183,20 @@ def test_corrected_certificate_constants(lib):
     assert not lib.scheme_certificate_corrected(lib.gauge_apply(s1, P, P, P), 64)[0]
     assert lib.int8_gemm_corrected_workspace(s2, 64, 128, 64) > 0
     assert lib.int8_gemm_corrected_workspace(s2, 64, 100, 64) == 0
+
+
+def test_empty_and_maximum_sizes_are_rejected_before_any_launch(lib):
+    """Empty shapes and blocks beyond the kernels' 32-bit position index return no workspace (FMM_ERR_SHAPE)."""
+    s2 = lib.scheme_builtin("strassen444")
+    ok = lib.GemmDesc.make(4096, 4096, 4096, "bf16", "bf16", "bf16")
+    assert lib.scheme_gemm_workspace(s2, ok) > 0
+    for M, K, N in ((0, 64, 32), (64, 0, 32), (64, 64, 0)):
+        assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(M, K, N, "bf16", "bf16", "bf16")) == 0
+        assert lib.classical_gemm_workspace(lib.GemmDesc.make(M, K, N, "bf16", "bf16", "bf16")) == 0
+    # largest legal block: (M/4) * (K/4) * 2 / 16 vectors just under 2^31 - 4096; one step beyond is refused
+    big_ok = lib.GemmDesc.make(4 * (1 << 20), 4 * 16368, 32, "bf16", "bf16", "bf16")       # 2^20 * 16368 / 8 = 2.1453e9
+    assert (1 << 20) * 16368 // 8 < (1 << 31) - 4096 and lib.scheme_gemm_workspace(s2, big_ok) > 0
+    too_big = lib.GemmDesc.make(4 * (1 << 20), 4 * 16400, 32, "bf16", "bf16", "bf16")
+    assert (1 << 20) * 16400 // 8 >= (1 << 31) - 4096 and lib.scheme_gemm_workspace(s2, too_big) == 0
+    assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4 * (1 << 17), 64, 4 * (1 << 17), "bf16", "bf16", "bf16")) == 0   # products
+    assert lib.int8_gemm_workspace(s2, 0, 128, 64) == 0
