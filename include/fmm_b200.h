@@ -75,6 +75,12 @@ typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
                                  "encode B".  Weights are static, so their block sums can be
                                  formed once (the paper prepares weight block sums offline,
                                  Section 3.1 / Appendix C).                                   */
+#define FMM_FLAG_PRODUCTS_BF16 2 /* every block product M_r is rounded to bf16 before the combination,
+                                 as in the paper's model schedule, whose product kernel "returns each
+                                 product in bf16" (Appendix B.1); the combination stays in fp32.  Halves
+                                 the bytes the products move.  With scale_mode 1 the product of the codes
+                                 is rounded (the power-of-two scales commute with the rounding); with
+                                 scale_mode 2 the rounding follows the row / column scales.            */
 
 /* The float-path "quantisation specification" (Section 2.2 treats these choices as part of the
  * operator): shapes, dtypes, layout of B, scale rule. */

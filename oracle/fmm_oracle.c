@@ -366,6 +366,7 @@ static void matmul_f64(const double* A, const double* B, double* C, int64_t M, i
  * and per column of each block sum of B, scale = max|x| / 448 in fp32 (1 for an all-zero
  * row), code = x / scale in fp32, then rounded to e4m3 (a reading: the paper states who
  * owns a scale, not its rule; max|x| / b is the rule of its int8 specification).
+ * md = dtype each product is rounded to before the combination (ORC_F64: none).
  * Optional outputs (may be NULL): Ahat [R][bm][bk], Bhat [R][bk][bn] (the rounded,
  * scaled block sums), sA[R], sB[R] (mode 2: sA[R][bm], sB[R][bn]), Mout [R][bm][bn]
  * (the fp64 products of the codes; mode 2: times the row and column scales).
@@ -374,7 +375,7 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
                     int64_t M, int64_t K, int64_t N, const double* A, const double* B,
                     int pd, int od, int scale_mode, double* C,
                     double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
-                    double* M_out) {
+                    double* M_out, int md) {
   if (M % m || K % k || N % n) return 1;
   int64_t bm = M / m, bk = K / k, bn = N / n;
   int quant = (pd != ORC_F64);
@@ -427,6 +428,11 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
     if (scale_mode == 2)
       for (int64_t p = 0; p < bm; ++p)
         for (int64_t q = 0; q < bn; ++q) Mr[p * bn + q] = (Mr[p * bn + q] * rs[p]) * cs[q];
+    /* model schedule (Appendix B.1): the product kernel returns each product in a storage dtype (bf16);
+     * md = ORC_F64 keeps the product as computed.  With per-tensor power-of-two scales the rounding of the
+     * product of the codes equals the rounding of the scaled product, so the order is immaterial.        */
+    if (md != ORC_F64)
+      for (int64_t x = 0; x < bm * bn; ++x) Mr[x] = orc_round(Mr[x], md);
     if (M_out) memcpy(M_out + (size_t)r * bm * bn, Mr, sizeof(double) * bm * bn);
     /* decode, ascending r: C_ij += w_{r,ij} * (sA_r sB_r) * M_r */
     for (int i = 0; i < m; ++i)

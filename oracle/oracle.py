@@ -63,7 +63,7 @@ def _L():
         lib.orc_criteria.argtypes = [C.c_int] * 4 + [dp] * 4
         lib.orc_scheme_gemm.restype = C.c_int
         lib.orc_scheme_gemm.argtypes = ([C.c_int] * 4 + [dp] * 3 + [i64] * 3 + [dp] * 2 +
-                                        [C.c_int] * 3 + [dp] * 6)
+                                        [C.c_int] * 3 + [dp] * 6 + [C.c_int])
         lib.orc_classical_gemm.restype = C.c_int
         lib.orc_classical_gemm.argtypes = [i64] * 3 + [dp] * 2 + [C.c_int] * 3 + [dp]
         lib.orc_exact_gemm.argtypes = [i64] * 3 + [dp] * 3
@@ -222,8 +222,9 @@ def criteria(s: Scheme) -> dict:
     return dict(zip(keys, meta.tolist()))
 
 
-def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts: bool = False):
-    """Apply the algorithm with block sums rounded to ``pd``; returns C (values of ``od``).
+def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts: bool = False, md="f64"):
+    """Apply the algorithm with block sums rounded to ``pd``; returns C (values of ``od``).  ``md``: dtype each
+    product is rounded to before the combination ("f64": none; "bf16": the paper's model schedule).
     With ``parts`` also returns dict(Ahat, Bhat, sA, sB, M)."""
     m, k, n, R = s.dims
     A = _d(A); B = _d(B)
@@ -238,7 +239,7 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
         sA = np.empty((R, bm) if scale_mode == 2 else R); sB = np.empty((R, bn) if scale_mode == 2 else R)
     rc = _L().orc_scheme_gemm(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
                               _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
-                              _p(sB), _p(Mr))
+                              _p(sB), _p(Mr), _fmt(md))
     if rc:
         raise ValueError("matrix dimensions are not divisible by the block grid")
     if parts:

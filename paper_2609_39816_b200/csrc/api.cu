@@ -143,7 +143,7 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.sProd = bm * bn + kSlabPadBytes / 4;
   L.ahat = o; o += align_up((size_t)R * L.sAhat * ep);
   L.bhat = o; o += align_up((size_t)R * L.sBhat * ep);
-  L.prod = o; o += align_up((size_t)R * L.sProd * 4);
+  L.prod = o; o += align_up((size_t)R * L.sProd * ((d->flags & FMM_FLAG_PRODUCTS_BF16) ? 2 : 4));
   L.total = o;
   return L;
 }
@@ -201,6 +201,7 @@ fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   g.B = at<char>(r.ws, r.L.bhat); g.ldb = bk; g.b_batch = r.L.sBhat;
   g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = s->R;
   g.out = at<char>(r.ws, r.L.prod); g.ldo = bn; g.o_batch = r.L.sProd; g.out_mode = 0; g.output = FMM_F32;
+  if (r.d->flags & FMM_FLAG_PRODUCTS_BF16) { g.out_mode = 1; g.output = FMM_BF16; }   // one rounding of each product
   if (r.d->scale_mode == 2) {   // row / column scales are folded into the stored products
     g.row_scale = r.sA(); g.rs_batch = bm;
     g.col_scale = r.sB(); g.cs_batch = bn;
@@ -215,7 +216,8 @@ fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, doubl
   ProfScope ps(3, st);
   int np = 0;
   const bool per_product = r.d->scale_mode == 1;   // mode 2: the products already carry their scales
-  FMM_CUDA(launch_decode(r.d->output, at<float>(r.ws, r.L.prod), r.L.sProd, r.dW, r.hW, s->R, per_product ? r.sA() : nullptr,
+  FMM_CUDA(launch_decode(r.d->output, at<char>(r.ws, r.L.prod), (r.d->flags & FMM_FLAG_PRODUCTS_BF16) ? FMM_BF16 : FMM_F32,
+                         r.L.sProd, r.dW, r.hW, s->R, per_product ? r.sA() : nullptr,
                          per_product ? r.sB() : nullptr, s->m, s->n,
                          r.d->M / s->m, r.d->N / s->n, C, r.d->ldc, cstar32, at<double>(r.ws, r.L.partials), &np, st));
   if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(r.ws, r.L.partials), np, err_out, st));

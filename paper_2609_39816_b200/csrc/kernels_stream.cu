@@ -398,15 +398,27 @@ struct DecSmemHead {
   double red[kDecThreads / 32];
 };  // followed by int2 ent[] {byte offset of product r's slab, scaled coefficient bits}, then the stage
 
-template <typename OutT, bool kStore, bool kErr, int kDecSplit>
+// four consecutive products of one row, staged as 16 bytes (fp32) or 8 bytes (bf16)
+__device__ __forceinline__ float4 staged_quad(const unsigned char* p, const float*) {
+  return *reinterpret_cast<const float4*>(p);
+}
+__device__ __forceinline__ float4 staged_quad(const unsigned char* p, const __nv_bfloat16*) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+  const __nv_bfloat162 hi = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+  return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
+
+template <typename OutT, bool kStore, bool kErr, int kDecSplit, typename ProdT>
 __global__ void __launch_bounds__(kDecThreads)
-decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
+decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
               const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
               OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
               double* __restrict__ partials, int tiles_per_block, int64_t rstride) {
   constexpr int kDecPos = kDecThreads / kDecSplit;
   constexpr int kCellsPerThread = 16 / kDecSplit;
-  constexpr int kSlab = kDecPos * 16;
+  constexpr int kVecBytes = 4 * (int)sizeof(ProdT);   // one position quad of products: 16 bytes (fp32) or 8 (bf16)
+  constexpr int kSlab = kDecPos * kVecBytes;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   DecSmemHead& sm = *reinterpret_cast<DecSmemHead*>(smem_raw);
   const int ncell = d_tab->R;                  // number of lists = number of C blocks
@@ -418,7 +430,7 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
   const int pq = threadIdx.x - g * kDecPos;
   const int vec_per_row = (int)(bn >> 2);      // 32-bit index arithmetic: bm * bn / 4 < 2^31 (checked by the host)
   const int nvec = (int)bm * vec_per_row;
-  unsigned char* my_stage = stage + pq * 16;
+  unsigned char* my_stage = stage + pq * kVecBytes;
   const uint32_t dst0 = (uint32_t)__cvta_generic_to_shared(my_stage);
   // element offsets of the output cells this thread forms (cells g, g+4, ...), computed once
   int64_t out_base[kCellsPerThread], cs_base[kCellsPerThread];
@@ -438,15 +450,23 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
     const int q = live ? (idx - p * vec_per_row) << 2 : 0;
     if (it > 0) __syncthreads();               // previous tile's readers are done with the stage
     {
-      const float* src = prod + (int64_t)p * bn + q;
-      const int nbytes = live ? 16 : 0;        // 0 source bytes -> the 16 destination bytes are zero-filled
-      for (int r = g; r < R; r += kDecSplit)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
-                     "r"(nbytes) : "memory");
+      const ProdT* src = prod + (int64_t)p * bn + q;
+      const int nbytes = live ? kVecBytes : 0;  // 0 source bytes -> the destination bytes are zero-filled
+      for (int r = g; r < R; r += kDecSplit) {
+        if (kVecBytes == 16)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
+                       "r"(nbytes) : "memory");
+        else
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
+                       "r"(nbytes) : "memory");
+      }
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (it == 0) {                             // table set-up overlaps the first tile's copies
-      if (g == 0) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (g == 0) {
+        if (kVecBytes == 16) *reinterpret_cast<float4*>(my_stage + R * kSlab) = make_float4(0.f, 0.f, 0.f, 0.f);
+        else *reinterpret_cast<uint2*>(my_stage + R * kSlab) = make_uint2(0u, 0u);
+      }
       for (int i = threadIdx.x; i <= ncell; i += kDecThreads) sm.off[i] = d_tab->off[i];
       for (int i = threadIdx.x; i < total; i += kDecThreads) {
         const int r = d_tab->cell[i];
@@ -474,7 +494,7 @@ decode_kernel(const float* __restrict__ prod, const CoefTable* __restrict__ d_ta
           en[u + 1] = make_int2(two.z, two.w);
         }
 #pragma unroll
-        for (int u = 0; u < kChunk; ++u) v[u] = *reinterpret_cast<const float4*>(my_stage + en[u].x);
+        for (int u = 0; u < kChunk; ++u) v[u] = staged_quad(my_stage + en[u].x, (const ProdT*)nullptr);
 #pragma unroll
         for (int u = 0; u < kChunk; ++u) {
           const float w = __int_as_float(en[u].y);
@@ -649,21 +669,21 @@ int decode_grid(int64_t bm, int64_t bn) {
   return grid;
 }
 
-template <typename OutT, int kSplit>
-static cudaError_t launch_decode_t(const float* prod, int64_t prod_stride, const CoefTable* d_tab, int R, int nnz, const float* sA,
+template <typename OutT, int kSplit, typename ProdT>
+static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const CoefTable* d_tab, int R, int nnz, const float* sA,
                                    const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
                                    const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
   constexpr int kDecPos = kDecThreads / kSplit;
-  const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 16;
+  const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 4 * sizeof(ProdT);
   if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
   int grid, tpb;
   split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
   if (n_partials) *n_partials = grid;
   const int64_t ldcs = (int64_t)n * bn;
-  static bool attr_done[3] = {false, false, false};
+  static bool attr_done[3] = {false, false, false};   // per template instantiation
 #define FMM_DECODE_LAUNCH(STORE, ERR, SLOT)                                                                      \
   {                                                                                                              \
-    auto k = decode_kernel<OutT, STORE, ERR, kSplit>;                                                            \
+    auto k = decode_kernel<OutT, STORE, ERR, kSplit, ProdT>;                                                         \
     if (!attr_done[SLOT]) {                                                                                      \
       cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);          \
       if (e != cudaSuccess) return e;                                                                            \
@@ -680,20 +700,32 @@ static cudaError_t launch_decode_t(const float* prod, int64_t prod_stride, const
   return cudaGetLastError();
 }
 
-cudaError_t launch_decode(int output, const float* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
-                          const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
-                          int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
+template <typename ProdT>
+static cudaError_t launch_decode_p(int output, const ProdT* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
+                                   const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
+                                   int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   // small schemes (at most 8 products, 4 output cells): one thread per position quad; otherwise four share one
   const bool small = R <= 8 && m * n <= 4;
   if (output == FMM_F32)
-    return small ? launch_decode_t<float, 1>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
-                 : launch_decode_t<float, 4>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
+    return small ? launch_decode_t<float, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
+                 : launch_decode_t<float, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
   if (output == FMM_BF16)
-    return small ? launch_decode_t<__nv_bfloat16, 1>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
-                 : launch_decode_t<__nv_bfloat16, 4>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
+    return small ? launch_decode_t<__nv_bfloat16, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
+                 : launch_decode_t<__nv_bfloat16, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_decode(int output, const void* prod, int prod_dtype, int64_t prod_stride, const CoefTable* d_tab,
+                          const CoefTable* h_tab, int R, const float* sA, const float* sB, int m, int n, int64_t bm,
+                          int64_t bn, void* C, int64_t ldc, const float* cstar32, double* partials, int* n_partials,
+                          cudaStream_t st) {
+  if (prod_dtype == FMM_BF16)
+    return launch_decode_p<__nv_bfloat16>(output, (const __nv_bfloat16*)prod, prod_stride, d_tab, h_tab, R, sA, sB, m, n, bm, bn, C, ldc,
+                                          cstar32, partials, n_partials, st);
+  return launch_decode_p<float>(output, (const float*)prod, prod_stride, d_tab, h_tab, R, sA, sB, m, n, bm, bn, C, ldc, cstar32,
+                                partials, n_partials, st);
 }
 
 cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st) {

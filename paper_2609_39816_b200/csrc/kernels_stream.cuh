@@ -28,14 +28,15 @@ cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, 
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
                              cudaStream_t st);
 
-// Decode (+ optional error reduction).  prod: R blocks [bm][bn] fp32, prod_stride elements apart.  If C != nullptr the rounded result is stored
+// Decode (+ optional error reduction).  prod: R blocks [bm][bn] of prod_dtype (FMM_F32 or FMM_BF16), prod_stride elements apart.  If C != nullptr the rounded result is stored
 // (dtype `output`, leading dimension ldc).  If cstar32 != nullptr the per-block partial sums of
 // (rnd_O(c) - C*)^2 are written to partials[gridDim.x] and *n_partials receives gridDim.x.
 // d_tab is the CELL-MAJOR decode table (list c = the (r, w) pairs feeding C block c, ascending r); R is the
 // number of products; h_tab is the host copy of d_tab (its list lengths size the shared memory).
-cudaError_t launch_decode(int output, const float* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
-                          const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
-                          int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st);
+cudaError_t launch_decode(int output, const void* prod, int prod_dtype, int64_t prod_stride, const CoefTable* d_tab,
+                          const CoefTable* h_tab, int R, const float* sA, const float* sB, int m, int n, int64_t bm,
+                          int64_t bn, void* C, int64_t ldc, const float* cstar32, double* partials, int* n_partials,
+                          cudaStream_t st);
 int decode_grid(int64_t bm, int64_t bn);
 
 // out[0] = sum of partials[0..n) in a fixed order (single block).

@@ -59,7 +59,7 @@ def run_scheme_gemm(s, A_t, B_t, S, Pd, O, weight_layout=False, scale_mode=0, fl
     p = dict(
         Ahat=grab(off["Ahat"], off["stride_Ahat"], bm, bk, pdt),
         BhatT=grab(off["Bhat"], off["stride_Bhat"], bn, bk, pdt),
-        M=grab(off["M"], off["stride_M"], bm, bn, torch.float32),
+        M=grab(off["M"], off["stride_M"], bm, bn, torch.bfloat16 if flags & 2 else torch.float32),
     )
     if scale_mode == 1:
         p["sA"] = ws[off["sA"]:off["sA"] + 4 * R].view(torch.float32).to(torch.float64).cpu().numpy()

@@ -76,6 +76,30 @@ def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     assert gu.rel_fro(C, Co) <= TOL_FRO
 
 
+@pytest.mark.parametrize("scheme,M,K,N,S,Pd,O,kind,scale", [
+    ("strassen444", 1024, 1024, 2048, "bf16", "bf16", "bf16", "llm", 0),    # CTA-pair kernel, bf16 products
+    ("strassen444", 384, 320, 288, "bf16", "bf16", "f32", "llm", 0),        # ragged tiles
+    ("strassen444", 512, 1024, 544, "bf16", "e4m3", "bf16", "t3", 1),       # per-tensor scales folded into the decode
+    ("strassen222", 200, 2240, 272, "bf16", "e4m3", "f32", "llm", 2),       # row / column scales applied before the rounding
+])
+def test_products_returned_in_bf16(lib, scheme, M, K, N, S, Pd, O, kind, scale):
+    """FMM_FLAG_PRODUCTS_BF16, the paper's model schedule: every product rounded once to bf16, combined in fp32.
+    The device rounds an fp32 accumulation where the oracle rounds an fp64 one, so a few products may land one
+    bf16 step apart: the products are compared in norm, and at most 1 in 1000 of them may differ at all."""
+    At, Bt, A64, B64 = _inputs(3, M, K, N, S, kind)
+    s, so = lib.scheme_builtin(scheme), gu.oracle_scheme(scheme)
+    C, p, _ = gu.run_scheme_gemm(s, At, Bt, S, Pd, O, scale_mode=scale, flags=lib.FLAG_PRODUCTS_BF16, parts=True)
+    Co, po = oracle.scheme_gemm(so, A64, B64, pd=Pd, od=O, scale_mode=scale, parts=True, md="bf16")
+    assert np.array_equal(p["Ahat"], po["Ahat"])
+    assert np.mean(p["M"] != po["M"]) <= 1e-3
+    # never more than one bf16 step, plus the fp32 accumulation error where a product cancels to almost nothing
+    assert np.all(np.abs(p["M"] - po["M"]) <= 2.0 ** -7 * np.abs(po["M"]) + 1e-5 * np.abs(po["M"]).max())
+    assert gu.rel_fro(C, Co) <= TOL_FRO
+    # and it is a different operator from the fp32-product default
+    C32 = gu.run_scheme_gemm(s, At, Bt, S, Pd, O, scale_mode=scale)
+    assert not np.array_equal(C, C32)
+
+
 @pytest.mark.parametrize("scheme,M,K,N,S,Pd,O,bound", [
     ("strassen222", 256, 256, 256, "f32", "bf16", "f32", 8),       # config 1 shape, L*b <= 2^8
     ("strassen444", 512, 512, 384, "bf16", "bf16", "f32", 7),      # two-level, 16*bk*(4*7)^2 < 2^24

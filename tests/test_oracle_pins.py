@@ -376,3 +376,24 @@ def test_generators_are_counter_based():
     assert np.linalg.cond(gen.gauge_cond_limited(0, 0, 2)) <= 10.0
     conds = [np.linalg.cond(gen.gauge_log_uniform_cond(1, i, 2)) for i in range(64)]
     assert 1.0 <= min(conds) < 3.0 and 300.0 < max(conds) <= 1000.0 + 1e-6
+
+
+def test_products_rounded_to_bf16_special_cases():
+    """Model schedule (Appendix B.1: each product is returned in bf16).  For the classical algorithm <1,1,1;1> the
+    only product is A B itself, so the result is the exact product rounded once to bf16 (a library matmul plus
+    the separately pinned rounding); on small integers the rounding is the identity; in general the result moves
+    by at most sum_r |w_r| half-ulps of the largest product."""
+    A = gen.integer_matrix(31, 1, (16, 32), 40).astype(np.float64)
+    B = gen.integer_matrix(31, 2, (32, 24), 40).astype(np.float64)
+    one = oracle.classical_scheme(1, 1, 1)
+    got = oracle.scheme_gemm(one, A, B, "f64", "f64", md="bf16")
+    assert np.array_equal(got, oracle.round_to(A @ B, "bf16")) and not np.array_equal(got, A @ B)
+    s2 = oracle.kron(oracle.strassen(), oracle.strassen())
+    a = gen.integer_matrix(32, 1, (8, 16), 1).astype(np.float64)
+    b = gen.integer_matrix(32, 2, (16, 8), 1).astype(np.float64)
+    assert np.array_equal(oracle.scheme_gemm(s2, a, b, "bf16", "f32", md="bf16"), a @ b)       # |M_r| <= 4*4*4 = 64: exact
+    X = gen.normal(33, 1, (64, 64)); Y = gen.normal(33, 2, (64, 64))
+    C0, p0 = oracle.scheme_gemm(s2, X, Y, "bf16", "f64", parts=True)
+    C1, p1 = oracle.scheme_gemm(s2, X, Y, "bf16", "f64", parts=True, md="bf16")
+    assert np.array_equal(p1["M"], oracle.round_to(p0["M"], "bf16"))
+    assert 0 < np.abs(C1 - C0).max() <= 16 * 2.0 ** -9 * np.abs(p0["M"]).max()
