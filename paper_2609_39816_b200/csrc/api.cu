@@ -168,6 +168,18 @@ fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, in
   return FMM_OK;
 }
 
+// The classical control's operand: the whole matrix as one block with coefficient 1.
+fmm_status quantize_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int64_t rows, int64_t cols, void* hat,
+                            unsigned* amax, float* scale, cudaStream_t st) {
+  const int mode = d->scale_mode;
+  if (mode != 0) {
+    FMM_CUDA(cudaMemsetAsync(amax, 0, (mode == 2 ? (size_t)rows : (size_t)FMM_MAX_R) * 4, st));
+    FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, true, mode, st));
+  }
+  FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, false, mode, st));
+  return FMM_OK;
+}
+
 // One scheme applied to one operand pair inside one workspace: the pieces every stage needs.
 struct SchemeRun {
   const fmm_scheme* s;
@@ -273,13 +285,6 @@ fmm_status check_ws(const void* ws, size_t have, size_t need) {
   return FMM_OK;
 }
 
-fmm_scheme classical_scheme_111() {
-  fmm_scheme c;
-  c.m = c.k = c.n = c.R = 1;
-  c.U = {1.0}; c.V = {1.0}; c.W = {1.0};
-  return c;
-}
-
 // Workspace of the classical product.
 struct ClassicalLayout { size_t status, tab, amaxA, amaxB, sA, sB, bt, ahat, bhat, total; bool direct; };
 
@@ -315,19 +320,12 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     g.A = A; g.lda = d->lda; g.a_batch = 0;
     g.B = bk_ptr; g.ldb = bk_ld; g.b_batch = 0;
   } else {
-    fmm_scheme one = classical_scheme_111();
-    CoefTable t;
-    std::memset(&t, 0, sizeof(t));
-    fmm_build_tables(one, &t, nullptr, nullptr);
-    FMM_CUDA(cudaMemcpyAsync(at<char>(ws, L.tab), &t, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
     const bool scaled = d->scale_mode != 0;
     float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
     float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
     ProfScope pe(5, st);
-    FMM_TRY(encode_operand(d, A, d->lda, 1, 1, d->M, d->K, at<CoefTable>(ws, L.tab), &t, at<char>(ws, L.ahat),
-                           d->M * d->K, at<unsigned>(ws, L.amaxA), sA, st));
-    FMM_TRY(encode_operand(d, bk_ptr, bk_ld, 1, 1, d->N, d->K, at<CoefTable>(ws, L.tab), &t, at<char>(ws, L.bhat),
-                           d->N * d->K, at<unsigned>(ws, L.amaxB), sB, st));
+    FMM_TRY(quantize_operand(d, A, d->lda, d->M, d->K, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
+    FMM_TRY(quantize_operand(d, bk_ptr, bk_ld, d->N, d->K, at<char>(ws, L.bhat), at<unsigned>(ws, L.amaxB), sB, st));
     g.A = at<char>(ws, L.ahat); g.lda = d->K; g.a_batch = 0;
     g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
     if (d->scale_mode == 2) { g.row_scale = sA; g.col_scale = sB; g.rs_batch = 0; g.cs_batch = 0; }

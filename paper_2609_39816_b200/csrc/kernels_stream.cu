@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdlib>
 
@@ -308,6 +309,110 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     __syncthreads();
     if (threadIdx.x < R && sm.amax[threadIdx.x] != 0u) atomicMax(&amax_bits[threadIdx.x], sm.amax[threadIdx.x]);
   }
+}
+
+// ------------------------------------------------------------------------------------------
+// Plain quantisation of one operand (the classical control: one cell, coefficient 1): rows x cols of SrcT ->
+// DstT with no scale (mode 0), one power-of-two scale per tensor (mode 1) or one scale per row (mode 2), the same
+// decisions as encode_kernel takes for a 1 x 1 grid.  A pure stream: each thread keeps four independent 16-byte
+// loads in flight, no shared memory.
+// ------------------------------------------------------------------------------------------
+template <typename SrcT, typename DstT, bool kAmaxOnly>
+__global__ void __launch_bounds__(256)
+quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols, DstT* __restrict__ out,
+                      unsigned* __restrict__ amax_bits, float* __restrict__ scale_out, int mode) {
+  constexpr int VE = Vec16<SrcT>::kElems;
+  constexpr int NP = VE / 2;
+  constexpr int kU = 4;
+  __shared__ unsigned s_amax;
+  const int64_t vec_per_row = cols / VE;
+  const int64_t nvec = rows * vec_per_row;
+  const int64_t stride = (int64_t)gridDim.x * 256;
+  float s = 1.0f, inv = 1.0f;
+  bool use_mul = true;
+  if (!kAmaxOnly && mode == 1) {
+    s = pow2_scale_448(__uint_as_float(amax_bits[0]));
+    inv = 1.0f / s;
+    use_mul = isfinite(inv) && inv * s == 1.0f && fabsf(inv) >= 1.17549435e-38f;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && scale_out) scale_out[0] = s;
+  }
+  if (kAmaxOnly && threadIdx.x == 0) s_amax = 0u;
+  if (kAmaxOnly) __syncthreads();
+  float tmax = 0.0f;
+  for (int64_t base = (int64_t)blockIdx.x * 256 + threadIdx.x; base < nvec; base += kU * stride) {
+    uint4 raw[kU];
+    int64_t row[kU];
+    int col[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const int64_t i = base + u * stride;
+      const bool on = i < nvec;
+      row[u] = on ? i / vec_per_row : 0;
+      col[u] = on ? (int)(i - row[u] * vec_per_row) * VE : 0;
+      raw[u] = on ? __ldcs(reinterpret_cast<const uint4*>(X + row[u] * ldx + col[u])) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const bool on = base + u * stride < nvec;
+      float2 v[NP];
+      Vec16<SrcT>::unpack(raw[u], v);
+      if (kAmaxOnly) {
+        float a = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(v[i].x), fabsf(v[i].y)));
+        if (mode == 2) {
+          if ((vec_per_row & 31) == 0) {   // a warp's 32 consecutive vectors lie in one row
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+            if ((threadIdx.x & 31) == 0 && on && a > 0.0f) atomicMax(&amax_bits[row[u]], __float_as_uint(a));
+          } else if (on && a > 0.0f) {
+            atomicMax(&amax_bits[row[u]], __float_as_uint(a));
+          }
+        } else {
+          tmax = fmaxf(tmax, a);
+        }
+      } else if (on) {
+        if (mode == 2) {
+          const float amax = __uint_as_float(amax_bits[row[u]]);
+          const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+          if (col[u] == 0 && scale_out) scale_out[row[u]] = sc;
+        } else if (mode == 1) {
+          if (use_mul) {
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { v[i].x *= inv; v[i].y *= inv; }
+          } else {
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, s); v[i].y = __fdiv_rn(v[i].y, s); }
+          }
+        }
+        store_vec<NP>(out + row[u] * cols + col[u], v, true);
+      }
+    }
+  }
+  if (kAmaxOnly && mode != 2) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    if ((threadIdx.x & 31) == 0 && tmax > 0.0f) atomicMax(&s_amax, __float_as_uint(tmax));
+    __syncthreads();
+    if (threadIdx.x == 0 && s_amax != 0u) atomicMax(&amax_bits[0], s_amax);
+  }
+}
+
+template <typename SrcT, typename DstT>
+static cudaError_t launch_quantize_plain_t(const void* X, int64_t ldx, int64_t rows, int64_t cols, void* out,
+                                           unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st) {
+  constexpr int VE = Vec16<SrcT>::kElems;
+  const int64_t nvec = rows * (cols / VE);
+  if (nvec == 0) return cudaSuccess;
+  const int grid = (int)std::min<int64_t>((nvec + 256 * 4 - 1) / (256 * 4), 148 * 16);
+  if (amax_only)
+    quantize_plain_kernel<SrcT, DstT, true><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode);
+  else
+    quantize_plain_kernel<SrcT, DstT, false><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode);
+  ++fmm_launch_counter();
+  return cudaGetLastError();
 }
 
 // Blocks of a streaming pass: enough to fill the machine about four times over, each block walking a
@@ -620,6 +725,20 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 }
 
 }  // namespace
+
+cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64_t ldx, int64_t rows, int64_t cols,
+                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st) {
+  if (storage == FMM_F32 && product == FMM_BF16)
+    return launch_quantize_plain_t<float, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+  if (storage == FMM_BF16 && product == FMM_BF16)
+    return launch_quantize_plain_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+  if (storage == FMM_F32 && product == FMM_E4M3)
+    return launch_quantize_plain_t<float, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+  if (storage == FMM_BF16 && product == FMM_E4M3)
+    return launch_quantize_plain_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+  return cudaErrorInvalidValue;
+}
+
 
 // ------------------------------------------------------------------------------------------
 // launch wrappers

@@ -24,6 +24,11 @@ cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, 
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
                           unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st);
 
+// The same decisions for a whole operand taken as one block with coefficient 1 (the classical control): rows x cols
+// of `storage` -> `product` dtype, mode 0 / 1 / 2 as use_scale above (amax_bits, scale: one word, or one per row).
+cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64_t ldx, int64_t rows, int64_t cols,
+                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st);
+
 // Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
                              cudaStream_t st);
