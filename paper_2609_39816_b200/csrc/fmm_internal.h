@@ -8,7 +8,7 @@
 
 constexpr int kMaxCells = FMM_MAX_GRID * FMM_MAX_GRID;  // blocks in one operand grid
 constexpr int kMaxNnz = FMM_MAX_R * kMaxCells;          // entries in one table (padding included)
-constexpr int kTablePad = 4;                            // every list is padded to a multiple of this
+constexpr int kTablePad = 2;                            // every list is padded to a multiple of this
 
 struct fmm_scheme {
   int m = 0, k = 0, n = 0, R = 0;

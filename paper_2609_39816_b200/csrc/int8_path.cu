@@ -210,7 +210,7 @@ decode_group_kernel(const float* __restrict__ prod, int64_t pstride, int G, cons
         }
         x = make_float4((float)xi.x, (float)xi.y, (float)xi.z, (float)xi.w);
       } else {
-        for (int e = sm.off[c]; e < e1; e += 2) {   // lists are padded to a multiple of four entries
+        for (int e = sm.off[c]; e < e1; e += 2) {   // lists are padded to an even number of entries
           const int4 two = *reinterpret_cast<const int4*>(&ent[e]);
           const float4 v0 = *reinterpret_cast<const float4*>(cur + two.x);
           const float4 v1 = *reinterpret_cast<const float4*>(cur + two.z);

@@ -214,50 +214,27 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     const unsigned char* my_stage = stage + (it & 1) * kStageBytes + pv * 16;
 
     DstT* dst = out + (int64_t)p * bc + t;
-    // two products per iteration (r and r + kEncSplit): their loads are issued together so that the two
-    // FMA chains overlap each other's shared-memory latency
-    for (int r0 = g; r0 < R; r0 += 2 * kEncSplit) {
-      const int r1 = r0 + kEncSplit;
-      const bool two = r1 < R;
+    // one product at a time, its list walked two entries per step (lists are padded to an even length with
+    // (zero slab, 0.0f) entries, which add exactly nothing); the four accumulator pairs are independent chains
+    for (int r0 = g; r0 < R; r0 += kEncSplit) {
+      constexpr bool two = false;
+      const int r1 = r0;
       float2 acc[2][NP];
 #pragma unroll
-      for (int j = 0; j < 2; ++j)
+      for (int i = 0; i < NP; ++i) acc[0][i] = make_float2(0.0f, 0.0f);
+      const int eend = sm.off[r0 + 1];
+      for (int e = sm.off[r0]; e < eend; e += 2) {
+        const int4 pair = *reinterpret_cast<const int4*>(&ent[e]);
+        const uint4 raw0 = *reinterpret_cast<const uint4*>(my_stage + pair.x);
+        const uint4 raw1 = *reinterpret_cast<const uint4*>(my_stage + pair.z);
+        float2 v[NP];
+        const float c0 = __int_as_float(pair.y), c1 = __int_as_float(pair.w);
+        Vec16<SrcT>::unpack(raw0, v);
 #pragma unroll
-        for (int i = 0; i < NP; ++i) acc[j][i] = make_float2(0.0f, 0.0f);
-      int e[2] = {sm.off[r0], two ? sm.off[r1] : 0};
-      const int eend[2] = {sm.off[r0 + 1], two ? sm.off[r1 + 1] : 0};
-      while (e[0] < eend[0] || e[1] < eend[1]) {
-        int2 en[2][kChunk];
-        uint4 raw[2][kChunk];
+        for (int i = 0; i < NP; ++i) acc[0][i] = __ffma2_rn(make_float2(c0, c0), v[i], acc[0][i]);
+        Vec16<SrcT>::unpack(raw1, v);
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const bool on = e[j] < eend[j];
-#pragma unroll
-          for (int u = 0; u < kChunk; u += 2) {
-            // an exhausted list reads the padding pattern (zero slab, 0.0f): adds exactly nothing
-            const int4 pair = on ? *reinterpret_cast<const int4*>(&ent[e[j] + u])
-                                 : make_int4(ncell * kSlab, 0, ncell * kSlab, 0);
-            en[j][u] = make_int2(pair.x, pair.y);
-            en[j][u + 1] = make_int2(pair.z, pair.w);
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-          for (int u = 0; u < kChunk; ++u) raw[j][u] = *reinterpret_cast<const uint4*>(my_stage + en[j][u].x);
-#pragma unroll
-        for (int u = 0; u < kChunk; ++u)
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const float c = __int_as_float(en[j][u].y);
-            const float2 cc = make_float2(c, c);
-            float2 v[NP];
-            Vec16<SrcT>::unpack(raw[j][u], v);
-#pragma unroll
-            for (int i = 0; i < NP; ++i) acc[j][i] = __ffma2_rn(cc, v[i], acc[j][i]);
-          }
-        e[0] += kChunk;
-        e[1] += kChunk;
+        for (int i = 0; i < NP; ++i) acc[0][i] = __ffma2_rn(make_float2(c1, c1), v[i], acc[0][i]);
       }
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
@@ -278,9 +255,9 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
             }
             continue;
           }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-          if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(&sm.amax[r], __float_as_uint(a));
+          // non-negative floats order like their bit patterns: one warp-wide integer max
+          const unsigned wmax = __reduce_max_sync(0xffffffffu, __float_as_uint(a));
+          if ((threadIdx.x & 31) == 0 && wmax != 0u) atomicMax(&sm.amax[r], wmax);
         } else if (live) {
           if (use_scale == 2) {
             // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
