@@ -60,12 +60,13 @@ __device__ __forceinline__ double block_sum_double(double v, double* red /* >= 8
 // encode: block sums of Eq. 1 (inner parentheses), scale, one rounding to the product dtype.
 // A block of 256 threads owns 64 "position vectors" (16 bytes = 8 bf16 or 4 fp32 consecutive
 // inner-dimension elements of one block row).  Four threads share each position vector:
-//   1. together they load the vectors of all grid cells at that position, convert them to fp32 once and
-//      park them in shared memory ([cell][half][position], conflict free; slab `ncell` holds zeros);
+//   1. together they copy the raw 16-byte vectors of all grid cells at that position into shared memory with
+//      cp.async ([cell][position], conflict free; slab `ncell` holds zeros), two stages deep, so the copies of
+//      the next tile overlap the arithmetic and the stores of this one;
 //   2. thread g of the four then forms the products r = g, g+4, g+8, ...: it walks the coefficient list
-//      of r in chunks of kChunk entries (lists are padded to a multiple of kChunk with (zero slab, 0.0f)
-//      entries, which add exactly nothing), an fp32 FMA chain in list order, two lanes per instruction
-//      (packed fma.rn.f32x2: each lane is an ordinary IEEE fp32 FMA), and stores 16 / 8 bytes.
+//      of r two entries per step (lists are padded to an even length with (zero slab, 0.0f) entries, which
+//      add exactly nothing), an fp32 FMA chain in list order, two lanes per instruction (packed
+//      fma.rn.f32x2: each lane is an ordinary IEEE fp32 FMA), and stores 16 / 8 bytes.
 // ------------------------------------------------------------------------------------------
 constexpr int kEncThreads = 256;
 // kEncSplit threads share one position vector (4 for the 4 x 4 grids / 49 products; 1 when the scheme is small,
@@ -216,14 +217,12 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     DstT* dst = out + (int64_t)p * bc + t;
     // one product at a time, its list walked two entries per step (lists are padded to an even length with
     // (zero slab, 0.0f) entries, which add exactly nothing); the four accumulator pairs are independent chains
-    for (int r0 = g; r0 < R; r0 += kEncSplit) {
-      constexpr bool two = false;
-      const int r1 = r0;
-      float2 acc[2][NP];
+    for (int r = g; r < R; r += kEncSplit) {
+      float2 acc[NP];
 #pragma unroll
-      for (int i = 0; i < NP; ++i) acc[0][i] = make_float2(0.0f, 0.0f);
-      const int eend = sm.off[r0 + 1];
-      for (int e = sm.off[r0]; e < eend; e += 2) {
+      for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
+      const int eend = sm.off[r + 1];
+      for (int e = sm.off[r]; e < eend; e += 2) {
         const int4 pair = *reinterpret_cast<const int4*>(&ent[e]);
         const uint4 raw0 = *reinterpret_cast<const uint4*>(my_stage + pair.x);
         const uint4 raw1 = *reinterpret_cast<const uint4*>(my_stage + pair.z);
@@ -231,54 +230,48 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
         const float c0 = __int_as_float(pair.y), c1 = __int_as_float(pair.w);
         Vec16<SrcT>::unpack(raw0, v);
 #pragma unroll
-        for (int i = 0; i < NP; ++i) acc[0][i] = __ffma2_rn(make_float2(c0, c0), v[i], acc[0][i]);
+        for (int i = 0; i < NP; ++i) acc[i] = __ffma2_rn(make_float2(c0, c0), v[i], acc[i]);
         Vec16<SrcT>::unpack(raw1, v);
 #pragma unroll
-        for (int i = 0; i < NP; ++i) acc[0][i] = __ffma2_rn(make_float2(c1, c1), v[i], acc[0][i]);
+        for (int i = 0; i < NP; ++i) acc[i] = __ffma2_rn(make_float2(c1, c1), v[i], acc[i]);
       }
+      if (kAmaxOnly) {
+        float a = 0.0f;
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int r = j == 0 ? r0 : r1;
-        if (j == 1 && !two) break;
-        if (kAmaxOnly) {
-          float a = 0.0f;
-#pragma unroll
-          for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[j][i].x), fabsf(acc[j][i].y)));   // fmaxf drops NaN
-          if (use_scale == 2) {
-            // one scale per row of the block sum: largest magnitude of row p of product r
-            if ((vec_per_row & 31) == 0) {       // a warp's 32 consecutive vectors lie in one row
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
-              if ((threadIdx.x & 31) == 0 && live && a > 0.0f) atomicMax(&amax_bits[(int64_t)r * br + p], __float_as_uint(a));
-            } else if (live && a > 0.0f) {
-              atomicMax(&amax_bits[(int64_t)r * br + p], __float_as_uint(a));
-            }
-            continue;
+        for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
+        if (use_scale == 2) {
+          // one scale per row of the block sum: largest magnitude of row p of product r
+          if ((vec_per_row & 31) == 0) {       // a warp's 32 consecutive vectors lie in one row
+            const unsigned wmax = __reduce_max_sync(0xffffffffu, live ? __float_as_uint(a) : 0u);
+            if ((threadIdx.x & 31) == 0 && wmax != 0u) atomicMax(&amax_bits[(int64_t)r * br + p], wmax);
+          } else if (live && a > 0.0f) {
+            atomicMax(&amax_bits[(int64_t)r * br + p], __float_as_uint(a));
           }
+        } else {
           // non-negative floats order like their bit patterns: one warp-wide integer max
           const unsigned wmax = __reduce_max_sync(0xffffffffu, __float_as_uint(a));
           if ((threadIdx.x & 31) == 0 && wmax != 0u) atomicMax(&sm.amax[r], wmax);
-        } else if (live) {
-          if (use_scale == 2) {
-            // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
-            const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
-            const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
-#pragma unroll
-            for (int i = 0; i < NP; ++i) { acc[j][i].x = __fdiv_rn(acc[j][i].x, sc); acc[j][i].y = __fdiv_rn(acc[j][i].y, sc); }
-            if (t == 0 && scale_out) scale_out[(int64_t)r * br + p] = sc;
-          } else if (use_scale) {
-            if (sm.use_mul[r]) {
-              const float inv = sm.inv_scale[r];
-#pragma unroll
-              for (int i = 0; i < NP; ++i) { acc[j][i].x *= inv; acc[j][i].y *= inv; }
-            } else {
-              const float sc = sm.scale[r];
-#pragma unroll
-              for (int i = 0; i < NP; ++i) { acc[j][i].x = __fdiv_rn(acc[j][i].x, sc); acc[j][i].y = __fdiv_rn(acc[j][i].y, sc); }
-            }
-          }
-          store_vec<NP>(dst + r * rstride, acc[j], stream_out != 0);
         }
+      } else if (live) {
+        if (use_scale == 2) {
+          // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
+          const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
+          const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+          if (t == 0 && scale_out) scale_out[(int64_t)r * br + p] = sc;
+        } else if (use_scale) {
+          if (sm.use_mul[r]) {
+            const float inv = sm.inv_scale[r];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { acc[i].x *= inv; acc[i].y *= inv; }
+          } else {
+            const float sc = sm.scale[r];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+          }
+        }
+        store_vec<NP>(dst + r * rstride, acc, stream_out != 0);
       }
     }
   }
