@@ -310,26 +310,31 @@ def run_ours(args):
     # Every step still copies all of its inputs from pinned host memory and its whole result back.
     def e2e_pipelined(steps):
         main = torch.cuda.current_stream()
-        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        s_in, s_in2, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         sets = [(A, B, C, ws, C_h)]
         sets.append((torch.empty_like(A), torch.empty_like(B), torch.empty_like(C), torch.empty_like(ws),
                      torch.empty_like(C_h).pin_memory()))
         ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_in2 = [torch.cuda.Event() for _ in range(2)]
         ev_comp = [torch.cuda.Event() for _ in range(2)]
         ev_out = [torch.cuda.Event() for _ in range(2)]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record(main)
-        s_in.wait_event(e0); s_out.wait_event(e0)
+        s_in.wait_event(e0); s_in2.wait_event(e0); s_out.wait_event(e0)
         for i in range(steps):
             Ad, Bd, Cd, wsd, Chd = sets[i % 2]
             with torch.cuda.stream(s_in):
                 if i >= 2:
                     s_in.wait_event(ev_comp[i % 2])        # step i-2 has finished reading this buffer set
                 Ad.copy_(A_h, non_blocking=True)
-                Bd.copy_(B_h, non_blocking=True)
                 ev_in[i % 2].record(s_in)
-            main.wait_event(ev_in[i % 2])
+            with torch.cuda.stream(s_in2):                 # the two operands travel on two copy streams
+                if i >= 2:
+                    s_in2.wait_event(ev_comp[i % 2])
+                Bd.copy_(B_h, non_blocking=True)
+                ev_in2[i % 2].record(s_in2)
+            main.wait_event(ev_in[i % 2]); main.wait_event(ev_in2[i % 2])
             if i >= 2:
                 main.wait_event(ev_out[i % 2])             # step i-2's result has left this C buffer
             flush.zero_()                                  # L2 discipline as in the device-timed region
