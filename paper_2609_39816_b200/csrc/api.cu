@@ -82,7 +82,7 @@ bool concurrency_enabled() {
 
 namespace {
 
-inline size_t align_up(size_t x, size_t a = 1024) { return (x + a - 1) / a * a; }
+inline size_t align_up(size_t x, size_t a = kPackedAlign) { return (x + a - 1) / a * a; }
 inline int esize(int dt) { return dt == FMM_F32 ? 4 : dt == FMM_BF16 ? 2 : 1; }
 
 constexpr int kMaxStreamPartials = 148 * 8;
@@ -402,14 +402,18 @@ fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* 
   FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool skip_b = (d->flags & FMM_FLAG_REUSE_BHAT) != 0;
-  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
-  CoefTable tA, tB, tW;
-  std::memset(&tA, 0, sizeof(tA)); std::memset(&tB, 0, sizeof(tB)); std::memset(&tW, 0, sizeof(tW));
-  fmm_build_tables(*s, &tA, &tB, &tW);
+  // one copy brings a zeroed status block and the three kernel tables (cached in the handle) to the head of the
+  // workspace, whose layout they mirror
+  const std::vector<unsigned char>& packed = fmm_packed_tables(*s);
+  if (L.status != 0 || L.tabA != kPackedStatusBytes || L.tabB != L.tabA + fmm_packed_table_stride() ||
+      L.tabW != L.tabB + fmm_packed_table_stride() || sizeof(DeviceStatus) > kPackedStatusBytes)
+    return FMM_ERR_CUDA;
+  FMM_CUDA(cudaMemcpyAsync(d_ws, packed.data(), packed.size(), cudaMemcpyHostToDevice, st));
   const void* bk_ptr; int64_t bk_ld;
   FMM_TRY(kmajor_b(d, dB, d_ws, L.bt, &bk_ptr, &bk_ld, skip_b, st));
-  return run_scheme(s, d, L, &tA, &tB, &tW, nullptr, nullptr, nullptr, dA, bk_ptr, bk_ld, dC, nullptr, nullptr, d_ws,
-                    skip_b, st);
+  return run_scheme(s, d, L, fmm_packed_table(*s, 0), fmm_packed_table(*s, 1), fmm_packed_table(*s, 2),
+                    at<CoefTable>(d_ws, L.tabA), at<CoefTable>(d_ws, L.tabB), at<CoefTable>(d_ws, L.tabW), dA, bk_ptr, bk_ld, dC,
+                    nullptr, nullptr, d_ws, skip_b, st);
 }
 
 fmm_status fmm_device_status(const void* d_ws, void* cuda_stream) {

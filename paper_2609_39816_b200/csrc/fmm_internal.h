@@ -2,6 +2,7 @@
 #pragma once
 #include <cstdint>
 #include <memory>
+#include <mutex>
 #include <vector>
 
 #include "fmm_b200.h"
@@ -10,11 +11,25 @@ constexpr int kMaxCells = FMM_MAX_GRID * FMM_MAX_GRID;  // blocks in one operand
 constexpr int kMaxNnz = FMM_MAX_R * kMaxCells;          // entries in one table (padding included)
 constexpr int kTablePad = 2;                            // every list is padded to a multiple of this
 
+struct CoefTable;
+
 struct fmm_scheme {
   int m = 0, k = 0, n = 0, R = 0;
   std::vector<double> U, V, W;                 // [R][m][k], [R][k][n], [R][m][n]
   std::unique_ptr<fmm_scheme> outer, inner;    // factors, when built by scheme_kron
+  // Kernel tables of this scheme, built once on first use (a handle's coefficients never change): a zeroed
+  // device-status block followed by the encode-A, encode-B and decode tables, laid out exactly as the head of a
+  // scheme_gemm workspace so that one copy uploads all of it.
+  mutable std::once_flag tables_once;
+  mutable std::vector<unsigned char> packed_tables;
 };
+
+// Offsets inside fmm_scheme::packed_tables (and inside the head of a scheme_gemm workspace).
+constexpr size_t kPackedAlign = 1024;           // alignment of every region of a workspace
+constexpr size_t kPackedStatusBytes = 1024;     // the status block's slot (the block itself is 256 bytes)
+size_t fmm_packed_table_stride();              // sizeof(CoefTable) rounded up to kPackedAlign
+const std::vector<unsigned char>& fmm_packed_tables(const fmm_scheme& s);
+const CoefTable* fmm_packed_table(const fmm_scheme& s, int which);   // 0: A, 1: B, 2: W (host copies)
 
 // Sparse coefficient table as the kernels read it: R lists of (slab, coefficient) pairs in the order in
 // which they are to be accumulated, each list padded to a multiple of kTablePad with (ncell, 0.0f).

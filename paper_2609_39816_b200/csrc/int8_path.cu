@@ -439,12 +439,13 @@ struct Int8Layout {
   bool trivial;
 };
 
-fmm_scheme trivial_scheme() {
-  fmm_scheme c;
-  c.m = c.k = c.n = c.R = 1;
-  c.U = {1.0}; c.V = {1.0}; c.W = {1.0};
-  return c;
-}
+// the classical algorithm <1,1,1;1> as a scheme
+struct TrivialScheme : fmm_scheme {
+  TrivialScheme() {
+    m = k = n = R = 1;
+    U = {1.0}; V = {1.0}; W = {1.0};
+  }
+};
 
 fmm_status int8_shape_ok(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
   if (M <= 0 || K <= 0 || N <= 0 || K % kGroup) return FMM_ERR_SHAPE;
@@ -540,7 +541,7 @@ bool corrected_certificate(const fmm_scheme& s, int h, double cert[4]) {
 extern "C" {
 
 int scheme_certificate(const fmm_scheme* s, int bA, int bB, int h, int g, int acc_bits, double cert[4]) {
-  fmm_scheme one = trivial_scheme();
+  TrivialScheme one;
   const fmm_scheme& sc = s ? *s : one;
   double meta[8];
   if (scheme_info(&sc, nullptr, meta) != FMM_OK) return 0;
@@ -572,7 +573,7 @@ fmm_status int8_quantize(const void* d_X, int storage, int64_t rows, int64_t K, 
 }
 
 size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N) {
-  fmm_scheme one = trivial_scheme();
+  TrivialScheme one;
   const fmm_scheme& sc = s ? *s : one;
   if (int8_shape_ok(sc, M, K, N) != FMM_OK) return 0;
   return int8_layout(sc, M, K, N).total;
@@ -584,7 +585,7 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
   if (!d_cA || !d_dA || !d_cB || !d_dB || !d_C) return FMM_ERR_ARG;
   if (output != FMM_F32 && output != FMM_BF16) return FMM_ERR_DTYPE;
   if (code_bound < 1 || code_bound > 127) return FMM_ERR_ARG;
-  fmm_scheme one = trivial_scheme();
+  TrivialScheme one;
   const fmm_scheme& sc = s ? *s : one;
   FMM_TRY(int8_shape_ok(sc, M, K, N));
   const int eo = output == FMM_F32 ? 4 : 2;

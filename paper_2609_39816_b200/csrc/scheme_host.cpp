@@ -226,6 +226,23 @@ void fmm_build_tables(const fmm_scheme& s, CoefTable* tA, CoefTable* tB, CoefTab
   }
 }
 
+size_t fmm_packed_table_stride() { return (sizeof(CoefTable) + kPackedAlign - 1) / kPackedAlign * kPackedAlign; }
+
+const std::vector<unsigned char>& fmm_packed_tables(const fmm_scheme& s) {
+  std::call_once(s.tables_once, [&s] {
+    const size_t stride = fmm_packed_table_stride();
+    s.packed_tables.assign(kPackedStatusBytes + 3 * stride, 0);
+    CoefTable* t = reinterpret_cast<CoefTable*>(s.packed_tables.data() + kPackedStatusBytes);
+    auto tab = [&](int w) { return reinterpret_cast<CoefTable*>(reinterpret_cast<unsigned char*>(t) + w * stride); };
+    fmm_build_tables(s, tab(0), tab(1), tab(2));
+  });
+  return s.packed_tables;
+}
+
+const CoefTable* fmm_packed_table(const fmm_scheme& s, int which) {
+  return reinterpret_cast<const CoefTable*>(fmm_packed_tables(s).data() + kPackedStatusBytes + which * fmm_packed_table_stride());
+}
+
 fmm_status fmm_gauge_core(const fmm_scheme& in, int level, const double* P, const double* Q, const double* S,
                           double cond_limit, fmm_scheme** out) {
   std::unique_ptr<fmm_scheme> res(new (std::nothrow) fmm_scheme);
