@@ -204,6 +204,26 @@ fmm_status stage_encode_b(const SchemeRun& r, const void* Bk, int64_t ldbk, cuda
   return encode_operand(r.d, Bk, ldbk, s->n, s->k, r.d->N / s->n, r.d->K / s->k, r.dB, r.hB, at<char>(r.ws, r.L.bhat),
                         r.L.sBhat, at<unsigned>(r.ws, r.L.amaxB), r.sB(), st);
 }
+// Both operands in one launch per pass (amax pass if scaled, then the encode pass), on one stream.
+fmm_status stage_encode_pair(const SchemeRun& r, const void* A, const void* Bk, int64_t ldbk, cudaStream_t st) {
+  const fmm_scheme* s = r.s;
+  const fmm_gemm_desc* d = r.d;
+  const int64_t bm = d->M / s->m, bk = d->K / s->k, bn = d->N / s->n;
+  const EncodeOperand oa{A, d->lda, s->m, s->k, bm, bk, r.dA, r.hA, at<char>(r.ws, r.L.ahat), r.L.sAhat,
+                         at<unsigned>(r.ws, r.L.amaxA), r.sA()};
+  const EncodeOperand ob{Bk, ldbk, s->n, s->k, bn, bk, r.dB, r.hB, at<char>(r.ws, r.L.bhat), r.L.sBhat,
+                         at<unsigned>(r.ws, r.L.amaxB), r.sB()};
+  ProfScope ps(0, st);
+  const int mode = d->scale_mode;
+  if (mode != 0) {
+    // amaxA and amaxB are neighbours in the workspace: one memset clears both
+    FMM_CUDA(cudaMemsetAsync(at<char>(r.ws, r.L.amaxA), 0, r.L.sA - r.L.amaxA, st));
+    FMM_CUDA(launch_encode_pair(d->storage, d->product, oa, &ob, true, mode, st));
+  }
+  FMM_CUDA(launch_encode_pair(d->storage, d->product, oa, &ob, false, mode, st));
+  return FMM_OK;
+}
+
 fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   const fmm_scheme* s = r.s;
   const int64_t bm = r.d->M / s->m, bk = r.d->K / s->k, bn = r.d->N / s->n;
@@ -255,16 +275,24 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
     dW_tab = at<CoefTable>(ws, L.tabW);
   }
   const SchemeRun r{s, d, L, ws, hA, hB, hW, dA_tab, dB_tab, dW_tab};
-  // encode A on the caller's stream and encode B beside it on the side stream (they share nothing)
-  SideStream* side = (!skip_b && concurrency_enabled()) ? side_stream() : nullptr;
-  cudaStream_t stB = st;
-  if (side) {
-    if (!stream_wait(side, st, side->stream)) return FMM_ERR_CUDA;
-    stB = side->stream;
+  // encode A and encode B side by side: one launch whose blocks split between the two operands (they share nothing);
+  // with the side stream enabled by the environment the two run as separate launches on two streams instead
+  static const bool two_streams = [] { const char* e = std::getenv("FMM_B200_ENCODE_TWO_STREAMS"); return e && e[0] == '1'; }();
+  if (skip_b) {
+    FMM_TRY(stage_encode_a(r, A, st));
+  } else if (!two_streams) {
+    FMM_TRY(stage_encode_pair(r, A, Bsrc_kmajor, ldb_kmajor, st));
+  } else {
+    SideStream* side = concurrency_enabled() ? side_stream() : nullptr;
+    cudaStream_t stB = st;
+    if (side) {
+      if (!stream_wait(side, st, side->stream)) return FMM_ERR_CUDA;
+      stB = side->stream;
+    }
+    FMM_TRY(stage_encode_b(r, Bsrc_kmajor, ldb_kmajor, stB));
+    FMM_TRY(stage_encode_a(r, A, st));
+    if (side && !stream_wait(side, side->stream, st)) return FMM_ERR_CUDA;
   }
-  if (!skip_b) FMM_TRY(stage_encode_b(r, Bsrc_kmajor, ldb_kmajor, stB));
-  FMM_TRY(stage_encode_a(r, A, st));
-  if (side && !stream_wait(side, side->stream, st)) return FMM_ERR_CUDA;
   FMM_TRY(stage_products(r, st));
   return stage_decode(r, C, cstar32, err_out, st);
 }

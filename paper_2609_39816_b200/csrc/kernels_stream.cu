@@ -131,11 +131,30 @@ template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* 
   }
 }
 
+// One operand of an encode launch.  A launch carries up to two (A and B of one product): blocks [0, a.blocks) work
+// on the first, the rest on the second, so both operands are encoded side by side without a second stream.
+struct EncodeJob {
+  const void* X; int64_t ldx; int gc; int64_t br, bc;
+  const CoefTable* tab; void* out; unsigned* amax_bits; float* scale_out;
+  int tiles_per_block; int64_t rstride; int stream_out; int blocks;
+};
+
 template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
 __global__ void __launch_bounds__(kEncThreads)
-encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64_t bc,
-              const CoefTable* __restrict__ d_tab, DstT* __restrict__ out, unsigned* __restrict__ amax_bits,
-              float* __restrict__ scale_out, int use_scale, int tiles_per_block, int64_t rstride, int stream_out) {
+encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
+  const bool second = (int)blockIdx.x >= job_a.blocks;
+  const int bid = (int)blockIdx.x - (second ? job_a.blocks : 0);
+  const SrcT* __restrict__ X = static_cast<const SrcT*>(second ? job_b.X : job_a.X);
+  const int64_t ldx = second ? job_b.ldx : job_a.ldx;
+  const int gc = second ? job_b.gc : job_a.gc;
+  const int64_t br = second ? job_b.br : job_a.br, bc = second ? job_b.bc : job_a.bc;
+  const CoefTable* __restrict__ d_tab = second ? job_b.tab : job_a.tab;
+  DstT* __restrict__ out = static_cast<DstT*>(second ? job_b.out : job_a.out);
+  unsigned* __restrict__ amax_bits = second ? job_b.amax_bits : job_a.amax_bits;
+  float* __restrict__ scale_out = second ? job_b.scale_out : job_a.scale_out;
+  const int tiles_per_block = second ? job_b.tiles_per_block : job_a.tiles_per_block;
+  const int64_t rstride = second ? job_b.rstride : job_a.rstride;
+  const int stream_out = second ? job_b.stream_out : job_a.stream_out;
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kEncSplit;
   constexpr int kCellsPerThread = 16 / kEncSplit; // grids have at most 16 cells
@@ -161,7 +180,7 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
     sm.use_mul[threadIdx.x] = (isfinite(inv) && inv * s == 1.0f && fabsf(inv) >= 1.17549435e-38f);
     sm.inv_scale[threadIdx.x] = inv;
     sm.amax[threadIdx.x] = 0u;
-    if (!kAmaxOnly && use_scale == 1 && blockIdx.x == 0 && scale_out) scale_out[threadIdx.x] = s;
+    if (!kAmaxOnly && use_scale == 1 && bid == 0 && scale_out) scale_out[threadIdx.x] = s;
   }
 
   const int g = threadIdx.x / kEncPos;           // which share of the cells / products this thread handles
@@ -185,7 +204,7 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   // asynchronous copies of this thread's cells of tile `it` into stage `it & 1` (16 bytes each, L2 only)
   auto issue_copies = [&](int it) {
     if (it < tiles_per_block) {
-      const int idx = (blockIdx.x * tiles_per_block + it) * kEncPos + pv;
+      const int idx = (bid * tiles_per_block + it) * kEncPos + pv;
       const bool live = idx < nvec;
       const int p = live ? idx / vec_per_row : 0;
       const int t = live ? (idx - p * vec_per_row) * VE : 0;
@@ -205,7 +224,7 @@ encode_kernel(const SrcT* __restrict__ X, int64_t ldx, int gc, int64_t br, int64
   issue_copies(0);
 
   for (int it = 0; it < tiles_per_block; ++it) {
-    const int idx = (blockIdx.x * tiles_per_block + it) * kEncPos + pv;
+    const int idx = (bid * tiles_per_block + it) * kEncPos + pv;
     const bool live = idx < nvec;
     const int p = live ? idx / vec_per_row : 0;
     const int t = live ? (idx - p * vec_per_row) * VE : 0;
@@ -396,22 +415,33 @@ static void split_tiles(int64_t tiles, int* grid, int* tiles_per_block) {
 
 static int padded_entries(const CoefTable& t) { return t.off[t.R]; }   // lists arrive padded from the host
 
+// Host description of one operand of an encode launch (see launch_encode_pair).
 template <typename SrcT, typename DstT, int kSplit>
-cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
-                            const CoefTable* d_tab, int padded, int lists, void* out, int64_t out_stride,
-                            unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
+static bool make_job(const EncodeOperand& o, EncodeJob* j, size_t* smem) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kSplit;
-  const size_t smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 +
-                      2 * (size_t)(gr * gc + 1) * kEncPos * 16;
-  const int64_t vecs = br * (bc / VE);
-  if (vecs == 0) return cudaSuccess;
-  if (vecs + kEncThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // kernels index positions in 32 bits
-  int grid, tpb;
-  split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
+  const int padded = padded_entries(*o.h_tab);
+  *smem = ((sizeof(EncSmemHead) + (size_t)padded * 8 + 15) / 16) * 16 + 2 * (size_t)(o.gr * o.gc + 1) * kEncPos * 16;
+  const int64_t vecs = o.br * (o.bc / VE);
+  if (vecs + kEncThreads * 8 >= (int64_t)1 << 31) return false;   // kernels index positions in 32 bits
+  int grid = 0, tpb = 1;
+  if (vecs > 0) split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
   // outputs larger than the part of L2 that keeps shared data (~60 MB) will have left it before they are read
-  int stream_out = (int64_t)lists * out_stride * (int64_t)sizeof(DstT) > ((int64_t)48 << 20) ? 1 : 0;
+  int stream_out = (int64_t)o.h_tab->R * o.out_stride * (int64_t)sizeof(DstT) > ((int64_t)48 << 20) ? 1 : 0;
   if (const char* e = std::getenv("FMM_B200_ENC_STREAM")) stream_out = std::atoi(e);
+  *j = EncodeJob{o.X, o.ldx, o.gc, o.br, o.bc, o.d_tab, o.out, o.amax_bits, o.scale, tpb, o.out_stride, stream_out, grid};
+  return true;
+}
+
+template <typename SrcT, typename DstT, int kSplit>
+cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool amax_only, int use_scale, cudaStream_t st) {
+  EncodeJob ja{}, jb{};
+  size_t smem_a = 0, smem_b = 0;
+  if (!make_job<SrcT, DstT, kSplit>(a, &ja, &smem_a)) return cudaErrorInvalidValue;
+  if (b && !make_job<SrcT, DstT, kSplit>(*b, &jb, &smem_b)) return cudaErrorInvalidValue;
+  const int grid = ja.blocks + jb.blocks;
+  if (grid == 0) return cudaSuccess;
+  const size_t smem = std::max(smem_a, smem_b);
   static bool attr_done[2] = {false, false};
   if (amax_only) {
     auto k = encode_kernel<SrcT, DstT, true, kSplit>;
@@ -420,7 +450,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[0] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride, stream_out);
+    k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
   } else {
     auto k = encode_kernel<SrcT, DstT, false, kSplit>;
     if (!attr_done[1]) {
@@ -428,7 +458,7 @@ cudaError_t launch_encode_t(const void* X, int64_t ldx, int gr, int gc, int64_t 
       if (e != cudaSuccess) return e;
       attr_done[1] = true;
     }
-    k<<<grid, kEncThreads, smem, st>>>((const SrcT*)X, ldx, gc, br, bc, d_tab, (DstT*)out, amax_bits, scale, use_scale, tpb, out_stride, stream_out);
+    k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
   }
   ++fmm_launch_counter();
   return cudaGetLastError();
@@ -714,28 +744,33 @@ cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64
 // launch wrappers
 // ------------------------------------------------------------------------------------------
 template <int kSplit>
-static cudaError_t launch_encode_split(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
-                                       int64_t bc, const CoefTable* d_tab, int nnz, int lists, void* out, int64_t out_stride,
-                                       unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
+static cudaError_t launch_encode_split(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
+                                       int use_scale, cudaStream_t st) {
   if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_encode_t<float, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_bfloat16, kSplit>(a, b, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_encode_t<__nv_bfloat16, __nv_bfloat16, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_bfloat16, kSplit>(a, b, amax_only, use_scale, st);
   if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_encode_t<float, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<float, __nv_fp8_storage_t, kSplit>(a, b, amax_only, use_scale, st);
   if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t, kSplit>(X, ldx, gr, gc, br, bc, d_tab, nnz, lists, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+    return launch_encode_t<__nv_bfloat16, __nv_fp8_storage_t, kSplit>(a, b, amax_only, use_scale, st);
   return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
+                               int use_scale, cudaStream_t st) {
+  // both operands of a product share the thread split: small schemes (at most 4 cells in either grid): one thread
+  // per position vector; otherwise four threads share one
+  const int cells = std::max(a.gr * a.gc, b ? b->gr * b->gc : 0);
+  if (cells <= 4) return launch_encode_split<1>(storage, product, a, b, amax_only, use_scale, st);
+  return launch_encode_split<4>(storage, product, a, b, amax_only, use_scale, st);
 }
 
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
                           unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
-  const int nnz = padded_entries(*h_tab);
-  // small schemes (at most 4 cells): one thread per position vector; otherwise four threads share one
-  if (gr * gc <= 4)
-    return launch_encode_split<1>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, h_tab->R, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
-  return launch_encode_split<4>(storage, product, X, ldx, gr, gc, br, bc, d_tab, nnz, h_tab->R, out, out_stride, amax_bits, scale, amax_only, use_scale, st);
+  const EncodeOperand a{X, ldx, gr, gc, br, bc, d_tab, h_tab, out, out_stride, amax_bits, scale};
+  return launch_encode_pair(storage, product, a, nullptr, amax_only, use_scale, st);
 }
 
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,

@@ -29,6 +29,15 @@ cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, 
 cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64_t ldx, int64_t rows, int64_t cols,
                                   void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st);
 
+// Two operands in one launch (A and B of one product, encoded side by side); b may be null.  Fields as the arguments
+// of launch_encode.
+struct EncodeOperand {
+  const void* X; int64_t ldx; int gr, gc; int64_t br, bc;
+  const CoefTable* d_tab; const CoefTable* h_tab; void* out; int64_t out_stride; unsigned* amax_bits; float* scale;
+};
+cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
+                               int use_scale, cudaStream_t st);
+
 // Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
                              cudaStream_t st);
