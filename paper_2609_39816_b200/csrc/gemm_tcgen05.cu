@@ -252,6 +252,7 @@ __global__ void __launch_bounds__(kNumThreads, 1)
 block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                       void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
                       TileParams tp, DeviceStatus* status) {
+  grid_launch_dependents();   // the decode may set up while this grid drains; it waits before reading the products
   using L = SmemLayout<BN>;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment of the swizzled tiles
@@ -290,6 +291,7 @@ block_products_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dependency_wait();     // operands and scales come from the previous kernel of the stream
 
   const int num_kb = (tp.kbytes + BKB - 1) / BKB;
   const int tiles_per_batch = tp.tiles_m * tp.tiles_n;
@@ -489,6 +491,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                            void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
                            TileParams tp, DeviceStatus* status) {
+  grid_launch_dependents();   // the decode may set up while this grid drains; it waits before reading the products
   using L = PairLayout;
   constexpr int BN = L::BN;
   extern __shared__ unsigned char smem_raw[];
@@ -529,6 +532,7 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
   cluster_sync_all();   // both CTAs' barriers are initialised before anything signals across the pair
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  grid_dependency_wait();     // operands and scales come from the previous kernel of the stream
 
   const int num_kb = (tp.kbytes + BKB - 1) / BKB;
   const int tiles_m = (tp.rows_a + 2 * BM - 1) / (2 * BM);
@@ -733,7 +737,8 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   const int grid = (int)(total < sms ? total : sms);
   auto k = block_products_kernel<BN, kFp8>;
   if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
-  k<<<grid, kNumThreads, L::kTotal, st>>>(ma, mb, a.out, a.sA, a.sB, tp, a.status);
+  if (launch_dependent(k, dim3(grid), dim3(kNumThreads), (size_t)L::kTotal, st, ma, mb, a.out, a.sA, a.sB, tp, a.status) != cudaSuccess)
+    return FMM_ERR_CUDA;
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
@@ -770,7 +775,8 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
     attr_done = true;
   }
-  k<<<(unsigned)(2 * pairs), kNumThreads, L::kTotal, st>>>(ma, mb, a.out, a.sA, a.sB, tp, a.status);
+  if (launch_dependent(k, dim3((unsigned)(2 * pairs)), dim3(kNumThreads), (size_t)L::kTotal, st, ma, mb, a.out, a.sA, a.sB, tp, a.status) != cudaSuccess)
+    return FMM_ERR_CUDA;
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }

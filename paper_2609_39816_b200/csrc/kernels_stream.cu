@@ -15,6 +15,11 @@ int64_t& fmm_launch_counter() {
   return c;
 }
 
+bool fmm_pdl_enabled() {
+  static const bool on = [] { const char* e = std::getenv("FMM_B200_NO_PDL"); return !(e && e[0] == '1'); }();
+  return on;
+}
+
 namespace {
 
 
@@ -142,6 +147,7 @@ struct EncodeJob {
 template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
+  grid_launch_dependents();   // the block products may set up while this grid drains; they wait before reading
   const bool second = (int)blockIdx.x >= job_a.blocks;
   const int bid = (int)blockIdx.x - (second ? job_a.blocks : 0);
   const SrcT* __restrict__ X = static_cast<const SrcT*>(second ? job_b.X : job_a.X);
@@ -522,6 +528,7 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
               double* __restrict__ partials, int tiles_per_block, int64_t rstride) {
   constexpr int kDecPos = kDecThreads / kDecSplit;
   constexpr int kCellsPerThread = 16 / kDecSplit;
+  grid_dependency_wait();     // the products (and scales) come from the previous kernel of the stream
   constexpr int kVecBytes = 4 * (int)sizeof(ProdT);   // one position quad of products: 16 bytes (fp32) or 8 (bf16)
   constexpr int kSlab = kDecPos * kVecBytes;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -813,7 +820,9 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
       if (e != cudaSuccess) return e;                                                                            \
       attr_done[SLOT] = true;                                                                                    \
     }                                                                                                            \
-    k<<<grid, kDecThreads, smem, st>>>(prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, cstar32, ldcs, partials, tpb, prod_stride); \
+    cudaError_t le = launch_dependent(k, dim3(grid), dim3(kDecThreads), smem, st, prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, \
+                                      cstar32, ldcs, partials, tpb, prod_stride);                                 \
+    if (le != cudaSuccess) return le;                                                                            \
   }
   if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true, 0)
   else if (C != nullptr) FMM_DECODE_LAUNCH(true, false, 1)

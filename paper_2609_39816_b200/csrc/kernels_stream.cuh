@@ -13,6 +13,28 @@ struct DeviceStatus {
 
 int64_t& fmm_launch_counter();
 
+// Programmatic dependent launch: a kernel launched with launch_dependent may begin (prologue: barrier set-up,
+// TMEM allocation, table loads) while the previous kernel of the same stream drains; it must execute
+// grid_dependency_wait() before it touches anything that kernel wrote.  Kernels that may be followed by such a launch
+// call grid_launch_dependents() early.  Both are no-ops when the launch carries no programmatic dependency.
+// FMM_B200_NO_PDL=1 in the environment turns the attribute off (ordinary stream order).
+bool fmm_pdl_enabled();
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = fmm_pdl_enabled() ? 1 : 0;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // X: source matrix (storage dtype), rows x cols with leading dimension ldx, split into a gr x gc grid of
 // br x bc blocks.  out: R blocks [br][bc] in the product dtype, out_stride elements apart.  With amax_only the kernel only accumulates
 // max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).
