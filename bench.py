@@ -165,6 +165,8 @@ def run_reference(args):
         return
     import oracle
     oracle.build()
+    # all host cores, also under launchers that export OMP_NUM_THREADS=1 for their workers
+    oracle.set_num_threads(len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1))
     _, _, A64, B64 = c2_inputs(0)
     rpb = 256
     val, t, cores, rows = time_oracle(A64, B64, rpb, args.steps, args.warmup)
