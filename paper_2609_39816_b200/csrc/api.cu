@@ -596,10 +596,16 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
                         d_tabs + 3 * g, d_tabs + 3 * g + 1, d_tabs + 3 * g + 2};
       // encode: the products of gauge g-2 must have finished reading this buffer's Ahat / Bhat
       if (evG[b] && cudaStreamWaitEvent(sE, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
-      // two launches here, not the paired one: beside the products and decode of the neighbouring gauges the two
-      // smaller kernels pack better (measured 8.06 k against 7.71 k gauges/s at the benchmark shape)
-      FMM_TRY(stage_encode_b(r, bk_ptr, bk_ld, sE));
-      FMM_TRY(stage_encode_a(r, dA, sE));
+      // Large operands: two launches, not the paired one — beside the products and decode of the neighbouring gauges
+      // the two smaller kernels pack better (measured 8.06 k against 7.71 k gauges/s at 2048 x 4096 x 4096).  Small
+      // operands are launch-bound: one paired launch (19.8 k against 14.1 k realisations/s at 128^3).
+      const bool small_operands = (d->M + d->N) * d->K * (int64_t)esize(d->storage) < ((int64_t)16 << 20);
+      if (small_operands) {
+        FMM_TRY(stage_encode_pair(r, dA, bk_ptr, bk_ld, sE));
+      } else {
+        FMM_TRY(stage_encode_b(r, bk_ptr, bk_ld, sE));
+        FMM_TRY(stage_encode_a(r, dA, sE));
+      }
       cudaEvent_t evE = record_event(side, sE);
       // products: need this gauge's encode, and the decode of gauge g-2 must be done with this product buffer
       if (!evE || cudaStreamWaitEvent(sG, evE, 0) != cudaSuccess) return FMM_ERR_CUDA;
