@@ -276,7 +276,8 @@ size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N)
 
 /* The int8 operator on quantised operands: d_cA int8 [M][K] with scales d_dA [M][K/128], d_cB int8 [N][K]
  * with d_dB [N][K/128] (all DEVICE, code pointers 8-byte aligned); d_C: DEVICE [M][ldc] of `output` (FMM_F32
- * or FMM_BF16, 16-byte aligned rows).  s == NULL computes every group's integer product classically; otherwise
+ * or FMM_BF16, 16-byte aligned rows).  s == NULL computes every group's integer product classically, in one kernel
+ * (int8 tensor-core products with int32 accumulators, the rescale in its epilogue; code pointers 16-byte aligned); otherwise
  * each group's product is computed by one call of s on the group's 128 inner indices split into k blocks of
  * length 128/k (which must be 32, 64 or 128), rows into m and columns into n contiguous blocks.  Codes, block
  * sums and all partial sums are integers held exactly (bf16 operands <= 127, fp32 accumulators < 2^24), so

@@ -126,6 +126,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
@@ -790,7 +799,261 @@ bool pair_kernel_enabled() {
   return on == 1;
 }
 
+// ---------------------------------------------------------------- group-scaled int8 GEMM
+// The classical int8 operator of the quantisation specification (Appendix D) as one kernel:
+//     C[t][j] = rnd_O( sum over groups g, ascending, of (float(P_g[t][j]) * dA[t][g]) * dB[j][g] ),
+//     P_g = exact integer product of the int8 codes of group g (128 inner indices).
+// One CTA owns a 128 x 128 output tile.  Warp 0 streams, per group, the 128 x 128-byte code tiles of A and B (one
+// 128-byte swizzle span = one group) through a shared-memory ring; one lane of warp 1 issues four tcgen05.mma
+// kind::i8 (K = 32 each) per group into one of two int32 accumulator buffers in TMEM, a FRESH accumulator per group;
+// warps 2-5 read the finished group's accumulator, convert it exactly to fp32, apply the two scales with two separate
+// roundings, and add to 128 fp32 accumulators per thread (one output row each); after the last group one rounding to
+// the output dtype.  The MMA of group g+1 overlaps the rescale of group g.
+struct Int8Layout {
+  static constexpr int BN = 128;
+  static constexpr int kStages = 5;
+  static constexpr int kABytes = BM * BKB;
+  static constexpr int kBBytes = BN * BKB;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarBytes = 256;
+  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;
+};
+
+struct Int8Params {
+  int M, N, G;                  // rows of A, rows of B (= output columns), groups of 128 along K
+  int tiles_m, tiles_n;
+  long long ldc;
+  int out_bf16;
+  int wide;                     // every output row starts on a 32-byte boundary
+  const float* dAt;             // [G][M] row scales, group-major
+  const float* dBt;             // [G][N] column scales, group-major
+  unsigned long long wait_limit_ns;
+};
+
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+constexpr int kInt8Threads = 320;   // 10 warps: TMA, MMA, and 8 rescale warps (two per TMEM lane quarter, 64 columns each)
+
+__global__ void __launch_bounds__(kInt8Threads, 1)
+int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                       void* __restrict__ out, Int8Params p, DeviceStatus* status) {
+  using L = Int8Layout;
+  constexpr int BN = L::BN;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - raw_addr);
+  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
+  const uint32_t bar_base = smem_u32(bar_mem);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr uint32_t kTmemCols = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int total_tiles = p.tiles_m * p.tiles_n;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+        for (int g = 0; g < p.G; ++g) {
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x41, status, p.wait_limit_ns);
+          if (!ok) break;
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::kStageBytes);
+          tma_load_3d(sa, &map_a, full_bar(stage), g * BKB, tm * BM, 0);
+          tma_load_3d(sa + L::kABytes, &map_b, full_bar(stage), g * BKB, tn * BN, 0);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        for (int s = 0; s < L::kStages; ++s) {
+          const uint32_t last_parity = (s < stage) ? phase : (phase ^ 1u);
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(s), last_parity)) {
+            if (global_timer_ns() - t0 > 20000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer: one fresh accumulator per group
+    if (lane == 0) {
+      // int32 accumulator (c format 2), signed 8-bit A and B (format 1), K-major, N >> 3, M >> 4
+      constexpr uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int g = 0; g < p.G; ++g) {
+          ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x52, status, p.wait_limit_ns);
+          if (!ok) break;
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x51, status, p.wait_limit_ns);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + L::kABytes);
+#pragma unroll
+          for (int k = 0; k < BKB / UMMA_KB; ++k)
+            tc_mma_i8(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc, k != 0 ? 1u : 0u);
+          tc_commit(empty_bar(stage));
+          tc_commit(tfull_bar(acc));
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        tc_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0)) {
+          if (global_timer_ns() - t0 > 20000000ull) break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ rescale and accumulate (warps 2..9)
+    const int quad = warp & 3;             // TMEM lanes [32*quad, 32*quad+32) are the ones this warp may read
+    const int half = (warp - 2) >> 2;      // which 64 of the tile's 128 columns
+    constexpr int HN = BN / 2;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
+      const int row = tm * BM + quad * 32 + lane;
+      const bool row_ok = row < p.M;
+      const int col_base = tn * BN + half * HN;
+      float sum[HN];
+#pragma unroll
+      for (int j = 0; j < HN; ++j) sum[j] = 0.0f;
+      for (int g = 0; g < p.G; ++g) {
+        ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x63, status, p.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const float da = row_ok ? p.dAt[(long long)g * p.M + row] : 0.0f;
+        const float* dbp = p.dBt + (long long)g * p.N + col_base;
+#pragma unroll
+        for (int c = 0; c < HN / 16; ++c) {
+          uint32_t v[16];
+          tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + half * HN + c * 16), v);
+          tc_wait_ld();
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int col = col_base + c * 16 + q4 * 4;
+            const float4 db = col < p.N ? *reinterpret_cast<const float4*>(dbp + c * 16 + q4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float dbv[4] = {db.x, db.y, db.z, db.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // exact int -> float for |P| < 2^22 (a group product is at most 128 * 127^2): add the integer to the bits
+              // of 1.5 * 2^23, subtract that constant
+              const float pf = __fsub_rn(__uint_as_float(v[q4 * 4 + e] + 0x4B400000u), 12582912.0f);
+              const float x = __fmul_rn(__fmul_rn(pf, da), dbv[e]);
+              sum[c * 16 + q4 * 4 + e] = __fadd_rn(sum[c * 16 + q4 * 4 + e], x);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) break;
+      if (row_ok) {
+        const long long row_off = (long long)row * p.ldc;
+#pragma unroll
+        for (int c = 0; c < HN / 32; ++c) {
+          const int col0 = col_base + c * 32;
+          if (col0 < p.N) {
+            uint32_t w[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) w[j] = __float_as_uint(sum[c * 32 + j]);
+            store_row_chunk(out, row_off + col0, min(32, p.N - col0), w, 1, p.out_bf16, 1.0f, p.wide != 0);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
 }  // namespace
+
+fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const float* dAt, const float* dBt, int64_t M,
+                                  int64_t K, int64_t N, int output, void* C, int64_t ldc, DeviceStatus* status, cudaStream_t st) {
+  using L = Int8Layout;
+  if (M > 0x7fffffff || N > 0x7fffffff || K % BKB || K / BKB > 0x7fffffff) return FMM_ERR_SHAPE;
+  CUtensorMap ma, mb;
+  if (!make_operand_map(&ma, true, cA, M, K, K, 0, 1, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, true, cB, N, K, K, 0, 1, L::BN)) return FMM_ERR_CUDA;
+  Int8Params p;
+  p.M = (int)M; p.N = (int)N; p.G = (int)(K / BKB);
+  p.tiles_m = (int)((M + BM - 1) / BM);
+  p.tiles_n = (int)((N + L::BN - 1) / L::BN);
+  p.ldc = ldc; p.out_bf16 = output == FMM_BF16;
+  const int es = p.out_bf16 ? 2 : 4;
+  p.wide = (reinterpret_cast<uintptr_t>(C) % 32 == 0) && ((ldc * es) % 32 == 0);
+  p.dAt = dAt; p.dBt = dBt;
+  p.wait_limit_ns = kDefaultWaitLimitNs;
+  const long long total = (long long)p.tiles_m * p.tiles_n;
+  if (total <= 0) return FMM_OK;
+  const int sms = sm_count();
+  if (sms <= 0) return FMM_ERR_CUDA;
+  const int grid = (int)(total < sms ? total : sms);
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(int8_group_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
+      return FMM_ERR_CUDA;
+    attr_done = true;
+  }
+  int8_group_gemm_kernel<<<grid, kInt8Threads, L::kTotal, st>>>(ma, mb, C, p, status);
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
 
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
   if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim > 0x3fffffff) return FMM_ERR_SHAPE;

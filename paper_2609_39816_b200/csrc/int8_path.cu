@@ -536,6 +536,42 @@ bool corrected_certificate(const fmm_scheme& s, int h, double cert[4]) {
          (int64_t)s.k * h == kGroup;
 }
 
+// Workspace of the fused classical operator: status word and the two transposed scale arrays.
+struct FusedLayout { size_t status, dAt, dBt, total; };
+
+FusedLayout fused_layout(int64_t M, int64_t K, int64_t N) {
+  FusedLayout L;
+  const size_t G = (size_t)(K / kGroup);
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.dAt = o; o += align_up((size_t)M * G * 4);
+  L.dBt = o; o += align_up((size_t)N * G * 4);
+  L.total = o;
+  return L;
+}
+
+// The classical int8 operator in one tensor-core kernel (int8 MMAs, int32 accumulators, rescale in the epilogue).
+fmm_status int8_classical_fused(const int8_t* d_cA, const float* d_dA, const int8_t* d_cB, const float* d_dB, int64_t M,
+                                int64_t K, int64_t N, int output, void* d_C, int64_t ldc, void* d_ws, size_t ws_bytes,
+                                cudaStream_t st) {
+  const FusedLayout L = fused_layout(M, K, N);
+  if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(d_cA) % 16) || (reinterpret_cast<uintptr_t>(d_cB) % 16)) return FMM_ERR_SHAPE;
+  const int G = (int)(K / kGroup);
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  {
+    ProfScope ps(5, st);
+    transpose_scales_kernel<<<stream_blocks(M * G, 256), 256, 0, st>>>(d_dA, M, G, at<float>(d_ws, L.dAt));
+    ++fmm_launch_counter();
+    transpose_scales_kernel<<<stream_blocks(N * G, 256), 256, 0, st>>>(d_dB, N, G, at<float>(d_ws, L.dBt));
+    ++fmm_launch_counter();
+    FMM_CUDA(cudaGetLastError());
+  }
+  ProfScope ps(4, st);
+  return launch_int8_group_gemm(d_cA, d_cB, at<float>(d_ws, L.dAt), at<float>(d_ws, L.dBt), M, K, N, output, d_C, ldc,
+                                at<DeviceStatus>(d_ws, L.status), st);
+}
+
 }  // namespace
 
 extern "C" {
@@ -576,6 +612,7 @@ size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N)
   TrivialScheme one;
   const fmm_scheme& sc = s ? *s : one;
   if (int8_shape_ok(sc, M, K, N) != FMM_OK) return 0;
+  if (!s) return fused_layout(M, K, N).total;
   return int8_layout(sc, M, K, N).total;
 }
 
@@ -593,6 +630,8 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
   if ((reinterpret_cast<uintptr_t>(d_cA) % 8) || (reinterpret_cast<uintptr_t>(d_cB) % 8)) return FMM_ERR_SHAPE;
   // Proposition 1 for this realisation: int8 block sums, integers exact in the fp32 accumulators (24 bits)
   if (!scheme_certificate(&sc, code_bound, code_bound, kGroup / sc.k, kGroup, 24, nullptr)) return FMM_ERR_CERTIFICATE;
+  if (!s)   // the classical operator: one fused tensor-core kernel
+    return int8_classical_fused(d_cA, d_dA, d_cB, d_dB, M, K, N, output, d_C, ldc, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
   const Int8Layout L = int8_layout(sc, M, K, N);
   if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

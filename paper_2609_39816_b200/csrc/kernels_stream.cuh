@@ -115,6 +115,12 @@ struct BlockProductArgs {
 };
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
 
+// The group-scaled int8 operator in one kernel (tcgen05 kind::i8, int32 accumulators in TMEM, rescale in the epilogue):
+// cA [M][K], cB [N][K] int8 codes (K % 128 == 0, rows 16-byte aligned), dAt [K/128][M] and dBt [K/128][N] fp32 scales,
+// C [M][ldc] of `output` (FMM_F32 / FMM_BF16).  N must be a multiple of 4.
+fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const float* dAt, const float* dBt, int64_t M,
+                                  int64_t K, int64_t N, int output, void* C, int64_t ldc, DeviceStatus* status, cudaStream_t st);
+
 // Phase timing (see fmm_profile_enable): RAII bracket of a region of the caller's stream.
 struct ProfScope {
   ProfScope(int kind, cudaStream_t st);

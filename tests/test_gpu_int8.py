@@ -67,8 +67,10 @@ def test_classical_and_certified_match_oracle_and_each_other(M, K, N):
     oA, odA = oracle.quantize_rows(A, 31)
     oB, odB = oracle.quantize_rows(B, 31)
     want = oracle.int8_classical(oA, odA, oB, odB)
-    got_cl = _gemm(lib, None, 31, cA, dA, cB, dB)
+    got_cl = _gemm(lib, None, 31, cA, dA, cB, dB)          # one fused kernel: int8 MMAs, rescale in the epilogue
     assert np.array_equal(got_cl, want)
+    one = lib.scheme_load(np.ones((1, 1, 1)), np.ones((1, 1, 1)), np.ones((1, 1, 1)))
+    assert np.array_equal(_gemm(lib, one, 31, cA, dA, cB, dB), want)   # <1,1,1;1> through the materialised pipeline
     s2 = _lib_scheme(lib, S2)
     got = _gemm(lib, s2, 31, cA, dA, cB, dB)
     assert np.array_equal(got, want)
