@@ -126,15 +126,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the 128-byte
@@ -838,7 +829,26 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
       : "memory");
 }
 
-constexpr int kInt8Threads = 320;   // 10 warps: TMA, MMA, and 8 rescale warps (two per TMEM lane quarter, 64 columns each)
+// Packed fp32 pairs, each lane one IEEE operation.  Measured on this toolchain: a packed multiply followed by a
+// packed add IS merged into a packed fused multiply-add even with the rounding mode spelled out on both, so the
+// accumulation that must round twice (product, then sum) uses scalar __fadd_rn; the packed forms are used only
+// where merging is impossible (multiply after multiply) or harmless (an exact subtraction).
+__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float2 add2_rn(float2 a, float2 b) {
+  float2 d;
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+
+constexpr int kInt8Threads = 576;   // 18 warps: TMA, MMA, and 16 rescale warps (four per TMEM lane quarter, 32 columns each)
 
 __global__ void __launch_bounds__(kInt8Threads, 1)
 int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -864,7 +874,7 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -949,10 +959,10 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       }
     }
   } else {
-    // ------------------------------------------------------------ rescale and accumulate (warps 2..9)
+    // ------------------------------------------------------------ rescale and accumulate (warps 2..17)
     const int quad = warp & 3;             // TMEM lanes [32*quad, 32*quad+32) are the ones this warp may read
-    const int half = (warp - 2) >> 2;      // which 64 of the tile's 128 columns
-    constexpr int HN = BN / 2;
+    const int part = (warp - 2) >> 2;      // which 32 of the tile's 128 columns
+    constexpr int PN = 32;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -960,55 +970,49 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
       const int row = tm * BM + quad * 32 + lane;
       const bool row_ok = row < p.M;
-      const int col_base = tn * BN + half * HN;
-      float sum[HN];
+      const int col_base = tn * BN + part * PN;
+      float2 sum[PN / 2];
 #pragma unroll
-      for (int j = 0; j < HN; ++j) sum[j] = 0.0f;
+      for (int j = 0; j < PN / 2; ++j) sum[j] = make_float2(0.0f, 0.0f);
       for (int g = 0; g < p.G; ++g) {
+        // the row scale does not depend on the products: fetch it before waiting for the accumulator
+        const float da = row_ok ? p.dAt[(long long)g * p.M + row] : 0.0f;
+        const float* dbp = p.dBt + (long long)g * p.N + col_base;
         ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x63, status, p.wait_limit_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const float da = row_ok ? p.dAt[(long long)g * p.M + row] : 0.0f;
-        const float* dbp = p.dBt + (long long)g * p.N + col_base;
-#pragma unroll
-        for (int c = 0; c < HN / 16; ++c) {
-          uint32_t v[16];
-          tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + half * HN + c * 16), v);
-          tc_wait_ld();
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int col = col_base + c * 16 + q4 * 4;
-            const float4 db = col < p.N ? *reinterpret_cast<const float4*>(dbp + c * 16 + q4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float dbv[4] = {db.x, db.y, db.z, db.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              // exact int -> float for |P| < 2^22 (a group product is at most 128 * 127^2): add the integer to the bits
-              // of 1.5 * 2^23, subtract that constant
-              const float pf = __fsub_rn(__uint_as_float(v[q4 * 4 + e] + 0x4B400000u), 12582912.0f);
-              const float x = __fmul_rn(__fmul_rn(pf, da), dbv[e]);
-              sum[c * 16 + q4 * 4 + e] = __fadd_rn(sum[c * 16 + q4 * 4 + e], x);
-            }
-          }
-        }
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + part * PN), v);
+        tc_wait_ld();
+        // the accumulator is in registers: hand the buffer back before the arithmetic
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        const float2 da2 = make_float2(da, da);
+        const float2 neg_magic = make_float2(-12582912.0f, -12582912.0f);
+#pragma unroll
+        for (int q4 = 0; q4 < PN / 4; ++q4) {
+          // exact int -> float for |P| < 2^22 (a group product is at most 128 * 127^2): add the integer to the bits
+          // of 1.5 * 2^23, subtract that constant (exact).  Then two separately rounded multiplications and a
+          // separately rounded addition, as the specification orders them.
+          float2 p0 = make_float2(__uint_as_float(v[q4 * 4 + 0] + 0x4B400000u), __uint_as_float(v[q4 * 4 + 1] + 0x4B400000u));
+          float2 p1 = make_float2(__uint_as_float(v[q4 * 4 + 2] + 0x4B400000u), __uint_as_float(v[q4 * 4 + 3] + 0x4B400000u));
+          p0 = add2_rn(p0, neg_magic); p1 = add2_rn(p1, neg_magic);
+          p0 = mul2_rn(p0, da2); p1 = mul2_rn(p1, da2);
+          const float4 db = col_base + q4 * 4 < p.N ? *reinterpret_cast<const float4*>(dbp + q4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          p0 = mul2_rn(p0, make_float2(db.x, db.y)); p1 = mul2_rn(p1, make_float2(db.z, db.w));
+          sum[q4 * 2].x = __fadd_rn(sum[q4 * 2].x, p0.x); sum[q4 * 2].y = __fadd_rn(sum[q4 * 2].y, p0.y);
+          sum[q4 * 2 + 1].x = __fadd_rn(sum[q4 * 2 + 1].x, p1.x); sum[q4 * 2 + 1].y = __fadd_rn(sum[q4 * 2 + 1].y, p1.y);
+        }
       }
       if (!ok) break;
-      if (row_ok) {
-        const long long row_off = (long long)row * p.ldc;
+      if (row_ok && col_base < p.N) {
+        uint32_t w[32];
 #pragma unroll
-        for (int c = 0; c < HN / 32; ++c) {
-          const int col0 = col_base + c * 32;
-          if (col0 < p.N) {
-            uint32_t w[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) w[j] = __float_as_uint(sum[c * 32 + j]);
-            store_row_chunk(out, row_off + col0, min(32, p.N - col0), w, 1, p.out_bf16, 1.0f, p.wide != 0);
-          }
-        }
+        for (int j = 0; j < PN / 2; ++j) { w[2 * j] = __float_as_uint(sum[j].x); w[2 * j + 1] = __float_as_uint(sum[j].y); }
+        store_row_chunk(out, (long long)row * p.ldc + col_base, min(32, p.N - col_base), w, 1, p.out_bf16, 1.0f, p.wide != 0);
       }
     }
   }
