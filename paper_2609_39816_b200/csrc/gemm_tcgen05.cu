@@ -802,12 +802,14 @@ bool pair_kernel_enabled() {
 // the output dtype.  The MMA of group g+1 overlaps the rescale of group g.
 struct Int8Layout {
   static constexpr int BN = 128;
-  static constexpr int kStages = 5;
+  static constexpr int kStages = 4;
   static constexpr int kABytes = BM * BKB;
   static constexpr int kBBytes = BN * BKB;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kBarBytes = 256;
-  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;
+  static constexpr int kMaxGroupsStaged = 64;                 // column scales of a tile staged in shared memory up to this many groups
+  static constexpr int kScaleBytes = kMaxGroupsStaged * BN * 4;
+  static constexpr int kTotal = kStages * kStageBytes + kBarBytes + kScaleBytes + 1024;
 };
 
 struct Int8Params {
@@ -829,25 +831,10 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
       : "memory");
 }
 
-// Packed fp32 pairs, each lane one IEEE operation.  Measured on this toolchain: a packed multiply followed by a
-// packed add IS merged into a packed fused multiply-add even with the rounding mode spelled out on both, so the
-// accumulation that must round twice (product, then sum) uses scalar __fadd_rn; the packed forms are used only
-// where merging is impossible (multiply after multiply) or harmless (an exact subtraction).
-__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b) {
-  float2 d;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "mul.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-  return d;
-}
-__device__ __forceinline__ float2 add2_rn(float2 a, float2 b) {
-  float2 d;
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
-      "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-  return d;
-}
-
+// Packed fp32 pairs (__fmul2_rn, __fadd2_rn): each lane one IEEE operation.  Measured on this toolchain: a packed
+// multiply followed by a packed add IS merged into a packed fused multiply-add, even when both are written with an
+// explicit rounding mode, so the accumulation that must round twice (product, then sum) uses scalar __fadd_rn; the
+// packed forms are used only where merging is impossible (multiply after multiply) or harmless (an exact subtraction).
 constexpr int kInt8Threads = 576;   // 18 warps: TMA, MMA, and 16 rescale warps (four per TMEM lane quarter, 32 columns each)
 
 __global__ void __launch_bounds__(kInt8Threads, 1)
@@ -868,6 +855,9 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+  float* scale_sm = reinterpret_cast<float*>(bar_mem + L::kBarBytes);   // [group][BN] column scales of the current tile
+  const uint32_t sfull_bar = bar_base + 8u * (2 * L::kStages + 7);      // the tile's scales are staged (16 warps arrive)
+  const uint32_t sempty_bar = bar_base + 8u * (2 * L::kStages + 8);     // the tile's scales are no longer read
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr uint32_t kTmemCols = 2 * BN;
@@ -876,6 +866,7 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
     mbar_init(drain_bar, 1);
+    mbar_init(sfull_bar, 16); mbar_init(sempty_bar, 16);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -965,6 +956,7 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
     constexpr int PN = 32;
     int acc = 0;
     uint32_t acc_phase = 0;
+    uint32_t scale_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int tm = tile / p.tiles_n, tn = tile - tm * p.tiles_n;
@@ -974,10 +966,32 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
       float2 sum[PN / 2];
 #pragma unroll
       for (int j = 0; j < PN / 2; ++j) sum[j] = make_float2(0.0f, 0.0f);
+      // column scales of this tile: [group][128] into shared memory (zero beyond N), by the 512 rescale threads
+      const bool staged = p.G <= L::kMaxGroupsStaged;
+      if (staged) {
+        // bounded waits on mbarriers, not a named barrier: a warp that gives up elsewhere must not strand the others
+        ok = mbar_wait(sempty_bar, scale_phase ^ 1u, abort_flag, 0x64, status, p.wait_limit_ns);   // previous tile's readers are done
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const int et = threadIdx.x - 64;                  // 0 .. 511
+        for (int i = et; i < p.G * (BN / 4); i += 512) {
+          const int g = i / (BN / 4), c4 = (i - g * (BN / 4)) * 4;
+          const int col = tn * BN + c4;
+          const float4 val = col < p.N ? *reinterpret_cast<const float4*>(p.dBt + (long long)g * p.N + col) : make_float4(0.f, 0.f, 0.f, 0.f);
+          *reinterpret_cast<float4*>(scale_sm + g * BN + c4) = val;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sfull_bar);            // release: this warp's share is written
+        ok = mbar_wait(sfull_bar, scale_phase, abort_flag, 0x65, status, p.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      float da_next = row_ok ? p.dAt[row] : 0.0f;
       for (int g = 0; g < p.G; ++g) {
-        // the row scale does not depend on the products: fetch it before waiting for the accumulator
-        const float da = row_ok ? p.dAt[(long long)g * p.M + row] : 0.0f;
-        const float* dbp = p.dBt + (long long)g * p.N + col_base;
+        // the row scale does not depend on the products: the next group's is fetched a step ahead
+        const float da = da_next;
+        if (g + 1 < p.G) da_next = row_ok ? p.dAt[(long long)(g + 1) * p.M + row] : 0.0f;
+        const float* dbp = staged ? scale_sm + g * BN + part * PN : p.dBt + (long long)g * p.N + col_base;
         ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x63, status, p.wait_limit_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -999,15 +1013,20 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           // separately rounded addition, as the specification orders them.
           float2 p0 = make_float2(__uint_as_float(v[q4 * 4 + 0] + 0x4B400000u), __uint_as_float(v[q4 * 4 + 1] + 0x4B400000u));
           float2 p1 = make_float2(__uint_as_float(v[q4 * 4 + 2] + 0x4B400000u), __uint_as_float(v[q4 * 4 + 3] + 0x4B400000u));
-          p0 = add2_rn(p0, neg_magic); p1 = add2_rn(p1, neg_magic);
-          p0 = mul2_rn(p0, da2); p1 = mul2_rn(p1, da2);
-          const float4 db = col_base + q4 * 4 < p.N ? *reinterpret_cast<const float4*>(dbp + q4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-          p0 = mul2_rn(p0, make_float2(db.x, db.y)); p1 = mul2_rn(p1, make_float2(db.z, db.w));
+          p0 = __fadd2_rn(p0, neg_magic); p1 = __fadd2_rn(p1, neg_magic);
+          p0 = __fmul2_rn(p0, da2); p1 = __fmul2_rn(p1, da2);
+          const float4 db = (staged || col_base + q4 * 4 < p.N) ? *reinterpret_cast<const float4*>(dbp + q4 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          p0 = __fmul2_rn(p0, make_float2(db.x, db.y)); p1 = __fmul2_rn(p1, make_float2(db.z, db.w));
           sum[q4 * 2].x = __fadd_rn(sum[q4 * 2].x, p0.x); sum[q4 * 2].y = __fadd_rn(sum[q4 * 2].y, p0.y);
           sum[q4 * 2 + 1].x = __fadd_rn(sum[q4 * 2 + 1].x, p1.x); sum[q4 * 2 + 1].y = __fadd_rn(sum[q4 * 2 + 1].y, p1.y);
         }
       }
       if (!ok) break;
+      if (staged) {                                        // this warp no longer reads the tile's scales
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sempty_bar);
+        scale_phase ^= 1u;
+      }
       if (row_ok && col_base < p.N) {
         uint32_t w[32];
 #pragma unroll
