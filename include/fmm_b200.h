@@ -36,6 +36,11 @@
  *     ((M/m) * (N/n) / 4); M/m, N/n < 2^31 - 4096 and K/k < 2^30.  Larger shapes, empty shapes
  *     (M, K or N <= 0) included, return FMM_ERR_SHAPE (the workspace queries return 0) and launch nothing;
  *   - NaN/Inf in operands propagate; e4m3 conversion saturates at +-448.
+ *   - devices and threads: a call works on the current device of the calling thread; kernels are configured per
+ *     device on first use.  The library keeps process-wide state (two helper streams with an event ring for
+ *     error_sweep, the launch counter, the phase-timing record), created on the device that first needs it: use
+ *     one device per process (the multi-GPU model here is one process per GPU) and do not call into the library
+ *     from two host threads at once.  Scheme handles are immutable after creation and may be shared.
  */
 #ifndef FMM_B200_H
 #define FMM_B200_H

@@ -736,7 +736,8 @@ fmm_status launch_t(const BlockProductArgs& a, cudaStream_t st) {
   if (sms <= 0) return FMM_ERR_CUDA;
   const int grid = (int)(total < sms ? total : sms);
   auto k = block_products_kernel<BN, kFp8>;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
+  static unsigned long long smem_ok = 0;   // per template instantiation, one bit per device
+  if (fmm_allow_dynamic_smem(k, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
   if (launch_dependent(k, dim3(grid), dim3(kNumThreads), (size_t)L::kTotal, st, ma, mb, a.out, a.sA, a.sB, tp, a.status) != cudaSuccess)
     return FMM_ERR_CUDA;
   ++fmm_launch_counter();
@@ -770,11 +771,8 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   if (sms < 2) return FMM_ERR_CUDA;
   const long long pairs = std::min<long long>(total, sms / 2);
   auto k = block_products_pair_kernel<kFp8>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess) return FMM_ERR_CUDA;
-    attr_done = true;
-  }
+  static unsigned long long smem_ok = 0;
+  if (fmm_allow_dynamic_smem(k, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
   if (launch_dependent(k, dim3((unsigned)(2 * pairs)), dim3(kNumThreads), (size_t)L::kTotal, st, ma, mb, a.out, a.sA, a.sB, tp, a.status) != cudaSuccess)
     return FMM_ERR_CUDA;
   ++fmm_launch_counter();
@@ -1067,12 +1065,8 @@ fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const floa
   const int sms = sm_count();
   if (sms <= 0) return FMM_ERR_CUDA;
   const int grid = (int)(total < sms ? total : sms);
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(int8_group_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
-      return FMM_ERR_CUDA;
-    attr_done = true;
-  }
+  static unsigned long long smem_ok = 0;
+  if (fmm_allow_dynamic_smem(int8_group_gemm_kernel, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
   int8_group_gemm_kernel<<<grid, kInt8Threads, L::kTotal, st>>>(ma, mb, C, p, status);
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;

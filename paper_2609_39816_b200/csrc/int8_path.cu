@@ -362,7 +362,8 @@ cudaError_t launch_encode_split(const int8_t* codes, int64_t K, int gr, int gc, 
   const size_t smem = ((size_t)(h_tab->R + 1) * 4 + 15) / 16 * 16 + (size_t)h_tab->off[h_tab->R] * 8 +
                       (size_t)(gr * gc + 1) * kSplitThreads * 4;
   if (smem > 96 * 1024) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(encode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  static unsigned long long smem_ok = 0;
+  cudaError_t e = fmm_allow_dynamic_smem(encode_split_kernel, 96 * 1024, &smem_ok);
   if (e != cudaSuccess) return e;
   const int64_t grid = (nquad + kSplitThreads - 1) / kSplitThreads;
   if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
@@ -384,7 +385,8 @@ cudaError_t launch_decode_group_t(const float* prod, int64_t pstride, int G, con
   if (nvec + kDecThreads >= (int64_t)1 << 31 || smem > 200 * 1024) return cudaErrorInvalidValue;
   if (m * n > kSplit * kCells) return cudaErrorInvalidValue;
   auto k = decode_group_kernel<OutT, kSplit, kStages, kCells, kIntAcc>;
-  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  static unsigned long long smem_ok = 0;   // per template instantiation, one bit per device
+  cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok);
   if (e != cudaSuccess) return e;
   const unsigned grid = (unsigned)((nvec + kPos - 1) / kPos);
   k<<<grid, kDecThreads, smem, st>>>(prod, pstride, G, d_tab, R, dAt, dBt, (int64_t)m * bm, (int64_t)n * bn, n, bm, bn,

@@ -448,22 +448,16 @@ cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool
   const int grid = ja.blocks + jb.blocks;
   if (grid == 0) return cudaSuccess;
   const size_t smem = std::max(smem_a, smem_b);
-  static bool attr_done[2] = {false, false};
+  static unsigned long long smem_ok[2] = {0, 0};   // per template instantiation, one bit per device
   if (amax_only) {
     auto k = encode_kernel<SrcT, DstT, true, kSplit>;
-    if (!attr_done[0]) {
-      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-      if (e != cudaSuccess) return e;
-      attr_done[0] = true;
-    }
+    cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[0]);
+    if (e != cudaSuccess) return e;
     k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
   } else {
     auto k = encode_kernel<SrcT, DstT, false, kSplit>;
-    if (!attr_done[1]) {
-      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-      if (e != cudaSuccess) return e;
-      attr_done[1] = true;
-    }
+    cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[1]);
+    if (e != cudaSuccess) return e;
     k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
   }
   ++fmm_launch_counter();
@@ -811,14 +805,13 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
   split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
   if (n_partials) *n_partials = grid;
   const int64_t ldcs = (int64_t)n * bn;
-  static bool attr_done[3] = {false, false, false};   // per template instantiation
+  static unsigned long long smem_ok[3] = {0, 0, 0};   // per template instantiation, one bit per device
 #define FMM_DECODE_LAUNCH(STORE, ERR, SLOT)                                                                      \
   {                                                                                                              \
     auto k = decode_kernel<OutT, STORE, ERR, kSplit, ProdT>;                                                         \
-    if (!attr_done[SLOT]) {                                                                                      \
-      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);          \
+    {                                                                                                            \
+      cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[SLOT]);                                     \
       if (e != cudaSuccess) return e;                                                                            \
-      attr_done[SLOT] = true;                                                                                    \
     }                                                                                                            \
     cudaError_t le = launch_dependent(k, dim3(grid), dim3(kDecThreads), smem, st, prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, \
                                       cstar32, ldcs, partials, tpb, prod_stride);                                 \

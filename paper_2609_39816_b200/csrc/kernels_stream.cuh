@@ -19,6 +19,19 @@ int64_t& fmm_launch_counter();
 // call grid_launch_dependents() early.  Both are no-ops when the launch carries no programmatic dependency.
 // FMM_B200_NO_PDL=1 in the environment turns the attribute off (ordinary stream order).
 bool fmm_pdl_enabled();
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per (kernel, device): `done_mask` is the caller's static word for
+// one kernel, bit d set once device d has been configured (devices beyond 63 are configured on every call).
+template <typename Kernel>
+cudaError_t fmm_allow_dynamic_smem(Kernel kernel, int bytes, unsigned long long* done_mask) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 64 && (*done_mask >> dev) & 1ull) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && dev < 64) *done_mask |= 1ull << dev;
+  return e;
+}
 #ifdef __CUDACC__
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
