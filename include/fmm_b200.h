@@ -138,6 +138,13 @@ fmm_status scheme_builtin(const char* name, fmm_scheme** out);
  * remembers its factors (see gauge_apply, level 1).                                         */
 fmm_status scheme_kron(const fmm_scheme* outer, const fmm_scheme* inner, fmm_scheme** out);
 
+/* The same algorithm with its products renumbered: product r of *out is product perm[r] of `in` (perm: HOST,
+ * a permutation of 0..R-1, else FMM_ERR_ARG).  The decode adds the products in ascending r, so the order of the
+ * fp32 additions is part of the operator (Appendix B.1 reports perplexity spans from the summation order alone):
+ * in exact arithmetic nothing changes, in fp32 the result may move in its last bits.  The handle is flat (no
+ * outer / inner factors for gauge_apply at level 1).                                                        */
+fmm_status scheme_permute_products(const fmm_scheme* in, const int* perm, fmm_scheme** out);
+
 /* Gauge transform (Section 2.1).  With P[m][m], Q[k][k], S[n][n] (HOST, fp64, row-major,
  * invertible):  U'_r = P^T U_r Q^-T,  V'_r = Q^T V_r S^-T,  W'_r = P^-1 W_r S, which for diagonal
  * sign matrices D,E,F is the paper's sign variant d_i e_l u, e_l f_j v, d_i f_j w.

@@ -19,7 +19,7 @@ FLAG_PRODUCTS_BF16 = 2
 _DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
 
 EXPORTED_SYMBOLS = [
-    "scheme_load", "scheme_builtin", "scheme_kron", "gauge_apply", "scheme_info", "scheme_coefficients",
+    "scheme_load", "scheme_builtin", "scheme_kron", "scheme_permute_products", "gauge_apply", "scheme_info", "scheme_coefficients",
     "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status",
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
@@ -74,6 +74,7 @@ _vp, _dp, _sz = C.c_void_p, C.POINTER(C.c_double), C.c_size_t
 _lib.scheme_load.argtypes = [C.c_int] * 4 + [_dp] * 3 + [C.c_double, C.POINTER(_vp)]
 _lib.scheme_builtin.argtypes = [C.c_char_p, C.POINTER(_vp)]
 _lib.scheme_kron.argtypes = [_vp, _vp, C.POINTER(_vp)]
+_lib.scheme_permute_products.argtypes = [_vp, C.POINTER(C.c_int), C.POINTER(_vp)]
 _lib.gauge_apply.argtypes = [_vp, C.c_int, _dp, _dp, _dp, C.c_double, C.POINTER(_vp)]
 _lib.scheme_info.argtypes = [_vp, C.POINTER(C.c_int), _dp]
 _lib.scheme_coefficients.argtypes = [_vp, _dp, _dp, _dp]
@@ -201,6 +202,17 @@ def scheme_builtin(name: str) -> Scheme:
 def scheme_kron(outer: Scheme, inner: Scheme) -> Scheme:
     h = _vp()
     _check(_lib.scheme_kron(outer.handle, inner.handle, C.byref(h)), "scheme_kron")
+    return Scheme(h)
+
+
+def scheme_permute_products(s: Scheme, perm) -> Scheme:
+    """The same algorithm with product r taken from product perm[r] (changes only the order of the decode's sums)."""
+    perm = [int(x) for x in perm]
+    arr = (C.c_int * len(perm))(*perm)
+    if len(perm) != s.dims[3]:
+        raise ValueError("perm must have R entries")
+    h = _vp()
+    _check(_lib.scheme_permute_products(s.handle, arr, C.byref(h)), "scheme_permute_products")
     return Scheme(h)
 
 

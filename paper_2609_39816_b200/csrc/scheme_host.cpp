@@ -323,6 +323,27 @@ fmm_status scheme_kron(const fmm_scheme* outer, const fmm_scheme* inner, fmm_sch
   return FMM_OK;
 }
 
+fmm_status scheme_permute_products(const fmm_scheme* in, const int* perm, fmm_scheme** out) {
+  if (!in || !perm || !out) return FMM_ERR_ARG;
+  const int R = in->R, m = in->m, k = in->k, n = in->n;
+  std::vector<char> seen(R, 0);
+  for (int r = 0; r < R; ++r) {
+    if (perm[r] < 0 || perm[r] >= R || seen[perm[r]]) return FMM_ERR_ARG;
+    seen[perm[r]] = 1;
+  }
+  std::unique_ptr<fmm_scheme> s(new (std::nothrow) fmm_scheme);
+  if (!s) return FMM_ERR_ARG;
+  s->m = m; s->k = k; s->n = n; s->R = R;
+  s->U.resize(in->U.size()); s->V.resize(in->V.size()); s->W.resize(in->W.size());
+  for (int r = 0; r < R; ++r) {   // product r of the result is product perm[r] of the input
+    std::copy_n(in->U.begin() + (size_t)perm[r] * m * k, (size_t)m * k, s->U.begin() + (size_t)r * m * k);
+    std::copy_n(in->V.begin() + (size_t)perm[r] * k * n, (size_t)k * n, s->V.begin() + (size_t)r * k * n);
+    std::copy_n(in->W.begin() + (size_t)perm[r] * m * n, (size_t)m * n, s->W.begin() + (size_t)r * m * n);
+  }
+  *out = s.release();
+  return FMM_OK;
+}
+
 fmm_status gauge_apply(const fmm_scheme* in, int level, const double* P, const double* Q, const double* S,
                        double cond_limit, fmm_scheme** out) {
   if (!in || !P || !Q || !S || !out) return FMM_ERR_ARG;

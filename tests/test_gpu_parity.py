@@ -370,3 +370,19 @@ def test_sign_variant_ensemble_on_the_device(lib):
         stats[kind] = (avg.max() / avg.min(), float(np.corrcoef(errs[:, 0::2].mean(axis=1), errs[:, 1::2].mean(axis=1))[0, 1]))
     assert abs(stats["u01"][0] - 2.59) < 0.12 * 2.59 and stats["u01"][1] > 0.99, stats
     assert 1.0 <= stats["upm1"][0] < 1.03 and abs(stats["upm1"][1]) < 0.6, stats
+
+
+def test_decode_order_is_part_of_the_operator(lib):
+    """Products renumbered (Appendix B.1's summation-order observation): exact on integers, equal to the oracle run on
+    the same renumbered coefficients, and on real data a different fp32 result from the original order."""
+    s2, o2 = lib.scheme_builtin("strassen444"), gu.oracle_scheme("strassen444")
+    perm = np.random.default_rng(9).permutation(49)
+    sp = lib.scheme_permute_products(s2, perm)
+    op = oracle.Scheme(o2.U[perm], o2.V[perm], o2.W[perm])
+    At, Bt, A64, B64 = _inputs(15, 256, 512, 256, "bf16", "int", 4)
+    assert np.array_equal(gu.run_scheme_gemm(sp, At, Bt, "bf16", "bf16", "f32"), A64 @ B64)
+    At, Bt, A64, B64 = _inputs(16, 512, 1024, 512, "bf16", "llm")
+    C0 = gu.run_scheme_gemm(s2, At, Bt, "bf16", "bf16", "f32")
+    C1 = gu.run_scheme_gemm(sp, At, Bt, "bf16", "bf16", "f32")
+    assert gu.rel_fro(C1, oracle.scheme_gemm(op, A64, B64, "bf16", "f32")) <= TOL_FRO
+    assert not np.array_equal(C0, C1) and gu.rel_fro(C0, C1) < 1e-5

@@ -200,3 +200,19 @@ def test_empty_and_maximum_sizes_are_rejected_before_any_launch(lib):
     assert (1 << 20) * 16400 // 8 >= (1 << 31) - 4096 and lib.scheme_gemm_workspace(s2, too_big) == 0
     assert lib.scheme_gemm_workspace(s2, lib.GemmDesc.make(4 * (1 << 17), 64, 4 * (1 << 17), "bf16", "bf16", "bf16")) == 0   # products
     assert lib.int8_gemm_workspace(s2, 0, 128, 64) == 0
+
+
+def test_permuted_products_are_the_same_algorithm(lib):
+    """Renumbering the products keeps the Brent equations and every criterion; bad permutations are refused."""
+    s2 = lib.scheme_builtin("strassen444")
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(49)
+    sp = lib.scheme_permute_products(s2, perm)
+    U, V, W = s2.coefficients()
+    Up, Vp, Wp = sp.coefficients()
+    assert np.array_equal(Up, U[perm]) and np.array_equal(Vp, V[perm]) and np.array_equal(Wp, W[perm])
+    assert sp.info == s2.info
+    assert oracle.brent_residual(oracle.Scheme(Up, Vp, Wp)) == 0.0
+    for bad in ([0] * 49, list(range(48)) + [49], list(range(48)) + [-1]):
+        with pytest.raises(lib.FmmError):
+            lib.scheme_permute_products(s2, bad)
