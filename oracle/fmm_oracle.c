@@ -359,6 +359,52 @@ static void matmul_f64(const double* A, const double* B, double* C, int64_t M, i
   }
 }
 
+/* Model schedule of Appendix B.1 (scale_mode 3).  Ah is bm x bk (rows of an A block sum), Bh is bk x bn (a weight
+ * block sum).  A: e4m3 codes with one scale for every 128 consecutive entries of a row.  B: first stored in bf16,
+ * then e4m3 codes with one scale for every 128 x 128 block (128 inner indices x 128 output columns).  Scale rule (a
+ * reading, as in mode 2): s = max|x| / 448 in fp32, 1 for an all-zero group; code = x / s in fp32, one rounding.
+ * The product kernel accumulates each 128-group of inner indices on its own, multiplies by the two scales and adds
+ * the groups in ascending order: Mr = sum_g (Aq_g Bq_g^T) * sA[p][g] * sB[c/128][g]  (fp64 here).
+ * Ah and Bh are overwritten with the codes; sa is [bm][G], sb is [ceil(bn/128)][G], G = ceil(bk/128).            */
+static void model_schedule_product(double* Ah, double* Bh, int64_t bm, int64_t bk, int64_t bn, int pd,
+                                   double* sa, double* sb, double* Mr) {
+  const int64_t G = (bk + 127) / 128, CB = (bn + 127) / 128;
+  for (int64_t p = 0; p < bm; ++p)
+    for (int64_t g = 0; g < G; ++g) {
+      const int64_t t0 = g * 128, t1 = t0 + 128 < bk ? t0 + 128 : bk;
+      float amax = 0.0f;
+      for (int64_t t = t0; t < t1; ++t) { float a = fabsf((float)Ah[p * bk + t]); if (a > amax) amax = a; }
+      float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+      sa[p * G + g] = (double)d;
+      for (int64_t t = t0; t < t1; ++t) Ah[p * bk + t] = orc_round((double)((float)Ah[p * bk + t] / d), pd);
+    }
+  for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x], ORC_BF16);   /* weights' block sums first stored in bf16 */
+  for (int64_t cb = 0; cb < CB; ++cb)
+    for (int64_t g = 0; g < G; ++g) {
+      const int64_t t0 = g * 128, t1 = t0 + 128 < bk ? t0 + 128 : bk;
+      const int64_t c0 = cb * 128, c1 = c0 + 128 < bn ? c0 + 128 : bn;
+      float amax = 0.0f;
+      for (int64_t t = t0; t < t1; ++t)
+        for (int64_t c = c0; c < c1; ++c) { float a = fabsf((float)Bh[t * bn + c]); if (a > amax) amax = a; }
+      float d = amax > 0.0f ? amax / 448.0f : 1.0f;
+      sb[cb * G + g] = (double)d;
+      for (int64_t t = t0; t < t1; ++t)
+        for (int64_t c = c0; c < c1; ++c) Bh[t * bn + c] = orc_round((double)((float)Bh[t * bn + c] / d), pd);
+    }
+#pragma omp parallel for schedule(static)
+  for (int64_t p = 0; p < bm; ++p)
+    for (int64_t c = 0; c < bn; ++c) {
+      double tot = 0.0;
+      for (int64_t g = 0; g < G; ++g) {
+        const int64_t t0 = g * 128, t1 = t0 + 128 < bk ? t0 + 128 : bk;
+        double part = 0.0;
+        for (int64_t t = t0; t < t1; ++t) part += Ah[p * bk + t] * Bh[t * bn + c];
+        tot += (part * sa[p * G + g]) * sb[(c / 128) * G + g];
+      }
+      Mr[p * bn + c] = tot;
+    }
+}
+
 /* Apply an algorithm <m,k,n;R> to A (M x K) and B (K x N); C is M x N.
  * pd = product dtype the block sums are rounded to, od = output dtype,
  * scale_mode 0: no scales; 1: per-encoded-tensor power-of-two scale (e4m3); 2: the
@@ -367,8 +413,10 @@ static void matmul_f64(const double* A, const double* B, double* C, int64_t M, i
  * row), code = x / scale in fp32, then rounded to e4m3 (a reading: the paper states who
  * owns a scale, not its rule; max|x| / b is the rule of its int8 specification).
  * md = dtype each product is rounded to before the combination (ORC_F64: none).
+ * scale_mode 3: the model schedule of Appendix B.1 (see model_schedule_product).
  * Optional outputs (may be NULL): Ahat [R][bm][bk], Bhat [R][bk][bn] (the rounded,
- * scaled block sums), sA[R], sB[R] (mode 2: sA[R][bm], sB[R][bn]), Mout [R][bm][bn]
+ * scaled block sums), sA[R], sB[R] (mode 2: sA[R][bm], sB[R][bn]; mode 3: sA[R][bm][G],
+ * sB[R][ceil(bn/128)][G], G = ceil(bk/128)), Mout [R][bm][bn]
  * (the fp64 products of the codes; mode 2: times the row and column scales).
  * Returns 0, or 1 if a dimension does not divide.                                 */
 int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V, const double* W,
@@ -413,7 +461,7 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
       }
       if (sA_out) memcpy(sA_out + (size_t)r * bm, rs, sizeof(double) * bm);
       if (sB_out) memcpy(sB_out + (size_t)r * bn, cs, sizeof(double) * bn);
-    } else {
+    } else if (scale_mode != 3) {
       if (quant) {
         for (int64_t x = 0; x < bm * bk; ++x) Ah[x] = orc_round(Ah[x] / sa, pd);
         for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x] / sb, pd);
@@ -421,10 +469,19 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
       if (sA_out) sA_out[r] = sa;
       if (sB_out) sB_out[r] = sb;
     }
+    if (scale_mode == 3) {
+      const int64_t G3 = (bk + 127) / 128, CB3 = (bn + 127) / 128;
+      double* sa3 = (double*)malloc(sizeof(double) * bm * G3);
+      double* sb3 = (double*)malloc(sizeof(double) * CB3 * G3);
+      model_schedule_product(Ah, Bh, bm, bk, bn, pd, sa3, sb3, Mr);
+      if (sA_out) memcpy(sA_out + (size_t)r * bm * G3, sa3, sizeof(double) * bm * G3);
+      if (sB_out) memcpy(sB_out + (size_t)r * CB3 * G3, sb3, sizeof(double) * CB3 * G3);
+      free(sa3); free(sb3);
+    }
     if (Ahat_out) memcpy(Ahat_out + (size_t)r * bm * bk, Ah, sizeof(double) * bm * bk);
     if (Bhat_out) memcpy(Bhat_out + (size_t)r * bk * bn, Bh, sizeof(double) * bk * bn);
     /* product */
-    matmul_f64(Ah, Bh, Mr, bm, bk, bn);
+    if (scale_mode != 3) matmul_f64(Ah, Bh, Mr, bm, bk, bn);
     if (scale_mode == 2)
       for (int64_t p = 0; p < bm; ++p)
         for (int64_t q = 0; q < bn; ++q) Mr[p * bn + q] = (Mr[p * bn + q] * rs[p]) * cs[q];
@@ -460,6 +517,17 @@ int orc_classical_gemm(int64_t M, int64_t K, int64_t N, const double* A, const d
   double* Bh = (double*)malloc(sizeof(double) * K * N);
   double* acc = (double*)malloc(sizeof(double) * M * N);
   double sa = 1.0, sb = 1.0;
+  if (scale_mode == 3) {   /* the deployed FP8 kernel's schedule: 1 x 128 scales for A, 128 x 128 for B */
+    const int64_t G3 = (K + 127) / 128, CB3 = (N + 127) / 128;
+    double* sa3 = (double*)malloc(sizeof(double) * M * G3);
+    double* sb3 = (double*)malloc(sizeof(double) * CB3 * G3);
+    for (int64_t x = 0; x < M * K; ++x) Ah[x] = A[x];
+    for (int64_t x = 0; x < K * N; ++x) Bh[x] = B[x];
+    model_schedule_product(Ah, Bh, M, K, N, pd, sa3, sb3, acc);
+    for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x], od);
+    free(sa3); free(sb3); free(Ah); free(Bh); free(acc);
+    return 0;
+  }
   if (scale_mode == 2) {
     double* rs = (double*)malloc(sizeof(double) * M);
     double* cs = (double*)malloc(sizeof(double) * N);

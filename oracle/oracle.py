@@ -236,7 +236,9 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
     if parts:
         bm, bk, bn = M // m, K // k, N // n
         Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
-        sA = np.empty((R, bm) if scale_mode == 2 else R); sB = np.empty((R, bn) if scale_mode == 2 else R)
+        G3, CB3 = -(-bk // 128), -(-bn // 128)
+        sA = np.empty({2: (R, bm), 3: (R, bm, G3)}.get(scale_mode, (R,)))
+        sB = np.empty({2: (R, bn), 3: (R, CB3, G3)}.get(scale_mode, (R,)))
     rc = _L().orc_scheme_gemm(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
                               _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
                               _p(sB), _p(Mr), _fmt(md))

@@ -397,3 +397,40 @@ def test_products_rounded_to_bf16_special_cases():
     C1, p1 = oracle.scheme_gemm(s2, X, Y, "bf16", "f64", parts=True, md="bf16")
     assert np.array_equal(p1["M"], oracle.round_to(p0["M"], "bf16"))
     assert 0 < np.abs(C1 - C0).max() <= 16 * 2.0 ** -9 * np.abs(p0["M"]).max()
+
+
+def test_model_schedule_group_scales_invariances():
+    """scale_mode 3 (Appendix B.1: e4m3 block sums of the input with one scale per 128 consecutive entries of a row,
+    weight block sums first stored in bf16 then one scale per 128 x 128 block, groups accumulated separately).
+    What the definition fixes without any reference values: (a) a power of two applied to one row position of A moves
+    only scales, so those output rows scale exactly and the others keep their bits; (b) a power of two moved from one
+    128-group of inner indices of A to the same group of B is absorbed by the two scales: identical bits; (c) on
+    {-1, 0, 1} inputs every code is +-448 or 0 and the result is the exact product up to the fp32 rounding of 1/448;
+    (d) finer scales help: the error is below the per-tensor schedule's on outlier-heavy inputs."""
+    s2 = oracle.kron(oracle.strassen(), oracle.strassen())
+    M, K, N = 64, 1024, 512                       # bm = 16, bk = 256 (2 groups), bn = 128 (1 block)
+    A = gen.to_storage(gen.activations_outlier(41, 1, M, K, frac=0.02, factor=50.0), "bf16")[1]
+    B = gen.to_storage(gen.weights(41, 2, K, N), "bf16")[1]
+    C = oracle.scheme_gemm(s2, A, B, "e4m3", "f32", scale_mode=3)
+    # (a)
+    A2 = A.copy(); rows = [3 + i * 16 for i in range(4)]
+    A2[rows] *= 8.0
+    C2 = oracle.scheme_gemm(s2, A2, B, "e4m3", "f32", scale_mode=3)
+    keep = np.setdiff1d(np.arange(M), rows)
+    assert np.array_equal(C2[rows], 8.0 * C[rows]) and np.array_equal(C2[keep], C[keep])
+    # (b) group 1 of every block column of A (inner indices 128..255 of each 256-wide block) times 4, B rows divided
+    idx = np.concatenate([l * 256 + np.arange(128, 256) for l in range(4)])
+    A3 = A.copy(); B3 = B.copy()
+    A3[:, idx] *= 4.0; B3[idx, :] /= 4.0
+    assert np.array_equal(oracle.scheme_gemm(s2, A3, B3, "e4m3", "f32", scale_mode=3), C)
+    assert np.array_equal(oracle.classical_gemm(A3, B3, "e4m3", "f32", 3), oracle.classical_gemm(A, B, "e4m3", "f32", 3))
+    # (c)
+    a = gen.integer_matrix(42, 1, (8, 512), 1).astype(np.float64); b = gen.integer_matrix(42, 2, (512, 128), 1).astype(np.float64)
+    got = oracle.classical_gemm(a, b, "e4m3", "f32", 3)
+    assert np.abs(got - a @ b).max() <= 1e-5 * np.abs(a @ b).max()
+    # (d)
+    Cs = A @ B
+    e3 = oracle.rel_error(C, Cs); e1 = oracle.rel_error(oracle.scheme_gemm(s2, A, B, "e4m3", "f32", scale_mode=1), Cs)
+    assert e3 < e1 and 1e-3 < e3 < 0.2
+    _, parts = oracle.scheme_gemm(s2, A, B, "e4m3", "f32", scale_mode=3, parts=True)
+    assert parts["sA"].shape == (49, 16, 2) and parts["sB"].shape == (49, 1, 2) and np.abs(parts["Ahat"]).max() == 448
