@@ -104,7 +104,16 @@ typedef struct {
                             scale per row of each block sum of A and per column of each block sum of
                             B, s = amax / 448 in fp32 (1 for an all-zero row), code = x / s in fp32,
                             then rounded; each product is stored as (M_r * s_row) * s_col.  In the
-                            workspace the scales are then [R][M/m] and [R][N/n] arrays */
+                            workspace the scales are then [R][M/m] and [R][N/n] arrays.
+                            3 (e4m3 only): the model schedule of Appendix B.1: block sums of A get one
+                            scale per row and per 128 consecutive inner indices; block sums of B are
+                            first rounded to bf16, then get one scale per 128 x 128 block (128 inner
+                            indices x 128 output columns); s = amax / 448 as in mode 2.  The product
+                            kernel accumulates every 128-group on its own, multiplies it by the two
+                            scales and adds the groups in ascending order in fp32.  Requires K/k to be
+                            a multiple of 128.  Scales in the workspace: [R][M/m][K/k/128] and
+                            [R][ceil(N/n/128)][K/k/128].  classical_gemm applies the same schedule to
+                            the operands themselves (the deployed FP8 kernel's layout of scales) */
   int32_t flags;         /* FMM_FLAG_* */
 } fmm_gemm_desc;
 

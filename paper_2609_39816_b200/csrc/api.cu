@@ -101,9 +101,10 @@ fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
   if (d->storage != FMM_F32 && d->storage != FMM_BF16) return FMM_ERR_DTYPE;
   if (d->product != FMM_BF16 && d->product != FMM_E4M3) return FMM_ERR_DTYPE;
   if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
-  if (d->scale_mode != 0 && !((d->scale_mode == 1 || d->scale_mode == 2) && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
+  if (d->scale_mode != 0 && !(d->scale_mode >= 1 && d->scale_mode <= 3 && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
   if (d->M % m || d->K % k || d->N % n) return FMM_ERR_SHAPE;
   if ((d->K / k) % 16 || (d->N / n) % 8) return FMM_ERR_SHAPE;
+  if (d->scale_mode == 3 && (d->K / k) % 128) return FMM_ERR_SHAPE;   // the model schedule scales groups of 128 inner indices
   const int es = esize(d->storage), eo = esize(d->output);
   const int64_t min_ldb = d->b_is_weight_layout ? d->K : d->N;
   if (d->lda < d->K || d->ldb < min_ldb || d->ldc < d->N) return FMM_ERR_SHAPE;
@@ -117,6 +118,13 @@ fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
   return FMM_OK;
 }
 
+// Number of amax / scale words of one operand: rows x inner extent of one block sum, R of them.
+size_t scale_words(int mode, int R, int64_t rows, int64_t inner, bool b_side) {
+  if (mode == 2) return (size_t)R * rows;
+  if (mode == 3) return (size_t)R * (b_side ? (rows + 127) / 128 : rows) * ((inner + 127) / 128);
+  return FMM_MAX_R;
+}
+
 GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   GemmLayout L;
   const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
@@ -127,7 +135,7 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.tabB = o; o += align_up(sizeof(CoefTable));
   L.tabW = o; o += align_up(sizeof(CoefTable));
   // scale_mode 2 keeps one amax / scale per row of every block sum: [R][bm] and [R][bn]
-  const size_t nsa = d->scale_mode == 2 ? (size_t)R * bm : FMM_MAX_R, nsb = d->scale_mode == 2 ? (size_t)R * bn : FMM_MAX_R;
+  const size_t nsa = scale_words(d->scale_mode, R, bm, bk, false), nsb = scale_words(d->scale_mode, R, bn, bk, true);
   L.amaxA = o; o += align_up(nsa * 4);
   L.amaxB = o; o += align_up(nsb * 4);
   L.sA = o; o += align_up(nsa * 4);
@@ -157,26 +165,27 @@ T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws)
 // Encode one operand: optional amax pass, then block sums -> product dtype.
 fmm_status encode_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
                           const CoefTable* d_tab, const CoefTable* h_tab, void* hat, int64_t hat_stride, unsigned* amax,
-                          float* scale, cudaStream_t st) {
-  const int mode = d->scale_mode;   // 0 none, 1 one power-of-two scale per encoded tensor, 2 one scale per row of it
+                          float* scale, bool b_side, cudaStream_t st) {
+  const int mode = d->scale_mode;   // 0 none, 1 per encoded tensor, 2 per row of it, 3 model schedule (128-groups)
+  const EncodeOperand o{X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, b_side ? 128 : 1, b_side ? 1 : 0};
   if (mode != 0) {
-    const size_t n_amax = mode == 2 ? (size_t)h_tab->R * br : FMM_MAX_R;
-    FMM_CUDA(cudaMemsetAsync(amax, 0, n_amax * 4, st));
-    FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, true, mode, st));
+    FMM_CUDA(cudaMemsetAsync(amax, 0, scale_words(mode, h_tab->R, br, bc, b_side) * 4, st));
+    FMM_CUDA(launch_encode_pair(d->storage, d->product, o, nullptr, true, mode, st));
   }
-  FMM_CUDA(launch_encode(d->storage, d->product, X, ldx, gr, gc, br, bc, d_tab, h_tab, hat, hat_stride, amax, scale, false, mode, st));
+  FMM_CUDA(launch_encode_pair(d->storage, d->product, o, nullptr, false, mode, st));
   return FMM_OK;
 }
 
 // The classical control's operand: the whole matrix as one block with coefficient 1.
 fmm_status quantize_operand(const fmm_gemm_desc* d, const void* X, int64_t ldx, int64_t rows, int64_t cols, void* hat,
-                            unsigned* amax, float* scale, cudaStream_t st) {
+                            unsigned* amax, float* scale, bool b_side, cudaStream_t st) {
   const int mode = d->scale_mode;
+  const int srows = b_side ? 128 : 1, bf16_first = b_side ? 1 : 0;   // model schedule only
   if (mode != 0) {
-    FMM_CUDA(cudaMemsetAsync(amax, 0, (mode == 2 ? (size_t)rows : (size_t)FMM_MAX_R) * 4, st));
-    FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, true, mode, st));
+    FMM_CUDA(cudaMemsetAsync(amax, 0, scale_words(mode, 1, rows, cols, b_side) * 4, st));
+    FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, true, mode, srows, bf16_first, st));
   }
-  FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, false, mode, st));
+  FMM_CUDA(launch_quantize_plain(d->storage, d->product, X, ldx, rows, cols, hat, amax, scale, false, mode, srows, bf16_first, st));
   return FMM_OK;
 }
 
@@ -196,13 +205,13 @@ fmm_status stage_encode_a(const SchemeRun& r, const void* A, cudaStream_t st) {
   const fmm_scheme* s = r.s;
   ProfScope ps(0, st);
   return encode_operand(r.d, A, r.d->lda, s->m, s->k, r.d->M / s->m, r.d->K / s->k, r.dA, r.hA, at<char>(r.ws, r.L.ahat),
-                        r.L.sAhat, at<unsigned>(r.ws, r.L.amaxA), r.sA(), st);
+                        r.L.sAhat, at<unsigned>(r.ws, r.L.amaxA), r.sA(), false, st);
 }
 fmm_status stage_encode_b(const SchemeRun& r, const void* Bk, int64_t ldbk, cudaStream_t st) {
   const fmm_scheme* s = r.s;
   ProfScope ps(1, st);
   return encode_operand(r.d, Bk, ldbk, s->n, s->k, r.d->N / s->n, r.d->K / s->k, r.dB, r.hB, at<char>(r.ws, r.L.bhat),
-                        r.L.sBhat, at<unsigned>(r.ws, r.L.amaxB), r.sB(), st);
+                        r.L.sBhat, at<unsigned>(r.ws, r.L.amaxB), r.sB(), true, st);
 }
 // Both operands in one launch per pass (amax pass if scaled, then the encode pass), on one stream.
 fmm_status stage_encode_pair(const SchemeRun& r, const void* A, const void* Bk, int64_t ldbk, cudaStream_t st) {
@@ -210,9 +219,9 @@ fmm_status stage_encode_pair(const SchemeRun& r, const void* A, const void* Bk, 
   const fmm_gemm_desc* d = r.d;
   const int64_t bm = d->M / s->m, bk = d->K / s->k, bn = d->N / s->n;
   const EncodeOperand oa{A, d->lda, s->m, s->k, bm, bk, r.dA, r.hA, at<char>(r.ws, r.L.ahat), r.L.sAhat,
-                         at<unsigned>(r.ws, r.L.amaxA), r.sA()};
+                         at<unsigned>(r.ws, r.L.amaxA), r.sA(), 1, 0};
   const EncodeOperand ob{Bk, ldbk, s->n, s->k, bn, bk, r.dB, r.hB, at<char>(r.ws, r.L.bhat), r.L.sBhat,
-                         at<unsigned>(r.ws, r.L.amaxB), r.sB()};
+                         at<unsigned>(r.ws, r.L.amaxB), r.sB(), 128, 1};
   ProfScope ps(0, st);
   const int mode = d->scale_mode;
   if (mode != 0) {
@@ -227,6 +236,18 @@ fmm_status stage_encode_pair(const SchemeRun& r, const void* A, const void* Bk, 
 fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   const fmm_scheme* s = r.s;
   const int64_t bm = r.d->M / s->m, bk = r.d->K / s->k, bn = r.d->N / s->n;
+  if (r.d->scale_mode == 3) {   // model schedule: every 128-group of inner indices is scaled on its own inside the product kernel
+    Fp8GroupArgs g{};
+    g.A = at<char>(r.ws, r.L.ahat); g.lda = bk; g.a_batch = r.L.sAhat;
+    g.B = at<char>(r.ws, r.L.bhat); g.ldb = bk; g.b_batch = r.L.sBhat;
+    g.rows_a = bm; g.rows_b = bn; g.kdim = bk; g.batches = s->R;
+    g.out = at<char>(r.ws, r.L.prod); g.ldo = bn; g.o_batch = r.L.sProd;
+    g.output = (r.d->flags & FMM_FLAG_PRODUCTS_BF16) ? FMM_BF16 : FMM_F32;
+    g.sA = r.sA(); g.sB = r.sB();
+    g.status = at<DeviceStatus>(r.ws, r.L.status);
+    ProfScope ps(2, st);
+    return launch_fp8_group_gemm(g, st);
+  }
   BlockProductArgs g{};
   g.product = r.d->product;
   g.A = at<char>(r.ws, r.L.ahat); g.lda = bk; g.a_batch = r.L.sAhat;
@@ -323,7 +344,7 @@ ClassicalLayout classical_layout(const fmm_gemm_desc* d) {
   size_t o = 0;
   L.status = o; o += align_up(sizeof(DeviceStatus));
   L.tab = o; o += align_up(sizeof(CoefTable));
-  const size_t nsa = d->scale_mode == 2 ? (size_t)d->M : FMM_MAX_R, nsb = d->scale_mode == 2 ? (size_t)d->N : FMM_MAX_R;
+  const size_t nsa = scale_words(d->scale_mode, 1, d->M, d->K, false), nsb = scale_words(d->scale_mode, 1, d->N, d->K, true);
   L.amaxA = o; o += align_up(nsa * 4);
   L.amaxB = o; o += align_up(nsb * 4);
   L.sA = o; o += align_up(nsa * 4);
@@ -352,10 +373,19 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
     float* sA = scaled ? at<float>(ws, L.sA) : nullptr;
     float* sB = scaled ? at<float>(ws, L.sB) : nullptr;
     ProfScope pe(5, st);
-    FMM_TRY(quantize_operand(d, A, d->lda, d->M, d->K, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, st));
-    FMM_TRY(quantize_operand(d, bk_ptr, bk_ld, d->N, d->K, at<char>(ws, L.bhat), at<unsigned>(ws, L.amaxB), sB, st));
+    FMM_TRY(quantize_operand(d, A, d->lda, d->M, d->K, at<char>(ws, L.ahat), at<unsigned>(ws, L.amaxA), sA, false, st));
+    FMM_TRY(quantize_operand(d, bk_ptr, bk_ld, d->N, d->K, at<char>(ws, L.bhat), at<unsigned>(ws, L.amaxB), sB, true, st));
     g.A = at<char>(ws, L.ahat); g.lda = d->K; g.a_batch = 0;
     g.B = at<char>(ws, L.bhat); g.ldb = d->K; g.b_batch = 0;
+    if (d->scale_mode == 3) {
+      Fp8GroupArgs q{};
+      q.A = g.A; q.lda = d->K; q.a_batch = 0; q.B = g.B; q.ldb = d->K; q.b_batch = 0;
+      q.rows_a = d->M; q.rows_b = d->N; q.kdim = d->K; q.batches = 1;
+      q.out = C; q.ldo = d->ldc; q.o_batch = 0; q.output = d->output;
+      q.sA = sA; q.sB = sB; q.status = g.status;
+      ProfScope ps(4, st);
+      return launch_fp8_group_gemm(q, st);
+    }
     if (d->scale_mode == 2) { g.row_scale = sA; g.col_scale = sB; g.rs_batch = 0; g.cs_batch = 0; }
     else { g.sA = sA; g.sB = sB; }
   }

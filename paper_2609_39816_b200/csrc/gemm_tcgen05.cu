@@ -1042,7 +1042,220 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   }
 }
 
+// ---------------------------------------------------------------- group-scaled fp8 GEMM (model schedule)
+// Batched block products under the model schedule of Appendix B.1: e4m3 codes of A with one scale per row and per
+// 128 inner indices, e4m3 codes of B with one scale per 128 x 128 block.  As in the int8 kernel every 128-group gets a
+// fresh fp32 accumulator in TMEM (four kind::f8f6f4 MMAs of K = 32); the epilogue multiplies the finished group by
+// s_A[row][g] * s_B[column block][g] and adds it to its fp32 running sums (one fused multiply-add per element and group);
+// after the last group one rounding to the output dtype (bf16 when the product kernel "returns each product in bf16").
+// One CTA per 128 x 128 tile of one product, so a tile's columns lie in one 128-column scale block.
+struct Fp8GroupParams {
+  int rows_a, rows_b, G, batches;   // extents of one product, 128-groups along K, number of products
+  int tiles_m, tiles_n;
+  long long ldo, o_batch;           // output strides in elements
+  int out_bf16, wide;
+  const float* sA; long long sa_batch;   // [batch][rows_a][G]
+  const float* sB; long long sb_batch;   // [batch][ceil(rows_b / 128)][G]
+  unsigned long long wait_limit_ns;
+};
+
+__global__ void __launch_bounds__(kInt8Threads, 1)
+fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                      void* __restrict__ out, Fp8GroupParams p, DeviceStatus* status) {
+  grid_launch_dependents();
+  using L = Int8Layout;             // same tile, ring and barrier block (the scale staging area is unused here)
+  constexpr int BN = L::BN;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - raw_addr);
+  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
+  const uint32_t bar_base = smem_u32(bar_mem);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr uint32_t kTmemCols = 2 * BN;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  grid_dependency_wait();           // codes and scales come from the previous kernel of the stream
+
+  const int tiles_per_batch = p.tiles_m * p.tiles_n;
+  const int total_tiles = tiles_per_batch * p.batches;
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int r = tile / tiles_per_batch;
+        const int rem = tile - r * tiles_per_batch;
+        const int tm = rem / p.tiles_n, tn = rem - tm * p.tiles_n;
+        for (int g = 0; g < p.G; ++g) {
+          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x71, status, p.wait_limit_ns);
+          if (!ok) break;
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::kStageBytes);
+          tma_load_3d(sa, &map_a, full_bar(stage), g * BKB, tm * BM, r);
+          tma_load_3d(sa + L::kABytes, &map_b, full_bar(stage), g * BKB, tn * BN, r);
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        for (int s = 0; s < L::kStages; ++s) {
+          const uint32_t last_parity = (s < stage) ? phase : (phase ^ 1u);
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(s), last_parity)) {
+            if (global_timer_ns() - t0 > 20000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer: one fresh accumulator per group
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(true, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int g = 0; g < p.G; ++g) {
+          ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x82, status, p.wait_limit_ns);
+          if (!ok) break;
+          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x81, status, p.wait_limit_ns);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t da = make_smem_desc(sa);
+          const uint64_t db = make_smem_desc(sa + L::kABytes);
+#pragma unroll
+          for (int k = 0; k < BKB / UMMA_KB; ++k)
+            tc_mma<true>(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc, k != 0 ? 1u : 0u);
+          tc_commit(empty_bar(stage));
+          tc_commit(tfull_bar(acc));
+          if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        tc_commit(drain_bar);
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(drain_bar, 0)) {
+          if (global_timer_ns() - t0 > 20000000ull) break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ scale and accumulate (warps 2..17)
+    const int quad = warp & 3;
+    const int part = (warp - 2) >> 2;
+    constexpr int PN = 32;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int r = tile / tiles_per_batch;
+      const int rem = tile - r * tiles_per_batch;
+      const int tm = rem / p.tiles_n, tn = rem - tm * p.tiles_n;
+      const int row = tm * BM + quad * 32 + lane;
+      const bool row_ok = row < p.rows_a;
+      const int col_base = tn * BN + part * PN;
+      const float* sa_row = p.sA + (long long)r * p.sa_batch + (long long)(row_ok ? row : 0) * p.G;
+      const float* sb_blk = p.sB + (long long)r * p.sb_batch + (long long)tn * p.G;   // BN = 128 = one scale block of columns
+      float sum[PN];
+#pragma unroll
+      for (int j = 0; j < PN; ++j) sum[j] = 0.0f;
+      float s_next = row_ok ? sa_row[0] * sb_blk[0] : 0.0f;
+      for (int g = 0; g < p.G; ++g) {
+        const float sc = s_next;      // the scales do not depend on the products: the next group's come a step ahead
+        if (g + 1 < p.G) s_next = row_ok ? sa_row[g + 1] * sb_blk[g + 1] : 0.0f;
+        ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x93, status, p.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + part * PN), v);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+#pragma unroll
+        for (int j = 0; j < PN; ++j) sum[j] = __fmaf_rn(__uint_as_float(v[j]), sc, sum[j]);
+      }
+      if (!ok) break;
+      if (row_ok && col_base < p.rows_b) {
+        uint32_t w[32];
+#pragma unroll
+        for (int j = 0; j < PN; ++j) w[j] = __float_as_uint(sum[j]);
+        store_row_chunk(out, (long long)r * p.o_batch + (long long)row * p.ldo + col_base, min(32, p.rows_b - col_base), w, 1,
+                        p.out_bf16, 1.0f, p.wide != 0);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
 }  // namespace
+
+fmm_status launch_fp8_group_gemm(const Fp8GroupArgs& a, cudaStream_t st) {
+  using L = Int8Layout;
+  if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim % BKB || a.kdim / BKB > 0x7fffffff) return FMM_ERR_SHAPE;
+  CUtensorMap ma, mb;
+  if (!make_operand_map(&ma, true, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, true, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, L::BN)) return FMM_ERR_CUDA;
+  Fp8GroupParams p;
+  p.rows_a = (int)a.rows_a; p.rows_b = (int)a.rows_b; p.G = (int)(a.kdim / BKB); p.batches = a.batches;
+  p.tiles_m = (int)((a.rows_a + BM - 1) / BM);
+  p.tiles_n = (int)((a.rows_b + L::BN - 1) / L::BN);
+  p.ldo = a.ldo; p.o_batch = a.o_batch; p.out_bf16 = a.output == FMM_BF16;
+  const int es = p.out_bf16 ? 2 : 4;
+  p.wide = (reinterpret_cast<uintptr_t>(a.out) % 32 == 0) && ((a.ldo * es) % 32 == 0) && ((a.o_batch * es) % 32 == 0);
+  p.sA = a.sA; p.sa_batch = a.rows_a * p.G;
+  p.sB = a.sB; p.sb_batch = (long long)p.tiles_n * p.G;
+  p.wait_limit_ns = kDefaultWaitLimitNs;
+  const long long total = (long long)p.tiles_m * p.tiles_n * p.batches;
+  if (total <= 0) return FMM_OK;
+  const int sms = sm_count();
+  if (sms <= 0) return FMM_ERR_CUDA;
+  const int grid = (int)(total < sms ? total : sms);
+  static unsigned long long smem_ok = 0;
+  if (fmm_allow_dynamic_smem(fp8_group_gemm_kernel, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
+  if (launch_dependent(fp8_group_gemm_kernel, dim3(grid), dim3(kInt8Threads), (size_t)L::kTotal, st, ma, mb, a.out, p, a.status) != cudaSuccess)
+    return FMM_ERR_CUDA;
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
 
 fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const float* dAt, const float* dBt, int64_t M,
                                   int64_t K, int64_t N, int output, void* C, int64_t ldc, DeviceStatus* status, cudaStream_t st) {

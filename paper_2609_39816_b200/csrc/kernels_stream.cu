@@ -142,6 +142,8 @@ struct EncodeJob {
   const void* X; int64_t ldx; int gc; int64_t br, bc;
   const CoefTable* tab; void* out; unsigned* amax_bits; float* scale_out;
   int tiles_per_block; int64_t rstride; int stream_out; int blocks;
+  int scale_rows;    // use_scale 3: rows of a block sum that share a scale (1: the input's 1 x 128 scales; 128: the weight's 128 x 128)
+  int bf16_first;    // use_scale 3: the block sum is first rounded to bf16 (weights are stored in bf16 before they are quantised)
 };
 
 template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
@@ -161,6 +163,8 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
   const int tiles_per_block = second ? job_b.tiles_per_block : job_a.tiles_per_block;
   const int64_t rstride = second ? job_b.rstride : job_a.rstride;
   const int stream_out = second ? job_b.stream_out : job_a.stream_out;
+  const int scale_rows = second ? job_b.scale_rows : job_a.scale_rows;
+  const int bf16_first = second ? job_b.bf16_first : job_a.bf16_first;
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int kEncPos = kEncThreads / kEncSplit;
   constexpr int kCellsPerThread = 16 / kEncSplit; // grids have at most 16 cells
@@ -260,11 +264,30 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
 #pragma unroll
         for (int i = 0; i < NP; ++i) acc[i] = __ffma2_rn(make_float2(c1, c1), v[i], acc[i]);
       }
+      // model schedule (use_scale 3): one scale per 128 consecutive entries of a row, shared by scale_rows rows
+      const int gk = (int)((bc + 127) >> 7);
+      const int64_t sidx3 = ((int64_t)r * ((br + scale_rows - 1) / scale_rows) + p / scale_rows) * gk + (t >> 7);
+      if (use_scale == 3 && bf16_first) {
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+          acc[i].x = __bfloat162float(__float2bfloat16_rn(acc[i].x));
+          acc[i].y = __bfloat162float(__float2bfloat16_rn(acc[i].y));
+        }
+      }
       if (kAmaxOnly) {
         float a = 0.0f;
 #pragma unroll
         for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
-        if (use_scale == 2) {
+        if (use_scale == 3) {
+          constexpr int kLanesPerGroup = 128 / VE;   // 16 (bf16 source) or 32 (fp32 source) lanes cover one 128-group
+          if ((vec_per_row & 31) == 0) {             // a warp's 32 consecutive vectors lie in one row
+            const unsigned mask = kLanesPerGroup == 32 ? 0xffffffffu : (0xffffu << (threadIdx.x & 16));
+            const unsigned wmax = __reduce_max_sync(mask, live ? __float_as_uint(a) : 0u);
+            if ((threadIdx.x & (kLanesPerGroup - 1)) == 0 && wmax != 0u) atomicMax(&amax_bits[sidx3], wmax);
+          } else if (live && a > 0.0f) {
+            atomicMax(&amax_bits[sidx3], __float_as_uint(a));
+          }
+        } else if (use_scale == 2) {
           // one scale per row of the block sum: largest magnitude of row p of product r
           if ((vec_per_row & 31) == 0) {       // a warp's 32 consecutive vectors lie in one row
             const unsigned wmax = __reduce_max_sync(0xffffffffu, live ? __float_as_uint(a) : 0u);
@@ -278,7 +301,13 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
           if ((threadIdx.x & 31) == 0 && wmax != 0u) atomicMax(&sm.amax[r], wmax);
         }
       } else if (live) {
-        if (use_scale == 2) {
+        if (use_scale == 3) {
+          const float amax = __uint_as_float(amax_bits[sidx3]);
+          const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+          if ((t & 127) == 0 && (p % scale_rows) == 0 && scale_out) scale_out[sidx3] = sc;
+        } else if (use_scale == 2) {
           // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
           const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
@@ -300,7 +329,7 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
       }
     }
   }
-  if (kAmaxOnly && use_scale != 2) {
+  if (kAmaxOnly && use_scale == 1) {
     __syncthreads();
     if (threadIdx.x < R && sm.amax[threadIdx.x] != 0u) atomicMax(&amax_bits[threadIdx.x], sm.amax[threadIdx.x]);
   }
@@ -315,7 +344,8 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
 template <typename SrcT, typename DstT, bool kAmaxOnly>
 __global__ void __launch_bounds__(256)
 quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int64_t cols, DstT* __restrict__ out,
-                      unsigned* __restrict__ amax_bits, float* __restrict__ scale_out, int mode) {
+                      unsigned* __restrict__ amax_bits, float* __restrict__ scale_out, int mode, int scale_rows,
+                      int bf16_first) {
   constexpr int VE = Vec16<SrcT>::kElems;
   constexpr int NP = VE / 2;
   constexpr int kU = 4;
@@ -351,11 +381,29 @@ quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int
       const bool on = base + u * stride < nvec;
       float2 v[NP];
       Vec16<SrcT>::unpack(raw[u], v);
+      // model schedule (mode 3): one scale per 128 consecutive entries of a row, shared by scale_rows rows
+      const int64_t sidx3 = (row[u] / scale_rows) * ((cols + 127) >> 7) + (col[u] >> 7);
+      if (mode == 3 && bf16_first) {
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+          v[i].x = __bfloat162float(__float2bfloat16_rn(v[i].x));
+          v[i].y = __bfloat162float(__float2bfloat16_rn(v[i].y));
+        }
+      }
       if (kAmaxOnly) {
         float a = 0.0f;
 #pragma unroll
         for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(v[i].x), fabsf(v[i].y)));
-        if (mode == 2) {
+        if (mode == 3) {
+          constexpr int kLanesPerGroup = 128 / VE;
+          if ((vec_per_row & 31) == 0) {   // a warp's 32 consecutive vectors lie in one row
+            const unsigned mask = kLanesPerGroup == 32 ? 0xffffffffu : (0xffffu << (threadIdx.x & 16));
+            const unsigned wmax = __reduce_max_sync(mask, on ? __float_as_uint(a) : 0u);
+            if ((threadIdx.x & (kLanesPerGroup - 1)) == 0 && wmax != 0u) atomicMax(&amax_bits[sidx3], wmax);
+          } else if (on && a > 0.0f) {
+            atomicMax(&amax_bits[sidx3], __float_as_uint(a));
+          }
+        } else if (mode == 2) {
           if ((vec_per_row & 31) == 0) {   // a warp's 32 consecutive vectors lie in one row
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
@@ -367,7 +415,13 @@ quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int
           tmax = fmaxf(tmax, a);
         }
       } else if (on) {
-        if (mode == 2) {
+        if (mode == 3) {
+          const float amax = __uint_as_float(amax_bits[sidx3]);
+          const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+#pragma unroll
+          for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+          if ((col[u] & 127) == 0 && (row[u] % scale_rows) == 0 && scale_out) scale_out[sidx3] = sc;
+        } else if (mode == 2) {
           const float amax = __uint_as_float(amax_bits[row[u]]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
 #pragma unroll
@@ -386,7 +440,7 @@ quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int
       }
     }
   }
-  if (kAmaxOnly && mode != 2) {
+  if (kAmaxOnly && mode != 2 && mode != 3) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
     if ((threadIdx.x & 31) == 0 && tmax > 0.0f) atomicMax(&s_amax, __float_as_uint(tmax));
@@ -397,15 +451,16 @@ quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int
 
 template <typename SrcT, typename DstT>
 static cudaError_t launch_quantize_plain_t(const void* X, int64_t ldx, int64_t rows, int64_t cols, void* out,
-                                           unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st) {
+                                           unsigned* amax_bits, float* scale, bool amax_only, int mode, int scale_rows,
+                                           int bf16_first, cudaStream_t st) {
   constexpr int VE = Vec16<SrcT>::kElems;
   const int64_t nvec = rows * (cols / VE);
   if (nvec == 0) return cudaSuccess;
   const int grid = (int)std::min<int64_t>((nvec + 256 * 4 - 1) / (256 * 4), 148 * 16);
   if (amax_only)
-    quantize_plain_kernel<SrcT, DstT, true><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode);
+    quantize_plain_kernel<SrcT, DstT, true><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode, scale_rows > 0 ? scale_rows : 1, bf16_first);
   else
-    quantize_plain_kernel<SrcT, DstT, false><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode);
+    quantize_plain_kernel<SrcT, DstT, false><<<grid, 256, 0, st>>>((const SrcT*)X, ldx, rows, cols, (DstT*)out, amax_bits, scale, mode, scale_rows > 0 ? scale_rows : 1, bf16_first);
   ++fmm_launch_counter();
   return cudaGetLastError();
 }
@@ -435,7 +490,8 @@ static bool make_job(const EncodeOperand& o, EncodeJob* j, size_t* smem) {
   // outputs larger than the part of L2 that keeps shared data (~60 MB) will have left it before they are read
   int stream_out = (int64_t)o.h_tab->R * o.out_stride * (int64_t)sizeof(DstT) > ((int64_t)48 << 20) ? 1 : 0;
   if (const char* e = std::getenv("FMM_B200_ENC_STREAM")) stream_out = std::atoi(e);
-  *j = EncodeJob{o.X, o.ldx, o.gc, o.br, o.bc, o.d_tab, o.out, o.amax_bits, o.scale, tpb, o.out_stride, stream_out, grid};
+  *j = EncodeJob{o.X, o.ldx, o.gc, o.br, o.bc, o.d_tab, o.out, o.amax_bits, o.scale, tpb, o.out_stride, stream_out, grid,
+                 o.scale_rows > 0 ? o.scale_rows : 1, o.bf16_first};
   return true;
 }
 
@@ -728,15 +784,16 @@ __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A,
 }  // namespace
 
 cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64_t ldx, int64_t rows, int64_t cols,
-                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st) {
+                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, int scale_rows,
+                                  int bf16_first, cudaStream_t st) {
   if (storage == FMM_F32 && product == FMM_BF16)
-    return launch_quantize_plain_t<float, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+    return launch_quantize_plain_t<float, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, scale_rows, bf16_first, st);
   if (storage == FMM_BF16 && product == FMM_BF16)
-    return launch_quantize_plain_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+    return launch_quantize_plain_t<__nv_bfloat16, __nv_bfloat16>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, scale_rows, bf16_first, st);
   if (storage == FMM_F32 && product == FMM_E4M3)
-    return launch_quantize_plain_t<float, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+    return launch_quantize_plain_t<float, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, scale_rows, bf16_first, st);
   if (storage == FMM_BF16 && product == FMM_E4M3)
-    return launch_quantize_plain_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, st);
+    return launch_quantize_plain_t<__nv_bfloat16, __nv_fp8_storage_t>(X, ldx, rows, cols, out, amax_bits, scale, amax_only, mode, scale_rows, bf16_first, st);
   return cudaErrorInvalidValue;
 }
 
@@ -770,7 +827,7 @@ cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a,
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
                           unsigned* amax_bits, float* scale, bool amax_only, int use_scale, cudaStream_t st) {
-  const EncodeOperand a{X, ldx, gr, gc, br, bc, d_tab, h_tab, out, out_stride, amax_bits, scale};
+  const EncodeOperand a{X, ldx, gr, gc, br, bc, d_tab, h_tab, out, out_stride, amax_bits, scale, 1, 0};
   return launch_encode_pair(storage, product, a, nullptr, amax_only, use_scale, st);
 }
 

@@ -53,7 +53,8 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 // max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).
 // With use_scale == 1, scale[r] is derived from amax_bits[r] (2^ceil(log2(amax/448)), 1 if amax==0),
 // written to scale[R] and divided out before rounding.  With use_scale == 2 there is one scale per row of every
-// block sum: amax_bits and scale are [R][br]; scale = amax / 448 in fp32 (1 for an all-zero row).
+// block sum: amax_bits and scale are [R][br]; scale = amax / 448 in fp32 (1 for an all-zero row).  use_scale == 3 (model
+// schedule): one scale per 128 consecutive entries of a row, see EncodeOperand::scale_rows.
 // h_tab = host copy of the same table (its list lengths size the kernel's shared memory).
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
@@ -62,13 +63,16 @@ cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, 
 // The same decisions for a whole operand taken as one block with coefficient 1 (the classical control): rows x cols
 // of `storage` -> `product` dtype, mode 0 / 1 / 2 as use_scale above (amax_bits, scale: one word, or one per row).
 cudaError_t launch_quantize_plain(int storage, int product, const void* X, int64_t ldx, int64_t rows, int64_t cols,
-                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, cudaStream_t st);
+                                  void* out, unsigned* amax_bits, float* scale, bool amax_only, int mode, int scale_rows,
+                                  int bf16_first, cudaStream_t st);
 
 // Two operands in one launch (A and B of one product, encoded side by side); b may be null.  Fields as the arguments
 // of launch_encode.
 struct EncodeOperand {
   const void* X; int64_t ldx; int gr, gc; int64_t br, bc;
   const CoefTable* d_tab; const CoefTable* h_tab; void* out; int64_t out_stride; unsigned* amax_bits; float* scale;
+  int scale_rows;   // use_scale 3 only: rows sharing a scale (1 or 128); amax_bits / scale are [R][ceil(br/scale_rows)][ceil(bc/128)]
+  int bf16_first;   // use_scale 3 only: round the block sum to bf16 before it is quantised
 };
 cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
                                int use_scale, cudaStream_t st);
@@ -127,6 +131,18 @@ struct BlockProductArgs {
   unsigned long long wait_limit_ns;    // 0: default (2 s)
 };
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
+
+// Batched block products under the model schedule (scale mode 3): e4m3 codes A [batches][rows_a][kdim] (K-major, lda) and
+// B [batches][rows_b][kdim], kdim % 128 == 0; scales sA [batches][rows_a][kdim/128], sB [batches][ceil(rows_b/128)][kdim/128];
+// out [batches][rows_a][ldo] of `output` (FMM_F32 / FMM_BF16), o_batch elements apart.
+struct Fp8GroupArgs {
+  const void* A; int64_t lda, a_batch; const void* B; int64_t ldb, b_batch;
+  int64_t rows_a, rows_b, kdim; int batches;
+  void* out; int64_t ldo, o_batch; int output;
+  const float* sA; const float* sB;
+  DeviceStatus* status;
+};
+fmm_status launch_fp8_group_gemm(const Fp8GroupArgs& a, cudaStream_t st);
 
 // The group-scaled int8 operator in one kernel (tcgen05 kind::i8, int32 accumulators in TMEM, rescale in the epilogue):
 // cA [M][K], cB [N][K] int8 codes (K % 128 == 0, rows 16-byte aligned), dAt [K/128][M] and dBt [K/128][N] fp32 scales,

@@ -64,6 +64,10 @@ def run_scheme_gemm(s, A_t, B_t, S, Pd, O, weight_layout=False, scale_mode=0, fl
     if scale_mode == 1:
         p["sA"] = ws[off["sA"]:off["sA"] + 4 * R].view(torch.float32).to(torch.float64).cpu().numpy()
         p["sB"] = ws[off["sB"]:off["sB"] + 4 * R].view(torch.float32).to(torch.float64).cpu().numpy()
+    elif scale_mode == 3:     # model schedule: [R][bm][G] and [R][ceil(bn/128)][G]
+        G3, CB3 = -(-bk // 128), -(-bn // 128)
+        p["sA"] = ws[off["sA"]:off["sA"] + 4 * R * bm * G3].view(torch.float32).to(torch.float64).cpu().numpy().reshape(R, bm, G3)
+        p["sB"] = ws[off["sB"]:off["sB"] + 4 * R * CB3 * G3].view(torch.float32).to(torch.float64).cpu().numpy().reshape(R, CB3, G3)
     elif scale_mode == 2:     # one scale per row of each block sum of A / per column of each block sum of B
         p["sA"] = ws[off["sA"]:off["sA"] + 4 * R * bm].view(torch.float32).to(torch.float64).cpu().numpy().reshape(R, bm)
         p["sB"] = ws[off["sB"]:off["sB"] + 4 * R * bn].view(torch.float32).to(torch.float64).cpu().numpy().reshape(R, bn)

@@ -60,6 +60,9 @@ def _inputs(seed, M, K, N, S, kind="normal", bound=None):
     ("strassen444", 128, 128, 128, "f32", "e4m3", "f32", "u01", 2),         # the ensemble's shape: row / column scales
     ("strassen444", 512, 1024, 544, "bf16", "e4m3", "bf16", "t3", 2),       # row / column scales, several tiles, CTA pairs
     ("strassen222", 200, 2240, 272, "bf16", "e4m3", "f32", "llm", 2),       # rows of 280 vectors: per-thread amax path
+    ("strassen444", 512, 1024, 512, "bf16", "e4m3", "f32", "t3", 3),        # model schedule: 2 groups, one 128-column block
+    ("strassen444", 256, 2048, 1088, "bf16", "e4m3", "bf16", "llm", 3),     # 4 groups, bn = 272: three column blocks, ragged
+    ("strassen222", 384, 768, 528, "f32", "e4m3", "f32", "llm", 3),         # fp32 source (weights rounded to bf16 first), 3 groups
 ])
 def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     At, Bt, A64, B64 = _inputs(3, M, K, N, S, kind)
@@ -188,6 +191,8 @@ def test_row_leak_pattern_on_gpu(lib):
     (384, 2240, 264, "bf16", "e4m3", "bf16", 1, False),    # fp8 with per-tensor scales
     (384, 2240, 264, "bf16", "e4m3", "f32", 2, False),     # fp8 with per-row / per-column scales
     (128, 128, 128, "f32", "e4m3", "f32", 2, True),
+    (384, 2048, 528, "bf16", "e4m3", "bf16", 3, True),     # the deployed FP8 kernel's schedule: 1 x 128 and 128 x 128 scales
+    (200, 1024, 264, "f32", "e4m3", "f32", 3, False),
 ])
 def test_classical_and_exact_match_oracle(lib, M, K, N, S, Pd, O, scale, wl):
     At, Bt, A64, B64 = _inputs(9, M, K, N, S, "llm")
