@@ -486,7 +486,7 @@ def run_workload(args):
         torch.cuda.synchronize()
         return float(np.median([a.elapsed_time(b) for a, b in evs]))
 
-    def one_gemm(scheme, T, K, N, S, Pd, O, scale, dist):
+    def one_gemm(scheme, T, K, N, S, Pd, O, scale, dist, flags=0):
         A = gen.activations_outlier(0, 1, T, K, dist=dist, frac=0.001 if dist == "t3" else 0.005,
                                     factor=300.0 if dist == "t3" else 100.0, at_least=1 if dist == "t3" else 0)
         if S == "f32":
@@ -496,12 +496,12 @@ def run_workload(args):
         Wt = gen.to_storage(W, S)[0].cuda()
         s = fmm.scheme_builtin(scheme)
         m, k, n, R = s.dims
-        d = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale)
+        d = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale, flags=flags)
         ws = torch.empty(fmm.scheme_gemm_workspace(s, d), dtype=torch.uint8, device="cuda")
         C = torch.empty((T, N), dtype=torch.float32 if O == "f32" else torch.bfloat16, device="cuda")
         t = timed(lambda: fmm.scheme_gemm(s, d, At, Wt, C, ws))
         fmm.device_status(ws)
-        dr = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale, flags=fmm.FLAG_REUSE_BHAT)
+        dr = fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale, flags=flags | fmm.FLAG_REUSE_BHAT)
         t_cached = timed(lambda: fmm.scheme_gemm(s, dr, At, Wt, C, ws))
         wsc = torch.empty(max(fmm.classical_gemm_workspace(d), 256), dtype=torch.uint8, device="cuda")
         t_cl = timed(lambda: fmm.classical_gemm(d, At, Wt, C, wsc))
@@ -520,6 +520,10 @@ def run_workload(args):
     elif wl == "c4":
         shapes = [(4096, 12288), (4096, 4096), (4096, 22016), (11008, 4096)]
         out["gemms"] = [one_gemm("strassen444", 2048, K, N, "bf16", "e4m3", "bf16", 1, "t3") for K, N in shapes]
+    elif wl == "c4m":   # the same shapes under the paper's model schedule: 1 x 128 / 128 x 128 scales, products in bf16
+        shapes = [(4096, 12288), (4096, 4096), (4096, 22016), (11008, 4096)]
+        out["gemms"] = [one_gemm("strassen444", 2048, K, N, "bf16", "e4m3", "bf16", 3, "t3", flags=fmm.FLAG_PRODUCTS_BF16)
+                        for K, N in shapes]
     elif wl == "c5":
         shapes = [(5120, 15360), (5120, 27648), (13824, 5120)]
         out["gemms"] = [one_gemm("strassen444", 8192, K, N, "bf16", pd, "bf16", 1 if pd == "e4m3" else 0, "t3")
@@ -653,7 +657,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=32, help="gauges per rank in the c3 sweep (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c5 | int8 | ensemble")
+    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c4m | c5 | int8 | ensemble")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

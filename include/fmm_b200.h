@@ -110,9 +110,9 @@ typedef struct {
                             first rounded to bf16, then get one scale per 128 x 128 block (128 inner
                             indices x 128 output columns); s = amax / 448 as in mode 2.  The product
                             kernel accumulates every 128-group on its own, multiplies it by the two
-                            scales and adds the groups in ascending order in fp32.  Requires K/k to be
-                            a multiple of 128.  Scales in the workspace: [R][M/m][K/k/128] and
-                            [R][ceil(N/n/128)][K/k/128].  classical_gemm applies the same schedule to
+                            scales and adds the groups in ascending order in fp32 (the last group may be
+                            shorter).  Scales in the workspace: [R][M/m][G] and [R][ceil(N/n/128)][G],
+                            G = ceil(K/k/128).  classical_gemm applies the same schedule to
                             the operands themselves (the deployed FP8 kernel's layout of scales) */
   int32_t flags;         /* FMM_FLAG_* */
 } fmm_gemm_desc;

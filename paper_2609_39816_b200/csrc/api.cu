@@ -104,7 +104,6 @@ fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
   if (d->scale_mode != 0 && !(d->scale_mode >= 1 && d->scale_mode <= 3 && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
   if (d->M % m || d->K % k || d->N % n) return FMM_ERR_SHAPE;
   if ((d->K / k) % 16 || (d->N / n) % 8) return FMM_ERR_SHAPE;
-  if (d->scale_mode == 3 && (d->K / k) % 128) return FMM_ERR_SHAPE;   // the model schedule scales groups of 128 inner indices
   const int es = esize(d->storage), eo = esize(d->output);
   const int64_t min_ldb = d->b_is_weight_layout ? d->K : d->N;
   if (d->lda < d->K || d->ldb < min_ldb || d->ldc < d->N) return FMM_ERR_SHAPE;

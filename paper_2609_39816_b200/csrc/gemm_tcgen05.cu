@@ -1230,12 +1230,12 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
 fmm_status launch_fp8_group_gemm(const Fp8GroupArgs& a, cudaStream_t st) {
   using L = Int8Layout;
-  if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim % BKB || a.kdim / BKB > 0x7fffffff) return FMM_ERR_SHAPE;
+  if (a.rows_a > 0x7fffffff || a.rows_b > 0x7fffffff || a.kdim <= 0 || a.kdim > 0x3fffffff) return FMM_ERR_SHAPE;
   CUtensorMap ma, mb;
   if (!make_operand_map(&ma, true, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
   if (!make_operand_map(&mb, true, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, L::BN)) return FMM_ERR_CUDA;
   Fp8GroupParams p;
-  p.rows_a = (int)a.rows_a; p.rows_b = (int)a.rows_b; p.G = (int)(a.kdim / BKB); p.batches = a.batches;
+  p.rows_a = (int)a.rows_a; p.rows_b = (int)a.rows_b; p.G = (int)((a.kdim + BKB - 1) / BKB); p.batches = a.batches;   // a ragged last group is zero-filled by the copies
   p.tiles_m = (int)((a.rows_a + BM - 1) / BM);
   p.tiles_n = (int)((a.rows_b + L::BN - 1) / L::BN);
   p.ldo = a.ldo; p.o_batch = a.o_batch; p.out_bf16 = a.output == FMM_BF16;

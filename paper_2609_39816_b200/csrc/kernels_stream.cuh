@@ -133,7 +133,7 @@ struct BlockProductArgs {
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
 
 // Batched block products under the model schedule (scale mode 3): e4m3 codes A [batches][rows_a][kdim] (K-major, lda) and
-// B [batches][rows_b][kdim], kdim % 128 == 0; scales sA [batches][rows_a][kdim/128], sB [batches][ceil(rows_b/128)][kdim/128];
+// B [batches][rows_b][kdim]; G = ceil(kdim / 128) groups; scales sA [batches][rows_a][G], sB [batches][ceil(rows_b/128)][G];
 // out [batches][rows_a][ldo] of `output` (FMM_F32 / FMM_BF16), o_batch elements apart.
 struct Fp8GroupArgs {
   const void* A; int64_t lda, a_batch; const void* B; int64_t ldb, b_batch;

@@ -63,6 +63,7 @@ def _inputs(seed, M, K, N, S, kind="normal", bound=None):
     ("strassen444", 512, 1024, 512, "bf16", "e4m3", "f32", "t3", 3),        # model schedule: 2 groups, one 128-column block
     ("strassen444", 256, 2048, 1088, "bf16", "e4m3", "bf16", "llm", 3),     # 4 groups, bn = 272: three column blocks, ragged
     ("strassen222", 384, 768, 528, "f32", "e4m3", "f32", "llm", 3),         # fp32 source (weights rounded to bf16 first), 3 groups
+    ("strassen444", 128, 11008, 512, "bf16", "e4m3", "f32", "t3", 3),       # K/4 = 2752 = 21.5 groups: ragged last group
 ])
 def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     At, Bt, A64, B64 = _inputs(3, M, K, N, S, kind)
@@ -84,6 +85,7 @@ def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     ("strassen444", 384, 320, 288, "bf16", "bf16", "f32", "llm", 0),        # ragged tiles
     ("strassen444", 512, 1024, 544, "bf16", "e4m3", "bf16", "t3", 1),       # per-tensor scales folded into the decode
     ("strassen222", 200, 2240, 272, "bf16", "e4m3", "f32", "llm", 2),       # row / column scales applied before the rounding
+    ("strassen444", 512, 2048, 1024, "bf16", "e4m3", "bf16", "t3", 3),      # the paper's whole model schedule: group scales, bf16 products
 ])
 def test_products_returned_in_bf16(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     """FMM_FLAG_PRODUCTS_BF16, the paper's model schedule: every product rounded once to bf16, combined in fp32.
@@ -391,3 +393,20 @@ def test_decode_order_is_part_of_the_operator(lib):
     C1 = gu.run_scheme_gemm(sp, At, Bt, "bf16", "bf16", "f32")
     assert gu.rel_fro(C1, oracle.scheme_gemm(op, A64, B64, "bf16", "f32")) <= TOL_FRO
     assert not np.array_equal(C0, C1) and gu.rel_fro(C0, C1) < 1e-5
+
+
+def test_sweep_under_the_model_schedule(lib):
+    """error_sweep with the model schedule (group scales, products returned in bf16): ratios against the oracle."""
+    At, Bt, A64, B64 = _inputs(19, 256, 1024, 512, "bf16", "t3")
+    var = oracle.sign_variants(4, 4, 4)[::85]
+    P = np.stack([np.diag(v[0]) for v in var]); Q = np.stack([np.diag(v[1]) for v in var]); S = np.stack([np.diag(v[2]) for v in var])
+    s2, o2 = lib.scheme_builtin("strassen444"), gu.oracle_scheme("strassen444")
+    d = lib.GemmDesc.make(256, 1024, 512, "bf16", "e4m3", "bf16", scale_mode=3, flags=lib.FLAG_PRODUCTS_BF16)
+    ws = gu.workspace(lib.error_sweep_workspace(s2, d, len(var)))
+    ratios, summ = lib.error_sweep(s2, 0, P, Q, S, d, At, Bt, ws)
+    Cs = A64 @ B64
+    Ecl = oracle.rel_error(oracle.classical_gemm(A64, B64, "e4m3", "bf16", 3), Cs)
+    assert math.isclose(summ["e_classical_rel"], Ecl, rel_tol=TOL_RATIO)
+    for r, v in zip(ratios, var):
+        E = oracle.rel_error(oracle.scheme_gemm(oracle.sign_variant(o2, *v), A64, B64, "e4m3", "bf16", 3, md="bf16"), Cs)
+        assert abs(r - E / Ecl) <= TOL_RATIO * E / Ecl
