@@ -146,7 +146,9 @@ struct EncodeJob {
   int bf16_first;    // use_scale 3: the block sum is first rounded to bf16 (weights are stored in bf16 before they are quantised)
 };
 
-template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit>
+// kM3: the model schedule (use_scale == 3) is compiled into its own instantiation so that the other modes carry none
+// of its index arithmetic.
+template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit, bool kM3>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
   grid_launch_dependents();   // the block products may set up while this grid drains; they wait before reading
@@ -244,6 +246,9 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
     const unsigned char* my_stage = stage + (it & 1) * kStageBytes + pv * 16;
 
     DstT* dst = out + (int64_t)p * bc + t;
+    const int m3_gk = (int)((bc + 127) >> 7);                                   // used by the model schedule only
+    const int64_t m3_row_groups = scale_rows == 1 ? br : (br + 127) >> 7;       // scale_rows is 1 or 128
+    const int64_t m3_row_group = scale_rows == 1 ? p : p >> 7;
     // one product at a time, its list walked two entries per step (lists are padded to an even length with
     // (zero slab, 0.0f) entries, which add exactly nothing); the four accumulator pairs are independent chains
     for (int r = g; r < R; r += kEncSplit) {
@@ -265,9 +270,9 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
         for (int i = 0; i < NP; ++i) acc[i] = __ffma2_rn(make_float2(c1, c1), v[i], acc[i]);
       }
       // model schedule (use_scale 3): one scale per 128 consecutive entries of a row, shared by scale_rows rows
-      const int gk = (int)((bc + 127) >> 7);
-      const int64_t sidx3 = ((int64_t)r * ((br + scale_rows - 1) / scale_rows) + p / scale_rows) * gk + (t >> 7);
-      if (use_scale == 3 && bf16_first) {
+      int64_t sidx3 = 0;
+      if constexpr (kM3) sidx3 = ((int64_t)r * m3_row_groups + m3_row_group) * m3_gk + (t >> 7);
+      if (kM3 && bf16_first) {
 #pragma unroll
         for (int i = 0; i < NP; ++i) {
           acc[i].x = __bfloat162float(__float2bfloat16_rn(acc[i].x));
@@ -278,7 +283,7 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
         float a = 0.0f;
 #pragma unroll
         for (int i = 0; i < NP; ++i) a = fmaxf(a, fmaxf(fabsf(acc[i].x), fabsf(acc[i].y)));   // fmaxf drops NaN
-        if (use_scale == 3) {
+        if (kM3) {
           constexpr int kLanesPerGroup = 128 / VE;   // 16 (bf16 source) or 32 (fp32 source) lanes cover one 128-group
           if ((vec_per_row & 31) == 0) {             // a warp's 32 consecutive vectors lie in one row
             const unsigned mask = kLanesPerGroup == 32 ? 0xffffffffu : (0xffffu << (threadIdx.x & 16));
@@ -301,12 +306,12 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
           if ((threadIdx.x & 31) == 0 && wmax != 0u) atomicMax(&sm.amax[r], wmax);
         }
       } else if (live) {
-        if (use_scale == 3) {
+        if (kM3) {
           const float amax = __uint_as_float(amax_bits[sidx3]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
 #pragma unroll
           for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
-          if ((t & 127) == 0 && (p % scale_rows) == 0 && scale_out) scale_out[sidx3] = sc;
+          if ((t & 127) == 0 && (p & (scale_rows - 1)) == 0 && scale_out) scale_out[sidx3] = sc;
         } else if (use_scale == 2) {
           // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
           const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
@@ -495,6 +500,16 @@ static bool make_job(const EncodeOperand& o, EncodeJob* j, size_t* smem) {
   return true;
 }
 
+template <typename SrcT, typename DstT, bool kAmaxOnly, int kSplit, bool kM3>
+static cudaError_t launch_encode_k(int grid, size_t smem, cudaStream_t st, const EncodeJob& ja, const EncodeJob& jb, int use_scale) {
+  auto k = encode_kernel<SrcT, DstT, kAmaxOnly, kSplit, kM3>;
+  static unsigned long long smem_ok = 0;   // per template instantiation, one bit per device
+  cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok);
+  if (e != cudaSuccess) return e;
+  k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
+  return cudaSuccess;
+}
+
 template <typename SrcT, typename DstT, int kSplit>
 cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool amax_only, int use_scale, cudaStream_t st) {
   EncodeJob ja{}, jb{};
@@ -504,18 +519,17 @@ cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool
   const int grid = ja.blocks + jb.blocks;
   if (grid == 0) return cudaSuccess;
   const size_t smem = std::max(smem_a, smem_b);
-  static unsigned long long smem_ok[2] = {0, 0};   // per template instantiation, one bit per device
-  if (amax_only) {
-    auto k = encode_kernel<SrcT, DstT, true, kSplit>;
-    cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[0]);
-    if (e != cudaSuccess) return e;
-    k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
-  } else {
-    auto k = encode_kernel<SrcT, DstT, false, kSplit>;
-    cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[1]);
-    if (e != cudaSuccess) return e;
-    k<<<grid, kEncThreads, smem, st>>>(ja, jb, use_scale);
-  }
+  // the model schedule exists for e4m3 block sums only
+  constexpr bool kCanM3 = sizeof(DstT) == 1;
+  if (use_scale == 3 && !kCanM3) return cudaErrorInvalidValue;
+  cudaError_t e;
+  if (use_scale == 3)
+    e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale)
+                  : launch_encode_k<SrcT, DstT, false, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale);
+  else
+    e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, false>(grid, smem, st, ja, jb, use_scale)
+                  : launch_encode_k<SrcT, DstT, false, kSplit, false>(grid, smem, st, ja, jb, use_scale);
+  if (e != cudaSuccess) return e;
   ++fmm_launch_counter();
   return cudaGetLastError();
 }
