@@ -538,6 +538,33 @@ def run_workload(args):
         return
     else:
         raise SystemExit(f"unknown workload {wl}")
+    if wl == "c5":
+        # the configuration's sweep: 512 gauges of <4,4,4;49>, applied to the outer factor, over the down projection
+        T, K, N, G = 8192, 13824, 5120, 512
+        A = gen.to_storage(gen.activations_outlier(0, 1, T, K, dist="t3", frac=0.001, factor=300.0, at_least=1), "bf16")[0].cuda()
+        W = gen.to_storage(gen.normal(0, 2, (N, K), std=0.02), "bf16")[0].cuda()
+        P, Q, S = sweep_gauges(G)
+        s1 = fmm.scheme_builtin("strassen222")
+        s2 = fmm.scheme_kron(s1, s1)
+        sweeps = []
+        for pd, scale in (("bf16", 0), ("e4m3", 1)):
+            d = fmm.GemmDesc.make(T, K, N, "bf16", pd, "bf16", weight_layout=True, scale_mode=scale)
+            ws = torch.empty(fmm.error_sweep_workspace(s2, d, G), dtype=torch.uint8, device="cuda")
+            Cs = torch.empty((T, N), dtype=torch.float64, device="cuda")
+            fmm.exact_gemm_f64(d, A, W, Cs)
+            fmm.error_sweep(s2, 1, P[:2], Q[:2], S[:2], d, A, W, ws, Cstar=Cs)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ratios, summ = fmm.error_sweep(s2, 1, P, Q, S, d, A, W, ws, Cstar=Cs)
+            e1.record(); torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) * 1e-3
+            sweeps.append({"product": pd, "gauges": G, "seconds": sec, "gauges_per_s": G / sec,
+                           "tensor_bound_gauges_per_s": peaks["bf16"] * (2 if pd == "e4m3" else 1) * 1e12 / (2.0 * 49 * (T // 4) * (K // 4) * (N // 4)),
+                           "min": summ["min"], "median": summ["median"], "max": summ["max"], "count_gt2": summ["count_gt2"],
+                           "e_classical_rel": summ["e_classical_rel"]})
+            del ws, Cs
+        out["sweep_down_projection"] = sweeps
     tot_t = sum(g["ms"] for g in out["gemms"])
     tot_f = sum(2.0 * g["shape"][0] * g["shape"][1] * g["shape"][2] for g in out["gemms"])
     out["metric"] = METRIC
@@ -655,7 +682,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sweep-gauges", type=int, default=32, help="gauges per rank in the c3 sweep (0 = skip)")
+    ap.add_argument("--sweep-gauges", type=int, default=512, help="gauges per rank in the c3 sweep (0 = skip); config 3 names 512")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c4m | c5 | int8 | ensemble")
     args = ap.parse_args()
