@@ -136,6 +136,33 @@ template <int NP> __device__ __forceinline__ void store_vec(__nv_fp8_storage_t* 
   }
 }
 
+// x / sc for values that are about to be rounded to e4m3, without eight IEEE divisions in the common case.  The exact
+// schedule is code = rnd_e4m3(fl32(x / sc)).  q = x * fl32(1 / sc) lies within 1.5 * 2^-23 (relative) of fl32(x / sc); rounding
+// to e4m3 is monotone, so if q (1 + 2^-21) and q (1 - 2^-21) round to the same code, so does fl32(x / sc), and q can stand
+// in for it.  Otherwise (a value that close to a rounding boundary: a few in a million) the vector is divided exactly.
+template <int NP>
+__device__ __forceinline__ void divide_for_e4m3(float2 (&a)[NP], float sc) {
+  const float r = __frcp_rn(sc);
+  const float2 up = make_float2(1.0f + 4.76837158203125e-7f, 1.0f + 4.76837158203125e-7f);
+  const float2 dn = make_float2(1.0f - 4.76837158203125e-7f, 1.0f - 4.76837158203125e-7f);
+  float2 q[NP];
+  bool same = true;
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    q[i] = __fmul2_rn(a[i], make_float2(r, r));
+    const unsigned hi = __nv_cvt_float2_to_fp8x2(__fmul2_rn(q[i], up), __NV_SATFINITE, __NV_E4M3);
+    const unsigned lo = __nv_cvt_float2_to_fp8x2(__fmul2_rn(q[i], dn), __NV_SATFINITE, __NV_E4M3);
+    same = same && (hi == lo);
+  }
+  if (same) {
+#pragma unroll
+    for (int i = 0; i < NP; ++i) a[i] = q[i];
+  } else {
+#pragma unroll
+    for (int i = 0; i < NP; ++i) { a[i].x = __fdiv_rn(a[i].x, sc); a[i].y = __fdiv_rn(a[i].y, sc); }
+  }
+}
+
 // One operand of an encode launch.  A launch carries up to two (A and B of one product): blocks [0, a.blocks) work
 // on the first, the rest on the second, so both operands are encoded side by side without a second stream.
 struct EncodeJob {
@@ -309,15 +336,23 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
         if (kM3) {
           const float amax = __uint_as_float(amax_bits[sidx3]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+          if constexpr (sizeof(DstT) == 1) {
+            divide_for_e4m3<NP>(acc, sc);
+          } else {
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+            for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+          }
           if ((t & 127) == 0 && (p & (scale_rows - 1)) == 0 && scale_out) scale_out[sidx3] = sc;
         } else if (use_scale == 2) {
           // scale = max|x| / 448 in fp32 (1 for an all-zero row), code = x / scale in fp32, then one rounding
           const float amax = __uint_as_float(amax_bits[(int64_t)r * br + p]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+          if constexpr (sizeof(DstT) == 1) {
+            divide_for_e4m3<NP>(acc, sc);
+          } else {
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+            for (int i = 0; i < NP; ++i) { acc[i].x = __fdiv_rn(acc[i].x, sc); acc[i].y = __fdiv_rn(acc[i].y, sc); }
+          }
           if (t == 0 && scale_out) scale_out[(int64_t)r * br + p] = sc;
         } else if (use_scale) {
           if (sm.use_mul[r]) {
@@ -423,14 +458,22 @@ quantize_plain_kernel(const SrcT* __restrict__ X, int64_t ldx, int64_t rows, int
         if (mode == 3) {
           const float amax = __uint_as_float(amax_bits[sidx3]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+          if constexpr (sizeof(DstT) == 1) {
+            divide_for_e4m3<NP>(v, sc);
+          } else {
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+            for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+          }
           if ((col[u] & 127) == 0 && (row[u] % scale_rows) == 0 && scale_out) scale_out[sidx3] = sc;
         } else if (mode == 2) {
           const float amax = __uint_as_float(amax_bits[row[u]]);
           const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+          if constexpr (sizeof(DstT) == 1) {
+            divide_for_e4m3<NP>(v, sc);
+          } else {
 #pragma unroll
-          for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+            for (int i = 0; i < NP; ++i) { v[i].x = __fdiv_rn(v[i].x, sc); v[i].y = __fdiv_rn(v[i].y, sc); }
+          }
           if (col[u] == 0 && scale_out) scale_out[row[u]] = sc;
         } else if (mode == 1) {
           if (use_mul) {
