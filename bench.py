@@ -315,7 +315,7 @@ def run_ours(args):
     # The same steps software-pipelined the way a caller streams requests: two sets of device buffers; the copies
     # of step i+1 (copy-in stream) and of step i-1's result (copy-out stream) run beside the kernels of step i.
     # Every step still copies all of its inputs from pinned host memory and its whole result back.
-    def e2e_pipelined(steps):
+    def e2e_pipelined(steps, weights_resident=False):
         main = torch.cuda.current_stream()
         s_in, s_in2, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         sets = [(A, B, C, ws, C_h)]
@@ -339,13 +339,14 @@ def run_ours(args):
             with torch.cuda.stream(s_in2):                 # the two operands travel on two copy streams
                 if i >= 2:
                     s_in2.wait_event(ev_comp[i % 2])
-                Bd.copy_(B_h, non_blocking=True)
+                if not weights_resident:
+                    Bd.copy_(B_h, non_blocking=True)
                 ev_in2[i % 2].record(s_in2)
             main.wait_event(ev_in[i % 2]); main.wait_event(ev_in2[i % 2])
             if i >= 2:
                 main.wait_event(ev_out[i % 2])             # step i-2's result has left this C buffer
             flush.zero_()                                  # L2 discipline as in the device-timed region
-            fmm.scheme_gemm(s, d, Ad, Bd, Cd, wsd)
+            fmm.scheme_gemm(s, d_reuse if weights_resident else d, Ad, Bd, Cd, wsd)
             ev_comp[i % 2].record(main)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_comp[i % 2])
@@ -361,6 +362,10 @@ def run_ours(args):
     e2e_pipelined(max(args.warmup, 3))
     barrier()
     t_e2e = max_over_ranks(e2e_pipelined(args.steps))
+    barrier()
+    # a serving deployment keeps the weights and their block sums on the device: only the activations travel.  The warm-up
+    # with the weights copied has left B and Bhat in both buffer sets.
+    t_e2e_wr = max_over_ranks(e2e_pipelined(args.steps, weights_resident=True))
     barrier()
 
     # ---- roofline of the dominant kernel (block products), timed live by the library's phase events
@@ -440,6 +445,9 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": world * flops_eff / (t_e2e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": t_e2e,
                     "mode": "double-buffered: copies of neighbouring steps overlap the kernels; K steps timed as one region",
+                    "weights_resident": {"value": world * flops_eff / (t_e2e_wr * 1e-3) / 1e12, "ms_per_step": t_e2e_wr,
+                                         "h2d_bytes_per_step": A_h.numel() * 2, "d2h_bytes_per_step": d2h,
+                                         "note": "weights and their block sums stay on the device; only A is copied in"},
                     "ms_per_step_serial": t_e2e_serial, "value_serial": world * flops_eff / (t_e2e_serial * 1e-3) / 1e12,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
