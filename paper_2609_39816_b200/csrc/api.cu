@@ -140,7 +140,7 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.sA = o; o += align_up(nsa * 4);
   L.sB = o; o += align_up(nsb * 4);
   L.n_partials = std::max(decode_grid(bm, bn), kMaxStreamPartials);
-  L.partials = o; o += align_up((size_t)L.n_partials * 8 * 2);
+  L.partials = o; o += align_up((size_t)L.n_partials * 8 * 4);   // up to four algorithms' error sums per decode launch
   L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
   // Consecutive products are spaced by the block size plus 256 bytes: block sizes are often powers of two, and
   // R streams written (or read) at the same offset of power-of-two-spaced slabs land on the same memory
@@ -263,7 +263,7 @@ fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   return launch_block_products(g, st);
 }
 // If C is null the result is not stored; if cstar32 is given the squared error is reduced into err_out[0].
-fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, double* err_out, cudaStream_t st) {
+fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, double* err_out, cudaStream_t st, int gauges = 1) {
   const fmm_scheme* s = r.s;
   ProfScope ps(3, st);
   int np = 0;
@@ -271,8 +271,8 @@ fmm_status stage_decode(const SchemeRun& r, void* C, const float* cstar32, doubl
   FMM_CUDA(launch_decode(r.d->output, at<char>(r.ws, r.L.prod), (r.d->flags & FMM_FLAG_PRODUCTS_BF16) ? FMM_BF16 : FMM_F32,
                          r.L.sProd, r.dW, r.hW, s->R, per_product ? r.sA() : nullptr,
                          per_product ? r.sB() : nullptr, s->m, s->n,
-                         r.d->M / s->m, r.d->N / s->n, C, r.d->ldc, cstar32, at<double>(r.ws, r.L.partials), &np, st));
-  if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(r.ws, r.L.partials), np, err_out, st));
+                         r.d->M / s->m, r.d->N / s->n, C, r.d->ldc, cstar32, at<double>(r.ws, r.L.partials), &np, st, gauges));
+  if (cstar32 && err_out) FMM_CUDA(launch_sum_partials(at<double>(r.ws, r.L.partials), np, err_out, st, gauges));
   return FMM_OK;
 }
 
@@ -393,6 +393,59 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
 }
 
 // Workspace of a sweep: the GEMM layout plus reference copies, classical result, tables and sums.
+// Gauge batching in the sweep.  Equivalent algorithms share their operands, so several of them can run as ONE set of
+// launches: the encode reads A and B once for all of them, the block products fill the machine with more tiles, the
+// decode walks the positions once.  `kb` algorithms become one table set with kb * R products; the decode table keeps
+// their C blocks apart (list c feeds block c / kb of algorithm c % kb).  Limits: kb * R <= FMM_MAX_R products,
+// kb * m * n <= 16 decode lists, kb in {1, 2, 4} (it must divide the decode's thread split).
+int sweep_batch(const fmm_scheme* s) {
+  static const bool off = [] { const char* e = std::getenv("FMM_B200_NO_GAUGE_BATCH"); return e && e[0] == '1'; }();
+  if (off) return 1;
+  for (int kb = 4; kb > 1; kb /= 2)
+    if (kb * s->R <= FMM_MAX_R && kb * s->m * s->n <= 16) return kb;
+  return 1;
+}
+
+// Merge the tables of kb algorithms (tabs[3*i .. 3*i+2] = encode A, encode B, decode of algorithm i).  Returns false if the
+// merged lists do not fit a table.
+bool merge_tables(const CoefTable* tabs, int kb, int R, CoefTable* mA, CoefTable* mB, CoefTable* mW) {
+  for (int which = 0; which < 2; ++which) {
+    CoefTable* out = which == 0 ? mA : mB;
+    std::memset(out, 0, sizeof(CoefTable));
+    out->ncell = tabs[which].ncell;
+    int n = 0, lists = 0;
+    for (int i = 0; i < kb; ++i) {
+      const CoefTable& t = tabs[3 * i + which];
+      for (int r = 0; r < t.R; ++r) {
+        out->off[lists++] = n;
+        for (int e = t.off[r]; e < t.off[r + 1]; ++e) {
+          if (n >= kMaxNnz) return false;
+          out->cell[n] = t.cell[e]; out->coef[n] = t.coef[e]; ++n;
+        }
+      }
+    }
+    out->off[lists] = n;
+    out->R = lists;
+  }
+  std::memset(mW, 0, sizeof(CoefTable));
+  const int cells = tabs[2].R;
+  mW->ncell = kb * R;                       // the padding slab sits behind all kb * R products
+  int n = 0, lists = 0;
+  for (int c = 0; c < cells; ++c)
+    for (int i = 0; i < kb; ++i) {
+      const CoefTable& t = tabs[3 * i + 2];
+      mW->off[lists++] = n;
+      for (int e = t.off[c]; e < t.off[c + 1]; ++e) {
+        if (n >= kMaxNnz) return false;
+        mW->cell[n] = t.cell[e] == t.ncell ? kb * R : t.cell[e] + i * R;
+        mW->coef[n] = t.coef[e]; ++n;
+      }
+    }
+  mW->off[lists] = n;
+  mW->R = lists;
+  return true;
+}
+
 struct SweepLayout {
   GemmLayout g; ClassicalLayout c;
   size_t gemm, gemm2, classical, cstar, cstar32, ccl, tables, sums, total;   // two GEMM workspaces: gauges are pipelined
@@ -400,7 +453,7 @@ struct SweepLayout {
 
 SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
   SweepLayout L;
-  L.g = gemm_layout(s->m, s->k, s->n, s->R, d);
+  L.g = gemm_layout(s->m, s->k, s->n, s->R * sweep_batch(s), d);   // room for a whole batch of algorithms
   L.c = classical_layout(d);
   size_t o = 0;
   L.gemm = o; o += align_up(L.g.total);
@@ -562,14 +615,32 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   const fmm_scheme* grid = level == 1 ? base->outer.get() : base;
   const int gm = grid->m, gk = grid->k, gn = grid->n;
 
-  // 1. gauge-transformed coefficient tables, built on the host and uploaded once
-  std::vector<CoefTable> tabs((size_t)G * 3);
-  std::memset(tabs.data(), 0, tabs.size() * sizeof(CoefTable));
+  // 1. gauge-transformed coefficient tables, built on the host, merged per batch of algorithms, uploaded once
+  std::vector<CoefTable> single((size_t)G * 3);
+  std::memset(single.data(), 0, single.size() * sizeof(CoefTable));
   for (int g = 0; g < G; ++g) {
     fmm_scheme* gs = nullptr;
     FMM_TRY(fmm_gauge_core(*base, level, P + (size_t)g * gm * gm, Q + (size_t)g * gk * gk, S + (size_t)g * gn * gn, 0.0, &gs));
-    fmm_build_tables(*gs, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2]);
+    fmm_build_tables(*gs, &single[3 * g], &single[3 * g + 1], &single[3 * g + 2]);
     scheme_free(gs);
+  }
+  struct Chunk { int g0, count; };
+  std::vector<Chunk> chunks;
+  std::vector<CoefTable> tabs;          // three tables per chunk
+  tabs.reserve((size_t)G * 3);
+  {
+    const int kb = sweep_batch(base);
+    int g = 0;
+    while (g < G) {
+      int kc = kb;
+      while (kc > G - g) kc /= 2;       // 4, 2 or 1 algorithms
+      CoefTable mA, mB, mW;
+      while (kc > 1 && !merge_tables(&single[3 * g], kc, base->R, &mA, &mB, &mW)) kc /= 2;   // lists too long: smaller batch
+      if (kc == 1) { mA = single[3 * g]; mB = single[3 * g + 1]; mW = single[3 * g + 2]; }
+      tabs.push_back(mA); tabs.push_back(mB); tabs.push_back(mW);
+      chunks.push_back({g, kc});
+      g += kc;
+    }
   }
   char* ws = static_cast<char*>(d_ws);
   void* gws = ws + L.gemm;
@@ -610,24 +681,30 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   void* gws2 = ws + L.gemm2;
   FMM_CUDA(cudaMemsetAsync(at<char>(gws2, L.g.status), 0, sizeof(DeviceStatus), st));
   SideStream* side = concurrency_enabled() ? side_stream() : nullptr;
+  fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
+  batched.m = base->m; batched.k = base->k; batched.n = base->n;
   if (side == nullptr) {
-    for (int g = 0; g < G; ++g) {
-      FMM_TRY(run_scheme(base, d, L.g, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2], d_tabs + 3 * g, d_tabs + 3 * g + 1,
-                         d_tabs + 3 * g + 2, dA, bk_ptr, bk_ld, nullptr, cstar32, sums + 8 + g, gws, false, st));
+    for (size_t c = 0; c < chunks.size(); ++c) {
+      batched.R = base->R * chunks[c].count;
+      const SchemeRun r{&batched, d, L.g, gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
+                        d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
+      FMM_TRY(stage_encode_pair(r, dA, bk_ptr, bk_ld, st));
+      FMM_TRY(stage_products(r, st));
+      FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, st, chunks[c].count));
     }
   } else {
     cudaStream_t sE = side->stream, sG = st, sD = side->stream2;
     if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;
     cudaEvent_t evG[2] = {nullptr, nullptr}, evD[2] = {nullptr, nullptr};
-    for (int g = 0; g < G; ++g) {
-      const int b = g & 1;
-      const SchemeRun r{base, d, L.g, b ? gws2 : gws, &tabs[3 * g], &tabs[3 * g + 1], &tabs[3 * g + 2],
-                        d_tabs + 3 * g, d_tabs + 3 * g + 1, d_tabs + 3 * g + 2};
-      // encode: the products of gauge g-2 must have finished reading this buffer's Ahat / Bhat
+    for (size_t c = 0; c < chunks.size(); ++c) {
+      const int b = (int)(c & 1);
+      batched.R = base->R * chunks[c].count;
+      const SchemeRun r{&batched, d, L.g, b ? gws2 : gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
+                        d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
+      // encode: the products of batch c-2 must have finished reading this buffer's Ahat / Bhat
       if (evG[b] && cudaStreamWaitEvent(sE, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
-      // Large operands: two launches, not the paired one — beside the products and decode of the neighbouring gauges
-      // the two smaller kernels pack better (measured 8.06 k against 7.71 k gauges/s at 2048 x 4096 x 4096).  Small
-      // operands are launch-bound: one paired launch (19.8 k against 14.1 k realisations/s at 128^3).
+      // Large operands: two launches, not the paired one — beside the products and decode of the neighbouring batches
+      // the two smaller kernels pack better.  Small operands are launch-bound: one paired launch.
       const bool small_operands = (d->M + d->N) * d->K * (int64_t)esize(d->storage) < ((int64_t)16 << 20);
       if (small_operands) {
         FMM_TRY(stage_encode_pair(r, dA, bk_ptr, bk_ld, sE));
@@ -636,14 +713,14 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
         FMM_TRY(stage_encode_a(r, dA, sE));
       }
       cudaEvent_t evE = record_event(side, sE);
-      // products: need this gauge's encode, and the decode of gauge g-2 must be done with this product buffer
+      // products: need this batch's encode, and the decode of batch c-2 must be done with this product buffer
       if (!evE || cudaStreamWaitEvent(sG, evE, 0) != cudaSuccess) return FMM_ERR_CUDA;
       if (evD[b] && cudaStreamWaitEvent(sG, evD[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
       FMM_TRY(stage_products(r, sG));
       evG[b] = record_event(side, sG);
-      // decode + error reduction
+      // decode + error reduction, one sum per algorithm of the batch
       if (!evG[b] || cudaStreamWaitEvent(sD, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
-      FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + g, sD));
+      FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, sD, chunks[c].count));
       evD[b] = record_event(side, sD);
       if (!evD[b]) return FMM_ERR_CUDA;
     }

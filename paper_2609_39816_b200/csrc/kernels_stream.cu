@@ -632,7 +632,10 @@ __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_tab, int R,
               const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
               OutT* __restrict__ C, int64_t ldc, const float* __restrict__ cstar32, int64_t ldcs,
-              double* __restrict__ partials, int tiles_per_block, int64_t rstride) {
+              double* __restrict__ partials, int tiles_per_block, int64_t rstride, int gauges) {
+  // gauges > 1 (error reduction only): the table describes `gauges` equivalent algorithms at once; list c belongs to
+  // C block c / gauges of algorithm c % gauges, and every algorithm gets its own error sum.  gauges divides kDecSplit,
+  // so a thread's lists (c = g, g + kDecSplit, ...) all belong to one algorithm.
   constexpr int kDecPos = kDecThreads / kDecSplit;
   constexpr int kCellsPerThread = 16 / kDecSplit;
   grid_dependency_wait();     // the products (and scales) come from the previous kernel of the stream
@@ -655,7 +658,7 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
   int64_t out_base[kCellsPerThread], cs_base[kCellsPerThread];
 #pragma unroll
   for (int u = 0; u < kCellsPerThread; ++u) {
-    const int c = g + u * kDecSplit;
+    const int c = (g + u * kDecSplit) / gauges;   // the C block this list feeds
     const int i = c / n, j = c - i * n;
     out_base[u] = (int64_t)i * bm * ldc + (int64_t)j * bn;
     cs_base[u] = (int64_t)i * bm * ldcs + (int64_t)j * bn;
@@ -736,21 +739,39 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
     }
   }
   if (kErr) {
-    const double tot = block_sum_double((double)err, sm.red);
-    if (threadIdx.x == 0) partials[blockIdx.x] = tot;
+    if (gauges == 1) {
+      const double tot = block_sum_double((double)err, sm.red);
+      if (threadIdx.x == 0) partials[blockIdx.x] = tot;
+    } else {
+      // one sum per algorithm: warps with the same (g % gauges); partials laid out [algorithm][block]
+      double v = (double)err;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      const int warp = threadIdx.x >> 5;
+      __syncthreads();
+      if ((threadIdx.x & 31) == 0) sm.red[warp] = v;
+      __syncthreads();
+      if (threadIdx.x < gauges) {
+        double tot = 0.0;
+        for (int w = 0; w < kDecThreads / 32; ++w)
+          if (((w * 32) / kDecPos) % gauges == (int)threadIdx.x) tot += sm.red[w];
+        partials[(size_t)threadIdx.x * gridDim.x + blockIdx.x] = tot;
+      }
+    }
   }
 }
 
 // ------------------------------------------------------------------------------------------
 // reductions
 // ------------------------------------------------------------------------------------------
+// block b sums partials[b * n .. b * n + n) into out[b]
 __global__ void __launch_bounds__(256) sum_partials_kernel(const double* __restrict__ partials, int n,
                                                            double* __restrict__ out) {
   __shared__ double red[8];
   double v = 0.0;
-  for (int i = threadIdx.x; i < n; i += 256) v += partials[i];
+  for (int i = threadIdx.x; i < n; i += 256) v += partials[(size_t)blockIdx.x * n + i];
   const double tot = block_sum_double(v, red);
-  if (threadIdx.x == 0) out[0] = tot;
+  if (threadIdx.x == 0) out[blockIdx.x] = tot;
 }
 
 __global__ void __launch_bounds__(256) cstar_prepare_kernel(const double* __restrict__ cstar, int64_t count,
@@ -911,7 +932,8 @@ int decode_grid(int64_t bm, int64_t bn) {
 template <typename OutT, int kSplit, typename ProdT>
 static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const CoefTable* d_tab, int R, int nnz, const float* sA,
                                    const float* sB, int m, int n, int64_t bm, int64_t bn, void* C, int64_t ldc,
-                                   const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
+                                   const float* cstar32, double* partials, int* n_partials, int gauges, cudaStream_t st) {
+  if (gauges < 1 || kSplit % gauges != 0 || (gauges > 1 && C != nullptr)) return cudaErrorInvalidValue;
   constexpr int kDecPos = kDecThreads / kSplit;
   const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 4 * sizeof(ProdT);
   if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
@@ -928,7 +950,7 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
       if (e != cudaSuccess) return e;                                                                            \
     }                                                                                                            \
     cudaError_t le = launch_dependent(k, dim3(grid), dim3(kDecThreads), smem, st, prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, \
-                                      cstar32, ldcs, partials, tpb, prod_stride);                                 \
+                                      cstar32, ldcs, partials, tpb, prod_stride, gauges);                         \
     if (le != cudaSuccess) return le;                                                                            \
   }
   if (C != nullptr && cstar32 != nullptr) FMM_DECODE_LAUNCH(true, true, 0)
@@ -943,33 +965,34 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
 template <typename ProdT>
 static cudaError_t launch_decode_p(int output, const ProdT* prod, int64_t prod_stride, const CoefTable* d_tab, const CoefTable* h_tab, int R,
                                    const float* sA, const float* sB, int m, int n, int64_t bm, int64_t bn, void* C,
-                                   int64_t ldc, const float* cstar32, double* partials, int* n_partials, cudaStream_t st) {
+                                   int64_t ldc, const float* cstar32, double* partials, int* n_partials, int gauges,
+                                   cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   // small schemes (at most 8 products, 4 output cells): one thread per position quad; otherwise four share one
-  const bool small = R <= 8 && m * n <= 4;
+  const bool small = R <= 8 && m * n * gauges <= 4 && gauges == 1;
   if (output == FMM_F32)
-    return small ? launch_decode_t<float, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
-                 : launch_decode_t<float, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
+    return small ? launch_decode_t<float, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, gauges, st)
+                 : launch_decode_t<float, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, gauges, st);
   if (output == FMM_BF16)
-    return small ? launch_decode_t<__nv_bfloat16, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st)
-                 : launch_decode_t<__nv_bfloat16, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, st);
+    return small ? launch_decode_t<__nv_bfloat16, 1, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, gauges, st)
+                 : launch_decode_t<__nv_bfloat16, 4, ProdT>(prod, prod_stride, d_tab, R, nnz, sA, sB, m, n, bm, bn, C, ldc, cstar32, partials, n_partials, gauges, st);
   return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_decode(int output, const void* prod, int prod_dtype, int64_t prod_stride, const CoefTable* d_tab,
                           const CoefTable* h_tab, int R, const float* sA, const float* sB, int m, int n, int64_t bm,
                           int64_t bn, void* C, int64_t ldc, const float* cstar32, double* partials, int* n_partials,
-                          cudaStream_t st) {
+                          cudaStream_t st, int gauges) {
   if (prod_dtype == FMM_BF16)
     return launch_decode_p<__nv_bfloat16>(output, (const __nv_bfloat16*)prod, prod_stride, d_tab, h_tab, R, sA, sB, m, n, bm, bn, C, ldc,
-                                          cstar32, partials, n_partials, st);
+                                          cstar32, partials, n_partials, gauges, st);
   return launch_decode_p<float>(output, (const float*)prod, prod_stride, d_tab, h_tab, R, sA, sB, m, n, bm, bn, C, ldc, cstar32,
-                                partials, n_partials, st);
+                                partials, n_partials, gauges, st);
 }
 
-cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st) {
-  sum_partials_kernel<<<1, 256, 0, st>>>(partials, n, out);
+cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st, int count) {
+  sum_partials_kernel<<<count, 256, 0, st>>>(partials, n, out);
   ++fmm_launch_counter();
   return cudaGetLastError();
 }

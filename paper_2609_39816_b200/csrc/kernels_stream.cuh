@@ -86,14 +86,17 @@ cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t
 // (rnd_O(c) - C*)^2 are written to partials[gridDim.x] and *n_partials receives gridDim.x.
 // d_tab is the CELL-MAJOR decode table (list c = the (r, w) pairs feeding C block c, ascending r); R is the
 // number of products; h_tab is the host copy of d_tab (its list lengths size the shared memory).
+// gauges > 1 (error reduction only, 1 / 2 / 4): the table holds that many equivalent algorithms, list c feeding C block
+// c / gauges of algorithm c % gauges with product indices offset by the algorithm; partials are [algorithm][block].
 cudaError_t launch_decode(int output, const void* prod, int prod_dtype, int64_t prod_stride, const CoefTable* d_tab,
                           const CoefTable* h_tab, int R, const float* sA, const float* sB, int m, int n, int64_t bm,
                           int64_t bn, void* C, int64_t ldc, const float* cstar32, double* partials, int* n_partials,
-                          cudaStream_t st);
+                          cudaStream_t st, int gauges = 1);
 int decode_grid(int64_t bm, int64_t bn);
 
 // out[0] = sum of partials[0..n) in a fixed order (single block).
-cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st);
+// out[b] = sum of partials[b*n .. b*n+n), b < count
+cudaError_t launch_sum_partials(const double* partials, int n, double* out, cudaStream_t st, int count = 1);
 
 // C*(fp64) -> fp32 copy, and partial sums of C*^2.
 cudaError_t launch_cstar_prepare(const double* cstar, int64_t count, float* cstar32, double* partials,
