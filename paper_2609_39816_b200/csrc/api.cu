@@ -615,25 +615,35 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   const fmm_scheme* grid = level == 1 ? base->outer.get() : base;
   const int gm = grid->m, gk = grid->k, gn = grid->n;
 
-  // 1. gauge-transformed coefficient tables, built on the host, merged per batch of algorithms, uploaded once
+  // 1. gauge-transformed coefficient tables: built on the host, merged per batch of algorithms and uploaded in groups
+  //    of kTableGroup gauges while the device works on the groups before (the first launch waits for one group only)
+  constexpr int kTableGroup = 32;
   std::vector<CoefTable> single((size_t)G * 3);
   std::memset(single.data(), 0, single.size() * sizeof(CoefTable));
-  for (int g = 0; g < G; ++g) {
-    fmm_scheme* gs = nullptr;
-    FMM_TRY(fmm_gauge_core(*base, level, P + (size_t)g * gm * gm, Q + (size_t)g * gk * gk, S + (size_t)g * gn * gn, 0.0, &gs));
-    fmm_build_tables(*gs, &single[3 * g], &single[3 * g + 1], &single[3 * g + 2]);
-    scheme_free(gs);
-  }
   struct Chunk { int g0, count; };
   std::vector<Chunk> chunks;
   std::vector<CoefTable> tabs;          // three tables per chunk
-  tabs.reserve((size_t)G * 3);
-  {
-    const int kb = sweep_batch(base);
-    int g = 0;
-    while (g < G) {
+  tabs.reserve((size_t)G * 3);          // never reallocates: launches keep pointers into it
+  const int kb = sweep_batch(base);
+  int next_gauge = 0;
+  char* ws = static_cast<char*>(d_ws);
+  void* gws = ws + L.gemm;
+  void* cws = ws + L.classical;
+  CoefTable* d_tabs = at<CoefTable>(ws, L.tables);
+  double* sums = at<double>(ws, L.sums);  // [0]=n*, [1]=e_cl, [2]=scratch, [8..8+G) = e_g
+  auto build_group = [&](cudaStream_t up) -> fmm_status {
+    const int g_end = std::min(G, next_gauge + kTableGroup);
+    for (int g = next_gauge; g < g_end; ++g) {
+      fmm_scheme* gs = nullptr;
+      FMM_TRY(fmm_gauge_core(*base, level, P + (size_t)g * gm * gm, Q + (size_t)g * gk * gk, S + (size_t)g * gn * gn, 0.0, &gs));
+      fmm_build_tables(*gs, &single[3 * g], &single[3 * g + 1], &single[3 * g + 2]);
+      scheme_free(gs);
+    }
+    const size_t first = chunks.size();
+    int g = next_gauge;
+    while (g < g_end) {
       int kc = kb;
-      while (kc > G - g) kc /= 2;       // 4, 2 or 1 algorithms
+      while (kc > g_end - g) kc /= 2;   // 4, 2 or 1 algorithms
       CoefTable mA, mB, mW;
       while (kc > 1 && !merge_tables(&single[3 * g], kc, base->R, &mA, &mB, &mW)) kc /= 2;   // lists too long: smaller batch
       if (kc == 1) { mA = single[3 * g]; mB = single[3 * g + 1]; mW = single[3 * g + 2]; }
@@ -641,13 +651,11 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
       chunks.push_back({g, kc});
       g += kc;
     }
-  }
-  char* ws = static_cast<char*>(d_ws);
-  void* gws = ws + L.gemm;
-  void* cws = ws + L.classical;
-  CoefTable* d_tabs = at<CoefTable>(ws, L.tables);
-  double* sums = at<double>(ws, L.sums);  // [0]=n*, [1]=e_cl, [2]=scratch, [8..8+G) = e_g
-  FMM_CUDA(cudaMemcpyAsync(d_tabs, tabs.data(), tabs.size() * sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+    next_gauge = g_end;
+    FMM_CUDA(cudaMemcpyAsync(d_tabs + 3 * first, tabs.data() + 3 * first, (tabs.size() - 3 * first) * sizeof(CoefTable),
+                             cudaMemcpyHostToDevice, up));
+    return FMM_OK;
+  };
   FMM_CUDA(cudaMemsetAsync(at<char>(gws, L.g.status), 0, sizeof(DeviceStatus), st));
   FMM_CUDA(cudaMemsetAsync(at<char>(cws, L.c.status), 0, sizeof(DeviceStatus), st));
 
@@ -684,7 +692,11 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
   batched.m = base->m; batched.k = base->k; batched.n = base->n;
   if (side == nullptr) {
-    for (size_t c = 0; c < chunks.size(); ++c) {
+    for (size_t c = 0;; ++c) {
+      if (c == chunks.size()) {
+        if (next_gauge >= G) break;
+        FMM_TRY(build_group(st));
+      }
       batched.R = base->R * chunks[c].count;
       const SchemeRun r{&batched, d, L.g, gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
                         d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
@@ -696,7 +708,11 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
     cudaStream_t sE = side->stream, sG = st, sD = side->stream2;
     if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;
     cudaEvent_t evG[2] = {nullptr, nullptr}, evD[2] = {nullptr, nullptr};
-    for (size_t c = 0; c < chunks.size(); ++c) {
+    for (size_t c = 0;; ++c) {
+      if (c == chunks.size()) {
+        if (next_gauge >= G) break;
+        FMM_TRY(build_group(sE));       // the encode stream reads the tables first; products and decode follow it
+      }
       const int b = (int)(c & 1);
       batched.R = base->R * chunks[c].count;
       const SchemeRun r{&batched, d, L.g, b ? gws2 : gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],

@@ -664,6 +664,13 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
     cs_base[u] = (int64_t)i * bm * ldcs + (int64_t)j * bn;
   }
 
+  // one algorithm per thread group: the reference values of C block g are staged once per position by thread group g
+  // and read by all groups, instead of every algorithm loading them again
+  const bool stage_cs = kErr && kDecSplit > 1 && gauges == kDecSplit;
+  unsigned char* cs_stage = stage + (size_t)(R + 1) * kSlab + pq * 16;
+  const bool cs_mine = stage_cs && g * gauges < ncell;
+  const int64_t cs_src = (int64_t)(g / n) * bm * ldcs + (int64_t)(g % n) * bn;
+
   float err = 0.0f;
   for (int it = 0; it < tiles_per_block; ++it) {
     const int idx = (blockIdx.x * tiles_per_block + it) * kDecPos + pq;
@@ -682,6 +689,9 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
           asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst0 + r * kSlab), "l"(src + r * rstride),
                        "r"(nbytes) : "memory");
       }
+      if (kErr && cs_mine)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(cs_stage + g * (kDecPos * 16))),
+                     "l"(cstar32 + cs_src + (int64_t)p * ldcs + q), "r"(live ? 16 : 0) : "memory");
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (it == 0) {                             // table set-up overlaps the first tile's copies
@@ -729,7 +739,8 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
         const float4 x = make_float4(x0.x, x0.y, x1.x, x1.y);
         if (kStore) store4(C + out_base[u4] + (int64_t)p * ldc + q, x);
         if (kErr) {
-          const float4 cs = __ldcs(reinterpret_cast<const float4*>(cstar32 + cs_base[u4] + (int64_t)p * ldcs + q));
+          const float4 cs = stage_cs ? *reinterpret_cast<const float4*>(cs_stage + u4 * (kDecPos * 16))
+                                     : __ldcs(reinterpret_cast<const float4*>(cstar32 + cs_base[u4] + (int64_t)p * ldcs + q));
           const float d0 = round_out(x.x, (OutT*)nullptr) - cs.x, d1 = round_out(x.y, (OutT*)nullptr) - cs.y;
           const float d2 = round_out(x.z, (OutT*)nullptr) - cs.z, d3 = round_out(x.w, (OutT*)nullptr) - cs.w;
           err = __fmaf_rn(d0, d0, err); err = __fmaf_rn(d1, d1, err);
@@ -936,6 +947,7 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
   if (gauges < 1 || kSplit % gauges != 0 || (gauges > 1 && C != nullptr)) return cudaErrorInvalidValue;
   constexpr int kDecPos = kDecThreads / kSplit;
   const size_t smem = ((sizeof(DecSmemHead) + (size_t)nnz * 8 + 15) / 16) * 16 + (size_t)(R + 1) * kDecPos * 4 * sizeof(ProdT);
+  const size_t smem_cs = (cstar32 != nullptr && kSplit > 1 && gauges == kSplit) ? (size_t)(16 / kSplit) * kDecPos * 16 : 0;
   if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // 32-bit position index
   int grid, tpb;
   split_tiles((bm * (bn >> 2) + kDecPos - 1) / kDecPos, &grid, &tpb);
@@ -949,7 +961,7 @@ static cudaError_t launch_decode_t(const ProdT* prod, int64_t prod_stride, const
       cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok[SLOT]);                                     \
       if (e != cudaSuccess) return e;                                                                            \
     }                                                                                                            \
-    cudaError_t le = launch_dependent(k, dim3(grid), dim3(kDecThreads), smem, st, prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, \
+    cudaError_t le = launch_dependent(k, dim3(grid), dim3(kDecThreads), smem + smem_cs, st, prod, d_tab, R, sA, sB, n, bm, bn, (OutT*)C, ldc, \
                                       cstar32, ldcs, partials, tpb, prod_stride, gauges);                         \
     if (le != cudaSuccess) return le;                                                                            \
   }
