@@ -29,6 +29,7 @@ __all__ = [
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
     "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "certificate",
+    "hadamard_matrix", "hadamard_rotate",
 ]
 
 
@@ -363,3 +364,37 @@ def int8_corrected(s: "Scheme", cA, dA, cB, dB, g: int = 128, od="bf16", product
     if rc:
         raise ValueError("shape does not divide, or coefficients are not integers")
     return (out, mx, P) if products else (out, mx)
+
+
+# ---------------------------------------------------------------------------- rotation pre-pass (Appendix B, "A rotation ...")
+def hadamard_matrix(h: int) -> np.ndarray:
+    """Sylvester's Hadamard matrix of order h (a power of two): H[i, j] = (-1)^popcount(i & j), entries +-1."""
+    if h < 1 or h & (h - 1):
+        raise ValueError("order must be a power of two")
+    i = np.arange(h)
+    bits = i[:, None] & i[None, :]
+    par = np.zeros((h, h), dtype=np.int64)
+    while bits.any():
+        par ^= bits & 1
+        bits >>= 1
+    return (1 - 2 * par).astype(np.float64)
+
+
+def hadamard_rotate(X, signs, h: int, fmt="f64") -> np.ndarray:
+    """Randomised Hadamard rotation along the inner dimension (Appendix B: A -> A H, B -> H^T B with H orthogonal).
+
+    X is [rows, K] with the inner dimension last (for B that is its transpose, so one routine serves both operands);
+    H = diag(signs) . blockdiag(H_h, ..., H_h) / sqrt(h) with K a multiple of h.  Computed in fp64 from the
+    definition, then rounded once to ``fmt`` (the storage type the rotated operand is kept in).
+    """
+    X = np.asarray(X, dtype=np.float64)
+    K = X.shape[1]
+    signs = np.asarray(signs, dtype=np.float64)
+    if K % h or signs.shape != (K,) or not np.all(np.abs(signs) == 1.0):
+        raise ValueError("K must be a multiple of h and signs must be K entries of +-1")
+    Hh = hadamard_matrix(h) / math.sqrt(h)
+    Y = np.empty_like(X)
+    for b in range(K // h):
+        sl = slice(b * h, (b + 1) * h)
+        Y[:, sl] = (X[:, sl] * signs[sl]) @ Hh
+    return round_to(Y, fmt)
