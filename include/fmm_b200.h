@@ -331,6 +331,21 @@ fmm_status int8_gemm_corrected(const fmm_scheme* s, const int8_t* d_cA, const fl
                                const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc,
                                void* d_ws, size_t ws_bytes, void* cuda_stream);
 
+/* Randomised Hadamard rotation of the inner dimension (Appendix B, "A rotation, other summation orders and repeated
+ * runs": A -> A H, B -> H^T B with H orthogonal leaves A B unchanged and changes what a fast algorithm's block sums
+ * round).  A pre-pass outside scheme_gemm: rotate both operands with the same h and signs, then call any product.
+ *     Y[t, :] = rnd_storage( (X[t, :] * signs) . blockdiag(H_h, ..., H_h) / sqrt(h) ),
+ * H_h Sylvester's Hadamard matrix of order h (H[i][j] = (-1)^popcount(i & j)).  Arithmetic: the fast Walsh-Hadamard
+ * recursion in fp32 (strides ascending), one multiplication by fl(1/sqrt(h)), one rounding to `storage`.
+ * dX, dY: DEVICE [rows][ld*] of `storage` (FMM_F32 or FMM_BF16), the inner dimension contiguous — A as stored, B in
+ * its [N, K] layout (rows = N); 16-byte aligned, ld* >= K and a multiple of 16 bytes; dY == dX rotates in place,
+ * any other overlap is undefined.  d_signs: DEVICE, K entries of +1 / -1 (only the sign is read), 16-byte aligned,
+ * or NULL for all +1.  h: a power of two, 2 <= h <= 1024, dividing K (K < 2^31).  The caller owns every buffer; the
+ * call only enqueues one kernel on `cuda_stream` (the current device's).  FMM_ERR_ARG: null operand;
+ * FMM_ERR_DTYPE: storage; FMM_ERR_SHAPE: sizes, divisibility or alignment (nothing is launched).             */
+fmm_status hadamard_rotate(int storage, const void* dX, int64_t ldx, int64_t rows, int64_t K, int h,
+                           const signed char* d_signs, void* dY, int64_t ldy, void* cuda_stream);
+
 const char* fmm_status_string(fmm_status st);
 
 /* Number of kernels this library has launched in this process (for benchmarks' accounting). */

@@ -392,9 +392,9 @@ def hadamard_rotate(X, signs, h: int, fmt="f64") -> np.ndarray:
     signs = np.asarray(signs, dtype=np.float64)
     if K % h or signs.shape != (K,) or not np.all(np.abs(signs) == 1.0):
         raise ValueError("K must be a multiple of h and signs must be K entries of +-1")
-    Hh = hadamard_matrix(h) / math.sqrt(h)
+    Hh = hadamard_matrix(h)
     Y = np.empty_like(X)
     for b in range(K // h):
         sl = slice(b * h, (b + 1) * h)
-        Y[:, sl] = (X[:, sl] * signs[sl]) @ Hh
+        Y[:, sl] = ((X[:, sl] * signs[sl]) @ Hh) / math.sqrt(h)     # +-1 sums first: exact cancellations stay exact
     return round_to(Y, fmt)

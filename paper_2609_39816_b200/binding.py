@@ -24,7 +24,7 @@ EXPORTED_SYMBOLS = [
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
-    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected",
+    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected", "hadamard_rotate",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
 ]
@@ -97,6 +97,7 @@ _lib.error_frobenius_noalloc.argtypes = [C.POINTER(GemmDesc), _vp, _vp, _vp, _vp
 _lib.error_frobenius_noalloc_max_elements.restype = C.c_int64
 _lib.scheme_certificate.argtypes = [_vp] + [C.c_int] * 5 + [_dp]
 _lib.scheme_certificate.restype = C.c_int
+_lib.hadamard_rotate.argtypes = [C.c_int, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, C.c_int64, _vp]
 _lib.int8_quantize.argtypes = [_vp, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, _vp]
 _lib.int8_gemm_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
 _lib.int8_gemm_workspace.restype = _sz
@@ -286,6 +287,19 @@ def int8_quantize(X, code_bound: int, codes, scales) -> None:
     st = F32 if X.dtype == torch.float32 else BF16
     _check(_lib.int8_quantize(_ptr(X), st, rows, K, X.stride(0), code_bound, _ptr(codes), _ptr(scales), _stream()),
            "int8_quantize")
+
+
+def hadamard_rotate(X, signs, h: int, out=None):
+    """Y = (X * signs) . blockdiag(H_h) / sqrt(h) along the last (contiguous) dimension; X [rows, K] fp32/bf16 on the
+    device, signs int8 [K] on the device (or None), out defaults to a new tensor (pass X to rotate in place)."""
+    import torch
+    rows, K = X.shape
+    if out is None:
+        out = torch.empty_like(X)
+    st = F32 if X.dtype == torch.float32 else BF16
+    _check(_lib.hadamard_rotate(st, _ptr(X), X.stride(0), rows, K, h, _ptr(signs) if signs is not None else None,
+                                _ptr(out), out.stride(0), _stream()), "hadamard_rotate")
+    return out
 
 
 def int8_gemm_workspace(s, M: int, K: int, N: int) -> int:

@@ -202,6 +202,21 @@ def test_empty_and_maximum_sizes_are_rejected_before_any_launch(lib):
     assert lib.int8_gemm_workspace(s2, 0, 128, 64) == 0
 
 
+def test_rotation_argument_checks_need_no_device(lib):
+    """hadamard_rotate validates before it touches CUDA: bad arguments return their status and launch nothing."""
+    f = lib.binding._lib.hadamard_rotate
+    x = ctypes.c_void_p(1 << 20)                       # never dereferenced: every call below is refused
+    assert f(0, None, 64, 4, 64, 32, None, x, 64, None) == 1               # FMM_ERR_ARG: null operand
+    assert f(2, x, 64, 4, 64, 32, None, x, 64, None) == 5                  # FMM_ERR_DTYPE: e4m3 storage
+    for h in (0, 1, 3, 48, 2048):
+        assert f(0, x, 64, 4, 64, h, None, x, 64, None) == 2               # FMM_ERR_SHAPE: h
+    assert f(0, x, 64, 0, 64, 32, None, x, 64, None) == 2                  # empty
+    assert f(0, x, 48, 4, 48, 32, None, x, 48, None) == 2                  # K % h
+    assert f(0, x, 32, 4, 64, 32, None, x, 64, None) == 2                  # ld < K
+    assert f(1, x, 68, 4, 64, 32, None, x, 64, None) == 2                  # bf16 rows not 16-byte multiples
+    assert f(0, ctypes.c_void_p((1 << 20) + 4), 64, 4, 64, 32, None, x, 64, None) == 2   # misaligned base
+
+
 def test_permuted_products_are_the_same_algorithm(lib):
     """Renumbering the products keeps the Brent equations and every criterion; bad permutations are refused."""
     s2 = lib.scheme_builtin("strassen444")
