@@ -540,6 +540,21 @@ def run_workload(args):
         out.update(ensemble_workload(fmm, gen, torch))
         print(json.dumps(out))
         return
+    elif wl == "rotation":   # the Hadamard pre-pass: a streaming kernel, one read and one write per element
+        rows_out = []
+        for dt, T, K, h in ((torch.bfloat16, 4096, 4096, 128), (torch.bfloat16, 8192, 13824, 128),
+                            (torch.bfloat16, 8192, 13824, 512), (torch.float32, 8192, 8192, 128)):
+            X = torch.randn((T, K), dtype=torch.float32, device="cuda").to(dt)
+            sg = (torch.randint(0, 2, (K,), device="cuda") * 2 - 1).to(torch.int8)
+            Y = torch.empty_like(X)
+            t = timed(lambda: fmm.hadamard_rotate(X, sg, h, out=Y))
+            nbytes = 2.0 * X.numel() * X.element_size()
+            rows_out.append({"shape": [T, K], "dtype": str(dt).split(".")[-1], "h": h, "ms": t, "gb_per_s": nbytes / t / 1e6,
+                             "frac_of_hbm_peak": nbytes / t / 1e6 / peaks["hbm"]})
+        out["rotation"] = rows_out
+        out["unit"] = "GB/s"
+        print(json.dumps(out))
+        return
     elif wl == "int8":
         out.update(int8_workload(fmm, gen, torch, timed, peaks))
         print(json.dumps(out))
@@ -692,7 +707,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=512, help="gauges per rank in the c3 sweep (0 = skip); config 3 names 512")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c4m | c5 | int8 | ensemble")
+    ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c4m | c5 | int8 | ensemble | rotation")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
