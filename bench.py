@@ -415,6 +415,28 @@ def run_ours(args):
         e1.record()
         barrier()
         t_sweep = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+        # phase table of the sweep: a second, event-instrumented pass over a few batches (stages back to back)
+        sweep_phases = None
+        if rank == 0:
+            Gp = min(len(mine), 64)
+            fmm.profile_enable(True); fmm.profile_collect()
+            fmm.error_sweep(s1, 0, P[mine][:Gp], Q[mine][:Gp], S[mine][:Gp], d3, A3, B3, ws3, Cstar=Cs)
+            ph3 = fmm.profile_collect(); fmm.profile_enable(False)
+            bm3, bk3, bn3 = C3["M"] // 2, C3["K"] // 2, C3["N"] // 2
+            kb = 4                                               # algorithms per launch set for <2,2,2;7>
+            enc_b = (C3["M"] * C3["K"] + C3["N"] * C3["K"]) * 2 / kb + 7 * (bm3 * bk3 + bn3 * bk3) * 2
+            dec_b = 7 * bm3 * bn3 * 4 + C3["M"] * C3["N"] * 4 / kb
+            enc_us = (ph3["encode_a"][0] + ph3["encode_b"][0]) * 1e3 / Gp
+            prod_us = ph3["products"][0] * 1e3 / Gp
+            dec_us = ph3["decode"][0] * 1e3 / Gp
+            tf = 2.0 * 7 * bm3 * bk3 * bn3 / (prod_us * 1e-6) / 1e12 if prod_us > 0 else 0.0
+            sweep_phases = {
+                "note": f"{Gp} gauges, stages back to back on one stream, {kb} algorithms per launch set; per gauge",
+                "encode": {"us": enc_us, "gb_per_s": enc_b / enc_us / 1e3 if enc_us > 0 else 0.0,
+                           "frac_of_hbm_peak": enc_b / enc_us / 1e3 / peaks["hbm"] if enc_us > 0 else 0.0},
+                "products": {"us": prod_us, "tflops": tf, "frac_of_bf16_peak": tf / peaks["bf16"]},
+                "decode_error": {"us": dec_us, "gb_per_s": dec_b / dec_us / 1e3 if dec_us > 0 else 0.0,
+                                 "frac_of_hbm_peak": dec_b / dec_us / 1e3 / peaks["hbm"] if dec_us > 0 else 0.0}}
         full = gather_ratios(torch.from_numpy(ratios), mine, G, rank, world, device=dev).cpu().numpy()
         srt = np.sort(full)
         sweep = {"workload": "c3: <2,2,2;7> one level, bf16, A 2048x4096, B 4096x4096, log-uniform-cond GL2 gauges",
@@ -422,7 +444,8 @@ def run_ours(args):
                  "tensor_bound_gauges_per_s": peaks["bf16"] * 1e12 / (2.0 * 7 * 1024 * 2048 * 2048),
                  "min": float(srt[0]), "median": float(srt[G // 2]), "max": float(srt[-1]),
                  "count_gt2": int((full > 2).sum()), "e_classical_rel": summ["e_classical_rel"],
-                 "includes": "classical product + its error, reference norm, G x (encode A, encode B, 7 products, decode+error)"}
+                 "includes": "classical product + its error, reference norm, G x (encode A, encode B, 7 products, decode+error)",
+                 "phases": sweep_phases}
         del ws3, Cs, A3, B3
 
     # ---- CPU oracle timed beside it (rank 0, N=1 only)

@@ -688,7 +688,8 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   FMM_TRY(kmajor_b(d, dB, gws, L.g.bt, &bk_ptr, &bk_ld, false, st));
   void* gws2 = ws + L.gemm2;
   FMM_CUDA(cudaMemsetAsync(at<char>(gws2, L.g.status), 0, sizeof(DeviceStatus), st));
-  SideStream* side = concurrency_enabled() ? side_stream() : nullptr;
+  // with phase timing on, the stages run back to back on the caller's stream so that the bracketing events measure them
+  SideStream* side = (concurrency_enabled() && !g_prof_on) ? side_stream() : nullptr;
   fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
   batched.m = base->m; batched.k = base->k; batched.n = base->n;
   if (side == nullptr) {

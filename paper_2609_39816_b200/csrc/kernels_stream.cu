@@ -906,10 +906,12 @@ static cudaError_t launch_encode_split(int storage, int product, const EncodeOpe
 
 cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
                                int use_scale, cudaStream_t st) {
-  // both operands of a product share the thread split: small schemes (at most 4 cells in either grid): one thread
-  // per position vector; otherwise four threads share one
+  // both operands of a product share the thread split: small schemes (at most 4 cells in either grid and at most 8
+  // products): one thread per position vector; otherwise four threads share one (a batch of algorithms on a 2 x 2
+  // grid has 28 products: 28.8 against 36.5 us per algorithm with four threads per vector)
   const int cells = std::max(a.gr * a.gc, b ? b->gr * b->gc : 0);
-  if (cells <= 4) return launch_encode_split<1>(storage, product, a, b, amax_only, use_scale, st);
+  const int products = std::max(a.h_tab->R, b ? b->h_tab->R : 0);
+  if (cells <= 4 && products <= 8) return launch_encode_split<1>(storage, product, a, b, amax_only, use_scale, st);
   return launch_encode_split<4>(storage, product, a, b, amax_only, use_scale, st);
 }
 
