@@ -293,6 +293,22 @@ def test_sweep_log_uniform_gauges_bf16_and_outer_level_fp8(lib):
         assert abs(r - E / Ecl) <= TOL_RATIO * E / Ecl
 
 
+def test_sweep_batches_walk_several_tiles_per_block(lib):
+    """Blocks of 512 x 1024 outputs: every decode block of the batched sweep walks four tiles, so the double-buffered
+    stages (products and staged reference values) are reused; ratios against the oracle for 4 + 2 + 1 gauges."""
+    At, Bt, A64, B64 = _inputs(21, 1024, 256, 2048, "bf16", "llm")
+    G = 7
+    P = np.stack([gen.gauge_log_uniform_cond(2, 3 * g, 2) for g in range(G)])
+    Q = np.stack([gen.gauge_log_uniform_cond(2, 3 * g + 1, 2) for g in range(G)])
+    S = np.stack([gen.gauge_log_uniform_cond(2, 3 * g + 2, 2) for g in range(G)])
+    s1 = lib.scheme_builtin("strassen222")
+    d = lib.GemmDesc.make(1024, 256, 2048, "bf16", "bf16", "bf16")
+    ws = gu.workspace(lib.error_sweep_workspace(s1, d, G))
+    ratios, _ = lib.error_sweep(s1, 0, P, Q, S, d, At, Bt, ws)
+    want, _ = _oracle_ratios(oracle.strassen(), P, Q, S, A64, B64, "bf16", "bf16")
+    assert np.all(np.abs(ratios - want) <= TOL_RATIO * want)
+
+
 # ---------------------------------------------------------------------------- full size, sampled
 def test_config2_full_size_sampled_outputs(lib):
     """Config 2 at full size in the launch configuration the benchmark times (bf16, weight layout):
