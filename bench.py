@@ -386,6 +386,8 @@ def run_ours(args):
         "decode": 49 * bm * bn * 4 + M * N * 2,
     }
     phase_out = {}
+    if phases["encode_b"][1] == 0:      # A and B are encoded by one launch, recorded under encode_a: its bytes are both operands'
+        pass_bytes["encode_a"] += pass_bytes["encode_b"]
     for name in ("encode_a", "encode_b", "products", "decode"):
         ms, n = phases[name]
         per = ms / max(n, 1)
