@@ -307,6 +307,12 @@ def test_sweep_batches_walk_several_tiles_per_block(lib):
     ratios, _ = lib.error_sweep(s1, 0, P, Q, S, d, At, Bt, ws)
     want, _ = _oracle_ratios(oracle.strassen(), P, Q, S, A64, B64, "bf16", "bf16")
     assert np.all(np.abs(ratios - want) <= TOL_RATIO * want)
+    # repeated runs give the same bits (Appendix B, repeated runs); a gauge swept alone gives the same ratio up to the
+    # partition of its error sum (every C is the same bits, the squares are added in another grouping)
+    again, _ = lib.error_sweep(s1, 0, P, Q, S, d, At, Bt, ws)
+    assert np.array_equal(again, ratios)
+    alone = np.array([lib.error_sweep(s1, 0, P[g:g + 1], Q[g:g + 1], S[g:g + 1], d, At, Bt, ws)[0][0] for g in range(G)])
+    assert np.all(np.abs(alone - ratios) <= 1e-6 * ratios)
 
 
 # ---------------------------------------------------------------------------- full size, sampled
