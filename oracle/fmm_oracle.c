@@ -367,7 +367,7 @@ static void matmul_f64(const double* A, const double* B, double* C, int64_t M, i
  * the groups in ascending order: Mr = sum_g (Aq_g Bq_g^T) * sA[p][g] * sB[c/128][g]  (fp64 here).
  * Ah and Bh are overwritten with the codes; sa is [bm][G], sb is [ceil(bn/128)][G], G = ceil(bk/128).            */
 static void model_schedule_product(double* Ah, double* Bh, int64_t bm, int64_t bk, int64_t bn, int pd,
-                                   double* sa, double* sb, double* Mr) {
+                                   double* sa, double* sb, double* Mr, int weights_given) {
   const int64_t G = (bk + 127) / 128, CB = (bn + 127) / 128;
   for (int64_t p = 0; p < bm; ++p)
     for (int64_t g = 0; g < G; ++g) {
@@ -378,7 +378,10 @@ static void model_schedule_product(double* Ah, double* Bh, int64_t bm, int64_t b
       sa[p * G + g] = (double)d;
       for (int64_t t = t0; t < t1; ++t) Ah[p * bk + t] = orc_round((double)((float)Ah[p * bk + t] / d), pd);
     }
+  /* weights_given: Bh already holds the codes and sb their scales (a weight-only search chose them, see orc_joint_round) */
+  if (!weights_given)
   for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x], ORC_BF16);   /* weights' block sums first stored in bf16 */
+  if (!weights_given)
   for (int64_t cb = 0; cb < CB; ++cb)
     for (int64_t g = 0; g < G; ++g) {
       const int64_t t0 = g * 128, t1 = t0 + 128 < bk ? t0 + 128 : bk;
@@ -419,12 +422,13 @@ static void model_schedule_product(double* Ah, double* Bh, int64_t bm, int64_t b
  * sB[R][ceil(bn/128)][G], G = ceil(bk/128)), Mout [R][bm][bn]
  * (the fp64 products of the codes; mode 2: times the row and column scales).
  * Returns 0, or 1 if a dimension does not divide.                                 */
-int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+static int scheme_gemm_impl(int m, int k, int n, int R, const double* U, const double* V, const double* W,
                     int64_t M, int64_t K, int64_t N, const double* A, const double* B,
                     int pd, int od, int scale_mode, double* C,
                     double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
-                    double* M_out, int md) {
+                    double* M_out, int md, const double* Bq_in, const double* sB_in) {
   if (M % m || K % k || N % n) return 1;
+  if (Bq_in && scale_mode != 3) return 1;
   int64_t bm = M / m, bk = K / k, bn = N / n;
   int quant = (pd != ORC_F64);
   double* Ah = (double*)malloc(sizeof(double) * bm * bk);
@@ -473,7 +477,11 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
       const int64_t G3 = (bk + 127) / 128, CB3 = (bn + 127) / 128;
       double* sa3 = (double*)malloc(sizeof(double) * bm * G3);
       double* sb3 = (double*)malloc(sizeof(double) * CB3 * G3);
-      model_schedule_product(Ah, Bh, bm, bk, bn, pd, sa3, sb3, Mr);
+      if (Bq_in) {
+        memcpy(Bh, Bq_in + (size_t)r * bk * bn, sizeof(double) * bk * bn);
+        memcpy(sb3, sB_in + (size_t)r * CB3 * G3, sizeof(double) * CB3 * G3);
+      }
+      model_schedule_product(Ah, Bh, bm, bk, bn, pd, sa3, sb3, Mr, Bq_in != NULL);
       if (sA_out) memcpy(sA_out + (size_t)r * bm * G3, sa3, sizeof(double) * bm * G3);
       if (sB_out) memcpy(sB_out + (size_t)r * CB3 * G3, sb3, sizeof(double) * CB3 * G3);
       free(sa3); free(sb3);
@@ -508,6 +516,23 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
   return 0;
 }
 
+int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                    int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                    int pd, int od, int scale_mode, double* C,
+                    double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
+                    double* M_out, int md) {
+  return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, scale_mode, C, Ahat_out, Bhat_out, sA_out,
+                          sB_out, M_out, md, NULL, NULL);
+}
+
+/* The same under the model schedule (scale_mode 3) with the weight side given as codes Bq [R][bk][bn] and scales
+ * sBq [R][ceil(bn/128)][ceil(bk/128)], as orc_joint_round returns them.                                         */
+int orc_scheme_gemm_weights(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                            int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                            int pd, int od, double* C, double* M_out, int md, const double* Bq, const double* sBq) {
+  return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, 3, C, NULL, NULL, NULL, NULL, M_out, md, Bq, sBq);
+}
+
 /* Classical product at the same dtypes (the control): operands rounded to the product
  * dtype (after a per-tensor power-of-two scale in scale_mode 1, or per-row / per-column
  * scales max|x| / 448 in scale_mode 2), fp64 accumulation, one rounding to the output dtype. */
@@ -523,7 +548,7 @@ int orc_classical_gemm(int64_t M, int64_t K, int64_t N, const double* A, const d
     double* sb3 = (double*)malloc(sizeof(double) * CB3 * G3);
     for (int64_t x = 0; x < M * K; ++x) Ah[x] = A[x];
     for (int64_t x = 0; x < K * N; ++x) Bh[x] = B[x];
-    model_schedule_product(Ah, Bh, M, K, N, pd, sa3, sb3, acc);
+    model_schedule_product(Ah, Bh, M, K, N, pd, sa3, sb3, acc, 0);
     for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x], od);
     free(sa3); free(sb3); free(Ah); free(Bh); free(acc);
     return 0;
@@ -808,5 +833,134 @@ int orc_int8_corrected(int m, int k, int n, int R, const double* U, const double
   }
   free(A0); free(RA); free(B0); free(RB); free(acc);
   if (!Pout) free(P);
+  return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Joint rounding of the weight block sums (Appendix C, "The repair rules").   */
+/* ------------------------------------------------------------------------- */
+
+/* All finite e4m3 values in ascending order (253 of them: -448 ... 448, one zero). */
+static int e4m3_grid(double* g) {
+  int cnt = 0;
+  double pos[127];
+  for (int code = 0; code <= 0x7E; ++code) {
+    const int e = code >> 3, mnt = code & 7;
+    pos[code] = e == 0 ? ldexp((double)mnt / 8.0, -6) : ldexp(1.0 + (double)mnt / 8.0, e - 7);
+  }
+  for (int c = 0x7E; c >= 1; --c) g[cnt++] = -pos[c];
+  for (int c = 0; c <= 0x7E; ++c) g[cnt++] = pos[c];
+  return cnt;
+}
+
+static int grid_index(const double* g, int cnt, double v) {
+  int lo = 0, hi = cnt - 1;
+  while (lo < hi) { int mid = (lo + hi) / 2; if (g[mid] < v) lo = mid + 1; else hi = mid; }
+  return lo;   /* v is a grid value */
+}
+
+/* The weight-only search of the repair rules.  For every position (inner index t, output column c) of the weight's
+ * R block sums, under the model schedule (block sums stored in bf16, one e4m3 scale s_r per 128 x 128 block, rule
+ * s = max|b| / 448 in fp32):
+ *   - candidates of entry r: the two e4m3 codes whose decoded values s_r q bracket the bf16 value b_r; start at the
+ *     nearer one (the code plain rounding gives);
+ *   - e_r = s_r q_r - b_r;  H_rs = <w_r, w_s> <u_r, u_s> over the coefficient vectors of products r and s (Eq. 1);
+ *   - sweep r = 1..R in order; switching entry r to its other candidate changes e_r by delta and e^T H e by
+ *     2 delta (He)_r + delta^2 H_rr, computed in fp32; the switch is accepted when that is negative;
+ *   - stop after a sweep without a change, at most max_sweeps (the paper: 12) sweeps.
+ * Readings: (He)_r is an fp32 FMA chain over s ascending, recomputed at every visit; the change is
+ * fma(delta*delta, H_rr, (2 delta) * (He)_r) with both products rounded to fp32; e_r, delta and s_r q are fp32;
+ * H is computed in fp64 and rounded to fp32; an entry whose bf16 value is itself a decoded code, or whose other
+ * candidate would lie beyond +-448, has no alternative.
+ * B is K x N.  Bq_out [R][bk][bn]: the chosen codes (as values); sB_out [R][ceil(bn/128)][ceil(bk/128)]: the scales;
+ * stats[0..3]: sum over positions of e^T H e before / after (fp64), number of entries that ended on their other
+ * candidate, largest number of sweeps any position used.  Returns 0, or 1 if a dimension does not divide.       */
+int orc_joint_round(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                    int64_t K, int64_t N, const double* B, int max_sweeps,
+                    double* Bq_out, double* sB_out, double* stats) {
+  (void)m;
+  if (K % k || N % n || R > 256) return 1;
+  const int64_t bk = K / k, bn = N / n, G = (bk + 127) / 128, CB = (bn + 127) / 128;
+  double* bs = (double*)malloc(sizeof(double) * (size_t)R * bk * bn);     /* bf16 block sums */
+  double* cv = (double*)malloc(sizeof(double) * k * n);
+  for (int r = 0; r < R; ++r) {
+    for (int x = 0; x < k * n; ++x) cv[x] = (double)(float)V[r * k * n + x];
+    double* Bh = bs + (size_t)r * bk * bn;
+    block_sum(B, N, k, n, bk, bn, cv, 1, Bh);
+    for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x], ORC_BF16);
+    for (int64_t cb = 0; cb < CB; ++cb)
+      for (int64_t g = 0; g < G; ++g) {
+        const int64_t t0 = g * 128, t1 = t0 + 128 < bk ? t0 + 128 : bk;
+        const int64_t c0 = cb * 128, c1 = c0 + 128 < bn ? c0 + 128 : bn;
+        float amax = 0.0f;
+        for (int64_t t = t0; t < t1; ++t)
+          for (int64_t c = c0; c < c1; ++c) { float a = fabsf((float)Bh[t * bn + c]); if (a > amax) amax = a; }
+        sB_out[((size_t)r * CB + cb) * G + g] = (double)(amax > 0.0f ? amax / 448.0f : 1.0f);
+      }
+  }
+  free(cv);
+  /* H_rs = <w_r, w_s> <u_r, u_s> */
+  float* H = (float*)malloc(sizeof(float) * R * R);
+  const int mk = m * k, mn = m * n;
+  for (int r = 0; r < R; ++r)
+    for (int s = 0; s < R; ++s) {
+      double uu = 0.0, ww = 0.0;
+      for (int x = 0; x < mk; ++x) uu += U[r * mk + x] * U[s * mk + x];
+      for (int x = 0; x < mn; ++x) ww += W[r * mn + x] * W[s * mn + x];
+      H[r * R + s] = (float)(ww * uu);
+    }
+  double grid[256];
+  const int cnt = e4m3_grid(grid);
+  double obj0 = 0.0, obj1 = 0.0, moved = 0.0;
+  int worst = 0;
+#pragma omp parallel for schedule(static) reduction(+ : obj0, obj1, moved) reduction(max : worst)
+  for (int64_t pos = 0; pos < bk * bn; ++pos) {
+    const int64_t t = pos / bn, c = pos % bn;
+    float q[256], alt[256], e[256], b[256], sc[256];
+    int has[256], flipped[256];
+    for (int r = 0; r < R; ++r) {
+      b[r] = (float)bs[(size_t)r * bk * bn + pos];
+      sc[r] = (float)sB_out[((size_t)r * CB + c / 128) * G + t / 128];
+      q[r] = (float)orc_round((double)(b[r] / sc[r]), ORC_E4M3);
+      const float dq = sc[r] * q[r];
+      const int gi = grid_index(grid, cnt, (double)q[r]);
+      has[r] = 0; alt[r] = q[r]; flipped[r] = 0;
+      if (dq < b[r] && gi + 1 < cnt) { alt[r] = (float)grid[gi + 1]; has[r] = 1; }
+      if (dq > b[r] && gi > 0) { alt[r] = (float)grid[gi - 1]; has[r] = 1; }
+      e[r] = dq - b[r];
+    }
+    double o = 0.0;
+    for (int r = 0; r < R; ++r) for (int s = 0; s < R; ++s) o += (double)e[r] * (double)H[r * R + s] * (double)e[s];
+    obj0 += o;
+    int used = 0;
+    for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+      int changed = 0;
+      ++used;
+      for (int r = 0; r < R; ++r) {
+        if (!has[r]) continue;
+        const float delta = sc[r] * alt[r] - sc[r] * q[r];
+        float he = 0.0f;
+        for (int s = 0; s < R; ++s) he = fmaf(H[r * R + s], e[s], he);
+        const float change = fmaf(delta * delta, H[r * R + r], (2.0f * delta) * he);
+        if (change < 0.0f) {
+          const float tmp = q[r]; q[r] = alt[r]; alt[r] = tmp;
+          e[r] = sc[r] * q[r] - b[r];
+          flipped[r] ^= 1;
+          changed = 1;
+        }
+      }
+      if (!changed) break;
+    }
+    if (used > worst) worst = used;
+    o = 0.0;
+    for (int r = 0; r < R; ++r) for (int s = 0; s < R; ++s) o += (double)e[r] * (double)H[r * R + s] * (double)e[s];
+    obj1 += o;
+    for (int r = 0; r < R; ++r) {
+      Bq_out[(size_t)r * bk * bn + pos] = (double)q[r];
+      moved += flipped[r];
+    }
+  }
+  if (stats) { stats[0] = obj0; stats[1] = obj1; stats[2] = moved; stats[3] = (double)worst; }
+  free(bs); free(H);
   return 0;
 }

@@ -29,7 +29,7 @@ __all__ = [
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
     "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "certificate",
-    "hadamard_matrix", "hadamard_rotate",
+    "hadamard_matrix", "hadamard_rotate", "row_pow2_scales", "joint_round_weights", "scheme_gemm_weights",
 ]
 
 
@@ -75,6 +75,11 @@ def _L():
         lib.orc_int8_certified.argtypes = ([C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 3)
         lib.orc_int8_corrected.restype = C.c_int
         lib.orc_int8_corrected.argtypes = ([C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 2 + [dp] * 3)
+        lib.orc_scheme_gemm_weights.restype = C.c_int
+        lib.orc_scheme_gemm_weights.argtypes = ([C.c_int] * 4 + [dp] * 3 + [i64] * 3 + [dp] * 2 + [C.c_int] * 2 +
+                                                [dp] * 2 + [C.c_int] + [dp] * 2)
+        lib.orc_joint_round.restype = C.c_int
+        lib.orc_joint_round.argtypes = [C.c_int] * 4 + [dp] * 3 + [i64] * 2 + [dp] + [C.c_int] + [dp] * 3
         lib.orc_certificate.restype = C.c_int
         lib.orc_certificate.argtypes = [C.c_int] * 4 + [dp] * 3 + [C.c_int] * 5 + [dp]
         _lib = lib
@@ -398,3 +403,47 @@ def hadamard_rotate(X, signs, h: int, fmt="f64") -> np.ndarray:
         sl = slice(b * h, (b + 1) * h)
         Y[:, sl] = ((X[:, sl] * signs[sl]) @ Hh) / math.sqrt(h)     # +-1 sums first: exact cancellations stay exact
     return round_to(Y, fmt)
+
+
+# ---------------------------------------------------------------------------- the repair rules (Appendix C)
+def row_pow2_scales(A) -> np.ndarray:
+    """d_t = 2^ceil(log2(max(RMS(x_t), 1e-3))) for every row x_t of A, the RMS over the full row (Appendix C, "The
+    repair rules").  The row is divided by d_t before the block sums and its output row multiplied by d_t after the
+    combination; both are exact, d_t being a power of two."""
+    A = _d(A)
+    rms = np.sqrt(np.mean(A * A, axis=1))
+    out = np.empty(A.shape[0])
+    for t, v in enumerate(np.maximum(rms, 1e-3)):
+        f, e = math.frexp(float(v))            # v = f 2^e, f in [0.5, 1)
+        out[t] = math.ldexp(1.0, e - 1 if f == 0.5 else e)
+    return out
+
+
+def joint_round_weights(s: Scheme, B, max_sweeps: int = 12):
+    """Joint rounding of the weight's block sums under the model schedule (Appendix C, "The repair rules"): returns
+    (codes [R, bk, bn], scales [R, ceil(bn/128), ceil(bk/128)], dict(objective_before, objective_after, moved, sweeps))."""
+    m, k, n, R = s.dims
+    B = _d(B)
+    K, N = B.shape
+    bk, bn = K // k, N // n
+    Bq = np.empty((R, bk, bn)); sB = np.empty((R, -(-bn // 128), -(-bk // 128))); st = np.zeros(4)
+    rc = _L().orc_joint_round(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), K, N, _p(B), int(max_sweeps),
+                              _p(Bq), _p(sB), _p(st))
+    if rc:
+        raise ValueError("matrix dimensions are not divisible by the block grid")
+    return Bq, sB, dict(objective_before=st[0], objective_after=st[1], moved=int(st[2]), sweeps=int(st[3]))
+
+
+def scheme_gemm_weights(s: Scheme, A, B, Bq, sB, od="bf16", md="bf16", products: bool = False):
+    """The model schedule (scale_mode 3, e4m3) with the weight side given as codes and scales (joint_round_weights)."""
+    m, k, n, R = s.dims
+    A = _d(A); B = _d(B)
+    M, K = A.shape
+    N = B.shape[1]
+    Cm = np.empty((M, N))
+    Mr = np.empty((R, M // m, N // n)) if products else None
+    rc = _L().orc_scheme_gemm_weights(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
+                                      _fmt("e4m3"), _fmt(od), _p(Cm), _p(Mr), _fmt(md), _p(_d(Bq)), _p(_d(sB)))
+    if rc:
+        raise ValueError("matrix dimensions are not divisible by the block grid")
+    return (Cm, Mr) if products else Cm

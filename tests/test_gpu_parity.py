@@ -80,6 +80,29 @@ def test_every_step_matches_oracle(lib, scheme, M, K, N, S, Pd, O, kind, scale):
     assert gu.rel_fro(C, Co) <= TOL_FRO
 
 
+@pytest.mark.parametrize("order", ["strassen_outside", "classical_outside"])
+@pytest.mark.parametrize("Pd,scale", [("bf16", 0), ("e4m3", 1)])
+def test_hybrid_of_one_strassen_and_one_classical_level(lib, order, Pd, scale):
+    """One level of Strassen nested with one classical level, <4,4,4;56> (the nesting the paper's first repaired
+    algorithm uses, Appendix C): every step against the oracle's Kronecker scheme, in both nesting orders; the
+    classical level adds no block sums of its own, so the largest block sum has two terms, not four."""
+    At, Bt, A64, B64 = _inputs(17, 512, 768, 544, "bf16", "llm")
+    st, cl = lib.scheme_builtin("strassen222"), lib.scheme_builtin("classical222")
+    ost, ocl = oracle.strassen(), oracle.classical_scheme(2, 2, 2)
+    s = lib.scheme_kron(st, cl) if order == "strassen_outside" else lib.scheme_kron(cl, st)
+    so = oracle.kron(ost, ocl) if order == "strassen_outside" else oracle.kron(ocl, ost)
+    assert s.dims == (4, 4, 4, 56)
+    assert oracle.criteria(so)["L_A"] == 2
+    C, p, _ = gu.run_scheme_gemm(s, At, Bt, "bf16", Pd, "bf16", scale_mode=scale, parts=True)
+    Co, po = oracle.scheme_gemm(so, A64, B64, pd=Pd, od="bf16", scale_mode=scale, parts=True)
+    assert np.array_equal(p["Ahat"], po["Ahat"])
+    assert np.array_equal(p["BhatT"], po["Bhat"].transpose(0, 2, 1))
+    if scale:
+        assert np.array_equal(p["sA"], po["sA"]) and np.array_equal(p["sB"], po["sB"])
+    assert gu.rel_fro(p["M"], po["M"]) <= 1e-5
+    assert gu.rel_fro(C, Co) <= TOL_FRO
+
+
 @pytest.mark.parametrize("scheme,M,K,N,S,Pd,O,kind,scale", [
     ("strassen444", 1024, 1024, 2048, "bf16", "bf16", "bf16", "llm", 0),    # CTA-pair kernel, bf16 products
     ("strassen444", 384, 320, 288, "bf16", "bf16", "f32", "llm", 0),        # ragged tiles
