@@ -346,6 +346,31 @@ fmm_status int8_gemm_corrected(const fmm_scheme* s, const int8_t* d_cA, const fl
 fmm_status hadamard_rotate(int storage, const void* dX, int64_t ldx, int64_t rows, int64_t K, int h,
                            const signed char* d_signs, void* dY, int64_t ldy, void* cuda_stream);
 
+/* The repair rules of Appendix C ("The repair rules").
+ *
+ * Rule 1, row scale.  row_pow2_scale: for every row x_t of X (rows x K, `storage` FMM_F32 / FMM_BF16, DEVICE, ldx >= K)
+ * d_scale[t] = 2^ceil(log2(max(RMS(x_t), 1e-3))) (DEVICE fp32 [rows]; RMS over the full row, sum of squares in fp64)
+ * and Y[t, :] = X[t, :] / d_scale[t] (exact: a power of two; dY may equal dX).  row_unscale: C[t, :] *= d_scale[t] in
+ * place (C rows x N of `output`, DEVICE, ldc >= N) — applied to the product of the scaled rows it restores the scale
+ * of every output row; the multiplication commutes with the rounding to `output`, so it may follow scheme_gemm.
+ *
+ * Rule 2, joint rounding of the weight's block sums (model schedule only: d->scale_mode == 3, product FMM_E4M3, else
+ * FMM_ERR_DTYPE).  scheme_joint_round_weights fills the weight side of a scheme_gemm workspace — the e4m3 codes of
+ * the R block sums of B and their 128 x 128 block scales — and a following scheme_gemm with FMM_FLAG_REUSE_BHAT on
+ * the same descriptor and workspace multiplies with them.  Per position, every code starts at the nearer of the two
+ * e4m3 codes whose decoded values bracket the block sum's bf16 value (the code the plain schedule gives) and, in
+ * sweeps over r = 1..R, is switched to the other one when that lowers e^T H e, e_r = decoded - bf16 value,
+ * H_rs = <w_r, w_s> <u_r, u_s>; fp32 arithmetic: (He)_r an FMA chain over s ascending, the change
+ * fma(delta^2, H_rr, 2 delta (He)_r); a sweep without a switch ends the search, at most max_sweeps (the paper: 12;
+ * 0 gives the plain codes).  dB and d exactly as for scheme_gemm; d_ws: DEVICE, >= scheme_gemm_workspace bytes.
+ * A weight-only pass: no activations enter.                                                                     */
+fmm_status row_pow2_scale(int storage, const void* dX, int64_t ldx, int64_t rows, int64_t K, float* d_scale,
+                          void* dY, int64_t ldy, void* cuda_stream);
+fmm_status row_unscale(int output, void* dC, int64_t ldc, int64_t rows, int64_t N, const float* d_scale,
+                       void* cuda_stream);
+fmm_status scheme_joint_round_weights(const fmm_scheme* s, const fmm_gemm_desc* d, const void* dB, int max_sweeps,
+                                      void* d_ws, size_t ws_bytes, void* cuda_stream);
+
 const char* fmm_status_string(fmm_status st);
 
 /* Number of kernels this library has launched in this process (for benchmarks' accounting). */

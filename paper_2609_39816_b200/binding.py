@@ -24,7 +24,8 @@ EXPORTED_SYMBOLS = [
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
-    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected", "hadamard_rotate",
+    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected", "hadamard_rotate", "row_pow2_scale", "row_unscale",
+    "scheme_joint_round_weights",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
 ]
@@ -98,6 +99,9 @@ _lib.error_frobenius_noalloc_max_elements.restype = C.c_int64
 _lib.scheme_certificate.argtypes = [_vp] + [C.c_int] * 5 + [_dp]
 _lib.scheme_certificate.restype = C.c_int
 _lib.hadamard_rotate.argtypes = [C.c_int, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, C.c_int64, _vp]
+_lib.row_pow2_scale.argtypes = [C.c_int, _vp, C.c_int64, C.c_int64, C.c_int64, _vp, _vp, C.c_int64, _vp]
+_lib.row_unscale.argtypes = [C.c_int, _vp, C.c_int64, C.c_int64, C.c_int64, _vp, _vp]
+_lib.scheme_joint_round_weights.argtypes = [_vp, C.POINTER(GemmDesc), _vp, C.c_int, _vp, _sz, _vp]
 _lib.int8_quantize.argtypes = [_vp, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, _vp]
 _lib.int8_gemm_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
 _lib.int8_gemm_workspace.restype = _sz
@@ -300,6 +304,33 @@ def hadamard_rotate(X, signs, h: int, out=None):
     _check(_lib.hadamard_rotate(st, _ptr(X), X.stride(0), rows, K, h, _ptr(signs) if signs is not None else None,
                                 _ptr(out), out.stride(0), _stream()), "hadamard_rotate")
     return out
+
+
+def row_pow2_scale(X, out=None):
+    """(X / d, d) with d[t] = 2^ceil(log2(max(RMS(X[t]), 1e-3))); X [rows, K] fp32/bf16 on the device."""
+    import torch
+    rows, K = X.shape
+    if out is None:
+        out = torch.empty_like(X)
+    d = torch.empty(rows, dtype=torch.float32, device=X.device)
+    st = F32 if X.dtype == torch.float32 else BF16
+    _check(_lib.row_pow2_scale(st, _ptr(X), X.stride(0), rows, K, _ptr(d), _ptr(out), out.stride(0), _stream()),
+           "row_pow2_scale")
+    return out, d
+
+
+def row_unscale(Cmat, d) -> None:
+    """C[t, :] *= d[t] in place."""
+    import torch
+    rows, N = Cmat.shape
+    out = F32 if Cmat.dtype == torch.float32 else BF16
+    _check(_lib.row_unscale(out, _ptr(Cmat), Cmat.stride(0), rows, N, _ptr(d), _stream()), "row_unscale")
+
+
+def scheme_joint_round_weights(s, d, B, ws, max_sweeps: int = 12) -> None:
+    """Fill the workspace's weight side with jointly rounded codes; follow with scheme_gemm(..., flags |= FLAG_REUSE_BHAT)."""
+    _check(_lib.scheme_joint_round_weights(s.handle, C.byref(d), _ptr(B), int(max_sweeps), _ptr(ws),
+                                           ws.numel() * ws.element_size(), _stream()), "scheme_joint_round_weights")
 
 
 def int8_gemm_workspace(s, M: int, K: int, N: int) -> int:

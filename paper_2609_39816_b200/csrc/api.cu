@@ -526,6 +526,48 @@ fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* 
                     nullptr, nullptr, d_ws, skip_b, st);
 }
 
+fmm_status scheme_joint_round_weights(const fmm_scheme* s, const fmm_gemm_desc* d, const void* dB, int max_sweeps,
+                                      void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!s || !d || !dB || max_sweeps < 0) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, s->m, s->k, s->n));
+  if (d->scale_mode != 3 || d->product != FMM_E4M3) return FMM_ERR_DTYPE;
+  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d);
+  FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const std::vector<unsigned char>& packed = fmm_packed_tables(*s);
+  if (L.status != 0 || L.tabA != kPackedStatusBytes || L.tabB != L.tabA + fmm_packed_table_stride() ||
+      L.tabW != L.tabB + fmm_packed_table_stride() || sizeof(DeviceStatus) > kPackedStatusBytes)
+    return FMM_ERR_CUDA;
+  FMM_CUDA(cudaMemcpyAsync(d_ws, packed.data(), packed.size(), cudaMemcpyHostToDevice, st));
+  const void* bk_ptr; int64_t bk_ld;
+  FMM_TRY(kmajor_b(d, dB, d_ws, L.bt, &bk_ptr, &bk_ld, false, st));
+  // H_rs = <w_r, w_s> <u_r, u_s>, fp64 on the host, rounded to fp32; parked in the product buffer, which nothing uses yet
+  const int R = s->R, mk = s->m * s->k, mn = s->m * s->n;
+  std::vector<float> H((size_t)R * R);
+  for (int r = 0; r < R; ++r)
+    for (int q = 0; q < R; ++q) {
+      double uu = 0.0, ww = 0.0;
+      for (int x = 0; x < mk; ++x) uu += s->U[(size_t)r * mk + x] * s->U[(size_t)q * mk + x];
+      for (int x = 0; x < mn; ++x) ww += s->W[(size_t)r * mn + x] * s->W[(size_t)q * mn + x];
+      H[(size_t)r * R + q] = (float)(ww * uu);
+    }
+  float* d_H = at<float>(d_ws, L.prod);
+  if (L.total - L.prod < H.size() * sizeof(float)) return FMM_ERR_SHAPE;   // blocks of a few elements only
+  FMM_CUDA(cudaMemcpyAsync(d_H, H.data(), H.size() * sizeof(float), cudaMemcpyHostToDevice, st));   // pageable: staged before it returns
+  const int64_t bn = d->N / s->n, bk = d->K / s->k;
+  const CoefTable* hB = fmm_packed_table(*s, 1);
+  const CoefTable* dB_tab = at<CoefTable>(d_ws, L.tabB);
+  unsigned* amax = at<unsigned>(d_ws, L.amaxB);
+  float* sB = at<float>(d_ws, L.sB);
+  // the model schedule's amax pass over the bf16 block sums, then the search in place of the plain encode pass
+  const EncodeOperand ob{bk_ptr, bk_ld, s->n, s->k, bn, bk, dB_tab, hB, at<char>(d_ws, L.bhat), L.sBhat, amax, sB, 128, 1};
+  FMM_CUDA(cudaMemsetAsync(amax, 0, scale_words(3, R, bn, bk, true) * 4, st));
+  FMM_CUDA(launch_encode_pair(d->storage, d->product, ob, nullptr, true, 3, st));
+  FMM_CUDA(launch_joint_round(d->storage, bk_ptr, bk_ld, s->n, s->k, bn, bk, dB_tab, d_H, amax, sB, at<char>(d_ws, L.bhat),
+                              L.sBhat, max_sweeps, st));
+  return FMM_OK;
+}
+
 fmm_status fmm_device_status(const void* d_ws, void* cuda_stream) {
   if (!d_ws) return FMM_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

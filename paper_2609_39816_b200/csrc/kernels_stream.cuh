@@ -48,6 +48,14 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
 }
 #endif
 
+// Joint rounding of the weight's block sums under the model schedule (Appendix C, "The repair rules"): X, the grid and
+// d_tab as for launch_encode (the weight read K-major); amax_bits [R][ceil(br/128)][ceil(bc/128)] from the amax pass of
+// the model schedule; d_H: R x R fp32, H_rs = <w_r, w_s> <u_r, u_s>; writes the e4m3 codes to out (R blocks [br][bc],
+// out_stride elements apart) and the scales to scale_out (laid out like amax_bits).
+cudaError_t launch_joint_round(int storage, const void* X, int64_t ldx, int gr, int gc, int64_t br, int64_t bc,
+                               const CoefTable* d_tab, const float* d_H, const unsigned* amax_bits, float* scale_out,
+                               void* out, int64_t out_stride, int max_sweeps, cudaStream_t st);
+
 // X: source matrix (storage dtype), rows x cols with leading dimension ldx, split into a gr x gc grid of
 // br x bc blocks.  out: R blocks [br][bc] in the product dtype, out_stride elements apart.  With amax_only the kernel only accumulates
 // max|block sum| per product into amax_bits[R] (fp32 bit patterns of non-negative values).

@@ -217,6 +217,23 @@ def test_rotation_argument_checks_need_no_device(lib):
     assert f(0, ctypes.c_void_p((1 << 20) + 4), 64, 4, 64, 32, None, x, 64, None) == 2   # misaligned base
 
 
+def test_repair_entry_points_validate_before_any_launch(lib):
+    L = lib.binding._lib
+    x = ctypes.c_void_p(1 << 20)
+    assert L.row_pow2_scale(0, None, 64, 4, 64, x, x, 64, None) == 1            # FMM_ERR_ARG
+    assert L.row_pow2_scale(2, x, 64, 4, 64, x, x, 64, None) == 5               # FMM_ERR_DTYPE: e4m3 storage
+    assert L.row_pow2_scale(0, x, 32, 4, 64, x, x, 64, None) == 2               # FMM_ERR_SHAPE: ld < K
+    assert L.row_unscale(0, x, 64, 0, 64, x, None) == 2                         # empty
+    assert L.row_unscale(0, x, 64, 4, 64, None, None) == 1
+    s1 = lib.scheme_builtin("strassen222")
+    for pd, mode, want in (("bf16", 0, 5), ("e4m3", 1, 5), ("e4m3", 2, 5)):     # only the model schedule has the rule
+        d = lib.GemmDesc.make(64, 256, 256, "bf16", pd, "bf16", weight_layout=True, scale_mode=mode)
+        assert L.scheme_joint_round_weights(s1.handle, ctypes.byref(d), x, 12, x, 1 << 30, None) == want
+    d3 = lib.GemmDesc.make(64, 256, 256, "bf16", "e4m3", "bf16", weight_layout=True, scale_mode=3)
+    assert L.scheme_joint_round_weights(s1.handle, ctypes.byref(d3), x, -1, x, 1 << 30, None) == 1
+    assert L.scheme_joint_round_weights(s1.handle, ctypes.byref(d3), x, 12, x, 16, None) == 6   # FMM_ERR_WORKSPACE
+
+
 def test_permuted_products_are_the_same_algorithm(lib):
     """Renumbering the products keeps the Brent equations and every criterion; bad permutations are refused."""
     s2 = lib.scheme_builtin("strassen444")
