@@ -25,18 +25,100 @@ __device__ __forceinline__ void store_f32(__nv_bfloat16* p, float v) { *p = __fl
 // the integer decision ceil(log2(.)) agrees with an fp64 evaluation of the definition except when the RMS lies
 // within an fp64 rounding of a power of two.
 // ------------------------------------------------------------------------------------------
+template <typename T> struct RowVec;              // 16 bytes of a row
+template <> struct RowVec<float> { static constexpr int kElems = 4; };
+template <> struct RowVec<__nv_bfloat16> { static constexpr int kElems = 8; };
+
 template <typename T>
+__device__ __forceinline__ void unpack16(const uint4& raw, float (&v)[RowVec<T>::kElems]) {
+  if constexpr (sizeof(T) == 4) {
+    v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y); v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+  } else {
+    const unsigned w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+  }
+}
+template <typename T>
+__device__ __forceinline__ uint4 pack16(const float (&v)[RowVec<T>::kElems]) {
+  uint4 raw;
+  if constexpr (sizeof(T) == 4) {
+    raw = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+  } else {
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<const unsigned*>(&h);
+    }
+    raw = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  return raw;
+}
+
+// kVec: rows are read and written as 16-byte vectors (the host checks alignment and divisibility)
+template <typename T, bool kVec>
 __global__ void __launch_bounds__(256)
-row_scale_kernel(const T* __restrict__ X, int64_t ldx, int64_t rows, int64_t K, float* __restrict__ d_out,
-                 T* __restrict__ Y, int64_t ldy) {
+row_scale_kernel(const T* X, int64_t ldx, int64_t rows, int64_t K, float* __restrict__ d_out, T* Y, int64_t ldy) {   // Y may be X
+  constexpr int VE = RowVec<T>::kElems;
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * 8;
   for (int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5); row < rows; row += warps) {
     const T* x = X + row * ldx;
     double ss = 0.0;
-    for (int64_t t = lane; t < K; t += 32) {
-      const double v = (double)load_f32(x + t);
-      ss = fma(v, v, ss);
+    if (kVec && K <= 16 * 32 * VE) {
+      // rows of up to 8 KB stay in registers between the two passes: every load is issued before the first use
+      if constexpr (kVec) {
+        uint4 keep[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int64_t t = ((int64_t)j * 32 + lane) * VE;
+          keep[j] = t < K ? *reinterpret_cast<const uint4*>(x + t) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        double part[4] = {0.0, 0.0, 0.0, 0.0};           // four chains; the order of an fp64 sum of exact squares
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float v[VE];
+          unpack16<T>(keep[j], v);
+#pragma unroll
+          for (int i = 0; i < VE; ++i) part[j & 3] = fma((double)v[i], (double)v[i], part[j & 3]);
+        }
+        ss = (part[0] + part[1]) + (part[2] + part[3]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        const double rms = fmax(sqrt(ss / (double)K), 1e-3);
+        int e;
+        const double f = frexp(rms, &e);
+        const float d = ldexpf(1.0f, f == 0.5 ? e - 1 : e);
+        if (lane == 0) d_out[row] = d;
+        const float inv = 1.0f / d;
+        T* y = Y + row * ldy;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int64_t t = ((int64_t)j * 32 + lane) * VE;
+          if (t < K) {
+            float v[VE];
+            unpack16<T>(keep[j], v);
+#pragma unroll
+            for (int i = 0; i < VE; ++i) v[i] = __fmul_rn(v[i], inv);
+            *reinterpret_cast<uint4*>(y + t) = pack16<T>(v);
+          }
+        }
+      }
+      continue;
+    }
+    if constexpr (kVec) {
+      for (int64_t t = (int64_t)lane * VE; t < K; t += 32 * VE) {
+        float v[VE];
+        unpack16<T>(*reinterpret_cast<const uint4*>(x + t), v);
+#pragma unroll
+        for (int i = 0; i < VE; ++i) ss = fma((double)v[i], (double)v[i], ss);
+      }
+    } else {
+      for (int64_t t = lane; t < K; t += 32) {
+        const double v = (double)load_f32(x + t);
+        ss = fma(v, v, ss);
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -47,18 +129,38 @@ row_scale_kernel(const T* __restrict__ X, int64_t ldx, int64_t rows, int64_t K, 
     if (lane == 0) d_out[row] = d;
     const float inv = 1.0f / d;                        // a power of two: exact
     T* y = Y + row * ldy;
-    for (int64_t t = lane; t < K; t += 32) store_f32(y + t, __fmul_rn(load_f32(x + t), inv));
+    if constexpr (kVec) {
+      for (int64_t t = (int64_t)lane * VE; t < K; t += 32 * VE) {
+        float v[VE];
+        unpack16<T>(*reinterpret_cast<const uint4*>(x + t), v);
+#pragma unroll
+        for (int i = 0; i < VE; ++i) v[i] = __fmul_rn(v[i], inv);
+        *reinterpret_cast<uint4*>(y + t) = pack16<T>(v);
+      }
+    } else {
+      for (int64_t t = lane; t < K; t += 32) store_f32(y + t, __fmul_rn(load_f32(x + t), inv));
+    }
   }
 }
 
-template <typename T>
+template <typename T, bool kVec>
 __global__ void __launch_bounds__(256)
 row_unscale_kernel(T* __restrict__ C, int64_t ldc, int64_t rows, int64_t N, const float* __restrict__ d) {
-  const int64_t total = rows * N;
+  constexpr int VE = kVec ? RowVec<T>::kElems : 1;
+  const int64_t per_row = N / VE, total = rows * per_row;
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (int64_t)gridDim.x * 256) {
-    const int64_t row = i / N, col = i - row * N;
+    const int64_t row = i / per_row, col = (i - row * per_row) * VE;
     T* p = C + row * ldc + col;
-    store_f32(p, __fmul_rn(load_f32(p), d[row]));
+    const float dr = d[row];
+    if constexpr (kVec) {
+      float v[RowVec<T>::kElems];
+      unpack16<T>(*reinterpret_cast<const uint4*>(p), v);
+#pragma unroll
+      for (int k = 0; k < RowVec<T>::kElems; ++k) v[k] = __fmul_rn(v[k], dr);
+      *reinterpret_cast<uint4*>(p) = pack16<T>(v);
+    } else {
+      store_f32(p, __fmul_rn(load_f32(p), dr));
+    }
   }
 }
 
@@ -191,11 +293,16 @@ extern "C" fmm_status row_pow2_scale(int storage, const void* dX, int64_t ldx, i
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int64_t want = (rows + 7) / 8, cap = (int64_t)sm_count() * 8;
   const unsigned grid = (unsigned)(want < cap ? want : cap);
-  if (storage == FMM_F32)
-    row_scale_kernel<float><<<grid, 256, 0, st>>>((const float*)dX, ldx, rows, K, d_scale, (float*)dY, ldy);
-  else
-    row_scale_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)dX, ldx, rows, K, d_scale,
-                                                          (__nv_bfloat16*)dY, ldy);
+  const int64_t eb = storage == FMM_F32 ? 4 : 2;
+  const bool vec = (((uintptr_t)dX | (uintptr_t)dY) & 15u) == 0 && (ldx * eb) % 16 == 0 && (ldy * eb) % 16 == 0 &&
+                   (K * eb) % 16 == 0;
+  if (storage == FMM_F32) {
+    if (vec) row_scale_kernel<float, true><<<grid, 256, 0, st>>>((const float*)dX, ldx, rows, K, d_scale, (float*)dY, ldy);
+    else row_scale_kernel<float, false><<<grid, 256, 0, st>>>((const float*)dX, ldx, rows, K, d_scale, (float*)dY, ldy);
+  } else {
+    if (vec) row_scale_kernel<__nv_bfloat16, true><<<grid, 256, 0, st>>>((const __nv_bfloat16*)dX, ldx, rows, K, d_scale, (__nv_bfloat16*)dY, ldy);
+    else row_scale_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>((const __nv_bfloat16*)dX, ldx, rows, K, d_scale, (__nv_bfloat16*)dY, ldy);
+  }
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
@@ -206,12 +313,18 @@ extern "C" fmm_status row_unscale(int output, void* dC, int64_t ldc, int64_t row
   if (output != FMM_F32 && output != FMM_BF16) return FMM_ERR_DTYPE;
   if (rows <= 0 || N <= 0 || ldc < N) return FMM_ERR_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int64_t want = (rows * N + 255) / 256, cap = (int64_t)sm_count() * 16;
+  const int64_t eb = output == FMM_F32 ? 4 : 2;
+  const bool vec = ((uintptr_t)dC & 15u) == 0 && (ldc * eb) % 16 == 0 && (N * eb) % 16 == 0;
+  const int64_t items = vec ? rows * (N * eb / 16) : rows * N;
+  const int64_t want = (items + 255) / 256, cap = (int64_t)sm_count() * 16;
   const unsigned grid = (unsigned)(want < cap ? want : cap);
-  if (output == FMM_F32)
-    row_unscale_kernel<float><<<grid, 256, 0, st>>>((float*)dC, ldc, rows, N, d_scale);
-  else
-    row_unscale_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)dC, ldc, rows, N, d_scale);
+  if (output == FMM_F32) {
+    if (vec) row_unscale_kernel<float, true><<<grid, 256, 0, st>>>((float*)dC, ldc, rows, N, d_scale);
+    else row_unscale_kernel<float, false><<<grid, 256, 0, st>>>((float*)dC, ldc, rows, N, d_scale);
+  } else {
+    if (vec) row_unscale_kernel<__nv_bfloat16, true><<<grid, 256, 0, st>>>((__nv_bfloat16*)dC, ldc, rows, N, d_scale);
+    else row_unscale_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>((__nv_bfloat16*)dC, ldc, rows, N, d_scale);
+  }
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
