@@ -36,7 +36,7 @@ __all__ = [
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (no fast-math, no FP contraction)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O3", "-march=native", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+        cmd = ["gcc", "-O3", "-march=x86-64-v3", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
                "-shared", "-fPIC", "-std=c11", "-o", _SO, _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _SO
