@@ -339,6 +339,26 @@ def test_sweep_batches_walk_several_tiles_per_block(lib):
 
 
 # ---------------------------------------------------------------------------- full size, sampled
+def test_config3_full_size_sweep_against_the_oracle(lib):
+    """The sweep exactly as bench.py times it (A 2048 x 4096, B 4096 x 4096 stored [N, K], bf16, batches of four
+    algorithms, fourteen tiles per decode block): the ratios of five of the configuration's gauges against the
+    oracle's full-size products (a 4 + 1 split of the batch)."""
+    import bench
+    At_h, Bt_h = bench.c3_inputs(0)
+    At, Bt = At_h.cuda(), Bt_h.cuda()
+    A64, B64 = At_h.double().numpy(), Bt_h.double().numpy().T.copy()
+    P, Q, S = bench.sweep_gauges(512)
+    pick = [0, 100, 200, 300, 511]
+    P, Q, S = P[pick], Q[pick], S[pick]
+    s1 = lib.scheme_builtin("strassen222")
+    d = lib.GemmDesc.make(2048, 4096, 4096, "bf16", "bf16", "bf16", weight_layout=True)
+    ws = gu.workspace(lib.error_sweep_workspace(s1, d, len(pick)))
+    ratios, summ = lib.error_sweep(s1, 0, P, Q, S, d, At, Bt, ws)
+    want, Ecl = _oracle_ratios(oracle.strassen(), P, Q, S, A64, B64, "bf16", "bf16")
+    assert math.isclose(summ["e_classical_rel"], Ecl, rel_tol=TOL_RATIO)
+    assert np.all(np.abs(ratios - want) <= TOL_RATIO * want), (ratios, want)
+
+
 def test_config2_full_size_sampled_outputs(lib):
     """Config 2 at full size in the launch configuration the benchmark times (bf16, weight layout):
     sampled rows/columns recomputed by the oracle one by one (a scheme acts position-wise on blocks)."""
