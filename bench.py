@@ -368,6 +368,12 @@ def run_ours(args):
     t_e2e_wr = max_over_ranks(e2e_pipelined(args.steps, weights_resident=True))
     barrier()
 
+    # ---- the error side of the benchmark workload: rho of the scheme as given, against the classical product
+    rho_c2 = None
+    if rank == 0:
+        r_, e_ = rho_identity(fmm, torch, s, d, A, B)
+        rho_c2 = {"rho": r_, "e_classical_rel": e_, "note": "identity gauge on the benchmark operands; fp64 reference formed on the device"}
+
     # ---- roofline of the dominant kernel (block products), timed live by the library's phase events
     peaks = measured_peaks()
     bm_, bk_, bn_ = M // 4, K // 4, N // 4
@@ -488,6 +494,7 @@ def run_ours(args):
                                        "scheme_time_over_classical": float(np.mean(times)) / t_cl},
             "phases": phase_out,
             "sweep": sweep,
+            "rho_identity": rho_c2,
         }
         print(json.dumps(line))
     if world > 1:
@@ -495,6 +502,16 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------ other configurations (not the default line)
+def rho_identity(fmm, torch, scheme, d, At, Bt):
+    """Error-amplification ratio of the scheme as given (identity gauge) on these operands, and the classical error:
+    one error_sweep call with a single gauge, outside any timed region (it forms the fp64 reference itself)."""
+    m, k, n, _ = scheme.dims
+    ws = torch.empty(fmm.error_sweep_workspace(scheme, d, 1), dtype=torch.uint8, device=At.device)
+    ratios, summ = fmm.error_sweep(scheme, 0, np.eye(m)[None], np.eye(k)[None], np.eye(n)[None], d, At, Bt, ws)
+    del ws
+    return float(ratios[0]), float(summ["e_classical_rel"])
+
+
 def run_workload(args):
     """Throughput of the other benchmark configurations on one GPU; prints one JSON line for --workload."""
     import torch
@@ -540,7 +557,10 @@ def run_workload(args):
         t_cl = timed(lambda: fmm.classical_gemm(d, At, Wt, C, wsc))
         eff = 2.0 * T * K * N
         rfl = 2.0 * R * (T // m) * (K // k) * (N // n)
+        del ws, wsc
+        rho, ecl = rho_identity(fmm, torch, s, fmm.GemmDesc.make(T, K, N, S, Pd, O, weight_layout=True, scale_mode=scale), At, Wt)
         return {"shape": [T, K, N], "product": Pd, "ms": t, "eff_tflops": eff / t / 1e9, "r_tflops": rfl / t / 1e9,
+                "rho_identity": rho, "e_classical_rel": ecl,
                 "ms_weights_cached": t_cached, "eff_tflops_weights_cached": eff / t_cached / 1e9,
                 "classical_ms": t_cl, "classical_tflops": eff / t_cl / 1e9, "scheme_over_classical": t / t_cl}
 
