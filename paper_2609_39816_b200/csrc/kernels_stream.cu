@@ -775,6 +775,129 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
 // ------------------------------------------------------------------------------------------
 // reductions
 // ------------------------------------------------------------------------------------------
+// Error-only decode of a batch of four gauge-equivalent algorithms with at most kBatchR products and four output
+// cells each (one level on a 2 x 2 grid).  Thread group g (two warps) owns algorithm g: a thread keeps the
+// algorithm's products of its position quad in registers — 16-byte loads straight from the product buffers, all
+// issued before the first use — and forms every output cell as the same fp32 FMA chain in ascending r that the list
+// walk of decode_kernel performs (coefficients from a dense [algorithm][cell][r] copy of the table in shared memory;
+// absent entries are skipped, not multiplied).  The reference values of a position are staged once for the four
+// algorithms, two tiles deep.  The table is the merged one of the batch: list c * 4 + g holds cell c of algorithm g,
+// its products numbered g * RB .. g * RB + RB - 1.
+// ------------------------------------------------------------------------------------------
+constexpr int kBatchR = 8;
+
+template <typename OutT, typename ProdT>
+__global__ void __launch_bounds__(kDecThreads)
+decode_batch_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_tab, int RB,
+                    const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
+                    const float* __restrict__ cstar32, int64_t ldcs, double* __restrict__ partials,
+                    int tiles_per_block, int64_t rstride) {
+  constexpr int kGauges = 4, kPos = kDecThreads / kGauges;
+  grid_dependency_wait();
+  __shared__ float Wd[kGauges][4][kBatchR];
+  __shared__ __align__(16) float4 cs_stage[2][4][kPos];
+  __shared__ double red[kDecThreads / 32];
+  const int cells = d_tab->R / kGauges;           // output cells per algorithm (<= 4)
+  const int Rtot = RB * kGauges;
+  for (int i = threadIdx.x; i < kGauges * 4 * kBatchR; i += kDecThreads) (&Wd[0][0][0])[i] = 0.0f;
+  __syncthreads();
+  {
+    const int total = d_tab->off[d_tab->R];
+    for (int i = threadIdx.x; i < total; i += kDecThreads) {
+      const int r = d_tab->cell[i];
+      if (r >= Rtot) continue;                     // padding entry
+      int c = 0;                                   // the list this entry belongs to
+      while (d_tab->off[c + 1] <= i) ++c;
+      float w = d_tab->coef[i];
+      if (sA != nullptr) w *= sA[r] * sB[r];       // power-of-two scales fold exactly into the coefficient
+      const int g2 = c % kGauges;
+      Wd[g2][c / kGauges][r - g2 * RB] = w;
+    }
+  }
+  const int g = threadIdx.x / kPos;
+  const int pq = threadIdx.x - g * kPos;
+  const int vec_per_row = (int)(bn >> 2);
+  const int nvec = (int)bm * vec_per_row;
+  const bool cs_mine = g < cells;
+  const int64_t cs_src = (int64_t)(g / n) * bm * ldcs + (int64_t)(g % n) * bn;
+  const uint32_t cs_dst = (uint32_t)__cvta_generic_to_shared(&cs_stage[0][g][pq]);
+  constexpr uint32_t kCsBuf = 4 * kPos * 16;
+  auto issue_cs = [&](int it) {
+    if (it < tiles_per_block && cs_mine) {
+      const int idx = (blockIdx.x * tiles_per_block + it) * kPos + pq;
+      const bool live = idx < nvec;
+      const int p = live ? idx / vec_per_row : 0;
+      const int q = live ? (idx - p * vec_per_row) << 2 : 0;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(cs_dst + (it & 1) * kCsBuf),
+                   "l"(cstar32 + cs_src + (int64_t)p * ldcs + q), "r"(live ? 16 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  issue_cs(0);
+  float err = 0.0f;
+  const ProdT* my_prod = prod + (int64_t)g * RB * rstride;
+  for (int it = 0; it < tiles_per_block; ++it) {
+    const int idx = (blockIdx.x * tiles_per_block + it) * kPos + pq;
+    const bool live = idx < nvec;
+    const int p = live ? idx / vec_per_row : 0;
+    const int q = live ? (idx - p * vec_per_row) << 2 : 0;
+    float4 v[kBatchR];
+#pragma unroll
+    for (int r = 0; r < kBatchR; ++r) {
+      v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < RB && live) {
+        const ProdT* src = my_prod + (int64_t)r * rstride + (int64_t)p * bn + q;
+        if constexpr (sizeof(ProdT) == 4) {
+          v[r] = __ldcs(reinterpret_cast<const float4*>(src));
+        } else {
+          const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(src));
+          v[r] = staged_quad(reinterpret_cast<const unsigned char*>(&raw), (const ProdT*)nullptr);
+        }
+      }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();          // tile it's reference values have landed; everyone is done reading the other buffer
+    issue_cs(it + 1);
+    if (live) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if (c < cells) {
+          float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int r = 0; r < kBatchR; ++r) {
+            const float w = Wd[g][c][r];
+            if (w != 0.0f) {                       // warp-uniform: absent entries are skipped, as in the list walk
+              const float2 ww = make_float2(w, w);
+              x0 = __ffma2_rn(ww, make_float2(v[r].x, v[r].y), x0);
+              x1 = __ffma2_rn(ww, make_float2(v[r].z, v[r].w), x1);
+            }
+          }
+          const float4 cs = cs_stage[it & 1][c][pq];
+          const float d0 = round_out(x0.x, (OutT*)nullptr) - cs.x, d1 = round_out(x0.y, (OutT*)nullptr) - cs.y;
+          const float d2 = round_out(x1.x, (OutT*)nullptr) - cs.z, d3 = round_out(x1.y, (OutT*)nullptr) - cs.w;
+          err = __fmaf_rn(d0, d0, err); err = __fmaf_rn(d1, d1, err);
+          err = __fmaf_rn(d2, d2, err); err = __fmaf_rn(d3, d3, err);
+        }
+      }
+    }
+  }
+  // one sum per algorithm; partials laid out [algorithm][block]
+  double sv = (double)err;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sv += __shfl_xor_sync(0xffffffffu, sv, o);
+  const int warp = threadIdx.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[warp] = sv;
+  __syncthreads();
+  if (threadIdx.x < kGauges) {
+    double tot = 0.0;
+    for (int w = 0; w < kDecThreads / 32; ++w)
+      if ((w * 32) / kPos == (int)threadIdx.x) tot += red[w];
+    partials[(size_t)threadIdx.x * gridDim.x + blockIdx.x] = tot;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // block b sums partials[b * n .. b * n + n) into out[b]
 __global__ void __launch_bounds__(256) sum_partials_kernel(const double* __restrict__ partials, int n,
                                                            double* __restrict__ out) {
@@ -983,6 +1106,27 @@ static cudaError_t launch_decode_p(int output, const ProdT* prod, int64_t prod_s
                                    cudaStream_t st) {
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
+  // a batch of four small algorithms, error only: products straight into registers (decode_batch_kernel)
+  if (gauges == 4 && C == nullptr && R % 4 == 0 && R / 4 <= kBatchR && m * n <= 4 && h_tab->R == 4 * m * n &&
+      std::getenv("FMM_B200_NO_BATCH_DECODE") == nullptr) {
+    if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    int grid, tpb;
+    split_tiles((bm * (bn >> 2) + 63) / 64, &grid, &tpb);
+    if (n_partials) *n_partials = grid;
+    const int64_t ldcs = (int64_t)n * bn;
+    cudaError_t le;
+    if (output == FMM_F32)
+      le = launch_dependent(decode_batch_kernel<float, ProdT>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, R / 4, sA, sB, n,
+                            bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
+    else if (output == FMM_BF16)
+      le = launch_dependent(decode_batch_kernel<__nv_bfloat16, ProdT>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, R / 4, sA,
+                            sB, n, bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
+    else
+      return cudaErrorInvalidValue;
+    if (le != cudaSuccess) return le;
+    ++fmm_launch_counter();
+    return cudaGetLastError();
+  }
   // small schemes (at most 8 products, 4 output cells): one thread per position quad; otherwise four share one
   const bool small = R <= 8 && m * n * gauges <= 4 && gauges == 1;
   if (output == FMM_F32)
