@@ -175,7 +175,10 @@ struct EncodeJob {
 
 // kM3: the model schedule (use_scale == 3) is compiled into its own instantiation so that the other modes carry none
 // of its index arithmetic.
-template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit, bool kM3>
+// kDense: a grid of four cells whose every product reads all four, in one cell order shared by all lists (what a general
+// gauge on a 2 x 2 grid produces): the four source vectors are unpacked once per tile and every product is a four-term
+// chain on registers — the same FMAs in the same order as the list walk.
+template <typename SrcT, typename DstT, bool kAmaxOnly, int kEncSplit, bool kM3, bool kDense = false>
 __global__ void __launch_bounds__(kEncThreads)
 encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
   grid_launch_dependents();   // the block products may set up while this grid drains; they wait before reading
@@ -278,11 +281,26 @@ encode_kernel(const EncodeJob job_a, const EncodeJob job_b, int use_scale) {
     const int64_t m3_row_group = scale_rows == 1 ? p : p >> 7;
     // one product at a time, its list walked two entries per step (lists are padded to an even length with
     // (zero slab, 0.0f) entries, which add exactly nothing); the four accumulator pairs are independent chains
+    float2 src[kDense ? 4 : 1][NP];
+    if constexpr (kDense) {     // slab offsets of the list's four entries are the same for every product: take product 0's
+#pragma unroll
+      for (int c = 0; c < 4; ++c) Vec16<SrcT>::unpack(*reinterpret_cast<const uint4*>(my_stage + ent[c].x), src[c]);
+    }
     for (int r = g; r < R; r += kEncSplit) {
       float2 acc[NP];
 #pragma unroll
       for (int i = 0; i < NP; ++i) acc[i] = make_float2(0.0f, 0.0f);
       const int eend = sm.off[r + 1];
+      if constexpr (kDense) {
+        const int4 p0 = *reinterpret_cast<const int4*>(&ent[4 * r]);
+        const int4 p1 = *reinterpret_cast<const int4*>(&ent[4 * r + 2]);
+        const float cf[4] = {__int_as_float(p0.y), __int_as_float(p0.w), __int_as_float(p1.y), __int_as_float(p1.w)};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+          for (int i = 0; i < NP; ++i) acc[i] = __ffma2_rn(make_float2(cf[c], cf[c]), src[c][i], acc[i]);
+        }
+      } else
       for (int e = sm.off[r]; e < eend; e += 2) {
         const int4 pair = *reinterpret_cast<const int4*>(&ent[e]);
         const uint4 raw0 = *reinterpret_cast<const uint4*>(my_stage + pair.x);
@@ -543,9 +561,25 @@ static bool make_job(const EncodeOperand& o, EncodeJob* j, size_t* smem) {
   return true;
 }
 
-template <typename SrcT, typename DstT, bool kAmaxOnly, int kSplit, bool kM3>
+// every list of the table has exactly four entries over the four cells of the grid, in the same cell order
+static bool dense_four_cells(const CoefTable& t) {
+  if (t.ncell != 4 || t.R < 1 || t.off[t.R] != 4 * t.R) return false;
+  bool seen[4] = {false, false, false, false};
+  for (int c = 0; c < 4; ++c) {
+    if (t.cell[c] < 0 || t.cell[c] > 3 || seen[t.cell[c]]) return false;
+    seen[t.cell[c]] = true;
+  }
+  for (int r = 0; r < t.R; ++r) {
+    if (t.off[r] != 4 * r) return false;
+    for (int c = 0; c < 4; ++c)
+      if (t.cell[4 * r + c] != t.cell[c]) return false;
+  }
+  return true;
+}
+
+template <typename SrcT, typename DstT, bool kAmaxOnly, int kSplit, bool kM3, bool kDense = false>
 static cudaError_t launch_encode_k(int grid, size_t smem, cudaStream_t st, const EncodeJob& ja, const EncodeJob& jb, int use_scale) {
-  auto k = encode_kernel<SrcT, DstT, kAmaxOnly, kSplit, kM3>;
+  auto k = encode_kernel<SrcT, DstT, kAmaxOnly, kSplit, kM3, kDense>;
   static unsigned long long smem_ok = 0;   // per template instantiation, one bit per device
   cudaError_t e = fmm_allow_dynamic_smem(k, 200 * 1024, &smem_ok);
   if (e != cudaSuccess) return e;
@@ -569,6 +603,10 @@ cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool
   if (use_scale == 3)
     e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale)
                   : launch_encode_k<SrcT, DstT, false, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale);
+  else if (kSplit == 4 && dense_four_cells(*a.h_tab) && (b == nullptr || dense_four_cells(*b->h_tab)) &&
+           std::getenv("FMM_B200_NO_DENSE_ENCODE") == nullptr)
+    e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, false, true>(grid, smem, st, ja, jb, use_scale)
+                  : launch_encode_k<SrcT, DstT, false, kSplit, false, true>(grid, smem, st, ja, jb, use_scale);
   else
     e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, false>(grid, smem, st, ja, jb, use_scale)
                   : launch_encode_k<SrcT, DstT, false, kSplit, false>(grid, smem, st, ja, jb, use_scale);
