@@ -82,7 +82,7 @@ def sweep_gauges(G: int, seed: int = 1):
 
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -96,39 +96,53 @@ class ClockSampler:
             f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
             self.path = f.name
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=f,
+                                          "--format=csv,noheader,nounits", "-lms", "10"], stdout=f,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self) -> dict:
+    def stop(self, t0: float = None, t1: float = None) -> dict:
+        """Median SM clock and the throttle reasons over the samples taken inside the wall-clock window [t0, t1]
+        (the sampler is started well before it: nvidia-smi needs a moment to come up); if the window is shorter than
+        the sampling period and holds no sample, the two samples around it are used and `window` says so."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        rows = []
         try:
+            import datetime
             for line in open(self.path):
                 p = [x.strip() for x in line.split(",")]
-                if len(p) < 7:
+                if len(p) < 8:
                     continue
                 try:
-                    sm.append(float(p[0])); mx.append(float(p[1]))
+                    ts = datetime.datetime.strptime(p[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(p[1]), float(p[2]), [v.lower().startswith("active") for v in p[4:8]]))
                 except ValueError:
                     continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        if not rows:
+            return out
+        inside = [r for r in rows if t0 is None or (t0 <= r[0] <= t1)]
+        out["window"] = "inside the timed region"
+        if not inside:      # region shorter than the sampling period: the nearest sample before and after it
+            before = [r for r in rows if r[0] < t0][-1:]
+            after = [r for r in rows if r[0] > t1][:1]
+            inside = before + after
+            out["window"] = "nearest samples around the timed region"
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        reasons = {n for r in inside for n, on in zip(names, r[3]) if on}
+        if inside:
+            out.update(sm_mhz=float(np.median([r[1] for r in inside])), sm_max_mhz=float(max(r[2] for r in inside)),
+                       samples=len(inside))
         out["reasons"] = sorted(reasons)
         return out
 
@@ -266,9 +280,10 @@ def run_ours(args):
 
     # ---- timed region: K steps of the whole path, inputs resident in HBM
     sampler = ClockSampler(local)
+    sampler.start()                      # before the warm-up: the sampling process is up when the timed steps begin
     timed(step, 0, args.warmup)
     launches0 = fmm.launch_count()
-    sampler.start()
+    t_wall0 = time.time()
     times = timed(step, args.steps, 0)
     launches = fmm.launch_count() - launches0
     # the same K steps once more with the library's phase events on the stream: per-kernel durations for the
@@ -279,7 +294,7 @@ def run_ours(args):
     times_ev = timed(step, args.steps, 0)
     phases = fmm.profile_collect()
     fmm.profile_enable(False)
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_wall0, time.time())     # the K timed steps and their event-instrumented repeat
     fmm.device_status(ws)
     ms_step = max_over_ranks(float(np.mean(times)))
     ms_step_events = float(np.mean(times_ev))
@@ -799,7 +814,7 @@ def int8_workload(fmm, gen, torch, timed, peaks):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=512, help="gauges per rank in the c3 sweep (0 = skip); config 3 names 512")
