@@ -446,7 +446,7 @@ def run_ours(args):
             fmm.error_sweep(s1, 0, P[mine][:Gp], Q[mine][:Gp], S[mine][:Gp], d3, A3, B3, ws3, Cstar=Cs)
             ph3 = fmm.profile_collect(); fmm.profile_enable(False)
             bm3, bk3, bn3 = C3["M"] // 2, C3["K"] // 2, C3["N"] // 2
-            kb = 4                                               # algorithms per launch set for <2,2,2;7>
+            kb = 8                                               # algorithms per launch set for <2,2,2;7>
             enc_b = (C3["M"] * C3["K"] + C3["N"] * C3["K"]) * 2 / kb + 7 * (bm3 * bk3 + bn3 * bk3) * 2
             dec_b = 7 * bm3 * bn3 * 4 + C3["M"] * C3["N"] * 4 / kb
             enc_us = (ph3["encode_a"][0] + ph3["encode_b"][0]) * 1e3 / Gp

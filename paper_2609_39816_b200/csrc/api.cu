@@ -140,7 +140,7 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.sA = o; o += align_up(nsa * 4);
   L.sB = o; o += align_up(nsb * 4);
   L.n_partials = std::max(decode_grid(bm, bn), kMaxStreamPartials);
-  L.partials = o; o += align_up((size_t)L.n_partials * 8 * 4);   // up to four algorithms' error sums per decode launch
+  L.partials = o; o += align_up((size_t)L.n_partials * 8 * 8);   // up to eight algorithms' error sums per decode launch
   L.bt = o; o += d->b_is_weight_layout ? 0 : align_up((size_t)d->N * d->K * es);
   // Consecutive products are spaced by the block size plus 256 bytes: block sizes are often powers of two, and
   // R streams written (or read) at the same offset of power-of-two-spaced slabs land on the same memory
@@ -397,12 +397,18 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
 // launches: the encode reads A and B once for all of them, the block products fill the machine with more tiles, the
 // decode walks the positions once.  `kb` algorithms become one table set with kb * R products; the decode table keeps
 // their C blocks apart (list c feeds block c / kb of algorithm c % kb).  Limits: kb * R <= FMM_MAX_R products,
-// kb * m * n <= 16 decode lists, kb in {1, 2, 4} (it must divide the decode's thread split).
+// kb * m * n <= 16 decode lists, kb in {1, 2, 4} (it must divide the decode's thread split); eight algorithms of at
+// most 8 products and 4 output cells each also fit (32 lists: the register-resident batch decode takes them).
 int sweep_batch(const fmm_scheme* s) {
-  static const bool off = [] { const char* e = std::getenv("FMM_B200_NO_GAUGE_BATCH"); return e && e[0] == '1'; }();
-  if (off) return 1;
+  static const int cap = [] {
+    const char* e = std::getenv("FMM_B200_NO_GAUGE_BATCH");
+    if (e && e[0] == '1') return 1;
+    const char* m = std::getenv("FMM_B200_MAX_GAUGE_BATCH");
+    return m ? std::max(1, std::atoi(m)) : 8;
+  }();
+  if (cap >= 8 && 8 * s->R <= FMM_MAX_R && s->R <= 8 && s->m * s->n <= 4) return 8;
   for (int kb = 4; kb > 1; kb /= 2)
-    if (kb * s->R <= FMM_MAX_R && kb * s->m * s->n <= 16) return kb;
+    if (kb <= cap && kb * s->R <= FMM_MAX_R && kb * s->m * s->n <= 16) return kb;
   return 1;
 }
 
@@ -685,7 +691,7 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
     int g = next_gauge;
     while (g < g_end) {
       int kc = kb;
-      while (kc > g_end - g) kc /= 2;   // 4, 2 or 1 algorithms
+      while (kc > g_end - g) kc /= 2;   // 8, 4, 2 or 1 algorithms
       CoefTable mA, mB, mW;
       while (kc > 1 && !merge_tables(&single[3 * g], kc, base->R, &mA, &mB, &mW)) kc /= 2;   // lists too long: smaller batch
       if (kc == 1) { mA = single[3 * g]; mB = single[3 * g + 1]; mW = single[3 * g + 2]; }

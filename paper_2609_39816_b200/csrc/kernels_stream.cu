@@ -813,24 +813,24 @@ decode_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_ta
 // ------------------------------------------------------------------------------------------
 // reductions
 // ------------------------------------------------------------------------------------------
-// Error-only decode of a batch of four gauge-equivalent algorithms with at most kBatchR products and four output
-// cells each (one level on a 2 x 2 grid).  Thread group g (two warps) owns algorithm g: a thread keeps the
+// Error-only decode of a batch of four or eight gauge-equivalent algorithms with at most kBatchR products and four output
+// cells each (one level on a 2 x 2 grid).  Thread group g (two warps, or one for eight algorithms) owns algorithm g: a thread keeps the
 // algorithm's products of its position quad in registers — 16-byte loads straight from the product buffers, all
 // issued before the first use — and forms every output cell as the same fp32 FMA chain in ascending r that the list
 // walk of decode_kernel performs (coefficients from a dense [algorithm][cell][r] copy of the table in shared memory;
 // absent entries are skipped, not multiplied).  The reference values of a position are staged once for the four
-// algorithms, two tiles deep.  The table is the merged one of the batch: list c * 4 + g holds cell c of algorithm g,
+// algorithms, two tiles deep.  The table is the merged one of the batch: list c * kGauges + g holds cell c of algorithm g,
 // its products numbered g * RB .. g * RB + RB - 1.
 // ------------------------------------------------------------------------------------------
 constexpr int kBatchR = 8;
 
-template <typename OutT, typename ProdT>
+template <typename OutT, typename ProdT, int kGauges>
 __global__ void __launch_bounds__(kDecThreads)
 decode_batch_kernel(const ProdT* __restrict__ prod, const CoefTable* __restrict__ d_tab, int RB,
                     const float* __restrict__ sA, const float* __restrict__ sB, int n, int64_t bm, int64_t bn,
                     const float* __restrict__ cstar32, int64_t ldcs, double* __restrict__ partials,
                     int tiles_per_block, int64_t rstride) {
-  constexpr int kGauges = 4, kPos = kDecThreads / kGauges;
+  constexpr int kPos = kDecThreads / kGauges;          // 64 positions for four algorithms, 32 for eight
   grid_dependency_wait();
   __shared__ float Wd[kGauges][4][kBatchR];
   __shared__ __align__(16) float4 cs_stage[2][4][kPos];
@@ -1145,19 +1145,27 @@ static cudaError_t launch_decode_p(int output, const ProdT* prod, int64_t prod_s
   const int nnz = padded_entries(*h_tab);
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   // a batch of four small algorithms, error only: products straight into registers (decode_batch_kernel)
-  if (gauges == 4 && C == nullptr && R % 4 == 0 && R / 4 <= kBatchR && m * n <= 4 && h_tab->R == 4 * m * n &&
-      std::getenv("FMM_B200_NO_BATCH_DECODE") == nullptr) {
+  if ((gauges == 4 || gauges == 8) && C == nullptr && R % gauges == 0 && R / gauges <= kBatchR && m * n <= 4 &&
+      h_tab->R == gauges * m * n && std::getenv("FMM_B200_NO_BATCH_DECODE") == nullptr) {
     if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    const int pos = kDecThreads / gauges;
     int grid, tpb;
-    split_tiles((bm * (bn >> 2) + 63) / 64, &grid, &tpb);
+    split_tiles((bm * (bn >> 2) + pos - 1) / pos, &grid, &tpb);
     if (n_partials) *n_partials = grid;
     const int64_t ldcs = (int64_t)n * bn;
+    const int RB = R / gauges;
     cudaError_t le;
-    if (output == FMM_F32)
-      le = launch_dependent(decode_batch_kernel<float, ProdT>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, R / 4, sA, sB, n,
+    if (output == FMM_F32 && gauges == 4)
+      le = launch_dependent(decode_batch_kernel<float, ProdT, 4>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, RB, sA, sB, n,
                             bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
+    else if (output == FMM_F32)
+      le = launch_dependent(decode_batch_kernel<float, ProdT, 8>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, RB, sA, sB, n,
+                            bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
+    else if (output == FMM_BF16 && gauges == 4)
+      le = launch_dependent(decode_batch_kernel<__nv_bfloat16, ProdT, 4>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, RB, sA,
+                            sB, n, bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
     else if (output == FMM_BF16)
-      le = launch_dependent(decode_batch_kernel<__nv_bfloat16, ProdT>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, R / 4, sA,
+      le = launch_dependent(decode_batch_kernel<__nv_bfloat16, ProdT, 8>, dim3(grid), dim3(kDecThreads), 0, st, prod, d_tab, RB, sA,
                             sB, n, bm, bn, cstar32, ldcs, partials, tpb, prod_stride);
     else
       return cudaErrorInvalidValue;
