@@ -430,14 +430,18 @@ def run_ours(args):
         ws3 = torch.empty(fmm.error_sweep_workspace(s1, d3, len(mine)), dtype=torch.uint8, device=dev)
         Cs = torch.empty((C3["M"], C3["N"]), dtype=torch.float64, device=dev)
         fmm.exact_gemm_f64(d3, A3, B3, Cs)
-        fmm.error_sweep(s1, 0, P[mine][:2], Q[mine][:2], S[mine][:2], d3, A3, B3, ws3, Cstar=Cs)   # warm-up
+        sweep_sampler = ClockSampler(local)
+        sweep_sampler.start()
+        fmm.error_sweep(s1, 0, P[mine][:16], Q[mine][:16], S[mine][:16], d3, A3, B3, ws3, Cstar=Cs)   # warm-up
         barrier()
+        t_sw0 = time.time()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         ratios, summ = fmm.error_sweep(s1, 0, P[mine], Q[mine], S[mine], d3, A3, B3, ws3, Cstar=Cs)
         e1.record()
         barrier()
         t_sweep = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+        sweep_clocks = sweep_sampler.stop(t_sw0, time.time())
         # phase table of the sweep: a second, event-instrumented pass over a few batches (stages back to back)
         sweep_phases = None
         if rank == 0:
@@ -468,7 +472,7 @@ def run_ours(args):
                  "min": float(srt[0]), "median": float(srt[G // 2]), "max": float(srt[-1]),
                  "count_gt2": int((full > 2).sum()), "e_classical_rel": summ["e_classical_rel"],
                  "includes": "classical product + its error, reference norm, G x (encode A, encode B, 7 products, decode+error)",
-                 "phases": sweep_phases}
+                 "phases": sweep_phases, "clocks": sweep_clocks}
         del ws3, Cs, A3, B3
 
     # ---- CPU oracle timed beside it (rank 0, N=1 only)
