@@ -40,6 +40,20 @@ def test_row_scale_and_unscale_are_exact(lib, dtype):
     assert torch.equal(Xp[:, :K], Y)
 
 
+@pytest.mark.parametrize("dtype,rows,K", [("bf16", 5, 100), ("bf16", 9, 11008), ("f32", 7, 8192), ("f32", 3, 50), ("bf16", 1, 8)])
+def test_row_scale_paths_for_short_long_and_unaligned_rows(lib, dtype, rows, K):
+    """Rows that are not a whole number of 16-byte vectors (scalar path), rows longer than the register-resident
+    limit (two passes over memory), and a single short row."""
+    X = gen.normal(2, K, (rows, K)) * np.exp2(gen.uniform(2, K + 1, (rows, 1), -6, 6))
+    Xt, X64 = gu.storage_pair(X, dtype)
+    Y, d = lib.row_pow2_scale(Xt)
+    want_d = oracle.row_pow2_scales(X64)
+    assert np.array_equal(d.double().cpu().numpy(), want_d)
+    assert np.array_equal(Y.double().cpu().numpy(), X64 / want_d[:, None])
+    lib.row_unscale(Y, d)
+    assert np.array_equal(Y.double().cpu().numpy(), X64)
+
+
 def _schemes(lib, name):
     st, cl = lib.scheme_builtin("strassen222"), lib.scheme_builtin("classical222")
     ost, ocl = oracle.strassen(), oracle.classical_scheme(2, 2, 2)

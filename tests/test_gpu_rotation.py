@@ -85,6 +85,16 @@ def test_large_operand_spans_many_waves_and_keeps_the_product(lib):
     assert np.array_equal(Y, want1)
 
 
+def test_single_row_and_single_block(lib):
+    for dtype, K, h in (("f32", 4, 4), ("bf16", 8, 8), ("bf16", 1024, 1024), ("f32", 2, 2)):
+        Xt, X64 = gu.storage_pair(gen.normal(4, K, (1, K)), dtype)
+        if (K * Xt.element_size()) % 16:
+            continue                                   # rows must be whole 16-byte vectors: checked elsewhere
+        Y = lib.hadamard_rotate(Xt, None, h)
+        want = oracle.hadamard_rotate(X64, np.ones(K), h, dtype if dtype == "bf16" else "f64")
+        assert gu.rel_fro(Y.to(torch.float64).cpu().numpy(), want) <= (1e-6 if dtype == "f32" else 4e-3)
+
+
 def test_argument_checks_launch_nothing(lib):
     X = torch.zeros((4, 64), dtype=torch.float32, device="cuda")
     for h in (0, 1, 3, 48, 2048):
