@@ -264,7 +264,11 @@ size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int
  * classical one does).
  * P, Q, S: HOST, G stacked row-major matrices (dimension of the gauged grid).  dCstar: DEVICE fp64
  * M x N reference, or NULL to have it computed.  h_ratios: HOST, G doubles (may be NULL).
- * out: HOST.  Synchronises the stream once before returning.                                */
+ * out: HOST.  Synchronises the stream once before returning.
+ * Execution: equivalent algorithms share their operands, so up to eight of them (as many as fit the table limits:
+ * products of the batch <= FMM_MAX_R) run as one encode, one product launch and one error-only decode; every
+ * algorithm's arithmetic and summation order are those of a scheme_gemm call on it, and the call is bit-reproducible
+ * run to run.  FMM_B200_NO_GAUGE_BATCH=1 in the environment runs one algorithm per launch set.              */
 fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P, const double* Q,
                        const double* S, const fmm_gemm_desc* d, const void* dA, const void* dB,
                        const double* dCstar, double* h_ratios, fmm_sweep_summary* out, void* d_ws,
