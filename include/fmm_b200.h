@@ -253,6 +253,21 @@ fmm_status error_frobenius_noalloc(const fmm_gemm_desc* d, const void* dC, const
                                    void* cuda_stream);
 int64_t error_frobenius_noalloc_max_elements(void);
 
+/* scheme_gemm for operands in HOST memory — the end-to-end form of the path (Eq. 1, Appendix B.1): on `cuda_stream`,
+ * A and B are copied into dense device buffers inside the workspace, scheme_gemm runs on them, and C is copied back.
+ * hA, hB, hC: HOST, laid out as d says (lda / ldb / ldc in elements; pinned memory makes the copies asynchronous and
+ * lets calls on different streams overlap; pageable memory works and serialises).  With FMM_FLAG_REUSE_BHAT the
+ * weight is neither copied nor encoded (hB may be NULL): the previous call on this workspace left its block sums.
+ * d_ws: DEVICE, >= scheme_gemm_host_workspace bytes (the three device copies plus a scheme_gemm workspace), 256-byte
+ * aligned, owned by the caller; one workspace per stream in flight.  The call only enqueues; hC is valid once the
+ * stream has been synchronised.  scheme_gemm_host_status synchronises the stream and reports the device status of
+ * the calls on this workspace (FMM_OK or FMM_ERR_TIMEOUT), as fmm_device_status does for scheme_gemm.
+ * Errors as scheme_gemm.                                                                                       */
+size_t scheme_gemm_host_workspace(const fmm_scheme* s, const fmm_gemm_desc* d);
+fmm_status scheme_gemm_host_status(const fmm_scheme* s, const fmm_gemm_desc* d, const void* d_ws, void* cuda_stream);
+fmm_status scheme_gemm_host(const fmm_scheme* s, const fmm_gemm_desc* d, const void* hA, const void* hB, void* hC,
+                            void* d_ws, size_t ws_bytes, void* cuda_stream);
+
 size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int G);
 
 /* Sweep over G gauge-equivalent copies of one scheme (Section 3.3 / Table 3, model-free form of

@@ -21,6 +21,7 @@ _DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
 EXPORTED_SYMBOLS = [
     "scheme_load", "scheme_builtin", "scheme_kron", "scheme_permute_products", "gauge_apply", "scheme_info", "scheme_coefficients",
     "scheme_free", "scheme_gemm_workspace", "scheme_gemm_workspace_layout", "scheme_gemm", "fmm_device_status",
+    "scheme_gemm_host_workspace", "scheme_gemm_host", "scheme_gemm_host_status",
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
@@ -85,6 +86,10 @@ _lib.scheme_gemm_workspace.argtypes = [_vp, C.POINTER(GemmDesc)]
 _lib.scheme_gemm_workspace.restype = _sz
 _lib.scheme_gemm_workspace_layout.argtypes = [_vp, C.POINTER(GemmDesc), C.POINTER(_sz)]
 _lib.scheme_gemm.argtypes = [_vp, C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.scheme_gemm_host_workspace.argtypes = [_vp, C.POINTER(GemmDesc)]
+_lib.scheme_gemm_host_workspace.restype = _sz
+_lib.scheme_gemm_host.argtypes = [_vp, C.POINTER(GemmDesc), _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.scheme_gemm_host_status.argtypes = [_vp, C.POINTER(GemmDesc), _vp, _vp]
 _lib.fmm_device_status.argtypes = [_vp, _vp]
 _lib.fmm_selftest_timeout.argtypes = [_vp, _sz, C.c_uint, _vp]
 _lib.classical_gemm_workspace.argtypes = [C.POINTER(GemmDesc)]
@@ -249,6 +254,21 @@ def error_sweep_workspace(s: Scheme, d: GemmDesc, G: int) -> int:
 def scheme_gemm(s: Scheme, d: GemmDesc, A, B, Cout, ws) -> None:
     _check(_lib.scheme_gemm(s.handle, C.byref(d), _ptr(A), _ptr(B), _ptr(Cout), _ptr(ws),
                             ws.numel() * ws.element_size(), _stream()), "scheme_gemm")
+
+
+def scheme_gemm_host_workspace(s: Scheme, d: GemmDesc) -> int:
+    return int(_lib.scheme_gemm_host_workspace(s.handle, C.byref(d)))
+
+
+def scheme_gemm_host(s: Scheme, d: GemmDesc, A_host, B_host, C_host, ws) -> None:
+    """scheme_gemm on HOST tensors (pinned for asynchronous copies): copies in, the path, copy out, on the current
+    stream; C_host is valid after the stream has been synchronised.  B_host may be None with FLAG_REUSE_BHAT."""
+    _check(_lib.scheme_gemm_host(s.handle, C.byref(d), _ptr(A_host), _ptr(B_host) if B_host is not None else None,
+                                 _ptr(C_host), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "scheme_gemm_host")
+
+
+def scheme_gemm_host_status(s: Scheme, d: GemmDesc, ws) -> None:
+    _check(_lib.scheme_gemm_host_status(s.handle, C.byref(d), _ptr(ws), _stream()), "scheme_gemm_host_status")
 
 
 def classical_gemm(d: GemmDesc, A, B, Cout, ws) -> None:

@@ -574,6 +574,61 @@ fmm_status scheme_joint_round_weights(const fmm_scheme* s, const fmm_gemm_desc* 
   return FMM_OK;
 }
 
+// ---- scheme_gemm on operands in HOST memory: copies in, the whole path, copy out, all on one stream
+namespace {
+struct HostLayout { size_t a, b, c, ws, total; fmm_gemm_desc dev; };
+HostLayout host_layout(const fmm_scheme* s, const fmm_gemm_desc* d) {
+  HostLayout L;
+  L.dev = *d;                      // the device copies are dense
+  L.dev.lda = d->K;
+  L.dev.ldb = d->b_is_weight_layout ? d->K : d->N;
+  L.dev.ldc = d->N;
+  const size_t es = (size_t)esize(d->storage), eo = (size_t)esize(d->output);
+  size_t o = 0;
+  L.a = o; o += align_up((size_t)d->M * d->K * es);
+  L.b = o; o += align_up((size_t)d->K * d->N * es);
+  L.c = o; o += align_up((size_t)d->M * d->N * eo);
+  L.ws = o; o += gemm_layout(s->m, s->k, s->n, s->R, &L.dev).total;
+  L.total = o;
+  return L;
+}
+}  // namespace
+
+size_t scheme_gemm_host_workspace(const fmm_scheme* s, const fmm_gemm_desc* d) {
+  if (!s || check_desc(d, s->m, s->k, s->n) != FMM_OK) return 0;
+  return host_layout(s, d).total;
+}
+
+fmm_status scheme_gemm_host(const fmm_scheme* s, const fmm_gemm_desc* d, const void* hA, const void* hB, void* hC,
+                            void* d_ws, size_t ws_bytes, void* cuda_stream) {
+  if (!s || !d || !hA || !hC) return FMM_ERR_ARG;
+  const bool reuse_b = (d->flags & FMM_FLAG_REUSE_BHAT) != 0;
+  if (!hB && !reuse_b) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, s->m, s->k, s->n));
+  const HostLayout L = host_layout(s, d);
+  FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t es = (size_t)esize(d->storage), eo = (size_t)esize(d->output);
+  char* ws = static_cast<char*>(d_ws);
+  FMM_CUDA(cudaMemcpy2DAsync(ws + L.a, (size_t)d->K * es, hA, (size_t)d->lda * es, (size_t)d->K * es, (size_t)d->M,
+                             cudaMemcpyHostToDevice, st));
+  if (!reuse_b) {
+    const size_t rows = d->b_is_weight_layout ? d->N : d->K, cols = d->b_is_weight_layout ? d->K : d->N;
+    FMM_CUDA(cudaMemcpy2DAsync(ws + L.b, cols * es, hB, (size_t)d->ldb * es, cols * es, rows, cudaMemcpyHostToDevice, st));
+  }
+  FMM_TRY(scheme_gemm(s, &L.dev, ws + L.a, ws + L.b, ws + L.c, ws + L.ws, ws_bytes - L.ws, cuda_stream));
+  FMM_CUDA(cudaMemcpy2DAsync(hC, (size_t)d->ldc * eo, ws + L.c, (size_t)d->N * eo, (size_t)d->N * eo, (size_t)d->M,
+                             cudaMemcpyDeviceToHost, st));
+  return FMM_OK;
+}
+
+fmm_status fmm_device_status(const void* d_ws, void* cuda_stream);
+fmm_status scheme_gemm_host_status(const fmm_scheme* s, const fmm_gemm_desc* d, const void* d_ws, void* cuda_stream) {
+  if (!s || !d_ws) return FMM_ERR_ARG;
+  FMM_TRY(check_desc(d, s->m, s->k, s->n));
+  return fmm_device_status(static_cast<const char*>(d_ws) + host_layout(s, d).ws, cuda_stream);
+}
+
 fmm_status fmm_device_status(const void* d_ws, void* cuda_stream) {
   if (!d_ws) return FMM_ERR_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -316,6 +316,33 @@ def test_sweep_log_uniform_gauges_bf16_and_outer_level_fp8(lib):
         assert abs(r - E / Ecl) <= TOL_RATIO * E / Ecl
 
 
+def test_host_buffer_entry_point_is_the_same_operator(lib):
+    """scheme_gemm_host: operands in (pinned) host memory with padded leading dimensions, result copied back; the
+    same bits as scheme_gemm on device tensors, also with the weight's block sums reused and no weight passed."""
+    M, K, N = 384, 320, 288
+    At, Bt, A64, B64 = _inputs(5, M, K, N, "bf16", "llm")
+    s = lib.scheme_builtin("strassen444")
+    want = gu.run_scheme_gemm(s, At, Bt, "bf16", "e4m3", "bf16", scale_mode=1)
+    lda, ldb, ldc = K + 8, N + 16, N + 24
+    Ah = torch.zeros((M, lda), dtype=torch.bfloat16).pin_memory(); Ah[:, :K] = At.cpu()
+    Bh = torch.zeros((K, ldb), dtype=torch.bfloat16).pin_memory(); Bh[:, :N] = Bt.cpu()
+    Ch = torch.full((M, ldc), 7.0, dtype=torch.bfloat16).pin_memory()
+    d = lib.GemmDesc.make(M, K, N, "bf16", "e4m3", "bf16", scale_mode=1)
+    d.lda, d.ldb, d.ldc = lda, ldb, ldc
+    ws = gu.workspace(lib.scheme_gemm_host_workspace(s, d))
+    lib.scheme_gemm_host(s, d, Ah, Bh, Ch, ws)
+    lib.scheme_gemm_host_status(s, d, ws)
+    assert np.array_equal(Ch[:, :N].double().numpy(), want) and torch.all(Ch[:, N:] == 7.0)
+    d2 = lib.GemmDesc.make(M, K, N, "bf16", "e4m3", "bf16", scale_mode=1, flags=lib.FLAG_REUSE_BHAT)
+    d2.lda, d2.ldb, d2.ldc = lda, ldb, ldc
+    Ch.fill_(0.0)
+    lib.scheme_gemm_host(s, d2, Ah, None, Ch, ws)
+    lib.scheme_gemm_host_status(s, d2, ws)
+    assert np.array_equal(Ch[:, :N].double().numpy(), want)
+    with pytest.raises(lib.FmmError):
+        lib.scheme_gemm_host(s, d, Ah, None, Ch, ws)             # no weight and nothing to reuse
+
+
 def test_sweep_batches_walk_several_tiles_per_block(lib):
     """Blocks of 512 x 1024 outputs: every decode block of the batched sweep walks four tiles, so the double-buffered
     stages (products and staged reference values) are reused; ratios against the oracle for 4 + 2 + 1 gauges."""

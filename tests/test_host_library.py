@@ -234,6 +234,21 @@ def test_repair_entry_points_validate_before_any_launch(lib):
     assert L.scheme_joint_round_weights(s1.handle, ctypes.byref(d3), x, 12, x, 16, None) == 6   # FMM_ERR_WORKSPACE
 
 
+def test_host_buffer_entry_point_validates_before_any_copy(lib):
+    L = lib.binding._lib
+    s2 = lib.scheme_builtin("strassen444")
+    d = lib.GemmDesc.make(256, 256, 256, "bf16", "bf16", "bf16")
+    x = ctypes.c_void_p(1 << 20)
+    need = lib.scheme_gemm_host_workspace(s2, d)
+    assert need > lib.scheme_gemm_workspace(s2, d) + 3 * 256 * 256 * 2 - 1
+    assert L.scheme_gemm_host(s2.handle, ctypes.byref(d), None, x, x, x, need, None) == 1       # FMM_ERR_ARG
+    assert L.scheme_gemm_host(s2.handle, ctypes.byref(d), x, None, x, x, need, None) == 1       # no weight, no reuse flag
+    assert L.scheme_gemm_host(s2.handle, ctypes.byref(d), x, x, x, x, need - 1, None) == 6      # FMM_ERR_WORKSPACE
+    bad = lib.GemmDesc.make(250, 256, 256, "bf16", "bf16", "bf16")
+    assert lib.scheme_gemm_host_workspace(s2, bad) == 0
+    assert L.scheme_gemm_host(s2.handle, ctypes.byref(bad), x, x, x, x, need, None) == 2        # FMM_ERR_SHAPE
+
+
 def test_permuted_products_are_the_same_algorithm(lib):
     """Renumbering the products keeps the Brent equations and every criterion; bad permutations are refused."""
     s2 = lib.scheme_builtin("strassen444")
