@@ -1073,17 +1073,20 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   const uint32_t bar_base = smem_u32(bar_mem);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };
+  // four accumulator buffers (all 512 TMEM columns): the MMAs of the next three groups run while the rescale warps wait
+  // for the tcgen05.ld of a finished one — that latency, not the arithmetic, sets the pace of this kernel
+  constexpr int kAcc = 4;
   auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };
-  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };
-  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + kAcc + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 2 * kAcc);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 2 * kAcc + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 2 * kAcc + 1) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr uint32_t kTmemCols = 2 * BN;
+  constexpr uint32_t kTmemCols = kAcc * BN;
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
+    for (int b = 0; b < kAcc; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1158,7 +1161,7 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
           tc_commit(empty_bar(stage));
           tc_commit(tfull_bar(acc));
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
         }
       }
       if (!ok) {
@@ -1203,7 +1206,7 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
 #pragma unroll
         for (int j = 0; j < PN; ++j) sum[j] = __fmaf_rn(__uint_as_float(v[j]), sc, sum[j]);
       }
