@@ -1189,13 +1189,16 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
       const int col_base = tn * BN + part * PN;
       const float* sa_row = p.sA + (long long)r * p.sa_batch + (long long)(row_ok ? row : 0) * p.G;
       const float* sb_blk = p.sB + (long long)r * p.sb_batch + (long long)tn * p.G;   // BN = 128 = one scale block of columns
-      float sum[PN];
+      float2 sum[PN / 2];
 #pragma unroll
-      for (int j = 0; j < PN; ++j) sum[j] = 0.0f;
+      for (int j = 0; j < PN / 2; ++j) sum[j] = make_float2(0.0f, 0.0f);
+      // the scales do not depend on the products: they are fetched two groups ahead of their use
       float s_next = row_ok ? sa_row[0] * sb_blk[0] : 0.0f;
+      float s_next2 = (row_ok && p.G > 1) ? sa_row[1] * sb_blk[1] : 0.0f;
       for (int g = 0; g < p.G; ++g) {
-        const float sc = s_next;      // the scales do not depend on the products: the next group's come a step ahead
-        if (g + 1 < p.G) s_next = row_ok ? sa_row[g + 1] * sb_blk[g + 1] : 0.0f;
+        const float sc = s_next;
+        s_next = s_next2;
+        if (g + 2 < p.G) s_next2 = row_ok ? sa_row[g + 2] * sb_blk[g + 2] : 0.0f;
         ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 0x93, status, p.wait_limit_ns);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -1207,14 +1210,16 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(acc));
         if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
+        const float2 sc2 = make_float2(sc, sc);
 #pragma unroll
-        for (int j = 0; j < PN; ++j) sum[j] = __fmaf_rn(__uint_as_float(v[j]), sc, sum[j]);
+        for (int j = 0; j < PN / 2; ++j)      // one fused multiply-add per element, two elements per instruction
+          sum[j] = __ffma2_rn(make_float2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), sc2, sum[j]);
       }
       if (!ok) break;
       if (row_ok && col_base < p.rows_b) {
         uint32_t w[32];
 #pragma unroll
-        for (int j = 0; j < PN; ++j) w[j] = __float_as_uint(sum[j]);
+        for (int j = 0; j < PN / 2; ++j) { w[2 * j] = __float_as_uint(sum[j].x); w[2 * j + 1] = __float_as_uint(sum[j].y); }
         store_row_chunk(out, (long long)r * p.o_batch + (long long)row * p.ldo + col_base, min(32, p.rows_b - col_base), w, 1,
                         p.out_bf16, 1.0f, p.wide != 0);
       }
