@@ -848,21 +848,22 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
   const uint32_t bar_base = smem_u32(bar_mem);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };
+  constexpr int kAcc = 4;   // accumulator buffers: all 512 TMEM columns, so the MMAs run up to three groups ahead of the rescale
   auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };
-  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };
-  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + kAcc + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 2 * kAcc);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 2 * kAcc + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 2 * kAcc + 1) + 8);
   float* scale_sm = reinterpret_cast<float*>(bar_mem + L::kBarBytes);   // [group][BN] column scales of the current tile
-  const uint32_t sfull_bar = bar_base + 8u * (2 * L::kStages + 7);      // the tile's scales are staged (16 warps arrive)
-  const uint32_t sempty_bar = bar_base + 8u * (2 * L::kStages + 8);     // the tile's scales are no longer read
+  const uint32_t sfull_bar = bar_base + 8u * (2 * L::kStages + 2 * kAcc + 3);   // the tile's scales are staged (16 warps arrive)
+  const uint32_t sempty_bar = bar_base + 8u * (2 * L::kStages + 2 * kAcc + 4);  // the tile's scales are no longer read
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr uint32_t kTmemCols = 2 * BN;
+  constexpr uint32_t kTmemCols = kAcc * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
+    for (int b = 0; b < kAcc; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 16); }
     mbar_init(drain_bar, 1);
     mbar_init(sfull_bar, 16); mbar_init(sempty_bar, 16);
     *abort_flag = 0;
@@ -936,7 +937,7 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
           tc_commit(empty_bar(stage));
           tc_commit(tfull_bar(acc));
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
-          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+          if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
         }
       }
       if (!ok) {
@@ -1001,7 +1002,7 @@ int8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_c
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAcc) { acc = 0; acc_phase ^= 1u; }
         const float2 da2 = make_float2(da, da);
         const float2 neg_magic = make_float2(-12582912.0f, -12582912.0f);
 #pragma unroll
