@@ -797,13 +797,17 @@ def int8_workload(fmm, gen, torch, timed, peaks):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: 100; 5 for --impl reference, whose steps take most of a second)")
+    ap.add_argument("--warmup", type=int, default=None, help="untimed warm-up steps (default: 5; 1 for --impl reference)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep-gauges", type=int, default=512, help="gauges per rank in the c3 sweep (0 = skip); config 3 names 512")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="c2", help="c2 (default: the benchmark line) | c1 | c4 | c4m | c5 | int8 | ensemble | rotation | repairs")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 5 if args.impl == "reference" else 100
+    if args.warmup is None:
+        args.warmup = 1 if args.impl == "reference" else 5
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
