@@ -316,6 +316,48 @@ def test_sweep_log_uniform_gauges_bf16_and_outer_level_fp8(lib):
         assert abs(r - E / Ecl) <= TOL_RATIO * E / Ecl
 
 
+@pytest.mark.parametrize("Pd,scale", [("bf16", 0), ("e4m3", 1), ("e4m3", 2), ("e4m3", 3)])
+def test_all_zero_operands(lib, Pd, scale):
+    """Degenerate input: an all-zero operand gives scales of one (no division by a zero maximum), a zero product, and
+    a ratio of 1 in the sweep (both errors vanish)."""
+    M, K, N = 256, 512, 384
+    At, Bt, A64, B64 = _inputs(13, M, K, N, "bf16", "llm")
+    Z = torch.zeros_like(At)
+    s, so = lib.scheme_builtin("strassen444"), gu.oracle_scheme("strassen444")
+    C, p, _ = gu.run_scheme_gemm(s, Z, Bt, "bf16", Pd, "bf16", scale_mode=scale, parts=True)
+    Co, po = oracle.scheme_gemm(so, np.zeros_like(A64), B64, pd=Pd, od="bf16", scale_mode=scale, parts=True)
+    assert np.all(C == 0.0) and np.all(Co == 0.0)
+    assert np.all(p["Ahat"] == 0.0) and np.array_equal(p["BhatT"], po["Bhat"].transpose(0, 2, 1))
+    if scale:
+        assert np.all(p["sA"] == 1.0) and np.array_equal(p["sA"], po["sA"]) and np.array_equal(p["sB"], po["sB"])
+    d = lib.GemmDesc.make(M, K, N, "bf16", Pd, "bf16", scale_mode=scale)
+    I4 = np.eye(4)[None]
+    ws = gu.workspace(lib.error_sweep_workspace(s, d, 1))
+    ratios, summ = lib.error_sweep(s, 0, I4, I4, I4, d, Z, Bt, ws)
+    assert ratios[0] == 1.0 and summ["e_classical_rel"] == 0.0 and summ["norm_ref"] == 0.0
+
+
+def test_one_product_scheme_and_nan_containment(lib):
+    """<1,1,1;1> (one product, no block sums) and <2,2,2;8> are the classical algorithm written as schemes: every step
+    against the oracle.  A NaN in one block of A reaches exactly the outputs the oracle says it reaches: products whose
+    block sum does not read that block are untouched (zero coefficients are skipped, not multiplied)."""
+    At, Bt, A64, B64 = _inputs(14, 256, 256, 256, "bf16", "normal")
+    for name, so in (("classical111", oracle.classical_scheme(1, 1, 1)), ("classical222", oracle.classical_scheme(2, 2, 2))):
+        s = lib.scheme_builtin(name)
+        C, p, _ = gu.run_scheme_gemm(s, At, Bt, "bf16", "bf16", "f32", parts=True)
+        Co, po = oracle.scheme_gemm(so, A64, B64, pd="bf16", od="f32", parts=True)
+        assert np.array_equal(p["Ahat"], po["Ahat"]) and gu.rel_fro(p["M"], po["M"]) <= 1e-5 and gu.rel_fro(C, Co) <= TOL_FRO
+    An = At.clone(); An[3, 200] = float("nan")                 # block (0, 1) of a 2 x 2 grid
+    A64n = A64.copy(); A64n[3, 200] = np.nan
+    s1, o1 = lib.scheme_builtin("strassen222"), oracle.strassen()
+    C = gu.run_scheme_gemm(s1, An, Bt, "bf16", "bf16", "f32")
+    Co = oracle.scheme_gemm(o1, A64n, B64, "bf16", "f32")
+    assert np.array_equal(np.isnan(C), np.isnan(Co))
+    assert 0 < np.isnan(Co).sum() < Co.size                    # row 3 of the blocks fed by products that read A_12, nothing else
+    ok = ~np.isnan(Co)
+    assert gu.rel_fro(C[ok], Co[ok]) <= TOL_FRO
+
+
 def test_host_buffer_entry_point_is_the_same_operator(lib):
     """scheme_gemm_host: operands in (pinned) host memory with padded leading dimensions, result copied back; the
     same bits as scheme_gemm on device tensors, also with the weight's block sums reused and no weight passed."""
