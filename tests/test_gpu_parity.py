@@ -358,6 +358,31 @@ def test_one_product_scheme_and_nan_containment(lib):
     assert gu.rel_fro(C[ok], Co[ok]) <= TOL_FRO
 
 
+@pytest.mark.parametrize("scheme,M,K,N", [("strassen444", 4, 64, 32), ("strassen222", 2, 32, 16), ("strassen444", 12, 192, 96)])
+@pytest.mark.parametrize("Pd,scale", [("bf16", 0), ("e4m3", 1), ("e4m3", 3)])
+def test_smallest_legal_shapes(lib, scheme, M, K, N, Pd, scale):
+    """One row per block, sixteen inner indices, eight columns: far below one tile in every dimension."""
+    At, Bt, A64, B64 = _inputs(15, M, K, N, "bf16", "normal")
+    s, so = lib.scheme_builtin(scheme), gu.oracle_scheme(scheme)
+    C, p, _ = gu.run_scheme_gemm(s, At, Bt, "bf16", Pd, "f32", scale_mode=scale, parts=True)
+    Co, po = oracle.scheme_gemm(so, A64, B64, pd=Pd, od="f32", scale_mode=scale, parts=True)
+    assert np.array_equal(p["Ahat"], po["Ahat"]) and np.array_equal(p["BhatT"], po["Bhat"].transpose(0, 2, 1))
+    assert gu.rel_fro(p["M"], po["M"]) <= 1e-5 and gu.rel_fro(C, Co) <= TOL_FRO
+    m = so.dims[0]
+    # the sweep with bf16 outputs: with bf16 storage and products the classical error is the output rounding alone
+    d = lib.GemmDesc.make(M, K, N, "bf16", Pd, "bf16", scale_mode=scale)
+    G = 5
+    var = oracle.sign_variants(m, m, m)[:G]
+    P = np.stack([np.diag(v[0]) for v in var]); Q = np.stack([np.diag(v[1]) for v in var]); S = np.stack([np.diag(v[2]) for v in var])
+    ws = gu.workspace(lib.error_sweep_workspace(s, d, G))
+    ratios, _ = lib.error_sweep(s, 0, P, Q, S, d, At, Bt, ws)
+    Cs = A64 @ B64
+    Ecl = oracle.rel_error(oracle.classical_gemm(A64, B64, Pd, "bf16", scale), Cs)
+    for r, v in zip(ratios, var):
+        E = oracle.rel_error(oracle.scheme_gemm(oracle.sign_variant(so, *v), A64, B64, Pd, "bf16", scale), Cs)
+        assert abs(r - E / Ecl) <= TOL_RATIO * E / Ecl
+
+
 def test_host_buffer_entry_point_is_the_same_operator(lib):
     """scheme_gemm_host: operands in (pinned) host memory with padded leading dimensions, result copied back; the
     same bits as scheme_gemm on device tensors, also with the weight's block sums reused and no weight passed."""
