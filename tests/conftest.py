@@ -13,6 +13,12 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
+    # a per-test limit, so that a stuck test cannot eat a whole run (every device-side wait of the library is bounded
+    # to seconds, so a healthy test never comes near it)
+    if config.pluginmanager.hasplugin("timeout"):
+        for it in items:
+            if it.get_closest_marker("timeout") is None:
+                it.add_marker(pytest.mark.timeout(600))
     try:
         import torch
         has_gpu = torch.cuda.is_available()
