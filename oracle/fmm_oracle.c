@@ -18,10 +18,20 @@
  *
  * Precision choices (each is a stated reading, the paper being silent):
  *   - coefficients are held in fp64 and used as (double)(float)c;
- *   - a block sum is the decision that produces a quantised code, so it is formed
- *     in the precision the kernel uses: an fp32 fused-multiply-add chain over the
- *     nonzero coefficients in ascending row-major (i,l) order, then ONE rounding to
- *     the product dtype (after an exact power-of-two scale for e4m3);
+ *   - a block sum has two selectable forms (sum_mode).  ORC_SUM_F64 is the definition:
+ *     the sum of the products (double)(float)u * a over the nonzero coefficients,
+ *     carried in fp64 (exact for every input used here up to one fp64 rounding), then
+ *     ONE rounding to the product dtype.  ORC_SUM_F32CHAIN is the reading that lets the
+ *     quantised codes be compared bit for bit with a device that works in fp32: an
+ *     fp32 fused-multiply-add chain over the nonzero coefficients in ascending
+ *     row-major (i,l) order, then the one rounding (after an exact power-of-two scale
+ *     for e4m3).  The two differ only where the fp32 chain rounds before the product
+ *     dtype does (double rounding); tests measure how many codes that moves;
+ *   - nested algorithms are applied FLAT (the Kronecker coefficients, one rounding of
+ *     each block sum) unless orc_scheme_gemm_per_level is called, which rounds the
+ *     outer level's block sums to the product dtype, forms the inner level's block
+ *     sums of those rounded values and rounds again ("applied to its own blocks",
+ *     Section 1, taken literally);
  *   - products, decode, classical and exact references accumulate in fp64, in
  *     ascending inner index t and ascending product index r;
  *   - with product dtype "f64" nothing is rounded at all (exact-arithmetic mode,
@@ -54,6 +64,7 @@
 #endif
 
 enum { ORC_F32 = 0, ORC_BF16 = 1, ORC_E4M3 = 2, ORC_F64 = 3 };
+enum { ORC_SUM_F32CHAIN = 0, ORC_SUM_F64 = 1 };
 
 /* Thread count of the OpenMP loops (tiny problems run faster on one thread; the arithmetic is the same). */
 void orc_set_num_threads(int n) {
@@ -305,8 +316,8 @@ void orc_criteria(int m, int k, int n, int R, const double* U, const double* V, 
 /* One block sum, Eq. 1 inner parentheses: out[p][t] = sum_x coef[x] * blk_x[p][t] over the
  * nonzero coefficients in ascending x (row-major over the block grid).
  * src is the whole matrix (ld elements per row); block x = (x / gc, x % gc) of a grid with gc
- * block columns, block size br x bc.  f32chain selects the fp32 FMA chain (quantised modes) or
- * a plain fp64 sum (exact mode).                                                   */
+ * block columns, block size br x bc.  f32chain selects the fp32 FMA chain (ORC_SUM_F32CHAIN in a
+ * quantised mode); otherwise the sum is carried in fp64 (the definition, and the exact mode).   */
 static void block_sum(const double* src, int64_t ld, int gr, int gc, int64_t br, int64_t bc,
                       const double* coef, int f32chain, double* out) {
 #pragma omp parallel for schedule(static)
@@ -426,7 +437,7 @@ static int scheme_gemm_impl(int m, int k, int n, int R, const double* U, const d
                     int64_t M, int64_t K, int64_t N, const double* A, const double* B,
                     int pd, int od, int scale_mode, double* C,
                     double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
-                    double* M_out, int md, const double* Bq_in, const double* sB_in) {
+                    double* M_out, int md, const double* Bq_in, const double* sB_in, int sum_mode) {
   if (M % m || K % k || N % n) return 1;
   if (Bq_in && scale_mode != 3) return 1;
   int64_t bm = M / m, bk = K / k, bn = N / n;
@@ -444,8 +455,9 @@ static int scheme_gemm_impl(int m, int k, int n, int R, const double* U, const d
     for (int x = 0; x < m * k; ++x) cu[x] = quant ? (double)(float)U[r * m * k + x] : U[r * m * k + x];
     for (int x = 0; x < k * n; ++x) cv[x] = quant ? (double)(float)V[r * k * n + x] : V[r * k * n + x];
     /* encode: block sums, scale, one rounding to the product dtype */
-    block_sum(A, K, m, k, bm, bk, cu, quant, Ah);
-    block_sum(B, N, k, n, bk, bn, cv, quant, Bh);
+    const int chain = quant && sum_mode == ORC_SUM_F32CHAIN;
+    block_sum(A, K, m, k, bm, bk, cu, chain, Ah);
+    block_sum(B, N, k, n, bk, bn, cv, chain, Bh);
     double sa = 1.0, sb = 1.0;
     if (scale_mode == 1) { sa = pow2_scale_448(Ah, bm * bk); sb = pow2_scale_448(Bh, bk * bn); }
     if (scale_mode == 2) {
@@ -522,7 +534,95 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
                     double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
                     double* M_out, int md) {
   return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, scale_mode, C, Ahat_out, Bhat_out, sA_out,
-                          sB_out, M_out, md, NULL, NULL);
+                          sB_out, M_out, md, NULL, NULL, ORC_SUM_F32CHAIN);
+}
+
+/* The same with the form of the block sum chosen by the caller (ORC_SUM_F32CHAIN / ORC_SUM_F64).              */
+int orc_scheme_gemm_sum(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                        int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                        int pd, int od, int scale_mode, double* C,
+                        double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out,
+                        double* M_out, int md, int sum_mode) {
+  return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, scale_mode, C, Ahat_out, Bhat_out, sA_out,
+                          sB_out, M_out, md, NULL, NULL, sum_mode);
+}
+
+/* A nested algorithm (outer <m1,k1,n1;R1> applied to blocks that the inner <m2,k2,n2;R2> multiplies) with the
+ * block sums rounded AT EVERY LEVEL: for each outer product r1 the outer block sum of A (M/m1 x K/k1) is scaled
+ * (scale_mode 1: one power-of-two scale for this tensor) and rounded to pd; the inner block sums are formed of
+ * those rounded values, scaled again (their own power-of-two scale, in units of the outer codes) and rounded to
+ * pd again; likewise for B.  The product r = r1 R2 + r2 multiplies the twice-rounded operands, and the
+ * combination is the flat one: C_{(I,i),(J,j)} = sum_r (float)(w1_{r1,IJ} w2_{r2,ij}) sA_r sB_r M_r in ascending
+ * r, one rounding to od, with sA_r = (outer scale)(inner scale).  scale_mode 0 or 1 only.  pd = ORC_F64 rounds
+ * nothing and equals the flat algorithm.  Optional outputs as orc_scheme_gemm (Ahat [R][bm][bk], ..., sA[R]).   */
+int orc_scheme_gemm_per_level(int m1, int k1, int n1, int R1, const double* U1, const double* V1, const double* W1,
+                              int m2, int k2, int n2, int R2, const double* U2, const double* V2, const double* W2,
+                              int64_t M, int64_t K, int64_t N, const double* A, const double* B,
+                              int pd, int od, int scale_mode, int sum_mode, double* C,
+                              double* Ahat_out, double* Bhat_out, double* sA_out, double* sB_out, double* M_out) {
+  const int m = m1 * m2, k = k1 * k2, n = n1 * n2;
+  if (M % m || K % k || N % n) return 1;
+  if (scale_mode != 0 && scale_mode != 1) return 1;
+  const int64_t Bm = M / m1, Bk = K / k1, Bn = N / n1;      /* outer blocks */
+  const int64_t bm = M / m, bk = K / k, bn = N / n;          /* inner blocks */
+  const int quant = (pd != ORC_F64);
+  const int chain = quant && sum_mode == ORC_SUM_F32CHAIN;
+  double cu[256], cv[256];
+  if (m1 * k1 > 256 || k1 * n1 > 256 || m2 * k2 > 256 || k2 * n2 > 256) return 1;
+  double* A1 = (double*)malloc(sizeof(double) * Bm * Bk);
+  double* B1 = (double*)malloc(sizeof(double) * Bk * Bn);
+  double* Ah = (double*)malloc(sizeof(double) * bm * bk);
+  double* Bh = (double*)malloc(sizeof(double) * bk * bn);
+  double* Mr = (double*)malloc(sizeof(double) * bm * bn);
+  double* acc = (double*)calloc((size_t)M * N, sizeof(double));
+  for (int r1 = 0; r1 < R1; ++r1) {
+    /* outer level: block sums of the operands themselves, one rounding */
+    for (int x = 0; x < m1 * k1; ++x) cu[x] = quant ? (double)(float)U1[r1 * m1 * k1 + x] : U1[r1 * m1 * k1 + x];
+    for (int x = 0; x < k1 * n1; ++x) cv[x] = quant ? (double)(float)V1[r1 * k1 * n1 + x] : V1[r1 * k1 * n1 + x];
+    block_sum(A, K, m1, k1, Bm, Bk, cu, chain, A1);
+    block_sum(B, N, k1, n1, Bk, Bn, cv, chain, B1);
+    double sa1 = 1.0, sb1 = 1.0;
+    if (scale_mode == 1) { sa1 = pow2_scale_448(A1, Bm * Bk); sb1 = pow2_scale_448(B1, Bk * Bn); }
+    if (quant) {
+      for (int64_t x = 0; x < Bm * Bk; ++x) A1[x] = orc_round(A1[x] / sa1, pd);
+      for (int64_t x = 0; x < Bk * Bn; ++x) B1[x] = orc_round(B1[x] / sb1, pd);
+    }
+    for (int r2 = 0; r2 < R2; ++r2) {
+      const int r = r1 * R2 + r2;
+      /* inner level: block sums of the rounded outer sums, rounded again */
+      for (int x = 0; x < m2 * k2; ++x) cu[x] = quant ? (double)(float)U2[r2 * m2 * k2 + x] : U2[r2 * m2 * k2 + x];
+      for (int x = 0; x < k2 * n2; ++x) cv[x] = quant ? (double)(float)V2[r2 * k2 * n2 + x] : V2[r2 * k2 * n2 + x];
+      block_sum(A1, Bk, m2, k2, bm, bk, cu, chain, Ah);
+      block_sum(B1, Bn, k2, n2, bk, bn, cv, chain, Bh);
+      double sa2 = 1.0, sb2 = 1.0;
+      if (scale_mode == 1) { sa2 = pow2_scale_448(Ah, bm * bk); sb2 = pow2_scale_448(Bh, bk * bn); }
+      if (quant) {
+        for (int64_t x = 0; x < bm * bk; ++x) Ah[x] = orc_round(Ah[x] / sa2, pd);
+        for (int64_t x = 0; x < bk * bn; ++x) Bh[x] = orc_round(Bh[x] / sb2, pd);
+      }
+      const double sa = sa1 * sa2, sb = sb1 * sb2;
+      if (sA_out) sA_out[r] = sa;
+      if (sB_out) sB_out[r] = sb;
+      if (Ahat_out) memcpy(Ahat_out + (size_t)r * bm * bk, Ah, sizeof(double) * bm * bk);
+      if (Bhat_out) memcpy(Bhat_out + (size_t)r * bk * bn, Bh, sizeof(double) * bk * bn);
+      matmul_f64(Ah, Bh, Mr, bm, bk, bn);
+      if (M_out) memcpy(M_out + (size_t)r * bm * bn, Mr, sizeof(double) * bm * bn);
+      for (int I = 0; I < m1; ++I) for (int i = 0; i < m2; ++i)
+        for (int J = 0; J < n1; ++J) for (int j = 0; j < n2; ++j) {
+          const double w12 = W1[(r1 * m1 + I) * n1 + J] * W2[(r2 * m2 + i) * n2 + j];
+          const double w = quant ? (double)(float)w12 : w12;
+          if (w == 0.0) continue;
+          const double ws = w * (sa * sb);
+          const int64_t row0 = ((int64_t)I * m2 + i) * bm, col0 = ((int64_t)J * n2 + j) * bn;
+#pragma omp parallel for schedule(static)
+          for (int64_t p = 0; p < bm; ++p)
+            for (int64_t q = 0; q < bn; ++q) acc[(row0 + p) * N + col0 + q] += ws * Mr[p * bn + q];
+        }
+    }
+  }
+  for (int64_t x = 0; x < M * N; ++x) C[x] = orc_round(acc[x], od);
+  free(A1); free(B1); free(Ah); free(Bh); free(Mr); free(acc);
+  return 0;
 }
 
 /* The same under the model schedule (scale_mode 3) with the weight side given as codes Bq [R][bk][bn] and scales
@@ -530,7 +630,8 @@ int orc_scheme_gemm(int m, int k, int n, int R, const double* U, const double* V
 int orc_scheme_gemm_weights(int m, int k, int n, int R, const double* U, const double* V, const double* W,
                             int64_t M, int64_t K, int64_t N, const double* A, const double* B,
                             int pd, int od, double* C, double* M_out, int md, const double* Bq, const double* sBq) {
-  return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, 3, C, NULL, NULL, NULL, NULL, M_out, md, Bq, sBq);
+  return scheme_gemm_impl(m, k, n, R, U, V, W, M, K, N, A, B, pd, od, 3, C, NULL, NULL, NULL, NULL, M_out, md, Bq, sBq,
+                          ORC_SUM_F32CHAIN);
 }
 
 /* Classical product at the same dtypes (the control): operands rounded to the product

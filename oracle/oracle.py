@@ -27,7 +27,7 @@ _FMT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3, "f64": F64, "fp64":
 __all__ = [
     "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "set_num_threads", "round_to", "strassen",
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
-    "criteria", "scheme_gemm", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
+    "criteria", "scheme_gemm", "scheme_gemm_per_level", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
     "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "certificate",
     "hadamard_matrix", "hadamard_rotate", "row_pow2_scales", "joint_round_weights", "scheme_gemm_weights",
 ]
@@ -65,6 +65,12 @@ def _L():
         lib.orc_scheme_gemm.restype = C.c_int
         lib.orc_scheme_gemm.argtypes = ([C.c_int] * 4 + [dp] * 3 + [i64] * 3 + [dp] * 2 +
                                         [C.c_int] * 3 + [dp] * 6 + [C.c_int])
+        lib.orc_scheme_gemm_sum.restype = C.c_int
+        lib.orc_scheme_gemm_sum.argtypes = ([C.c_int] * 4 + [dp] * 3 + [i64] * 3 + [dp] * 2 +
+                                            [C.c_int] * 3 + [dp] * 6 + [C.c_int] * 2)
+        lib.orc_scheme_gemm_per_level.restype = C.c_int
+        lib.orc_scheme_gemm_per_level.argtypes = ([C.c_int] * 4 + [dp] * 3 + [C.c_int] * 4 + [dp] * 3 + [i64] * 3 +
+                                                  [dp] * 2 + [C.c_int] * 4 + [dp] * 6)
         lib.orc_classical_gemm.restype = C.c_int
         lib.orc_classical_gemm.argtypes = [i64] * 3 + [dp] * 2 + [C.c_int] * 3 + [dp]
         lib.orc_exact_gemm.argtypes = [i64] * 3 + [dp] * 3
@@ -228,9 +234,16 @@ def criteria(s: Scheme) -> dict:
     return dict(zip(keys, meta.tolist()))
 
 
-def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts: bool = False, md="f64"):
+_SUM = {"f32chain": 0, "f64": 1}
+
+
+def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts: bool = False, md="f64",
+                sum: str = "f32chain"):
     """Apply the algorithm with block sums rounded to ``pd``; returns C (values of ``od``).  ``md``: dtype each
     product is rounded to before the combination ("f64": none; "bf16": the paper's model schedule).
+    ``sum``: how a block sum is formed before its one rounding — "f64": the definition (fp64 sum of the products
+    coefficient x entry); "f32chain": an fp32 fused-multiply-add chain in ascending block order, the reading under
+    which quantised codes can be compared bit for bit with fp32 hardware.
     With ``parts`` also returns dict(Ahat, Bhat, sA, sB, M)."""
     m, k, n, R = s.dims
     A = _d(A); B = _d(B)
@@ -245,11 +258,41 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
         G3, CB3 = -(-bk // 128), -(-bn // 128)
         sA = np.empty({2: (R, bm), 3: (R, bm, G3)}.get(scale_mode, (R,)))
         sB = np.empty({2: (R, bn), 3: (R, CB3, G3)}.get(scale_mode, (R,)))
-    rc = _L().orc_scheme_gemm(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
-                              _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
-                              _p(sB), _p(Mr), _fmt(md))
+    rc = _L().orc_scheme_gemm_sum(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), M, K, N, _p(A), _p(B),
+                                  _fmt(pd), _fmt(od), int(scale_mode), _p(Cm), _p(Ah), _p(Bh), _p(sA),
+                                  _p(sB), _p(Mr), _fmt(md), _SUM[sum])
     if rc:
         raise ValueError("matrix dimensions are not divisible by the block grid")
+    if parts:
+        return Cm, dict(Ahat=Ah, Bhat=Bh, sA=sA, sB=sB, M=Mr)
+    return Cm
+
+
+def scheme_gemm_per_level(outer: Scheme, inner: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0,
+                          parts: bool = False, sum: str = "f32chain"):
+    """The nested algorithm outer (x) inner with the block sums rounded at EVERY level: the outer level's block
+    sums are rounded to ``pd``, the inner level's block sums are formed of those rounded values and rounded again
+    (Section 1, "applied to its own blocks", taken literally).  ``kron(outer, inner)`` through ``scheme_gemm`` is
+    the flat reading (one rounding of each of the R1 R2 block sums).  scale_mode 0 or 1."""
+    m1, k1, n1, R1 = outer.dims
+    m2, k2, n2, R2 = inner.dims
+    m, k, n, R = m1 * m2, k1 * k2, n1 * n2, R1 * R2
+    A = _d(A); B = _d(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    Cm = np.empty((M, N))
+    Ah = Bh = sA = sB = Mr = None
+    if parts:
+        bm, bk, bn = M // m, K // k, N // n
+        Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
+        sA = np.empty((R,)); sB = np.empty((R,))
+    rc = _L().orc_scheme_gemm_per_level(m1, k1, n1, R1, _p(_d(outer.U)), _p(_d(outer.V)), _p(_d(outer.W)),
+                                        m2, k2, n2, R2, _p(_d(inner.U)), _p(_d(inner.V)), _p(_d(inner.W)),
+                                        M, K, N, _p(A), _p(B), _fmt(pd), _fmt(od), int(scale_mode), _SUM[sum],
+                                        _p(Cm), _p(Ah), _p(Bh), _p(sA), _p(sB), _p(Mr))
+    if rc:
+        raise ValueError("dimensions not divisible by the block grid, or unsupported scale mode")
     if parts:
         return Cm, dict(Ahat=Ah, Bhat=Bh, sA=sA, sB=sB, M=Mr)
     return Cm

@@ -46,6 +46,30 @@ def test_builtin_schemes_match_oracle_tables(lib):
     assert lib.scheme_builtin("strassen444").info["Phi"] == 1024.0
 
 
+def _golden(name):
+    out = {}
+    with open(os.path.join(ROOT, "tests", "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                k, *v = line.split()
+                out[k] = [float(x) for x in v]
+    return out
+
+
+def test_scheme_info_against_printed_and_hand_derived_constants(lib):
+    """All eight metadata entries of scheme_info against the golden files (printed constants; Q and E evaluated by
+    hand from the printed product table), not against the oracle."""
+    g, h = _golden("two_level_strassen_constants.txt"), _golden("ballard_criteria_hand.txt")
+    two = lib.scheme_builtin("strassen444").info
+    for key in ("L_A", "L_B", "L_W", "Phi", "nnz", "maxabs"):
+        assert two[key] == g[key][0], key
+    assert two["Q"] == h["Q_two_level"][0] and two["E"] == h["E_two_level"][0]
+    one = lib.scheme_builtin("strassen222").info
+    assert one["Q"] == h["Q_one_level"][0] and one["E"] == h["E_one_level"][0]
+    assert (one["L_A"], one["L_B"], one["L_W"], one["nnz"], one["maxabs"]) == (2.0, 2.0, 4.0, 36.0, 1.0)
+
+
 def test_scheme_load_checks_brent(lib):
     o = oracle.strassen()
     s = lib.scheme_load(o.U, o.V, o.W)

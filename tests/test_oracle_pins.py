@@ -71,6 +71,11 @@ def test_printed_constants_two_level():
     assert h == g["h_max_int32"][0]
     assert round(127 / b, 4) == g["step_ratio"][0]
     assert len(oracle.sign_variants(4, 4, 4)) == g["sign_variants"][0]
+    # the two remaining metadata entries: hand-evaluated from the printed product table (the paper prints no value)
+    h = _golden("ballard_criteria_hand.txt")
+    assert c["Q"] == h["Q_two_level"][0] and c["E"] == h["E_two_level"][0]
+    c1 = oracle.criteria(S1)
+    assert c1["Q"] == h["Q_one_level"][0] and c1["E"] == h["E_one_level"][0]
 
 
 def test_strassen_reads_feeds_table():
