@@ -87,6 +87,12 @@ typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
                                  is rounded (the power-of-two scales commute with the rounding); with
                                  scale_mode 2 the rounding follows the row / column scales.            */
 
+#define FMM_FLAG_SWEEP_SERIAL 4 /* error_sweep only: run the stages of every gauge back to back on the caller's
+                                 stream instead of pipelining consecutive gauges over the library's helper
+                                 streams.  Same results bit for bit (the arithmetic and the order of every sum
+                                 are the same); slower.  For callers that want one stream only, and for checking
+                                 the pipelined path against.                                              */
+
 /* The float-path "quantisation specification" (Section 2.2 treats these choices as part of the
  * operator): shapes, dtypes, layout of B, scale rule. */
 typedef struct {
@@ -245,7 +251,8 @@ fmm_status error_frobenius(const fmm_gemm_desc* d, const void* dC, const double*
  *   - Size limit: M * N <= error_frobenius_noalloc_max_elements() (67,108,864); larger problems return
  *     FMM_ERR_LIMIT and nothing is launched.
  *   - First call on a device: looks up the array's device address (once per device, with that device
- *     current).  Make that first call outside any stream capture.
+ *     current).  Make that first call outside any stream capture.  The address is kept for the life of the
+ *     process and does not survive a cudaDeviceReset of that device.
  *   - All calls on a device share the one array.  Nothing in it needs clearing between calls (each block
  *     overwrites its own slot), but two calls whose kernels overlap on the GPU — different streams without an
  *     ordering between them — race on it: order such calls yourself.                                        */
@@ -280,6 +287,11 @@ size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int
  * P, Q, S: HOST, G stacked row-major matrices (dimension of the gauged grid).  dCstar: DEVICE fp64
  * M x N reference, or NULL to have it computed.  h_ratios: HOST, G doubles (may be NULL).
  * out: HOST.  Synchronises the stream once before returning.
+ * Errors: every gauge matrix is inverted on the host before anything is enqueued, so FMM_ERR_SINGULAR leaves the
+ * device untouched; a failure after that point returns only once the caller's stream is ordered behind all work the
+ * call enqueued on the library's helper streams (the workspace may then be reused or freed in stream order).
+ * NaN: ratios of operands that hold NaN are NaN; if any ratio is NaN, min / median / max / spread are NaN and
+ * count_gt2 counts the comparable ratios above 2.
  * Execution: equivalent algorithms share their operands, so up to eight of them (as many as fit the table limits:
  * products of the batch <= FMM_MAX_R) run as one encode, one product launch and one error-only decode; every
  * algorithm's arithmetic and summation order are those of a scheme_gemm call on it, and the call is bit-reproducible

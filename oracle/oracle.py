@@ -244,7 +244,7 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
     ``sum``: how a block sum is formed before its one rounding — "f64": the definition (fp64 sum of the products
     coefficient x entry); "f32chain": an fp32 fused-multiply-add chain in ascending block order, the reading under
     which quantised codes can be compared bit for bit with fp32 hardware.
-    With ``parts`` also returns dict(Ahat, Bhat, sA, sB, M)."""
+    With ``parts`` also returns dict(Ahat, Bhat, sA, sB, M); ``parts="scales"`` fills only sA and sB."""
     m, k, n, R = s.dims
     A = _d(A); B = _d(B)
     M, K = A.shape
@@ -254,7 +254,8 @@ def scheme_gemm(s: Scheme, A, B, pd="bf16", od="f32", scale_mode: int = 0, parts
     Ah = Bh = sA = sB = Mr = None
     if parts:
         bm, bk, bn = M // m, K // k, N // n
-        Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
+        if parts != "scales":      # "scales": only the scale arrays (full-size problems, where the rest is gigabytes)
+            Ah = np.empty((R, bm, bk)); Bh = np.empty((R, bk, bn)); Mr = np.empty((R, bm, bn))
         G3, CB3 = -(-bk // 128), -(-bn // 128)
         sA = np.empty({2: (R, bm), 3: (R, bm, G3)}.get(scale_mode, (R,)))
         sB = np.empty({2: (R, bn), 3: (R, CB3, G3)}.get(scale_mode, (R,)))
@@ -340,8 +341,13 @@ def error_ratio(E_scheme: float, E_classical: float) -> float:
 
 def summary(ratios) -> dict:
     """Smallest, median (upper of the two middle values when the count is even, Table 3
-    caption), largest, spread = largest/smallest, and the number of ratios above 2."""
-    r = np.sort(np.asarray(ratios, dtype=np.float64))
+    caption), largest, spread = largest/smallest, and the number of ratios above 2.  A set that holds NaN has no
+    order: its smallest, median, largest and spread are NaN; the count is over the comparable ratios."""
+    r = np.asarray(ratios, dtype=np.float64)
+    if np.isnan(r).any():
+        return dict(min=math.nan, median=math.nan, max=math.nan, spread=math.nan,
+                    count_gt2=int(np.sum(r[~np.isnan(r)] > 2.0)), G=int(r.size))
+    r = np.sort(r)
     G = r.size
     return dict(min=float(r[0]), median=float(r[G // 2]), max=float(r[-1]),
                 spread=float(r[-1] / r[0]) if r[0] > 0 else math.inf,

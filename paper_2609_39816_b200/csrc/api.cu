@@ -41,6 +41,9 @@ constexpr int kMaxDev = 64, kEventRing = 64;
 struct SideStream {
   cudaStream_t stream = nullptr;    // general side stream (encode B beside encode A)
   cudaStream_t stream2 = nullptr;   // second side stream (decode stage of a pipelined sweep)
+  cudaStream_t stream_hi = nullptr; // highest-priority stream (block products of a pipelined sweep: when the three
+                                    // stages of neighbouring batches become runnable together, the persistent
+                                    // tensor-core blocks are placed first and the streaming blocks fill in beside them)
   cudaEvent_t ev[kEventRing] = {};
   int next = 0;
 };
@@ -53,6 +56,9 @@ SideStream* side_stream() {
   if (s.stream == nullptr) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&s.stream2, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    int prio_lo = 0, prio_hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&s.stream_hi, cudaStreamNonBlocking, prio_hi) != cudaSuccess) return nullptr;
     for (int i = 0; i < kEventRing; ++i)
       if (cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
   }
@@ -717,6 +723,10 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const fmm_scheme* grid = level == 1 ? base->outer.get() : base;
   const int gm = grid->m, gk = grid->k, gn = grid->n;
+  // every gauge matrix is checked before the first launch: a singular one returns with nothing enqueued
+  for (int g = 0; g < G; ++g)
+    if (!fmm_gauge_invertible(gm, gk, gn, P + (size_t)g * gm * gm, Q + (size_t)g * gk * gk, S + (size_t)g * gn * gn))
+      return FMM_ERR_SINGULAR;
 
   // 1. gauge-transformed coefficient tables: built on the host, merged per batch of algorithms and uploaded in groups
   //    of kTableGroup gauges while the device works on the groups before (the first launch waits for one group only)
@@ -791,38 +801,43 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   FMM_TRY(kmajor_b(d, dB, gws, L.g.bt, &bk_ptr, &bk_ld, false, st));
   void* gws2 = ws + L.gemm2;
   FMM_CUDA(cudaMemsetAsync(at<char>(gws2, L.g.status), 0, sizeof(DeviceStatus), st));
-  // with phase timing on, the stages run back to back on the caller's stream so that the bracketing events measure them
-  SideStream* side = (concurrency_enabled() && !g_prof_on) ? side_stream() : nullptr;
+  // with phase timing on, or when the caller asks for it, the stages run back to back on the caller's stream
+  const bool serial = g_prof_on || (d->flags & FMM_FLAG_SWEEP_SERIAL) != 0 || !concurrency_enabled();
+  SideStream* side = serial ? nullptr : side_stream();
   fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
   batched.m = base->m; batched.k = base->k; batched.n = base->n;
+  fmm_status loop_rc = FMM_OK;
   if (side == nullptr) {
-    for (size_t c = 0;; ++c) {
+    for (size_t c = 0; loop_rc == FMM_OK; ++c) {
       if (c == chunks.size()) {
         if (next_gauge >= G) break;
-        FMM_TRY(build_group(st));
+        if ((loop_rc = build_group(st)) != FMM_OK) break;
       }
       batched.R = base->R * chunks[c].count;
       const SchemeRun r{&batched, d, L.g, gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
                         d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
-      FMM_TRY(stage_encode_pair(r, dA, bk_ptr, bk_ld, st));
-      FMM_TRY(stage_products(r, st));
-      FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, st, chunks[c].count));
+      if ((loop_rc = stage_encode_pair(r, dA, bk_ptr, bk_ld, st)) != FMM_OK) break;
+      if ((loop_rc = stage_products(r, st)) != FMM_OK) break;
+      loop_rc = stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, st, chunks[c].count);
     }
   } else {
-    cudaStream_t sE = side->stream, sG = st, sD = side->stream2;
-    if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;
+    static const bool hi_prio = [] { const char* e = std::getenv("FMM_X_PRIO"); return e && e[0] == '1'; }();
+    cudaStream_t sE = side->stream, sG = hi_prio ? side->stream_hi : st, sD = side->stream2;
+    if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;   // nothing of the sweep is enqueued yet
+    if (sG != st && !stream_wait(side, st, sG)) return FMM_ERR_CUDA;
     cudaEvent_t evG[2] = {nullptr, nullptr}, evD[2] = {nullptr, nullptr};
-    for (size_t c = 0;; ++c) {
-      if (c == chunks.size()) {
-        if (next_gauge >= G) break;
-        FMM_TRY(build_group(sE));       // the encode stream reads the tables first; products and decode follow it
-      }
+    // One step of the pipeline; any failure leaves the loop through the joins below, so that the caller's stream is
+    // ordered behind everything that was enqueued on the library's streams (the caller owns the workspace they use).
+    auto step = [&](size_t c) -> fmm_status {
       const int b = (int)(c & 1);
       batched.R = base->R * chunks[c].count;
       const SchemeRun r{&batched, d, L.g, b ? gws2 : gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
                         d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
-      // encode: the products of batch c-2 must have finished reading this buffer's Ahat / Bhat
+      // encode: the products of batch c-2 must have finished reading this buffer's Ahat / Bhat.  With one scale per
+      // encoded tensor (mode 1) the decode of batch c-2 still reads this buffer's scales, which the encode rewrites:
+      // then the encode waits for that decode too (the other modes fold their scales into the products).
       if (evG[b] && cudaStreamWaitEvent(sE, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
+      if (d->scale_mode == 1 && evD[b] && cudaStreamWaitEvent(sE, evD[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
       // Large operands: two launches, not the paired one — beside the products and decode of the neighbouring batches
       // the two smaller kernels pack better.  Small operands are launch-bound: one paired launch.
       const bool small_operands = (d->M + d->N) * d->K * (int64_t)esize(d->storage) < ((int64_t)16 << 20);
@@ -842,11 +857,25 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
       if (!evG[b] || cudaStreamWaitEvent(sD, evG[b], 0) != cudaSuccess) return FMM_ERR_CUDA;
       FMM_TRY(stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, sD, chunks[c].count));
       evD[b] = record_event(side, sD);
-      if (!evD[b]) return FMM_ERR_CUDA;
+      return evD[b] ? FMM_OK : FMM_ERR_CUDA;
+    };
+    for (size_t c = 0; loop_rc == FMM_OK; ++c) {
+      if (c == chunks.size()) {
+        if (next_gauge >= G) break;
+        // the encode stream reads the tables first; products and decode follow it
+        if ((loop_rc = build_group(sE)) != FMM_OK) break;
+      }
+      loop_rc = step(c);
     }
-    // join: the caller's stream continues after the last decode (the encode stream is ahead of it by construction)
-    if (!stream_wait(side, sD, st) || !stream_wait(side, sE, st)) return FMM_ERR_CUDA;
+    // join: the caller's stream continues after everything enqueued on the library's streams
+    bool joined = stream_wait(side, sD, st) && stream_wait(side, sE, st);
+    if (sG != st) joined = stream_wait(side, sG, st) && joined;
+    if (!joined) {   // last resort: nothing may still run on streams the caller cannot see
+      cudaStreamSynchronize(sE); cudaStreamSynchronize(sD); cudaStreamSynchronize(sG);
+      if (loop_rc == FMM_OK) loop_rc = FMM_ERR_CUDA;
+    }
   }
+  if (loop_rc != FMM_OK) return loop_rc;
 
   // 5. results to the host
   std::vector<double> h((size_t)G + 8);
@@ -865,12 +894,19 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
     rho[g] = (ecl == 0.0) ? (eg == 0.0 ? 1.0 : INFINITY) : std::sqrt(eg / ecl);
   }
   if (h_ratios) std::copy(rho.begin(), rho.end(), h_ratios);
-  std::vector<double> sorted = rho;
-  std::sort(sorted.begin(), sorted.end());
-  out->min = sorted.front();
-  out->max = sorted.back();
-  out->median = sorted[G / 2];  // upper of the two middle values when G is even
-  out->spread = sorted.front() > 0 ? sorted.back() / sorted.front() : INFINITY;
+  // NaN in the operands propagates into the ratios; a summary over a set that contains NaN is NaN (ordering NaN
+  // with operator< is undefined), the count of ratios above 2 is taken over the comparable ones
+  const bool any_nan = std::any_of(rho.begin(), rho.end(), [](double x) { return std::isnan(x); });
+  if (any_nan) {
+    out->min = out->max = out->median = out->spread = NAN;
+  } else {
+    std::vector<double> sorted = rho;
+    std::sort(sorted.begin(), sorted.end());
+    out->min = sorted.front();
+    out->max = sorted.back();
+    out->median = sorted[G / 2];  // upper of the two middle values when G is even
+    out->spread = sorted.front() > 0 ? sorted.back() / sorted.front() : INFINITY;
+  }
   out->count_gt2 = (int64_t)std::count_if(rho.begin(), rho.end(), [](double x) { return x > 2.0; });
   out->G = G;
   out->e_classical_rel = nref > 0 ? std::sqrt(ecl / nref) : 0.0;

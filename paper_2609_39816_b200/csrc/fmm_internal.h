@@ -49,5 +49,7 @@ struct CoefTable {
 // ascending (l,j) order of V; tW: cell-major decode table (R field = m*n lists, `cell` = product index r,
 // ascending).  Any pointer may be null.
 void fmm_build_tables(const fmm_scheme& s, CoefTable* tA, CoefTable* tB, CoefTable* tW);
+// true when P (m x m), Q (k x k) and S (n x n) can all be inverted (the test gauge_apply / fmm_gauge_core apply)
+bool fmm_gauge_invertible(int m, int k, int n, const double* P, const double* Q, const double* S);
 fmm_status fmm_gauge_core(const fmm_scheme& in, int level, const double* P, const double* Q, const double* S,
                           double cond_limit, fmm_scheme** out);

@@ -18,7 +18,9 @@ constexpr int kMaxBlocks = 2048;
 static __device__ __align__(256) double g_noalloc_partials[2 * kMaxBlocks];   // 32 KiB per GPU
 
 constexpr int kMaxDevices = 64;
-double* g_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+// Device address of the array, per device ordinal, kept for the life of the process: it does not survive a
+// cudaDeviceReset of that device by the host application (the library must not be used across one).
+double* g_scratch_ptr[kMaxDevices] = {};
 
 // In host code the array's name is only a handle for the runtime, not an address the GPU understands:
 // the device address has to be asked for, once per device, while that device is current.
@@ -45,8 +47,9 @@ fmm_status error_frobenius_noalloc(const fmm_gemm_desc* d, const void* dC, const
   if (!d || !dC || !dCstar || !d_out) return FMM_ERR_ARG;
   if (d->M <= 0 || d->N <= 0 || d->ldc < d->N) return FMM_ERR_SHAPE;
   if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
+  // would not fit the fixed array (tested by division: M * N itself may not fit 64 bits)
+  if (d->M > error_frobenius_noalloc_max_elements() / d->N) return FMM_ERR_LIMIT;
   const int64_t count = d->M * d->N;
-  if (count > error_frobenius_noalloc_max_elements()) return FMM_ERR_LIMIT;   // would not fit the fixed array
   double* scratch = nullptr;
   fmm_status s = scratch_for_current_device(&scratch);
   if (s != FMM_OK) return s;

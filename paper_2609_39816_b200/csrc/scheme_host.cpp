@@ -243,6 +243,12 @@ const CoefTable* fmm_packed_table(const fmm_scheme& s, int which) {
   return reinterpret_cast<const CoefTable*>(fmm_packed_tables(s).data() + kPackedStatusBytes + which * fmm_packed_table_stride());
 }
 
+bool fmm_gauge_invertible(int m, int k, int n, const double* P, const double* Q, const double* S) {
+  double inv[FMM_MAX_GRID * FMM_MAX_GRID];
+  if (m < 1 || k < 1 || n < 1 || m > FMM_MAX_GRID || k > FMM_MAX_GRID || n > FMM_MAX_GRID) return false;
+  return invert(m, P, inv) && invert(k, Q, inv) && invert(n, S, inv);
+}
+
 fmm_status fmm_gauge_core(const fmm_scheme& in, int level, const double* P, const double* Q, const double* S,
                           double cond_limit, fmm_scheme** out) {
   std::unique_ptr<fmm_scheme> res(new (std::nothrow) fmm_scheme);

@@ -349,6 +349,8 @@ def test_error_ratio_and_summary_rules():
     s = oracle.summary([5.0, 1.0, 3.0, 2.5])              # even count: upper of the two middle values
     assert (s["min"], s["median"], s["max"], s["spread"], s["count_gt2"]) == (1.0, 3.0, 5.0, 5.0, 3)
     assert oracle.summary([4.0, 1.0, 2.0])["median"] == 2.0
+    n = oracle.summary([4.0, math.nan, 1.0])              # a set with NaN has no order; the count skips it
+    assert all(math.isnan(n[k]) for k in ("min", "median", "max", "spread")) and n["count_gt2"] == 1 and n["G"] == 3
 
 
 def test_symmetric_vs_offset_operands_soft():

@@ -47,3 +47,8 @@ def test_noalloc_matches_workspace_variant_twice_in_a_row():
     with pytest.raises(lib.FmmError) as err:
         lib.error_frobenius_noalloc(too_big, Cbig, Cstar, got)
     assert err.value.code == 9
+    # also when M * N does not fit 64 bits
+    huge = lib.GemmDesc.make(2 ** 40, 16, 2 ** 40, "bf16", "bf16", "f32")
+    with pytest.raises(lib.FmmError) as err:
+        lib.error_frobenius_noalloc(huge, Cbig, Cstar, got)
+    assert err.value.code == 9
