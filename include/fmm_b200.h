@@ -93,6 +93,25 @@ typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
                                  are the same); slower.  For callers that want one stream only, and for checking
                                  the pipelined path against.                                              */
 
+#define FMM_FLAG_SWEEP_FUSED 16 /* error_sweep only (bf16 storage and products, no scales, one-level algorithms on a
+                                 2 x 2 grid, else ignored): run each batch's block products, the decode of the batch
+                                 before it and the encode of the batch after it as ONE kernel launch whose CTAs carry
+                                 the tensor-core roles and, beside them, warps that stream the other two passes.  Same
+                                 C bits per algorithm; each error sum is added over another partition of the outputs
+                                 (ratios agree to 1e-8, bit-reproducible run to run).  On a power-limited B200 it is
+                                 no faster than the default pipeline: the passes overlap and the clock drops.      */
+#define FMM_FLAG_ROUND_PER_LEVEL 8 /* scheme_gemm on a handle made by scheme_kron (or "strassen444"): round the block
+                                 sums at EVERY level.  The outer factor's block sums of A (and of B) are scaled
+                                 and rounded to the product dtype; the inner factor's block sums are formed of
+                                 those rounded values and rounded again; products and decode are unchanged
+                                 (decode uses the flat coefficients w1 w2 in ascending r).  This is "the algorithm
+                                 applied to its own blocks" (Section 1) taken literally — a different operator
+                                 from the default, flat one, which rounds each of the R1 R2 block sums of the
+                                 Kronecker coefficients once (what the paper's two-level algorithm does).
+                                 scale_mode 0 or 1 (mode 1: one power-of-two scale per outer tensor, then one per
+                                 inner tensor in units of it; sA_r is their product).  FMM_ERR_ARG for a flat
+                                 handle and in error_sweep.                                                  */
+
 /* The float-path "quantisation specification" (Section 2.2 treats these choices as part of the
  * operator): shapes, dtypes, layout of B, scale rule. */
 typedef struct {

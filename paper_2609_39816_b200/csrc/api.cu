@@ -41,9 +41,6 @@ constexpr int kMaxDev = 64, kEventRing = 64;
 struct SideStream {
   cudaStream_t stream = nullptr;    // general side stream (encode B beside encode A)
   cudaStream_t stream2 = nullptr;   // second side stream (decode stage of a pipelined sweep)
-  cudaStream_t stream_hi = nullptr; // highest-priority stream (block products of a pipelined sweep: when the three
-                                    // stages of neighbouring batches become runnable together, the persistent
-                                    // tensor-core blocks are placed first and the streaming blocks fill in beside them)
   cudaEvent_t ev[kEventRing] = {};
   int next = 0;
 };
@@ -56,9 +53,6 @@ SideStream* side_stream() {
   if (s.stream == nullptr) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&s.stream2, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    int prio_lo = 0, prio_hi = 0;
-    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) return nullptr;
-    if (cudaStreamCreateWithPriority(&s.stream_hi, cudaStreamNonBlocking, prio_hi) != cudaSuccess) return nullptr;
     for (int i = 0; i < kEventRing; ++i)
       if (cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
   }
@@ -99,6 +93,10 @@ struct GemmLayout {
   size_t status, tabA, tabB, tabW, amaxA, amaxB, sA, sB, partials, bt, ahat, bhat, prod, total;
   int64_t sAhat, sBhat, sProd;   // elements between consecutive products (block size + padding)
   int n_partials;
+  // FMM_FLAG_ROUND_PER_LEVEL: the outer level's rounded block sums (R1 tensors per operand), its tables, amax words
+  // and scales, and the inner level's tables
+  size_t lvl_tab_outer, lvl_tab_inner, lvl_amax, lvl_scale, lvl_a, lvl_b;
+  int64_t sLvlA, sLvlB;
 };
 
 fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
@@ -130,8 +128,8 @@ size_t scale_words(int mode, int R, int64_t rows, int64_t inner, bool b_side) {
   return FMM_MAX_R;
 }
 
-GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
-  GemmLayout L;
+GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d, const fmm_scheme* nested = nullptr) {
+  GemmLayout L{};
   const int64_t bm = d->M / m, bk = d->K / k, bn = d->N / n;
   const int ep = esize(d->product), es = esize(d->storage);
   size_t o = 0;
@@ -157,6 +155,17 @@ GemmLayout gemm_layout(int m, int k, int n, int R, const fmm_gemm_desc* d) {
   L.ahat = o; o += align_up((size_t)R * L.sAhat * ep);
   L.bhat = o; o += align_up((size_t)R * L.sBhat * ep);
   L.prod = o; o += align_up((size_t)R * L.sProd * ((d->flags & FMM_FLAG_PRODUCTS_BF16) ? 2 : 4));
+  if ((d->flags & FMM_FLAG_ROUND_PER_LEVEL) && nested && nested->outer && nested->inner) {
+    const fmm_scheme& so = *nested->outer;
+    L.lvl_tab_outer = o; o += 2 * align_up(sizeof(CoefTable));
+    L.lvl_tab_inner = o; o += 2 * align_up(sizeof(CoefTable));
+    L.lvl_amax = o; o += align_up(2 * FMM_MAX_R * 4);
+    L.lvl_scale = o; o += align_up(2 * FMM_MAX_R * 4);
+    L.sLvlA = (d->M / so.m) * (d->K / so.k) + kSlabPadBytes / ep;
+    L.sLvlB = (d->N / so.n) * (d->K / so.k) + kSlabPadBytes / ep;
+    L.lvl_a = o; o += align_up((size_t)so.R * L.sLvlA * ep);
+    L.lvl_b = o; o += align_up((size_t)so.R * L.sLvlB * ep);
+  }
   L.total = o;
   return L;
 }
@@ -238,6 +247,55 @@ fmm_status stage_encode_pair(const SchemeRun& r, const void* A, const void* Bk, 
   return FMM_OK;
 }
 
+// Block sums rounded at every level of a nested algorithm (FMM_FLAG_ROUND_PER_LEVEL): the outer factor's block sums
+// of the operand are scaled, rounded to the product dtype and kept as R1 tensors; for each of them the inner factor's
+// block sums are formed of those rounded values and rounded again into products r1 * R2 .. r1 * R2 + R2 - 1.  With one
+// scale per encoded tensor the inner pass works in units of the outer scale and writes the product of the two.
+fmm_status stage_encode_per_level(const SchemeRun& r, const void* X, int64_t ldx, bool b_side, cudaStream_t st) {
+  const fmm_scheme& so = *r.s->outer;
+  const fmm_scheme& si = *r.s->inner;
+  const fmm_gemm_desc* d = r.d;
+  const int mode = d->scale_mode;
+  const int gr1 = b_side ? so.n : so.m, gc1 = so.k, gr2 = b_side ? si.n : si.m, gc2 = si.k;
+  const int64_t Br = (b_side ? d->N : d->M) / gr1, Bc = d->K / gc1;      // outer blocks
+  const int64_t br = Br / gr2, bc = Bc / gc2;                            // inner blocks
+  const int which = b_side ? 1 : 0;
+  const size_t tstride = align_up(sizeof(CoefTable));
+  const CoefTable* h_out = fmm_packed_table(so, which);
+  const CoefTable* h_in = fmm_packed_table(si, which);
+  const CoefTable* d_out = at<CoefTable>(r.ws, r.L.lvl_tab_outer + which * tstride);
+  const CoefTable* d_in = at<CoefTable>(r.ws, r.L.lvl_tab_inner + which * tstride);
+  FMM_CUDA(cudaMemcpyAsync(const_cast<CoefTable*>(d_out), h_out, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(const_cast<CoefTable*>(d_in), h_in, sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  unsigned* amax1 = at<unsigned>(r.ws, r.L.lvl_amax) + which * FMM_MAX_R;
+  float* scale1 = at<float>(r.ws, r.L.lvl_scale) + which * FMM_MAX_R;
+  const int ep = esize(d->product);
+  char* lvl = at<char>(r.ws, b_side ? r.L.lvl_b : r.L.lvl_a);
+  const int64_t lvl_stride = b_side ? r.L.sLvlB : r.L.sLvlA;
+  ProfScope ps(b_side ? 1 : 0, st);
+  // outer level
+  const EncodeOperand o1{X, ldx, gr1, gc1, Br, Bc, d_out, h_out, lvl, lvl_stride, amax1, mode ? scale1 : nullptr, 1, 0, nullptr};
+  if (mode != 0) {
+    FMM_CUDA(cudaMemsetAsync(amax1, 0, FMM_MAX_R * 4, st));
+    FMM_CUDA(launch_encode_pair(d->storage, d->product, o1, nullptr, true, mode, st));
+  }
+  FMM_CUDA(launch_encode_pair(d->storage, d->product, o1, nullptr, false, mode, st));
+  // inner level, one outer product at a time: its source is the rounded outer block sum (product dtype)
+  char* hat = at<char>(r.ws, b_side ? r.L.bhat : r.L.ahat);
+  const int64_t hat_stride = b_side ? r.L.sBhat : r.L.sAhat;
+  unsigned* amax2 = at<unsigned>(r.ws, b_side ? r.L.amaxB : r.L.amaxA);
+  float* scale2 = b_side ? r.sB() : r.sA();
+  if (mode != 0) FMM_CUDA(cudaMemsetAsync(amax2, 0, FMM_MAX_R * 4, st));
+  for (int r1 = 0; r1 < so.R; ++r1) {
+    const EncodeOperand o2{lvl + (size_t)r1 * lvl_stride * ep, Bc, gr2, gc2, br, bc, d_in, h_in,
+                           hat + (size_t)r1 * si.R * hat_stride * ep, hat_stride, amax2 + r1 * si.R,
+                           mode ? scale2 + r1 * si.R : nullptr, 1, 0, mode ? scale1 + r1 : nullptr};
+    if (mode != 0) FMM_CUDA(launch_encode_pair(d->product, d->product, o2, nullptr, true, mode, st));
+    FMM_CUDA(launch_encode_pair(d->product, d->product, o2, nullptr, false, mode, st));
+  }
+  return FMM_OK;
+}
+
 fmm_status stage_products(const SchemeRun& r, cudaStream_t st) {
   const fmm_scheme* s = r.s;
   const int64_t bm = r.d->M / s->m, bk = r.d->K / s->k, bn = r.d->N / s->n;
@@ -304,7 +362,10 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
   // encode A and encode B side by side: one launch whose blocks split between the two operands (they share nothing);
   // with the side stream enabled by the environment the two run as separate launches on two streams instead
   static const bool two_streams = [] { const char* e = std::getenv("FMM_B200_ENCODE_TWO_STREAMS"); return e && e[0] == '1'; }();
-  if (skip_b) {
+  if (d->flags & FMM_FLAG_ROUND_PER_LEVEL) {
+    FMM_TRY(stage_encode_per_level(r, A, d->lda, false, st));
+    if (!skip_b) FMM_TRY(stage_encode_per_level(r, Bsrc_kmajor, ldb_kmajor, true, st));
+  } else if (skip_b) {
     FMM_TRY(stage_encode_a(r, A, st));
   } else if (!two_streams) {
     FMM_TRY(stage_encode_pair(r, A, Bsrc_kmajor, ldb_kmajor, st));
@@ -331,6 +392,15 @@ fmm_status kmajor_b(const fmm_gemm_desc* d, const void* B, void* ws, size_t bt_o
   ProfScope ps(1, st);
   if (!skip) FMM_CUDA(launch_transpose(esize(d->storage), B, d->ldb, d->K, d->N, bt, st));
   *out = bt; *ld = d->K;
+  return FMM_OK;
+}
+
+// FMM_FLAG_ROUND_PER_LEVEL needs a handle that remembers its factors, scale mode 0 or 1, and inner blocks the 16-byte
+// vectors of the product dtype tile (a multiple of 16 inner indices per inner block already holds)
+fmm_status check_per_level(const fmm_scheme* s, const fmm_gemm_desc* d) {
+  if (!(d->flags & FMM_FLAG_ROUND_PER_LEVEL)) return FMM_OK;
+  if (!s->outer || !s->inner) return FMM_ERR_ARG;
+  if (d->scale_mode != 0 && d->scale_mode != 1) return FMM_ERR_DTYPE;
   return FMM_OK;
 }
 
@@ -460,8 +530,9 @@ bool merge_tables(const CoefTable* tabs, int kb, int R, CoefTable* mA, CoefTable
 
 struct SweepLayout {
   GemmLayout g; ClassicalLayout c;
-  size_t gemm, gemm2, classical, cstar, cstar32, ccl, tables, sums, total;   // two GEMM workspaces: gauges are pipelined
+  size_t gemm, gemm2, classical, cstar, cstar32, ccl, tables, sums, fpart, total;   // two GEMM workspaces: gauges are pipelined
 };
+constexpr int kFusedPartialsPerGauge = 512;   // room for the streaming blocks of a fused launch (2 per SM)
 
 SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
   SweepLayout L;
@@ -476,6 +547,7 @@ SweepLayout sweep_layout(const fmm_scheme* s, const fmm_gemm_desc* d, int G) {
   L.ccl = o; o += align_up((size_t)d->M * d->N * esize(d->output));
   L.tables = o; o += align_up((size_t)G * 3 * sizeof(CoefTable));
   L.sums = o; o += align_up((size_t)(G + 8) * 8);
+  L.fpart = o; o += align_up((size_t)G * kFusedPartialsPerGauge * 8);
   L.total = o;
   return L;
 }
@@ -503,14 +575,15 @@ fmm_status fmm_profile_collect(double ms[8], int64_t count[8]) {
 }
 
 size_t scheme_gemm_workspace(const fmm_scheme* s, const fmm_gemm_desc* d) {
-  if (!s || check_desc(d, s->m, s->k, s->n) != FMM_OK) return 0;
-  return gemm_layout(s->m, s->k, s->n, s->R, d).total;
+  if (!s || check_desc(d, s->m, s->k, s->n) != FMM_OK || check_per_level(s, d) != FMM_OK) return 0;
+  return gemm_layout(s->m, s->k, s->n, s->R, d, s).total;
 }
 
 fmm_status scheme_gemm_workspace_layout(const fmm_scheme* s, const fmm_gemm_desc* d, size_t off[8]) {
   if (!s || !off) return FMM_ERR_ARG;
   FMM_TRY(check_desc(d, s->m, s->k, s->n));
-  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d);
+  FMM_TRY(check_per_level(s, d));
+  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d, s);
   off[0] = L.ahat; off[1] = L.bhat; off[2] = L.prod; off[3] = L.sA; off[4] = L.sB;
   off[5] = (size_t)L.sAhat; off[6] = (size_t)L.sBhat; off[7] = (size_t)L.sProd;
   return FMM_OK;
@@ -520,7 +593,8 @@ fmm_status scheme_gemm(const fmm_scheme* s, const fmm_gemm_desc* d, const void* 
                        void* d_ws, size_t ws_bytes, void* cuda_stream) {
   if (!s || !d || !dA || !dB || !dC) return FMM_ERR_ARG;
   FMM_TRY(check_desc(d, s->m, s->k, s->n));
-  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d);
+  FMM_TRY(check_per_level(s, d));
+  const GemmLayout L = gemm_layout(s->m, s->k, s->n, s->R, d, s);
   FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const bool skip_b = (d->flags & FMM_FLAG_REUSE_BHAT) != 0;
@@ -594,7 +668,7 @@ HostLayout host_layout(const fmm_scheme* s, const fmm_gemm_desc* d) {
   L.a = o; o += align_up((size_t)d->M * d->K * es);
   L.b = o; o += align_up((size_t)d->K * d->N * es);
   L.c = o; o += align_up((size_t)d->M * d->N * eo);
-  L.ws = o; o += gemm_layout(s->m, s->k, s->n, s->R, &L.dev).total;
+  L.ws = o; o += gemm_layout(s->m, s->k, s->n, s->R, &L.dev, s).total;
   L.total = o;
   return L;
 }
@@ -718,6 +792,7 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   if (level != 0 && level != 1) return FMM_ERR_ARG;
   if (level == 1 && (!base->outer || !base->inner)) return FMM_ERR_ARG;
   FMM_TRY(check_desc(d, base->m, base->k, base->n));
+  if (d->flags & FMM_FLAG_ROUND_PER_LEVEL) return FMM_ERR_ARG;   // the sweep runs the flat operator
   const SweepLayout L = sweep_layout(base, d, G);
   FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -807,8 +882,98 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
   batched.m = base->m; batched.k = base->k; batched.n = base->n;
   fmm_status loop_rc = FMM_OK;
+  // Fused pipeline (FMM_FLAG_SWEEP_FUSED; bf16 storage and products, no scales, batches of four or eight one-level
+  // algorithms): ONE launch per batch runs its block products together with the decode of the batch before and the
+  // encode of the batch after, in the same CTAs (launch_fused_sweep), on the caller's stream; the pipeline starts with a
+  // plain encode and ends with a decode-only launch.  Batches of one or two algorithms at the end of the list take the
+  // ordinary path below.  Measured on B200: the three passes do overlap inside the launch, and the chip answers by
+  // lowering its clock (the board's power limit: tensor cores and the memory system cannot both run flat out), so the
+  // sweep takes the same time as with the passes one after another — hence opt-in, not the default.
+  size_t first_plain_chunk = 0;
+  const int kFusedGroups = 2;
+  const int64_t bm_ = d->M / base->m, bn_ = d->N / base->n, bk_ = d->K / base->k;
+  const bool fused_ok = (d->flags & FMM_FLAG_SWEEP_FUSED) && !serial && kb >= 4 && d->storage == FMM_BF16 && d->product == FMM_BF16 && d->scale_mode == 0 &&
+                        !(d->flags & FMM_FLAG_PRODUCTS_BF16) && base->m * base->k <= 4 && base->n * base->k <= 4 &&
+                        base->m * base->n <= 4 && bm_ > 128 && bn_ > 128 &&
+                        fused_sweep_blocks(kFusedGroups) <= kFusedPartialsPerGauge && fused_sweep_blocks(kFusedGroups) >= 2 &&
+                        (int64_t)4 * base->R * ((bm_ + 255) / 256) * ((bn_ + 255) / 256) >= fused_sweep_blocks(1) / 2;
+  if (fused_ok) {
+    const int nblk = fused_sweep_blocks(kFusedGroups);
+    double* fpart = at<double>(ws, L.fpart);
+    auto chunk_ready = [&](size_t c) -> fmm_status {   // tables of chunk c built and uploaded (in groups, ahead of use)
+      while (c >= chunks.size() && next_gauge < G) FMM_TRY(build_group(st));
+      return FMM_OK;
+    };
+    auto run_of = [&](size_t c, int b) {
+      batched.R = base->R * chunks[c].count;
+      return SchemeRun{&batched, d, L.g, b ? gws2 : gws, &tabs[3 * c], &tabs[3 * c + 1], &tabs[3 * c + 2],
+                       d_tabs + 3 * c, d_tabs + 3 * c + 1, d_tabs + 3 * c + 2};
+    };
+    auto fusable = [&](size_t c) { return c < chunks.size() && chunks[c].count >= 4; };
+    loop_rc = chunk_ready(0);
+    size_t nf = 0;                     // fused chunks so far: chunk i lives in buffer i & 1
+    if (loop_rc == FMM_OK && fusable(0)) {
+      const SchemeRun r0 = run_of(0, 0);
+      loop_rc = stage_encode_pair(r0, dA, bk_ptr, bk_ld, st);
+      for (size_t c = 0; loop_rc == FMM_OK; ++c) {
+        if ((loop_rc = chunk_ready(c + 1)) != FMM_OK) break;
+        const int b = (int)(c & 1);
+        const bool more = fusable(c + 1);
+        FusedSweepArgs f{};
+        f.groups = kFusedGroups; f.output = d->output;
+        f.n = base->n; f.bm = bm_; f.bn = bn_; f.cstar32 = cstar32;
+        {  // products of chunk c
+          const SchemeRun r = run_of(c, b);
+          BlockProductArgs& g = f.products;
+          g.product = FMM_BF16;
+          g.A = at<char>(r.ws, L.g.ahat); g.lda = bk_; g.a_batch = L.g.sAhat;
+          g.B = at<char>(r.ws, L.g.bhat); g.ldb = bk_; g.b_batch = L.g.sBhat;
+          g.rows_a = bm_; g.rows_b = bn_; g.kdim = bk_; g.batches = base->R * chunks[c].count;
+          g.out = at<char>(r.ws, L.g.prod); g.ldo = bn_; g.o_batch = L.g.sProd; g.out_mode = 0; g.output = FMM_F32;
+          g.status = at<DeviceStatus>(r.ws, L.g.status);
+          f.have_products = 1;
+        }
+        if (c > 0) {  // decode of chunk c-1 out of the other buffer
+          const SchemeRun rp = run_of(c - 1, b ^ 1);
+          f.dec_gauges = chunks[c - 1].count;
+          f.dec_prod = at<float>(rp.ws, L.g.prod); f.dec_prod_stride = L.g.sProd; f.dec_tab = rp.dW; f.dec_RB = base->R;
+          f.partials = fpart + (size_t)chunks[c - 1].g0 * nblk;
+        }
+        if (more) {   // encode of chunk c+1 into the other buffer (its last reader was the previous launch)
+          const SchemeRun rn = run_of(c + 1, b ^ 1);
+          f.have_encode = 1;
+          f.enc_a = EncodeOperand{dA, d->lda, base->m, base->k, bm_, bk_, rn.dA, rn.hA, at<char>(rn.ws, L.g.ahat), L.g.sAhat,
+                                  nullptr, nullptr, 1, 0, nullptr};
+          f.enc_b = EncodeOperand{bk_ptr, bk_ld, base->n, base->k, bn_, bk_, rn.dB, rn.hB, at<char>(rn.ws, L.g.bhat), L.g.sBhat,
+                                  nullptr, nullptr, 128, 1, nullptr};
+        }
+        {
+          ProfScope ps(2, st);
+          loop_rc = launch_fused_sweep(f, st);
+        }
+        nf = c + 1;
+        if (!more) break;
+      }
+      if (loop_rc == FMM_OK && nf > 0) {   // tail of the pipeline: decode of the last fused chunk, then all its sums
+        const size_t c = nf - 1;
+        FusedSweepArgs f{};
+        f.groups = kFusedGroups; f.output = d->output;
+        f.n = base->n; f.bm = bm_; f.bn = bn_; f.cstar32 = cstar32;
+        const SchemeRun rp = run_of(c, (int)(c & 1));
+        f.products.status = at<DeviceStatus>(rp.ws, L.g.status);
+        f.dec_gauges = chunks[c].count;
+        f.dec_prod = at<float>(rp.ws, L.g.prod); f.dec_prod_stride = L.g.sProd; f.dec_tab = rp.dW; f.dec_RB = base->R;
+        f.partials = fpart + (size_t)chunks[c].g0 * nblk;
+        loop_rc = launch_fused_sweep(f, st);
+        const int gauges_done = chunks[c].g0 + chunks[c].count;
+        if (loop_rc == FMM_OK && launch_sum_partials(fpart, nblk, sums + 8, st, gauges_done) != cudaSuccess) loop_rc = FMM_ERR_CUDA;
+      }
+      first_plain_chunk = nf;
+    }
+  }
+  if (loop_rc != FMM_OK) return loop_rc;    // everything so far ran on the caller's stream
   if (side == nullptr) {
-    for (size_t c = 0; loop_rc == FMM_OK; ++c) {
+    for (size_t c = first_plain_chunk; loop_rc == FMM_OK; ++c) {
       if (c == chunks.size()) {
         if (next_gauge >= G) break;
         if ((loop_rc = build_group(st)) != FMM_OK) break;
@@ -821,8 +986,7 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
       loop_rc = stage_decode(r, nullptr, cstar32, sums + 8 + chunks[c].g0, st, chunks[c].count);
     }
   } else {
-    static const bool hi_prio = [] { const char* e = std::getenv("FMM_X_PRIO"); return e && e[0] == '1'; }();
-    cudaStream_t sE = side->stream, sG = hi_prio ? side->stream_hi : st, sD = side->stream2;
+    cudaStream_t sE = side->stream, sG = st, sD = side->stream2;
     if (!stream_wait(side, st, sE) || !stream_wait(side, st, sD)) return FMM_ERR_CUDA;   // nothing of the sweep is enqueued yet
     if (sG != st && !stream_wait(side, st, sG)) return FMM_ERR_CUDA;
     cudaEvent_t evG[2] = {nullptr, nullptr}, evD[2] = {nullptr, nullptr};
@@ -859,7 +1023,7 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
       evD[b] = record_event(side, sD);
       return evD[b] ? FMM_OK : FMM_ERR_CUDA;
     };
-    for (size_t c = 0; loop_rc == FMM_OK; ++c) {
+    for (size_t c = first_plain_chunk; loop_rc == FMM_OK; ++c) {
       if (c == chunks.size()) {
         if (next_gauge >= G) break;
         // the encode stream reads the tables first; products and decode follow it

@@ -19,9 +19,11 @@
 
 #include <algorithm>
 #include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "kernels_stream.cuh"
+#include "stream_bodies.cuh"
 
 namespace {
 
@@ -486,54 +488,33 @@ struct PairLayout {
   static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;
 };
 
+// The three roles of one CTA of a pair (producer warp 0, MMA warp 1, epilogue warps 2..5), given the CTA's ring,
+// barrier block and TMEM base.  `warp` is the warp's index among those six.
+struct PairCtx {
+  unsigned char* smem;        // 1024-byte aligned ring
+  uint32_t bar_base;          // shared-memory address of the barrier block behind it
+  volatile int* abort_flag;
+  uint32_t tmem_base;
+  uint32_t rank;              // CTA rank in the pair (0 = leader)
+};
+
 template <bool kFp8>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
-block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                           void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
-                           TileParams tp, DeviceStatus* status) {
-  grid_launch_dependents();   // the decode may set up while this grid drains; it waits before reading the products
+__device__ __forceinline__ void pair_roles(const int warp, const int lane, const PairCtx& cx, const CUtensorMap& map_a,
+                                           const CUtensorMap& map_b, void* __restrict__ out, const float* __restrict__ sA,
+                                           const float* __restrict__ sB, const TileParams& tp, DeviceStatus* status) {
   using L = PairLayout;
   constexpr int BN = L::BN;
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t raw_addr = smem_u32(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  unsigned char* smem = smem_raw + (base - raw_addr);
-  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
-  const uint32_t bar_base = smem_u32(bar_mem);
+  unsigned char* smem = cx.smem;
+  const uint32_t bar_base = cx.bar_base;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };                       // used in the leader only
   auto empty_bar = [&](int s) { return bar_base + 8u * (L::kStages + s); };       // one per CTA
   auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + b); };   // one per CTA
   auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * L::kStages + 2 + b); };  // used in the leader only
   const uint32_t drain_bar = bar_base + 8u * (2 * L::kStages + 4);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();   // 0 = leader
+  volatile int* abort_flag = cx.abort_flag;
+  const uint32_t tmem_base = cx.tmem_base;
+  const uint32_t rank = cx.rank;
   const bool leader = rank == 0;
-  constexpr uint32_t kTmemCols = 2 * BN;     // two accumulator buffers of 256 columns
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < L::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 8); }
-    mbar_init(drain_bar, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();   // both CTAs' barriers are initialised before anything signals across the pair
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  grid_dependency_wait();     // operands and scales come from the previous kernel of the stream
-
   const int num_kb = (tp.kbytes + BKB - 1) / BKB;
   const int tiles_m = (tp.rows_a + 2 * BM - 1) / (2 * BM);
   const int tiles_n = (tp.rows_b + BN - 1) / BN;
@@ -565,7 +546,20 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) __nanosleep(2000000);   // let copies already issued land before shared memory goes away
+      if (!ok && leader) {
+        // Let copies that were already issued land before shared memory goes away.  The copies of BOTH CTAs complete
+        // on the leader's full barriers, so the leader waits (bounded) for the most recent fill of every stage; its
+        // partner cannot leave before the leader does (the cluster barrier at the end of the kernel), so the partner's
+        // shared memory outlives its own copies too.  A fill the partner never issued leaves its barrier incomplete:
+        // that wait runs into its bound.
+        for (int s = 0; s < L::kStages; ++s) {
+          const uint32_t last_parity = (s < stage) ? phase : (phase ^ 1u);
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(s), last_parity)) {
+            if (global_timer_ns() - t0 > 20000000ull) break;  // 20 ms
+          }
+        }
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
@@ -650,13 +644,128 @@ block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
     }
   }
 
+}
+
+// Set-up shared by every kernel that runs the pair roles: barrier block, TMEM allocation (warp 1 of the CTA), and the
+// CTA- and cluster-wide barriers that make them visible.  Every thread of the CTA calls it, and pair_teardown at the end.
+__device__ __forceinline__ PairCtx pair_setup(unsigned char* smem_raw, const int warp) {
+  using L = PairLayout;
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* smem = smem_raw + (base - raw_addr);
+  unsigned char* bar_mem = smem + L::kStages * L::kStageBytes;
+  const uint32_t bar_base = smem_u32(bar_mem);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_mem + 8 * (2 * L::kStages + 5));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_mem + 8 * (2 * L::kStages + 5) + 8);
+  constexpr uint32_t kTmemCols = 2 * L::BN;     // two accumulator buffers of 256 columns
+  if (threadIdx.x == 0) {
+    for (int st = 0; st < L::kStages; ++st) {
+      mbar_init(bar_base + 8u * st, 1);                       // full (used in the leader only)
+      mbar_init(bar_base + 8u * (L::kStages + st), 1);        // empty
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_base + 8u * (2 * L::kStages + b), 1);     // accumulator full
+      mbar_init(bar_base + 8u * (2 * L::kStages + 2 + b), 8); // accumulator empty: four epilogue warps of each CTA
+    }
+    mbar_init(bar_base + 8u * (2 * L::kStages + 4), 1);       // drain
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();   // both CTAs' barriers are initialised before anything signals across the pair
+  tc_fence_after();
+  return PairCtx{smem, bar_base, abort_flag, *tmem_slot, cluster_ctarank()};
+}
+
+__device__ __forceinline__ void pair_teardown(const PairCtx& cx, const int warp) {
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();   // neither CTA frees TMEM / leaves while its partner may still touch it
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(cx.tmem_base), "r"(2 * PairLayout::BN) : "memory");
   }
+}
+
+template <bool kFp8>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+block_products_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                           void* __restrict__ out, const float* __restrict__ sA, const float* __restrict__ sB,
+                           TileParams tp, DeviceStatus* status) {
+  grid_launch_dependents();   // the decode may set up while this grid drains; it waits before reading the products
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const PairCtx cx = pair_setup(smem_raw, warp);
+  grid_dependency_wait();     // operands and scales come from the previous kernel of the stream
+  pair_roles<kFp8>(warp, lane, cx, map_a, map_b, out, sA, sB, tp, status);
+  pair_teardown(cx, warp);
+}
+
+// ---------------------------------------------------------------- fused sweep kernel
+// One launch of a gauge sweep's pipeline: the block products of batch c on the tensor cores (the pair roles above,
+// warps 0..5) and, beside them in the same CTAs, groups of eight warps that run the streaming passes of the neighbouring
+// batches — first the error-only decode of batch c-1 (its products were written by the previous launch), then the
+// encode of batch c+1 (its block sums are read by the next launch).  The three passes touch disjoint buffers, so no
+// CTA waits for another inside the launch; all dependencies are launch-to-launch in stream order.  Why: each pass alone
+// leaves most of the machine idle (the products use the tensor pipe and a sixth of the warp slots, the streaming passes
+// are bound by issue slots and memory latency at 0.65-0.72 of the HBM peak), and as separate kernels they cannot share
+// an SM, because a product CTA holds nearly all of its shared memory.
+// A streaming group is a virtual block of the pass: group g of CTA b is block b * kGroups + g of gridDim.x * kGroups.
+struct FusedStreamArgs {
+  // error-only batch decode of the previous batch (dec_gauges = 0: none).  Arguments as decode_batch_kernel's.
+  int dec_gauges;               // 4 or 8 algorithms in the batch
+  const float* prod; const CoefTable* tab_w; int RB; int n; long long bm, bn;
+  const float* cstar32; long long ldcs; double* partials; int dec_tiles_per_block; long long prod_stride;
+  // encode of the next batch (enc_dense < 0: none)
+  int enc_dense;                // 1: register-chain variant (every product reads the four cells in one order)
+  EncodeJob ja, jb;
+};
+
+template <int kGroups> struct FusedLayout {
+  static constexpr int kThreads = kNumThreads + 256 * kGroups;
+  static constexpr int kGroupBytes = 14 * 1024;   // one streaming group: the larger of its decode and encode needs
+  static constexpr int kTotal = PairLayout::kTotal + kGroups * kGroupBytes;
+};
+
+template <typename OutT, int kGroups>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(FusedLayout<kGroups>::kThreads, 1)
+fused_sweep_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                   void* __restrict__ out, TileParams tp, DeviceStatus* status, const FusedStreamArgs fa) {
+  grid_launch_dependents();
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const PairCtx cx = pair_setup(smem_raw, warp);
+  grid_dependency_wait();     // everything this launch reads was written by earlier work of the stream
+  if (warp < kNumThreads / 32) {
+    if (tp.batches > 0) pair_roles<false>(warp, lane, cx, map_a, map_b, out, nullptr, nullptr, tp, status);
+  } else {
+    const int grp = (warp - kNumThreads / 32) >> 3;
+    unsigned char* gsm = smem_raw + PairLayout::kTotal + grp * FusedLayout<kGroups>::kGroupBytes;
+    const StreamRole role{(int)threadIdx.x - kNumThreads - grp * 256, (int)blockIdx.x * kGroups + grp, (int)gridDim.x * kGroups,
+                          1 + grp};
+    if (fa.dec_gauges == 8)
+      decode_batch_body<OutT, float, 8>(role, *reinterpret_cast<DecBatchSmem<8>*>(gsm), fa.prod, fa.tab_w, fa.RB, nullptr, nullptr,
+                                        fa.n, fa.bm, fa.bn, fa.cstar32, fa.ldcs, fa.partials, fa.dec_tiles_per_block, fa.prod_stride);
+    else if (fa.dec_gauges == 4)
+      decode_batch_body<OutT, float, 4>(role, *reinterpret_cast<DecBatchSmem<4>*>(gsm), fa.prod, fa.tab_w, fa.RB, nullptr, nullptr,
+                                        fa.n, fa.bm, fa.bn, fa.cstar32, fa.ldcs, fa.partials, fa.dec_tiles_per_block, fa.prod_stride);
+    if (fa.enc_dense >= 0 && role.bid < fa.ja.blocks + fa.jb.blocks) {
+      role.sync();            // the group is done with the decode's shared memory
+      if (fa.enc_dense)
+        encode_body<__nv_bfloat16, __nv_bfloat16, false, 4, false, true>(role, gsm, fa.ja, fa.jb, 0);
+      else
+        encode_body<__nv_bfloat16, __nv_bfloat16, false, 4, false, false>(role, gsm, fa.ja, fa.jb, 0);
+    }
+  }
+  pair_teardown(cx, warp);
 }
 
 // ---------------------------------------------------------------- host side
@@ -774,6 +883,61 @@ fmm_status launch_pair(const BlockProductArgs& a, cudaStream_t st) {
   static unsigned long long smem_ok = 0;
   if (fmm_allow_dynamic_smem(k, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
   if (launch_dependent(k, dim3((unsigned)(2 * pairs)), dim3(kNumThreads), (size_t)L::kTotal, st, ma, mb, a.out, a.sA, a.sB, tp, a.status) != cudaSuccess)
+    return FMM_ERR_CUDA;
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+template <typename OutT, int kGroups>
+fmm_status launch_fused_t(const FusedSweepArgs& f, cudaStream_t st) {
+  using F = FusedLayout<kGroups>;
+  const BlockProductArgs& a = f.products;
+  CUtensorMap ma, mb;
+  TileParams tp{};
+  const int sms = sm_count();
+  if (sms < 2) return FMM_ERR_CUDA;
+  long long pairs = sms / 2;
+  if (f.have_products) {
+    if (!make_operand_map(&ma, false, a.A, a.rows_a, a.kdim, a.lda, a.a_batch, a.batches, BM)) return FMM_ERR_CUDA;
+    if (!make_operand_map(&mb, false, a.B, a.rows_b, a.kdim, a.ldb, a.b_batch, a.batches, PairLayout::BN / 2)) return FMM_ERR_CUDA;
+    tp.rows_a = (int)a.rows_a; tp.rows_b = (int)a.rows_b;
+    tp.elem_bytes = 2;
+    tp.kbytes = (int)a.kdim * 2;
+    tp.batches = a.batches;
+    tp.groups = 1;
+    tp.tiles_m = (int)((a.rows_a + 2 * BM - 1) / (2 * BM));
+    tp.tiles_n = (int)((a.rows_b + PairLayout::BN - 1) / PairLayout::BN);
+    tp.ldo = a.ldo; tp.o_batch = a.o_batch;
+    tp.out_mode = 0; tp.out_bf16 = 0;
+    tp.wide = rows_32b_aligned(a);
+    tp.wait_limit_ns = kDefaultWaitLimitNs;
+  } else {
+    std::memset(&ma, 0, sizeof(ma)); std::memset(&mb, 0, sizeof(mb));
+    tp.batches = 0;             // the tensor-core roles do nothing in this launch
+    tp.wait_limit_ns = kDefaultWaitLimitNs;
+  }
+  FusedStreamArgs fa{};
+  fa.dec_gauges = f.dec_gauges;
+  fa.prod = f.dec_prod; fa.tab_w = f.dec_tab; fa.RB = f.dec_RB; fa.n = f.n; fa.bm = f.bm; fa.bn = f.bn;
+  fa.cstar32 = f.cstar32; fa.ldcs = (long long)f.n * f.bn; fa.partials = f.partials; fa.prod_stride = f.dec_prod_stride;
+  const int nblocks = (int)(2 * pairs) * kGroups;
+  if (f.dec_gauges) {
+    const long long pos = 256 / f.dec_gauges;
+    const long long tiles = (f.bm * (f.bn >> 2) + pos - 1) / pos;
+    fa.dec_tiles_per_block = (int)((tiles + nblocks - 1) / nblocks);
+  }
+  fa.enc_dense = -1;
+  if (f.have_encode) {
+    size_t smem = 0; int dense = 0;
+    if (!fmm_encode_jobs_for_blocks(f.enc_a, f.enc_b, nblocks, &fa.ja, &fa.jb, &smem, &dense)) return FMM_ERR_SHAPE;
+    if (smem > (size_t)F::kGroupBytes) return FMM_ERR_SHAPE;
+    fa.enc_dense = dense;
+  }
+  static_assert(sizeof(DecBatchSmem<4>) <= F::kGroupBytes && sizeof(DecBatchSmem<8>) <= F::kGroupBytes, "group shared memory");
+  auto k = fused_sweep_kernel<OutT, kGroups>;
+  static unsigned long long smem_ok = 0;
+  if (fmm_allow_dynamic_smem(k, F::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
+  if (launch_dependent(k, dim3((unsigned)(2 * pairs)), dim3(F::kThreads), (size_t)F::kTotal, st, ma, mb, a.out, tp, a.status, fa) != cudaSuccess)
     return FMM_ERR_CUDA;
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
@@ -1305,4 +1469,16 @@ fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
   const bool narrow = a.rows_b <= 128;
   if (fp8) return narrow ? launch_t<128, true>(a, st) : launch_t<256, true>(a, st);
   return narrow ? launch_t<128, false>(a, st) : launch_t<256, false>(a, st);
+}
+
+int fused_sweep_blocks(int groups) { return (sm_count() / 2) * 2 * groups; }
+
+fmm_status launch_fused_sweep(const FusedSweepArgs& f, cudaStream_t st) {
+  if (f.output != FMM_F32 && f.output != FMM_BF16) return FMM_ERR_DTYPE;
+  if (f.dec_gauges != 0 && f.dec_gauges != 4 && f.dec_gauges != 8) return FMM_ERR_ARG;
+  if (f.groups == 1)
+    return f.output == FMM_F32 ? launch_fused_t<float, 1>(f, st) : launch_fused_t<__nv_bfloat16, 1>(f, st);
+  if (f.groups == 2)
+    return f.output == FMM_F32 ? launch_fused_t<float, 2>(f, st) : launch_fused_t<__nv_bfloat16, 2>(f, st);
+  return FMM_ERR_ARG;
 }

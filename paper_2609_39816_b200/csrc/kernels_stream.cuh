@@ -63,6 +63,7 @@ cudaError_t launch_joint_round(int storage, const void* X, int64_t ldx, int gr, 
 // written to scale[R] and divided out before rounding.  With use_scale == 2 there is one scale per row of every
 // block sum: amax_bits and scale are [R][br]; scale = amax / 448 in fp32 (1 for an all-zero row).  use_scale == 3 (model
 // schedule): one scale per 128 consecutive entries of a row, see EncodeOperand::scale_rows.
+// storage may also be FMM_E4M3 with product FMM_E4M3 (use_scale 0 or 1): the source holds codes, sixteen per vector.
 // h_tab = host copy of the same table (its list lengths size the kernel's shared memory).
 cudaError_t launch_encode(int storage, int product, const void* X, int64_t ldx, int gr, int gc, int64_t br,
                           int64_t bc, const CoefTable* d_tab, const CoefTable* h_tab, void* out, int64_t out_stride,
@@ -81,9 +82,31 @@ struct EncodeOperand {
   const CoefTable* d_tab; const CoefTable* h_tab; void* out; int64_t out_stride; unsigned* amax_bits; float* scale;
   int scale_rows;   // use_scale 3 only: rows sharing a scale (1 or 128); amax_bits / scale are [R][ceil(br/scale_rows)][ceil(bc/128)]
   int bf16_first;   // use_scale 3 only: round the block sum to bf16 before it is quantised
+  const float* pre_scale = nullptr;   // use_scale 1 only: DEVICE, one float; the source's codes are in units of it and
+                                      // scale[r] receives (this pass's scale) * pre_scale[0]
 };
 cudaError_t launch_encode_pair(int storage, int product, const EncodeOperand& a, const EncodeOperand* b, bool amax_only,
                                int use_scale, cudaStream_t st);
+
+// One operand of an encode launch.  A launch carries up to two (A and B of one product): blocks [0, a.blocks) work
+// on the first, the rest on the second, so both operands are encoded side by side without a second stream.
+struct EncodeJob {
+  const void* X; int64_t ldx; int gc; int64_t br, bc;
+  const CoefTable* tab; void* out; unsigned* amax_bits; float* scale_out;
+  int tiles_per_block; int64_t rstride; int stream_out; int blocks;
+  int scale_rows;    // use_scale 3: rows of a block sum that share a scale (1: the input's 1 x 128 scales; 128: the weight's 128 x 128)
+  int bf16_first;    // use_scale 3: the block sum is first rounded to bf16 (weights are stored in bf16 before they are quantised)
+  const float* pre_scale;   // use_scale 1: the source holds codes in units of *pre_scale (an outer level's scale); the
+                            // scale written out is the product of the two.  Null: 1.
+};
+
+// The two jobs of a bf16 -> bf16 encode without scales whose work is spread over `nblocks` blocks of 256 threads that
+// exist already (the streaming groups of the fused sweep kernel) instead of a grid of its own: blocks [0, ja->blocks)
+// take operand a, the next jb->blocks take b, in proportion to their sizes.  *smem_bytes: shared memory one block
+// needs; *dense: every list reads the four cells of a 2 x 2 grid in one order (the register-chain variant applies).
+// False if the tables do not fit this path (more than four cells per grid, positions beyond 32-bit indexing).
+bool fmm_encode_jobs_for_blocks(const EncodeOperand& a, const EncodeOperand& b, int nblocks, EncodeJob* ja, EncodeJob* jb,
+                                size_t* smem_bytes, int* dense);
 
 // Bt[N x K] = B[K x N]^T for 2- or 4-byte elements.
 cudaError_t launch_transpose(int elem_bytes, const void* B, int64_t ldb, int64_t K, int64_t N, void* Bt,
@@ -142,6 +165,25 @@ struct BlockProductArgs {
   unsigned long long wait_limit_ns;    // 0: default (2 s)
 };
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st);
+
+// One launch of a pipelined gauge sweep (bf16 storage and products, no scales, batches of four or eight one-level
+// algorithms): the block products of one batch on the tensor cores and, in the same CTAs, the error-only decode of the
+// batch before it and the encode of the batch after it.  Each of the three parts may be absent (pipeline head and tail).
+struct FusedSweepArgs {
+  int groups;                   // streaming groups (of eight warps) per CTA: 1 or 2
+  int output;                   // FMM_F32 / FMM_BF16: the dtype the decoded result is rounded to before the error is taken
+  int have_products;            // products: operands, batch count and output as for launch_block_products (bf16, out_mode 0)
+  BlockProductArgs products;
+  int dec_gauges;               // 0: no decode; 4 / 8: algorithms in the decoded batch
+  const float* dec_prod; int64_t dec_prod_stride; const CoefTable* dec_tab; int dec_RB;
+  int n; int64_t bm, bn;        // C grid columns and block size
+  const float* cstar32;
+  double* partials;             // [dec_gauges][fused_sweep_blocks(groups)] error partials of the decoded batch
+  int have_encode;              // encode: the two operands as for launch_encode_pair (bf16 -> bf16, 2 x 2 grids)
+  EncodeOperand enc_a, enc_b;
+};
+int fused_sweep_blocks(int groups);   // number of streaming blocks (= partial sums per algorithm) of a fused launch
+fmm_status launch_fused_sweep(const FusedSweepArgs& f, cudaStream_t st);
 
 // Batched block products under the model schedule (scale mode 3): e4m3 codes A [batches][rows_a][kdim] (K-major, lda) and
 // B [batches][rows_b][kdim]; G = ceil(kdim / 128) groups; scales sA [batches][rows_a][G], sB [batches][ceil(rows_b/128)][G];

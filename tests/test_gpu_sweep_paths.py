@@ -57,6 +57,30 @@ def test_pipelined_sweep_gives_the_bits_of_the_serial_one(lib, Pd, scale, level)
         assert np.array_equal(piped, serial)
 
 
+@pytest.mark.parametrize("M,K,N,G,O", [(2048, 2048, 2048, 27, "bf16"), (512, 1024, 768, 16, "f32"), (1024, 256, 2048, 9, "bf16")])
+def test_fused_sweep_launches_against_the_serial_path(lib, M, K, N, G, O):
+    """FMM_FLAG_SWEEP_FUSED: products of a batch, decode of the batch before and encode of the batch after in one launch.
+    Every algorithm's C is the same bits as on the serial path; its error sum is added over another partition of the
+    outputs (the fused launch has its own number of streaming blocks), so ratios agree to 1e-6, and run to run they are
+    bit-identical.  G = 27 leaves a batch of two and one of one behind the fused batches (8 + 8 + 8 | 2 + 1)."""
+    At, Wt = _ops(12, M, K, N)
+    P, Q, S = _gauges(G, seed=9)
+    s1 = lib.scheme_builtin("strassen222")
+    mk = lambda fl: lib.GemmDesc.make(M, K, N, "bf16", "bf16", O, weight_layout=True, flags=fl)
+    ws = gu.workspace(lib.error_sweep_workspace(s1, mk(0), G))
+    serial, ss = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_SERIAL), At, Wt, ws)
+    n0 = lib.launch_count()
+    fused, sf = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_FUSED), At, Wt, ws)
+    n_fused = lib.launch_count() - n0
+    n0 = lib.launch_count()
+    lib.error_sweep(s1, 0, P, Q, S, mk(0), At, Wt, ws)
+    assert n_fused < lib.launch_count() - n0              # the fused path really ran: far fewer launches
+    assert np.all(np.abs(fused - serial) <= 1e-6 * serial)
+    assert sf["count_gt2"] == ss["count_gt2"]
+    again, _ = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_FUSED), At, Wt, ws)
+    assert np.array_equal(again, fused)
+
+
 def test_sweep_in_two_calls_is_the_sweep_in_one(lib):
     """Resuming: gauges [0, G1) in one call and [G1, G) in a second (pointer offset into the gauge arrays) give the
     ratios of the single call, up to the grouping of a batch's error partials (1e-6), and the same summary."""
