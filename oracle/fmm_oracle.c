@@ -854,6 +854,78 @@ static int64_t split_high(int64_t x) {
   return y >= 0 ? y / 256 : -((-y + 255) / 256);
 }
 
+/* The control of Section 4.2 that BREAKS condition (iii) of Proposition 1: the scales sit on fine groups of h = g / k
+ * inner indices (one per block column of the call) while a call still spans g.  A block sum then mixes codes that
+ * carry different scales, so it cannot stay an integer: it is formed of the dequantised values code * scale (fp32,
+ * ascending (i,l)), and "rounded again with one scale, set by its largest magnitude" — one scale per block sum and
+ * call, s = max|x| / b2 in fp32 (1 if all zero), codes = rint(x / s): the quantiser's own rule with the full int8
+ * range b2 = 127 (a reading: the paper names neither).  The products of the new codes are exact integers; each is
+ * rescaled (P * sA) * sB in fp32 and combined with w in fp32, ascending r within a call, calls ascending.
+ * cA [M][K], cB [N][K]: codes; dA [M][K/h], dB [N][K/h]: fine-group scales.  The largest magnitude of a block sum
+ * depends on every row it reads, so changing one token row can move every output row.                           */
+int orc_int8_finegroup_control(int m, int k, int n, int R, const double* U, const double* V, const double* W,
+                               const double* cA, const double* dA, const double* cB, const double* dB, int64_t M,
+                               int64_t K, int64_t N, int g, int b2, int od, double* out) {
+  if (M % m || N % n || g % k || K % g) return 1;
+  const int64_t calls = K / g, bm = M / m, bn = N / n, Gf = K / (g / k);
+  const int h = g / k;
+  float* Sa = (float*)malloc(sizeof(float) * bm * h);
+  float* Sb = (float*)malloc(sizeof(float) * bn * h);
+  float* acc = (float*)calloc((size_t)M * N, sizeof(float));
+  for (int64_t q = 0; q < calls; ++q)
+    for (int r = 0; r < R; ++r) {
+      float amaxA = 0.0f, amaxB = 0.0f;
+      for (int64_t p = 0; p < bm; ++p)
+        for (int t = 0; t < h; ++t) {
+          float sum = 0.0f;
+          for (int i = 0; i < m; ++i)
+            for (int l = 0; l < k; ++l) {
+              const float u = (float)U[(r * m + i) * k + l];
+              if (u == 0.0f) continue;
+              const int64_t row = i * bm + p, col = q * g + l * h + t;
+              const float x = (float)cA[row * K + col] * (float)dA[row * Gf + col / h];   /* dequantised entry */
+              sum = fmaf(u, x, sum);
+            }
+          Sa[p * h + t] = sum;
+          if (fabsf(sum) > amaxA) amaxA = fabsf(sum);
+        }
+      for (int64_t c = 0; c < bn; ++c)
+        for (int t = 0; t < h; ++t) {
+          float sum = 0.0f;
+          for (int l = 0; l < k; ++l)
+            for (int j = 0; j < n; ++j) {
+              const float v = (float)V[(r * k + l) * n + j];
+              if (v == 0.0f) continue;
+              const int64_t row = j * bn + c, col = q * g + l * h + t;
+              const float x = (float)cB[row * K + col] * (float)dB[row * Gf + col / h];
+              sum = fmaf(v, x, sum);
+            }
+          Sb[c * h + t] = sum;
+          if (fabsf(sum) > amaxB) amaxB = fabsf(sum);
+        }
+      const float sA = amaxA == 0.0f ? 1.0f : amaxA / (float)b2;
+      const float sB = amaxB == 0.0f ? 1.0f : amaxB / (float)b2;
+      for (int64_t x = 0; x < bm * h; ++x) Sa[x] = rintf(Sa[x] / sA);   /* the second rounding: one scale per block sum */
+      for (int64_t x = 0; x < bn * h; ++x) Sb[x] = rintf(Sb[x] / sB);
+      for (int64_t p = 0; p < bm; ++p)
+        for (int64_t c = 0; c < bn; ++c) {
+          int64_t prod = 0;
+          for (int t = 0; t < h; ++t) prod += (int64_t)Sa[p * h + t] * (int64_t)Sb[c * h + t];
+          const float scaled = ((float)prod * sA) * sB;
+          for (int i = 0; i < m; ++i)
+            for (int j = 0; j < n; ++j) {
+              const float w = (float)W[(r * m + i) * n + j];
+              if (w == 0.0f) continue;
+              float* dst = &acc[(i * bm + p) * N + j * bn + c];
+              *dst = fmaf(w, scaled, *dst);
+            }
+        }
+    }
+  for (int64_t x = 0; x < M * N; ++x) out[x] = orc_round((double)acc[x], od);
+  free(Sa); free(Sb); free(acc);
+  return 0;
+}
+
 /* As orc_int8_certified, but every block sum of codes is split exactly, Ahat = A0 + 256 R_A with
  * R_A = floor((Ahat + 128) / 256) and A0 in [-128, 127], likewise Bhat, and each block product is rebuilt from
  * the four products of Eq. 2: A0 B0 + 256 (R_A B0 + A0 R_B) + 256^2 R_A R_B.  Arithmetic in 64-bit integers;

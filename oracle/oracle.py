@@ -28,7 +28,7 @@ __all__ = [
     "F32", "BF16", "E4M3", "F64", "Scheme", "build", "num_threads", "set_num_threads", "round_to", "strassen",
     "classical_scheme", "kron", "gauge", "sign_variant", "sign_variants", "brent_residual",
     "criteria", "scheme_gemm", "scheme_gemm_per_level", "classical_gemm", "exact_gemm", "fro_err", "rel_error",
-    "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "certificate",
+    "error_ratio", "summary", "quantize_rows", "int8_classical", "int8_certified", "int8_corrected", "int8_finegroup_control", "certificate",
     "hadamard_matrix", "hadamard_rotate", "row_pow2_scales", "joint_round_weights", "scheme_gemm_weights",
 ]
 
@@ -86,6 +86,8 @@ def _L():
                                                 [dp] * 2 + [C.c_int] + [dp] * 2)
         lib.orc_joint_round.restype = C.c_int
         lib.orc_joint_round.argtypes = [C.c_int] * 4 + [dp] * 3 + [i64] * 2 + [dp] + [C.c_int] + [dp] * 3
+        lib.orc_int8_finegroup_control.restype = C.c_int
+        lib.orc_int8_finegroup_control.argtypes = [C.c_int] * 4 + [dp] * 3 + [dp] * 4 + [i64] * 3 + [C.c_int] * 3 + [dp]
         lib.orc_certificate.restype = C.c_int
         lib.orc_certificate.argtypes = [C.c_int] * 4 + [dp] * 3 + [C.c_int] * 5 + [dp]
         _lib = lib
@@ -392,6 +394,22 @@ def int8_certified(s: "Scheme", cA, dA, cB, dB, g: int = 128, od="bf16", product
     if rc:
         raise ValueError("shape does not divide, or coefficients are not integers")
     return (out, mx, P) if products else (out, mx)
+
+
+def int8_finegroup_control(s: "Scheme", cA, dA, cB, dB, call: int = 128, b2: int = 127, od="bf16"):
+    """The control of Section 4.2 that breaks condition (iii): scales on fine groups of call / k inner indices (dA
+    [M, K / (call / k)], dB likewise) under calls of `call`; every mixed block sum is formed of dequantised values and
+    rounded again with ONE scale max|x| / b2 per block sum and call.  cA [M, K], cB [N, K] codes.  Returns [M, N]."""
+    m, k, n, R = s.dims
+    cA = _d(cA); cB = _d(cB); dA = _d(dA); dB = _d(dB)
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = np.empty((M, N))
+    rc = _L().orc_int8_finegroup_control(m, k, n, R, _p(_d(s.U)), _p(_d(s.V)), _p(_d(s.W)), _p(cA), _p(dA), _p(cB), _p(dB),
+                                         M, K, N, int(call), int(b2), _fmt(od), _p(out))
+    if rc:
+        raise ValueError("shape does not fit the call")
+    return out
 
 
 def certificate(s: "Scheme", bA: int, bB: int, h: int, g: int, acc_bits: int = 31):

@@ -104,12 +104,12 @@ def test_bound_is_sharp_and_violations_are_reported():
         oracle.int8_certified(oracle.gauge(S1, P, P, P), cA[:2], one[:2], cB[:2], one[:2])
 
 
-def _pairs_moved(run, A, rows=32):
+def _pairs_moved(run, A, rows=32, std=1.0):
     base = run(A)
     moved = set()
     for later in range(rows):
         A2 = A.copy()
-        A2[later] = gen.to_storage(gen.normal(77, 900 + later, (A.shape[1],)), "f32")[1]
+        A2[later] = gen.to_storage(gen.normal(77, 900 + later, (A.shape[1],), std=std), "f32")[1]
         out = run(A2)
         for earlier in range(later):
             if np.any(out[earlier] != base[earlier]):
@@ -130,6 +130,46 @@ def test_fp8_schedule_moves_exactly_the_48_same_offset_pairs():
         moved = _pairs_moved(lambda X: oracle.scheme_gemm(S2, X, B, "e4m3", "f32", scale_mode=mode), A)
         assert moved == want, (mode, len(moved))
     assert _pairs_moved(lambda X: oracle.classical_gemm(X, B, "e4m3", "f32", 2), A) == set()
+
+
+def test_fine_group_control_moves_all_496_pairs():
+    """Section 4.2, the control that breaks condition (iii): scales on groups of 32 indices while a call spans 128.
+    Every mixed block sum is rounded again with one scale set by its largest magnitude, which any of its rows can
+    change: all 496 (earlier, later) pairs move — the third of the printed counts 0 / 48 / 496.  With the scales on
+    groups of 128 (condition (iii) kept) the same inputs move none (test_row_locality_zero_of_496_pairs_move)."""
+    A = gen.to_storage(gen.normal(6, 1, (32, 128)), "f32")[1]
+    Bt = gen.to_storage(gen.normal(6, 2, (32, 128)), "f32")[1]
+    cB, dB = oracle.quantize_rows(Bt, 31, g=32)
+
+    def run(X):
+        cA, dA = oracle.quantize_rows(X, 31, g=32)
+        return oracle.int8_finegroup_control(S2, cA, dA, cB, dB, call=128, od="f32")
+    # "which any of its rows can change": a replacement row loud enough (N(0, 4^2) among N(0, 1) rows) to take over the
+    # largest magnitude of every block sum it enters changes every such scale, and every pair moves ...
+    assert len(_pairs_moved(run, A, std=4.0)) == 496
+    # ... while a replacement no louder than its neighbours changes a scale only when it held, or takes, the maximum:
+    # most pairs move, not all
+    quiet = len(_pairs_moved(run, A, std=1.0))
+    assert 350 < quiet < 496
+    # the same loud replacement leaves the two structural counts where they are: 0 for the certified call (scales on
+    # the call's own group of 128), 48 for block sums rounded to FP8
+    cB128, dB128 = oracle.quantize_rows(Bt, 31, g=128)
+
+    def run_cert(X):
+        cA, dA = oracle.quantize_rows(X, 31, g=128)
+        return oracle.int8_certified(S2, cA, dA, cB128, dB128, od="f32")[0]
+    assert _pairs_moved(run_cert, A, std=4.0) == set()
+    assert len(_pairs_moved(lambda X: oracle.scheme_gemm(S2, X, Bt.T.copy(), "e4m3", "f32"), A, std=4.0)) == 48
+    # the control is still a sound approximation of the product (it is the invariance that is lost, not the accuracy)
+    ref = A @ Bt.T
+    assert np.linalg.norm(run(A) - ref) <= 0.1 * np.linalg.norm(ref)     # code bound 31: a few per cent
+    # one fine group per call (call = 32 with a <1,1,1;1> algorithm) is the classical operator on groups of 32: row local
+    one = oracle.classical_scheme(1, 1, 1)
+
+    def run_cl(X):
+        cA, dA = oracle.quantize_rows(X, 31, g=32)
+        return oracle.int8_classical(cA, dA, cB, dB, g=32, od="f32")
+    assert _pairs_moved(run_cl, A, std=4.0) == set()
 
 
 def test_fp8_block_sums_leave_no_sign_variant_exact_on_integer_codes():
