@@ -93,13 +93,15 @@ typedef enum { FMM_F32 = 0, FMM_BF16 = 1, FMM_E4M3 = 2 } fmm_dtype;
                                  are the same); slower.  For callers that want one stream only, and for checking
                                  the pipelined path against.                                              */
 
-#define FMM_FLAG_SWEEP_FUSED 16 /* error_sweep only (bf16 storage and products, no scales, one-level algorithms on a
-                                 2 x 2 grid, else ignored): run each batch's block products, the decode of the batch
-                                 before it and the encode of the batch after it as ONE kernel launch whose CTAs carry
-                                 the tensor-core roles and, beside them, warps that stream the other two passes.  Same
-                                 C bits per algorithm; each error sum is added over another partition of the outputs
-                                 (ratios agree to 1e-8, bit-reproducible run to run).  On a power-limited B200 it is
-                                 no faster than the default pipeline: the passes overlap and the clock drops.      */
+#define FMM_FLAG_SWEEP_UNFUSED 16 /* error_sweep only: do not use the fused launches.  By default, where it applies (bf16
+                                 storage and products, no scales, one-level algorithms on a 2 x 2 grid, blocks larger
+                                 than 128 x 128), each batch's block products run as ONE kernel launch together with
+                                 the decode of the batch before it and the encode of the batch after it: the CTAs
+                                 carry the tensor-core roles and, beside them, warps that stream the other two passes.
+                                 Every algorithm's C is the same bits either way; its error sum is added over another
+                                 partition of the outputs (ratios agree to 1e-8; each path is bit-reproducible run to
+                                 run).  With this flag such sweeps take the three-stream pipeline that all other
+                                 sweeps use.                                                                    */
 #define FMM_FLAG_ROUND_PER_LEVEL 8 /* scheme_gemm on a handle made by scheme_kron (or "strassen444"): round the block
                                  sums at EVERY level.  The outer factor's block sums of A (and of B) are scaled
                                  and rounded to the product dtype; the inner factor's block sums are formed of
@@ -237,7 +239,10 @@ size_t classical_gemm_workspace(const fmm_gemm_desc* d);
 
 /* The classical product at the same dtypes (the paper's control, Section 3.1):
  * C = rnd_O( sA sB * rnd_Pd(A/sA) * rnd_Pd(B/sB) ), fp32 accumulation on the same tensor-core
- * kernel.  With storage == product == bf16 and weight layout the operands are read in place. */
+ * kernel.  With storage == product == bf16 the operands are read in place.  Operands that are already e4m3 codes
+ * (storage == product == FMM_E4M3, scale_mode 0, weight layout; one byte per element, leading dimensions a
+ * multiple of 16) are multiplied in place too: the tensor-core product of the codes alone, which is also how
+ * the library's own fp8 tensor rate is measured.                                                          */
 fmm_status classical_gemm(const fmm_gemm_desc* d, const void* dA, const void* dB, void* dC,
                           void* d_ws, size_t ws_bytes, void* cuda_stream);
 
@@ -314,7 +319,7 @@ size_t error_sweep_workspace(const fmm_scheme* base, const fmm_gemm_desc* d, int
  * Execution: equivalent algorithms share their operands, so up to eight of them (as many as fit the table limits:
  * products of the batch <= FMM_MAX_R) run as one encode, one product launch and one error-only decode; every
  * algorithm's arithmetic and summation order are those of a scheme_gemm call on it, and the call is bit-reproducible
- * run to run.  FMM_B200_NO_GAUGE_BATCH=1 in the environment runs one algorithm per launch set.              */
+ * run to run.                                                                                              */
 fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P, const double* Q,
                        const double* S, const fmm_gemm_desc* d, const void* dA, const void* dB,
                        const double* dCstar, double* h_ratios, fmm_sweep_summary* out, void* d_ws,

@@ -18,7 +18,7 @@ FLAG_REUSE_BHAT = 1
 FLAG_PRODUCTS_BF16 = 2
 FLAG_SWEEP_SERIAL = 4
 FLAG_ROUND_PER_LEVEL = 8
-FLAG_SWEEP_FUSED = 16
+FLAG_SWEEP_UNFUSED = 16
 _DT = {"f32": F32, "fp32": F32, "bf16": BF16, "e4m3": E4M3}
 
 EXPORTED_SYMBOLS = [

@@ -70,14 +70,6 @@ bool stream_wait(SideStream* s, cudaStream_t from, cudaStream_t to) {
   s->next = (s->next + 1) % kEventRing;
   return cudaEventRecord(e, from) == cudaSuccess && cudaStreamWaitEvent(to, e, 0) == cudaSuccess;
 }
-bool concurrency_enabled() {
-  static int on = -1;
-  if (on < 0) {
-    const char* e = std::getenv("FMM_B200_NO_OVERLAP");
-    on = (e && e[0] == '1') ? 0 : 1;
-  }
-  return on == 1;
-}
 }  // namespace
 
 namespace {
@@ -99,10 +91,12 @@ struct GemmLayout {
   int64_t sLvlA, sLvlB;
 };
 
-fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n) {
+// codes_ok: operands may already be e4m3 codes (classical_gemm on pre-quantised operands, read in place)
+fmm_status check_desc(const fmm_gemm_desc* d, int m, int k, int n, bool codes_ok = false) {
   if (!d) return FMM_ERR_ARG;
   if (d->M <= 0 || d->K <= 0 || d->N <= 0) return FMM_ERR_SHAPE;
-  if (d->storage != FMM_F32 && d->storage != FMM_BF16) return FMM_ERR_DTYPE;
+  const bool codes = codes_ok && d->storage == FMM_E4M3 && d->product == FMM_E4M3 && d->scale_mode == 0 && d->b_is_weight_layout;
+  if (d->storage != FMM_F32 && d->storage != FMM_BF16 && !codes) return FMM_ERR_DTYPE;
   if (d->product != FMM_BF16 && d->product != FMM_E4M3) return FMM_ERR_DTYPE;
   if (d->output != FMM_F32 && d->output != FMM_BF16) return FMM_ERR_DTYPE;
   if (d->scale_mode != 0 && !(d->scale_mode >= 1 && d->scale_mode <= 3 && d->product == FMM_E4M3)) return FMM_ERR_DTYPE;
@@ -359,26 +353,14 @@ fmm_status run_scheme(const fmm_scheme* s, const fmm_gemm_desc* d, const GemmLay
     dW_tab = at<CoefTable>(ws, L.tabW);
   }
   const SchemeRun r{s, d, L, ws, hA, hB, hW, dA_tab, dB_tab, dW_tab};
-  // encode A and encode B side by side: one launch whose blocks split between the two operands (they share nothing);
-  // with the side stream enabled by the environment the two run as separate launches on two streams instead
-  static const bool two_streams = [] { const char* e = std::getenv("FMM_B200_ENCODE_TWO_STREAMS"); return e && e[0] == '1'; }();
+  // encode A and encode B side by side: one launch whose blocks split between the two operands (they share nothing)
   if (d->flags & FMM_FLAG_ROUND_PER_LEVEL) {
     FMM_TRY(stage_encode_per_level(r, A, d->lda, false, st));
     if (!skip_b) FMM_TRY(stage_encode_per_level(r, Bsrc_kmajor, ldb_kmajor, true, st));
   } else if (skip_b) {
     FMM_TRY(stage_encode_a(r, A, st));
-  } else if (!two_streams) {
-    FMM_TRY(stage_encode_pair(r, A, Bsrc_kmajor, ldb_kmajor, st));
   } else {
-    SideStream* side = concurrency_enabled() ? side_stream() : nullptr;
-    cudaStream_t stB = st;
-    if (side) {
-      if (!stream_wait(side, st, side->stream)) return FMM_ERR_CUDA;
-      stB = side->stream;
-    }
-    FMM_TRY(stage_encode_b(r, Bsrc_kmajor, ldb_kmajor, stB));
-    FMM_TRY(stage_encode_a(r, A, st));
-    if (side && !stream_wait(side, side->stream, st)) return FMM_ERR_CUDA;
+    FMM_TRY(stage_encode_pair(r, A, Bsrc_kmajor, ldb_kmajor, st));
   }
   FMM_TRY(stage_products(r, st));
   return stage_decode(r, C, cstar32, err_out, st);
@@ -415,7 +397,7 @@ struct ClassicalLayout { size_t status, tab, amaxA, amaxB, sA, sB, bt, ahat, bha
 ClassicalLayout classical_layout(const fmm_gemm_desc* d) {
   ClassicalLayout L;
   const int ep = esize(d->product), es = esize(d->storage);
-  L.direct = d->storage == FMM_BF16 && d->product == FMM_BF16 && d->scale_mode == 0;
+  L.direct = d->storage == d->product && d->scale_mode == 0;   // bf16, or e4m3 codes: the operands are read in place
   size_t o = 0;
   L.status = o; o += align_up(sizeof(DeviceStatus));
   L.tab = o; o += align_up(sizeof(CoefTable));
@@ -476,12 +458,7 @@ fmm_status run_classical(const fmm_gemm_desc* d, const ClassicalLayout& L, const
 // kb * m * n <= 16 decode lists, kb in {1, 2, 4} (it must divide the decode's thread split); eight algorithms of at
 // most 8 products and 4 output cells each also fit (32 lists: the register-resident batch decode takes them).
 int sweep_batch(const fmm_scheme* s) {
-  static const int cap = [] {
-    const char* e = std::getenv("FMM_B200_NO_GAUGE_BATCH");
-    if (e && e[0] == '1') return 1;
-    const char* m = std::getenv("FMM_B200_MAX_GAUGE_BATCH");
-    return m ? std::max(1, std::atoi(m)) : 8;
-  }();
+  constexpr int cap = 8;
   if (cap >= 8 && 8 * s->R <= FMM_MAX_R && s->R <= 8 && s->m * s->n <= 4) return 8;
   for (int kb = 4; kb > 1; kb /= 2)
     if (kb <= cap && kb * s->R <= FMM_MAX_R && kb * s->m * s->n <= 16) return kb;
@@ -719,14 +696,14 @@ fmm_status fmm_device_status(const void* d_ws, void* cuda_stream) {
 }
 
 size_t classical_gemm_workspace(const fmm_gemm_desc* d) {
-  if (check_desc(d, 1, 1, 1) != FMM_OK) return 0;
+  if (check_desc(d, 1, 1, 1, true) != FMM_OK) return 0;
   return classical_layout(d).total;
 }
 
 fmm_status classical_gemm(const fmm_gemm_desc* d, const void* dA, const void* dB, void* dC, void* d_ws,
                           size_t ws_bytes, void* cuda_stream) {
   if (!d || !dA || !dB || !dC) return FMM_ERR_ARG;
-  FMM_TRY(check_desc(d, 1, 1, 1));
+  FMM_TRY(check_desc(d, 1, 1, 1, true));
   const ClassicalLayout L = classical_layout(d);
   FMM_TRY(check_ws(d_ws, ws_bytes, L.total));
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -877,22 +854,23 @@ fmm_status error_sweep(const fmm_scheme* base, int level, int G, const double* P
   void* gws2 = ws + L.gemm2;
   FMM_CUDA(cudaMemsetAsync(at<char>(gws2, L.g.status), 0, sizeof(DeviceStatus), st));
   // with phase timing on, or when the caller asks for it, the stages run back to back on the caller's stream
-  const bool serial = g_prof_on || (d->flags & FMM_FLAG_SWEEP_SERIAL) != 0 || !concurrency_enabled();
+  const bool serial = g_prof_on || (d->flags & FMM_FLAG_SWEEP_SERIAL) != 0;
   SideStream* side = serial ? nullptr : side_stream();
   fmm_scheme batched;                   // dimensions only: a batch of kc algorithms looks like one with kc * R products
   batched.m = base->m; batched.k = base->k; batched.n = base->n;
   fmm_status loop_rc = FMM_OK;
-  // Fused pipeline (FMM_FLAG_SWEEP_FUSED; bf16 storage and products, no scales, batches of four or eight one-level
+  // Fused pipeline (unless FMM_FLAG_SWEEP_UNFUSED; bf16 storage and products, no scales, batches of four or eight one-level
   // algorithms): ONE launch per batch runs its block products together with the decode of the batch before and the
   // encode of the batch after, in the same CTAs (launch_fused_sweep), on the caller's stream; the pipeline starts with a
   // plain encode and ends with a decode-only launch.  Batches of one or two algorithms at the end of the list take the
   // ordinary path below.  Measured on B200: the three passes do overlap inside the launch, and the chip answers by
   // lowering its clock (the board's power limit: tensor cores and the memory system cannot both run flat out), so the
-  // sweep takes the same time as with the passes one after another — hence opt-in, not the default.
+  // gain over the passes one after another is a few per cent (512 gauges of config 3: 42-43 ms against 44-46 ms after
+  // idle, 45.4 against 46.8-47.9 ms sustained), not the sum of the hidden passes.
   size_t first_plain_chunk = 0;
   const int kFusedGroups = 2;
   const int64_t bm_ = d->M / base->m, bn_ = d->N / base->n, bk_ = d->K / base->k;
-  const bool fused_ok = (d->flags & FMM_FLAG_SWEEP_FUSED) && !serial && kb >= 4 && d->storage == FMM_BF16 && d->product == FMM_BF16 && d->scale_mode == 0 &&
+  const bool fused_ok = !(d->flags & FMM_FLAG_SWEEP_UNFUSED) && !serial && kb >= 4 && d->storage == FMM_BF16 && d->product == FMM_BF16 && d->scale_mode == 0 &&
                         !(d->flags & FMM_FLAG_PRODUCTS_BF16) && base->m * base->k <= 4 && base->n * base->k <= 4 &&
                         base->m * base->n <= 4 && bm_ > 128 && bn_ > 128 &&
                         fused_sweep_blocks(kFusedGroups) <= kFusedPartialsPerGauge && fused_sweep_blocks(kFusedGroups) >= 2 &&

@@ -943,14 +943,6 @@ fmm_status launch_fused_t(const FusedSweepArgs& f, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
-bool pair_kernel_enabled() {
-  static int on = -1;
-  if (on < 0) {
-    const char* e = std::getenv("FMM_B200_NO_PAIR");
-    on = (e && e[0] == '1') ? 0 : 1;
-  }
-  return on == 1;
-}
 
 // ---------------------------------------------------------------- group-scaled int8 GEMM
 // The classical int8 operator of the quantisation specification (Appendix D) as one kernel:
@@ -1463,7 +1455,7 @@ fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {
   const bool fp8 = (a.product == FMM_E4M3);
   if (!fp8 && a.product != FMM_BF16) return FMM_ERR_DTYPE;
   // large problems: CTA pairs on 256 x 256 tiles (less L2 traffic per flop)
-  if (a.rows_a > 128 && a.rows_b > 128 && pair_kernel_enabled() && !a.selftest_no_producer)
+  if (a.rows_a > 128 && a.rows_b > 128 && !a.selftest_no_producer)
     return fp8 ? launch_pair<true>(a, st) : launch_pair<false>(a, st);
   // narrow problems use the 128-column tile (less padding, more tiles in flight)
   const bool narrow = a.rows_b <= 128;

@@ -17,10 +17,6 @@ int64_t& fmm_launch_counter() {
   return c;
 }
 
-bool fmm_pdl_enabled() {
-  static const bool on = [] { const char* e = std::getenv("FMM_B200_NO_PDL"); return !(e && e[0] == '1'); }();
-  return on;
-}
 
 namespace {
 
@@ -197,7 +193,6 @@ static bool make_job(const EncodeOperand& o, EncodeJob* j, size_t* smem) {
   if (vecs > 0) split_tiles((vecs + kEncPos - 1) / kEncPos, &grid, &tpb);
   // outputs larger than the part of L2 that keeps shared data (~60 MB) will have left it before they are read
   int stream_out = (int64_t)o.h_tab->R * o.out_stride * (int64_t)sizeof(DstT) > ((int64_t)48 << 20) ? 1 : 0;
-  if (const char* e = std::getenv("FMM_B200_ENC_STREAM")) stream_out = std::atoi(e);
   *j = EncodeJob{o.X, o.ldx, o.gc, o.br, o.bc, o.d_tab, o.out, o.amax_bits, o.scale, tpb, o.out_stride, stream_out, grid,
                  o.scale_rows > 0 ? o.scale_rows : 1, o.bf16_first, o.pre_scale};
   return true;
@@ -272,8 +267,7 @@ cudaError_t launch_encode_t(const EncodeOperand& a, const EncodeOperand* b, bool
   if (use_scale == 3)
     e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale)
                   : launch_encode_k<SrcT, DstT, false, kSplit, kCanM3>(grid, smem, st, ja, jb, use_scale);
-  else if (kSplit == 4 && dense_four_cells(*a.h_tab) && (b == nullptr || dense_four_cells(*b->h_tab)) &&
-           std::getenv("FMM_B200_NO_DENSE_ENCODE") == nullptr)
+  else if (kSplit == 4 && dense_four_cells(*a.h_tab) && (b == nullptr || dense_four_cells(*b->h_tab)))
     e = amax_only ? launch_encode_k<SrcT, DstT, true, kSplit, false, true>(grid, smem, st, ja, jb, use_scale)
                   : launch_encode_k<SrcT, DstT, false, kSplit, false, true>(grid, smem, st, ja, jb, use_scale);
   else
@@ -545,7 +539,7 @@ static cudaError_t launch_decode_p(int output, const ProdT* prod, int64_t prod_s
   if (C == nullptr && cstar32 == nullptr) return cudaErrorInvalidValue;
   // a batch of four small algorithms, error only: products straight into registers (decode_batch_kernel)
   if ((gauges == 4 || gauges == 8) && C == nullptr && R % gauges == 0 && R / gauges <= kBatchR && m * n <= 4 &&
-      h_tab->R == gauges * m * n && std::getenv("FMM_B200_NO_BATCH_DECODE") == nullptr) {
+      h_tab->R == gauges * m * n) {
     if (bm * (bn >> 2) + kDecThreads * 8 >= (int64_t)1 << 31) return cudaErrorInvalidValue;
     const int pos = kDecThreads / gauges;
     int grid, tpb;

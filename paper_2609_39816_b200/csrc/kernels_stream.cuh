@@ -17,8 +17,6 @@ int64_t& fmm_launch_counter();
 // TMEM allocation, table loads) while the previous kernel of the same stream drains; it must execute
 // grid_dependency_wait() before it touches anything that kernel wrote.  Kernels that may be followed by such a launch
 // call grid_launch_dependents() early.  Both are no-ops when the launch carries no programmatic dependency.
-// FMM_B200_NO_PDL=1 in the environment turns the attribute off (ordinary stream order).
-bool fmm_pdl_enabled();
 
 // cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per (kernel, device): `done_mask` is the caller's static word for
 // one kernel, bit d set once device d has been configured (devices beyond 63 are configured on every call).
@@ -42,7 +40,7 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = fmm_pdl_enabled() ? 1 : 0;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }

@@ -48,7 +48,7 @@ def test_pipelined_sweep_gives_the_bits_of_the_serial_one(lib, Pd, scale, level)
     P, Q, S = _gauges(G)
     s1 = lib.scheme_builtin("strassen222")
     s = lib.scheme_kron(s1, s1) if level == 1 else s1
-    d = lib.GemmDesc.make(M, K, N, "bf16", Pd, "bf16", weight_layout=True, scale_mode=scale)
+    d = lib.GemmDesc.make(M, K, N, "bf16", Pd, "bf16", weight_layout=True, scale_mode=scale, flags=lib.FLAG_SWEEP_UNFUSED)
     ds = lib.GemmDesc.make(M, K, N, "bf16", Pd, "bf16", weight_layout=True, scale_mode=scale, flags=lib.FLAG_SWEEP_SERIAL)
     ws = gu.workspace(lib.error_sweep_workspace(s, d, G))
     serial, _ = lib.error_sweep(s, level, P, Q, S, ds, At, Wt, ws)
@@ -57,9 +57,9 @@ def test_pipelined_sweep_gives_the_bits_of_the_serial_one(lib, Pd, scale, level)
         assert np.array_equal(piped, serial)
 
 
-@pytest.mark.parametrize("M,K,N,G,O", [(2048, 2048, 2048, 27, "bf16"), (512, 1024, 768, 16, "f32"), (1024, 256, 2048, 9, "bf16")])
+@pytest.mark.parametrize("M,K,N,G,O", [(2048, 2048, 2048, 27, "bf16"), (1024, 512, 1536, 16, "f32"), (1024, 256, 2048, 9, "bf16")])
 def test_fused_sweep_launches_against_the_serial_path(lib, M, K, N, G, O):
-    """FMM_FLAG_SWEEP_FUSED: products of a batch, decode of the batch before and encode of the batch after in one launch.
+    """The fused launches (default where they apply): products of a batch, decode of the batch before and encode of the batch after in one launch.
     Every algorithm's C is the same bits as on the serial path; its error sum is added over another partition of the
     outputs (the fused launch has its own number of streaming blocks), so ratios agree to 1e-6, and run to run they are
     bit-identical.  G = 27 leaves a batch of two and one of one behind the fused batches (8 + 8 + 8 | 2 + 1)."""
@@ -70,14 +70,15 @@ def test_fused_sweep_launches_against_the_serial_path(lib, M, K, N, G, O):
     ws = gu.workspace(lib.error_sweep_workspace(s1, mk(0), G))
     serial, ss = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_SERIAL), At, Wt, ws)
     n0 = lib.launch_count()
-    fused, sf = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_FUSED), At, Wt, ws)
+    fused, sf = lib.error_sweep(s1, 0, P, Q, S, mk(0), At, Wt, ws)
     n_fused = lib.launch_count() - n0
     n0 = lib.launch_count()
-    lib.error_sweep(s1, 0, P, Q, S, mk(0), At, Wt, ws)
+    piped, _ = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_UNFUSED), At, Wt, ws)
     assert n_fused < lib.launch_count() - n0              # the fused path really ran: far fewer launches
+    assert np.array_equal(piped, serial)                  # the three-stream pipeline uses the serial path's kernels
     assert np.all(np.abs(fused - serial) <= 1e-6 * serial)
     assert sf["count_gt2"] == ss["count_gt2"]
-    again, _ = lib.error_sweep(s1, 0, P, Q, S, mk(lib.FLAG_SWEEP_FUSED), At, Wt, ws)
+    again, _ = lib.error_sweep(s1, 0, P, Q, S, mk(0), At, Wt, ws)
     assert np.array_equal(again, fused)
 
 

@@ -129,6 +129,35 @@ def test_kron_and_gauges_match_oracle(lib):
         lib.gauge_apply(s1, np.eye(2), np.eye(2), np.eye(2), level=1)
 
 
+def test_gauge_apply_against_the_numpy_definition(lib):
+    """The library's gauge against the definition written with library routines of another kind (numpy's inverse and
+    einsum), not against the oracle's loops, which have the same shape as the library's: U'_r = P^T U_r Q^-T,
+    V'_r = Q^T V_r S^-T, W'_r = P^-1 W_r S; and running the gauged algorithm in exact arithmetic gives A B."""
+    s1 = lib.scheme_builtin("strassen222")
+    s2 = lib.scheme_builtin("strassen444")
+    U1, V1, W1 = s1.coefficients()
+    rng = np.random.default_rng(5)
+    for idx in range(3):
+        P, Q, S = (gen.gauge_log_uniform_cond(9, 3 * idx + i, 2) for i in range(3))
+        Pi, Qi, Si = np.linalg.inv(P), np.linalg.inv(Q), np.linalg.inv(S)
+        want = (np.einsum("ia,ril,bl->rab", P, U1, Qi), np.einsum("la,rlj,bj->rab", Q, V1, Si),
+                np.einsum("ai,rij,jb->rab", Pi, W1, S))
+        got = lib.gauge_apply(s1, P, Q, S).coefficients()
+        for a, b in zip(got, want):
+            assert np.allclose(a, b, rtol=1e-11, atol=1e-11 * np.abs(b).max())
+        # level 1 on the nested handle = Kronecker product of the gauged outer factor with the inner one
+        g2 = lib.gauge_apply(s2, P, Q, S, level=1).coefficients()
+        kron = lambda X, Y: np.einsum("pab,qcd->pqacbd", X, Y).reshape(49, 4, 4)
+        for a, X, Y in zip(g2, want, (U1, V1, W1)):
+            assert np.allclose(a, kron(X, Y), rtol=1e-11, atol=1e-11 * np.abs(X).max())
+        # Eq. 1 with the gauged coefficients, in fp64, on random 2 x 2 block matrices of scalars
+        A, B = rng.standard_normal((2, 2)), rng.standard_normal((2, 2))
+        Ug, Vg, Wg = got
+        Mr = np.einsum("ril,il->r", Ug, A) * np.einsum("rlj,lj->r", Vg, B)
+        C = np.einsum("rij,r->ij", Wg, Mr)
+        assert np.allclose(C, A @ B, rtol=0, atol=1e-9 * np.abs(Ug).max() * np.abs(Vg).max() * np.abs(Wg).max())
+
+
 def test_descriptor_validation_without_gpu(lib):
     s2 = lib.scheme_builtin("strassen444")
     ok = lib.GemmDesc.make(4096, 4096, 4096, "bf16", "bf16", "bf16")
