@@ -9,6 +9,7 @@ codes move, and assert that the result and the error-amplification ratio do not.
 """
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from fmm_inputs import generators as gen
@@ -129,3 +130,25 @@ def test_integer_domain_is_the_same_in_both_forms():
     ref = A @ B
     for mode in ("f32chain", "f64"):
         assert np.array_equal(oracle.scheme_gemm(S2, A, B, "bf16", "f32", sum=mode), ref)
+
+
+def test_two_term_sums_of_bf16_values_are_the_same_in_both_forms_at_any_exponent_gap():
+    """For TWO bf16 terms with coefficients +-1 the fp32 chain, the exact sum rounded once, and a single correctly
+    rounded bf16 addition all agree — the fp32 sum is exact up to
+    16 binades apart, and beyond that the small term cannot reach a rounding boundary of bf16.  One level of Strassen
+    has only one- and two-term sums; operands span 60 binades and include exact ties."""
+    rng = np.random.default_rng(3)
+    n = 64
+    mant = rng.integers(128, 256, size=(n, n)).astype(np.float64)            # 8 significant bits
+    A = np.ldexp(mant, rng.integers(-30, 30, size=(n, n))) * rng.choice([-1.0, 1.0], size=(n, n))
+    # force ties: A22 = half an ulp of A11 wherever the row index is even
+    e11 = np.floor(np.log2(np.abs(A[:n // 2, :n // 2])))
+    A[n // 2::2, n // 2:] = np.ldexp(1.0, (e11 - 8).astype(int))[::2]
+    B = np.eye(n)
+    _, pc = oracle.scheme_gemm(S1, A, B, "bf16", "f32", parts=True, sum="f32chain")
+    _, pd_ = oracle.scheme_gemm(S1, A, B, "bf16", "f32", parts=True, sum="f64")
+    assert np.array_equal(pc["Ahat"], pd_["Ahat"])
+    # and torch's own bf16 addition (a library routine: one rounding of the exact sum) gives the same codes for M1 = A11 + A22
+    a11 = torch.from_numpy(A[:n // 2, :n // 2]).to(torch.bfloat16)
+    a22 = torch.from_numpy(A[n // 2:, n // 2:]).to(torch.bfloat16)
+    assert np.array_equal((a11.double() + a22.double()).to(torch.bfloat16).double().numpy(), pc["Ahat"][0])
