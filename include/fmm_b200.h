@@ -386,6 +386,24 @@ fmm_status int8_gemm_corrected(const fmm_scheme* s, const int8_t* d_cA, const fl
                                const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc,
                                void* d_ws, size_t ws_bytes, void* cuda_stream);
 
+/* The control of the row-pair test that BREAKS condition (iii) of Proposition 1 (Section 4.2): scales on fine groups
+ * of h = call / k inner indices (one per block column of a call) while a call of the algorithm spans `call` indices.
+ * The operands are quantised here (rows of d_A and of d_B, the latter in the weight layout [N][K]; d = max|x| /
+ * code_bound per row and fine group, 1 if all zero, codes rounded to nearest even).  A block sum then mixes codes
+ * with different scales: it is formed of the dequantised values code * scale (fp32 chain, ascending block order) and
+ * rounded again with ONE scale per block sum and call, s = max|x| / second_bound (a reading: the paper names neither
+ * the rule nor the bound of this second rounding; this is its quantiser's rule).  Products of the new codes are exact
+ * integers, rescaled (P * sA) * sB and combined with w in fp32, ascending r within a call, calls ascending; one
+ * rounding to `output`.  Because a block sum's largest magnitude depends on every row it reads, changing one token
+ * row can move every output row: the paper counts all 496 pairs.  A demonstration on tiles (M * K, N * K < 2^31),
+ * plain kernels, not a fast path.  d_A [M][lda], d_B [N][ldb]: DEVICE fp32; d_C: DEVICE [M][ldc] of `output`
+ * (FMM_F32 / FMM_BF16).  Requires M % m == 0, N % n == 0, call % k == 0, K % call == 0.  Copies the coefficients to the
+ * workspace and synchronises the stream once before enqueueing its kernels.                                      */
+size_t int8_finegroup_control_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N, int call);
+fmm_status int8_finegroup_control(const fmm_scheme* s, int code_bound, int second_bound, const float* d_A, int64_t lda,
+                                  const float* d_B, int64_t ldb, int64_t M, int64_t K, int64_t N, int call, int output,
+                                  void* d_C, int64_t ldc, void* d_ws, size_t ws_bytes, void* cuda_stream);
+
 /* Randomised Hadamard rotation of the inner dimension (Appendix B, "A rotation, other summation orders and repeated
  * runs": A -> A H, B -> H^T B with H orthogonal leaves A B unchanged and changes what a fast algorithm's block sums
  * round).  A pre-pass outside scheme_gemm: rotate both operands with the same h and signs, then call any product.

@@ -11,4 +11,5 @@ from .binding import (  # noqa: F401
     F32, BF16, E4M3, FLAG_REUSE_BHAT, FLAG_PRODUCTS_BF16, FLAG_SWEEP_SERIAL, FLAG_ROUND_PER_LEVEL, FLAG_SWEEP_UNFUSED, EXPORTED_SYMBOLS, profile_enable, profile_collect, PHASES,
     scheme_certificate, int8_quantize, hadamard_rotate, row_pow2_scale, row_unscale, scheme_joint_round_weights, int8_gemm_workspace, int8_gemm,
     scheme_certificate_corrected, int8_gemm_corrected_workspace, int8_gemm_corrected,
+    int8_finegroup_control_workspace, int8_finegroup_control,
 )

@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INC = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libfmm_b200.so")
-SOURCES = ["api.cu", "kernels_stream.cu", "gemm_tcgen05.cu", "noalloc.cu", "int8_path.cu", "rotate.cu", "repairs.cu", "scheme_host.cpp"]
+SOURCES = ["api.cu", "kernels_stream.cu", "gemm_tcgen05.cu", "noalloc.cu", "int8_path.cu", "int8_control.cu", "rotate.cu", "repairs.cu", "scheme_host.cpp"]
 
 
 def _newest_source_mtime() -> float:

@@ -28,7 +28,8 @@ EXPORTED_SYMBOLS = [
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
-    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected", "hadamard_rotate", "row_pow2_scale", "row_unscale",
+    "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected",
+    "int8_finegroup_control_workspace", "int8_finegroup_control", "hadamard_rotate", "row_pow2_scale", "row_unscale",
     "scheme_joint_round_weights",
     "error_sweep_workspace", "error_sweep", "fmm_status_string", "fmm_launch_count", "fmm_profile_enable",
     "fmm_profile_collect",
@@ -121,6 +122,10 @@ _lib.int8_gemm_corrected_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_in
 _lib.int8_gemm_corrected_workspace.restype = _sz
 _lib.int8_gemm_corrected.argtypes = [_vp, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
                                      _vp, _sz, _vp]
+_lib.int8_finegroup_control_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64, C.c_int]
+_lib.int8_finegroup_control_workspace.restype = _sz
+_lib.int8_finegroup_control.argtypes = [_vp, C.c_int, C.c_int, _vp, C.c_int64, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_int, C.c_int, _vp, C.c_int64, _vp, _sz, _vp]
 _lib.error_sweep_workspace.argtypes = [_vp, C.POINTER(GemmDesc), C.c_int]
 _lib.error_sweep_workspace.restype = _sz
 _lib.error_sweep.argtypes = [_vp, C.c_int, C.c_int, _dp, _dp, _dp, C.POINTER(GemmDesc), _vp, _vp, _vp, _dp,
@@ -391,6 +396,22 @@ def int8_gemm_corrected(s, cA, dA, cB, dB, Cmat, ws) -> None:
     _check(_lib.int8_gemm_corrected(s.handle, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB), M, K, N, out, _ptr(Cmat),
                                     Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "int8_gemm_corrected")
+
+
+def int8_finegroup_control_workspace(s, M: int, K: int, N: int, call: int = 128) -> int:
+    return int(_lib.int8_finegroup_control_workspace(s.handle, M, K, N, call))
+
+
+def int8_finegroup_control(s, A, B, Cmat, ws, code_bound: int = 31, second_bound: int = 127, call: int = 128) -> None:
+    """The control that breaks condition (iii): fine-group scales (call / k indices) under calls of `call` indices, every
+    mixed block sum rounded again with one scale.  A [M, K], B [N, K]: fp32 CUDA tensors; Cmat [M, N] fp32 or bf16."""
+    import torch
+    M, K = A.shape
+    N = B.shape[0]
+    out = F32 if Cmat.dtype == torch.float32 else BF16
+    _check(_lib.int8_finegroup_control(s.handle, code_bound, second_bound, _ptr(A), A.stride(0), _ptr(B), B.stride(0), M, K, N,
+                                       call, out, _ptr(Cmat), Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(),
+                                       _stream()), "int8_finegroup_control")
 
 
 def error_sweep(base: Scheme, level: int, P, Q, S, d: GemmDesc, A, B, ws, Cstar=None):

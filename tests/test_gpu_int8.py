@@ -209,3 +209,45 @@ def test_overflow_corrected_full_range_codes(M, K, N):
     with pytest.raises(lib.FmmError) as ei:
         _gemm(lib, s2, 127, cA, dA, cB, dB)
     assert ei.value.code == 10
+
+
+def test_fine_group_control_on_the_device():
+    """Section 4.2, the control that breaks condition (iii) (scales on groups of 32 under a call of 128): the device's
+    result is the oracle's bit for bit, and with one token row replaced at a time by a loud one every one of the 496
+    (earlier, later) pairs moves — beside 0 for the certified call (test_row_locality...) and 48 for FP8 block sums."""
+    lib = fmm()
+    s1 = lib.scheme_builtin("strassen222")
+    s2 = lib.scheme_kron(s1, s1)
+    o2 = S2
+    A = gen.to_storage(gen.normal(6, 1, (32, 128)), "f32")[1]
+    Bt = gen.to_storage(gen.normal(6, 2, (32, 128)), "f32")[1]
+    Bd = torch.from_numpy(Bt).float().cuda()
+    ws = workspace(lib.int8_finegroup_control_workspace(s2, 32, 128, 32, 128))
+
+    def run(X):
+        C = torch.empty((32, 32), dtype=torch.float32, device="cuda")
+        lib.int8_finegroup_control(s2, torch.from_numpy(X).float().cuda(), Bd, C, ws)
+        return C.double().cpu().numpy()
+
+    cB, dB = oracle.quantize_rows(Bt, 31, g=32)
+    cA, dA = oracle.quantize_rows(A, 31, g=32)
+    assert np.array_equal(run(A), oracle.int8_finegroup_control(o2, cA, dA, cB, dB, call=128, od="f32"))
+    base = run(A)
+    moved = 0
+    for later in range(32):
+        A2 = A.copy()
+        A2[later] = gen.to_storage(gen.normal(77, 900 + later, (128,), std=4.0), "f32")[1]
+        out = run(A2)
+        moved += sum(int(np.any(out[e] != base[e])) for e in range(later))
+    assert moved == 496
+    # two calls along K, bf16 output, one level of Strassen (fine groups of 64): still the oracle's bits
+    A3 = gen.to_storage(gen.normal(8, 1, (16, 256)), "f32")[1]
+    B3 = gen.to_storage(gen.normal(8, 2, (24, 256)), "f32")[1]
+    C3 = torch.empty((16, 24), dtype=torch.bfloat16, device="cuda")
+    ws3 = workspace(lib.int8_finegroup_control_workspace(s1, 16, 256, 24, 128))
+    lib.int8_finegroup_control(s1, torch.from_numpy(A3).float().cuda(), torch.from_numpy(B3).float().cuda(), C3, ws3, code_bound=63)
+    c3a, d3a = oracle.quantize_rows(A3, 63, g=64)
+    c3b, d3b = oracle.quantize_rows(B3, 63, g=64)
+    want = oracle.int8_finegroup_control(oracle.strassen(), c3a, d3a, c3b, d3b, call=128, od="bf16")
+    assert np.array_equal(C3.double().cpu().numpy(), want)
+    assert lib.int8_finegroup_control_workspace(s2, 30, 128, 32, 128) == 0      # rows do not split into four blocks
