@@ -374,51 +374,60 @@ __global__ void __launch_bounds__(256) frob_err_kernel(const OutT* __restrict__ 
 }
 
 // ------------------------------------------------------------------------------------------
-// fp64 reference product: 64 x 64 tile per block, 4 x 4 per thread, ascending inner index
+// fp64 reference product: 128 x 128 tile per block of 256 threads, 8 x 8 outputs per thread (rows ty + 16 a,
+// columns tx + 16 b: a half-warp reads 16 consecutive doubles of the staged operands), inner index ascending,
+// one fused multiply-add per term; operands converted to fp64 when they are staged.
 // ------------------------------------------------------------------------------------------
+constexpr int kExT = 128, kExK = 16;
 template <typename T>
 __global__ void __launch_bounds__(256) exact_f64_kernel(const T* __restrict__ A, int64_t lda,
                                                         const T* __restrict__ B, int64_t ldb, int b_weight,
                                                         int64_t M, int64_t K, int64_t N, double* __restrict__ C) {
-  __shared__ double As[16][64 + 1];
-  __shared__ double Bs[16][64 + 1];
-  const int64_t m0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
+  __shared__ double As[kExK][kExT];
+  __shared__ double Bs[kExK][kExT];
+  const int64_t m0 = (int64_t)blockIdx.y * kExT, n0 = (int64_t)blockIdx.x * kExT;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  double acc[4][4] = {};
-  for (int64_t k0 = 0; k0 < K; k0 += 16) {
-    for (int i = threadIdx.x; i < 64 * 16; i += 256) {
+  double acc[8][8];
+#pragma unroll
+  for (int a = 0; a < 8; ++a)
+#pragma unroll
+    for (int b = 0; b < 8; ++b) acc[a][b] = 0.0;
+  for (int64_t k0 = 0; k0 < K; k0 += kExK) {
+    for (int i = threadIdx.x; i < kExT * kExK; i += 256) {
       {  // A tile: consecutive threads along the inner dimension
-        const int kk = i & 15, r = i >> 4;
+        const int kk = i & (kExK - 1), r = i >> 4;
         const int64_t row = m0 + r, t = k0 + kk;
         As[kk][r] = (row < M && t < K) ? (double)(float)A[row * lda + t] : 0.0;
       }
       if (b_weight) {
-        const int kk = i & 15, c = i >> 4;
+        const int kk = i & (kExK - 1), c = i >> 4;
         const int64_t col = n0 + c, t = k0 + kk;
         Bs[kk][c] = (col < N && t < K) ? (double)(float)B[col * ldb + t] : 0.0;
       } else {
-        const int c = i & 63, kk = i >> 6;
+        const int c = i & (kExT - 1), kk = i >> 7;
         const int64_t col = n0 + c, t = k0 + kk;
         Bs[kk][c] = (col < N && t < K) ? (double)(float)B[t * ldb + col] : 0.0;
       }
     }
     __syncthreads();
 #pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
-      double a[4], b[4];
+    for (int kk = 0; kk < kExK; ++kk) {
+      double a[8], b[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+      for (int x = 0; x < 8; ++x) { a[x] = As[kk][ty + 16 * x]; b[x] = Bs[kk][tx + 16 * x]; }
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int x = 0; x < 8; ++x)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+        for (int y = 0; y < 8; ++y) acc[x][y] = fma(a[x], b[y], acc[x][y]);
     }
     __syncthreads();
   }
-  for (int i = 0; i < 4; ++i)
-    for (int j = 0; j < 4; ++j) {
-      const int64_t row = m0 + ty * 4 + i, col = n0 + tx * 4 + j;
-      if (row < M && col < N) C[row * N + col] = acc[i][j];
+#pragma unroll
+  for (int x = 0; x < 8; ++x)
+#pragma unroll
+    for (int y = 0; y < 8; ++y) {
+      const int64_t row = m0 + ty + 16 * x, col = n0 + tx + 16 * y;
+      if (row < M && col < N) C[row * N + col] = acc[x][y];
     }
 }
 
@@ -639,7 +648,7 @@ cudaError_t launch_frob_err_fixed_grid(int output, const void* C, int64_t ldc, c
 
 cudaError_t launch_exact_f64(int storage, const void* A, int64_t lda, const void* B, int64_t ldb,
                              int b_weight_layout, int64_t M, int64_t K, int64_t N, double* C, cudaStream_t st) {
-  dim3 grid((unsigned)((N + 63) / 64), (unsigned)((M + 63) / 64));
+  dim3 grid((unsigned)((N + kExT - 1) / kExT), (unsigned)((M + kExT - 1) / kExT));
   if (storage == FMM_F32)
     exact_f64_kernel<float><<<grid, 256, 0, st>>>((const float*)A, lda, (const float*)B, ldb, b_weight_layout, M, K, N, C);
   else if (storage == FMM_BF16)
