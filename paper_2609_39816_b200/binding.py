@@ -28,6 +28,7 @@ EXPORTED_SYMBOLS = [
     "fmm_selftest_timeout", "classical_gemm_workspace",
     "classical_gemm", "exact_gemm_f64", "error_frobenius_workspace", "error_frobenius", "error_frobenius_noalloc",
     "error_frobenius_noalloc_max_elements", "scheme_certificate", "int8_quantize", "int8_gemm_workspace", "int8_gemm",
+    "int8_gemm_materialised_workspace", "int8_gemm_materialised",
     "scheme_certificate_corrected", "int8_gemm_corrected_workspace", "int8_gemm_corrected",
     "int8_finegroup_control_workspace", "int8_finegroup_control", "hadamard_rotate", "row_pow2_scale", "row_unscale",
     "scheme_joint_round_weights",
@@ -114,6 +115,10 @@ _lib.scheme_joint_round_weights.argtypes = [_vp, C.POINTER(GemmDesc), _vp, C.c_i
 _lib.int8_quantize.argtypes = [_vp, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, _vp, _vp]
 _lib.int8_gemm_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
 _lib.int8_gemm_workspace.restype = _sz
+_lib.int8_gemm_materialised_workspace.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64]
+_lib.int8_gemm_materialised_workspace.restype = _sz
+_lib.int8_gemm_materialised.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
+                                        _vp, _sz, _vp]
 _lib.int8_gemm.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, _vp, C.c_int64,
                            _vp, _sz, _vp]
 _lib.scheme_certificate_corrected.argtypes = [_vp, C.c_int, _dp]
@@ -173,7 +178,7 @@ class Scheme:
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
+        if h and _lib is not None:      # at interpreter shutdown the module's globals may already be gone
             _lib.scheme_free(h)
 
     @property
@@ -374,6 +379,21 @@ def int8_gemm(s, code_bound: int, cA, dA, cB, dB, Cmat, ws) -> None:
     _check(_lib.int8_gemm(s.handle if s is not None else None, code_bound, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB), M, K, N,
                           out, _ptr(Cmat), Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "int8_gemm")
+
+
+def int8_gemm_materialised_workspace(s, M: int, K: int, N: int) -> int:
+    return int(_lib.int8_gemm_materialised_workspace(s.handle if s is not None else None, M, K, N))
+
+
+def int8_gemm_materialised(s, code_bound: int, cA, dA, cB, dB, Cmat, ws) -> None:
+    """The same operator as int8_gemm through the pipeline that writes every per-group block product to memory."""
+    import torch
+    M, K = cA.shape
+    N = cB.shape[0]
+    out = F32 if Cmat.dtype == torch.float32 else BF16
+    _check(_lib.int8_gemm_materialised(s.handle if s is not None else None, code_bound, _ptr(cA), _ptr(dA), _ptr(cB), _ptr(dB),
+                                       M, K, N, out, _ptr(Cmat), Cmat.stride(0), _ptr(ws), ws.numel() * ws.element_size(),
+                                       _stream()), "int8_gemm_materialised")
 
 
 def scheme_certificate_corrected(s, h: int):

@@ -1391,6 +1391,8 @@ fp8_group_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
   }
 }
 
+#include "int8_certified.inc"
+
 }  // namespace
 
 fmm_status launch_fp8_group_gemm(const Fp8GroupArgs& a, cudaStream_t st) {
@@ -1448,6 +1450,48 @@ fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const floa
   int8_group_gemm_kernel<<<grid, kInt8Threads, L::kTotal, st>>>(ma, mb, C, p, status);
   ++fmm_launch_counter();
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+fmm_status launch_int8_certified(const Int8CertArgs& a, cudaStream_t st) {
+  using L = CertLayout;
+  if (a.h != 32 && a.h != 64 && a.h != 128) return FMM_ERR_SHAPE;
+  if (a.m * a.n > L::kMaxBlocks || a.R > FMM_MAX_R || a.n_entries > L::kMaxEntries) return FMM_ERR_LIMIT;
+  if (a.bm * a.G > 0x7fffffff || a.bn * a.G > 0x7fffffff || a.M > 0x7fffffff || a.N > 0x7fffffff) return FMM_ERR_SHAPE;
+  const int per = BKB / a.h;
+  const int row_stages = (a.R + per - 1) / per;
+  CUtensorMap ma, mb;
+  if (!make_operand_map(&ma, true, a.Ahat, a.bm * a.G, BKB, BKB, a.bm * a.G * BKB, row_stages, BM)) return FMM_ERR_CUDA;
+  if (!make_operand_map(&mb, true, a.Bhat, a.bn * a.G, BKB, BKB, a.bn * a.G * BKB, row_stages, L::BN)) return FMM_ERR_CUDA;
+  CertParams p{};
+  p.M = (int)a.M; p.N = (int)a.N; p.m = a.m; p.n = a.n; p.bm = (int)a.bm; p.bn = (int)a.bn;
+  p.G = a.G; p.R = a.R; p.h = a.h; p.per = per; p.ksteps = a.h / UMMA_KB;
+  int8_certified_passes(a.R, per, &p.passes, &p.pass_len);
+  p.tiles_m = (int)((a.bm + BM - 1) / BM);
+  p.tiles_n = (int)((a.bn + L::BN - 1) / L::BN);
+  p.ldc = a.ldc; p.out_bf16 = a.output == FMM_BF16;
+  p.dAt = a.dAt; p.dBt = a.dBt;
+  p.entries = a.d_entries; p.pass_off = a.d_pass_off; p.owned = a.d_owned; p.n_entries = a.n_entries;
+  p.wait_limit_ns = kDefaultWaitLimitNs;
+  const long long total = (long long)p.tiles_m * p.tiles_n;
+  if (total <= 0) return FMM_OK;
+  const int sms = sm_count();
+  if (sms <= 0) return FMM_ERR_CUDA;
+  const int grid = (int)(total < sms ? total : sms);
+  static unsigned long long smem_ok = 0;
+  if (fmm_allow_dynamic_smem(int8_certified_kernel, L::kTotal, &smem_ok) != cudaSuccess) return FMM_ERR_CUDA;
+  int8_certified_kernel<<<grid, kCertThreads, L::kTotal, st>>>(ma, mb, a.C, p, a.status);
+  ++fmm_launch_counter();
+  return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
+}
+
+// The R products of a group go through TMEM in ceil(R / kPass) passes of equal length (a multiple of the products per
+// ring stage), the last one taking the remainder, when that fits a buffer; otherwise in passes of kPass.
+void int8_certified_passes(int R, int per, int* passes, int* pass_len) {
+  const int n = (R + CertLayout::kPass - 1) / CertLayout::kPass;
+  int len = R / n / per * per;
+  if (len == 0 || R - len * (n - 1) > CertLayout::kPass) len = CertLayout::kPass;
+  *passes = n;
+  *pass_len = len;
 }
 
 fmm_status launch_block_products(const BlockProductArgs& a, cudaStream_t st) {

@@ -17,6 +17,8 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <memory>
+#include <vector>
 
 #include "fmm_internal.h"
 #include "kernels_stream.cuh"
@@ -372,6 +374,72 @@ cudaError_t launch_encode_split(const int8_t* codes, int64_t K, int gr, int gc, 
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// Block sums of int8 codes as int8 (certificate (i): |sum| <= 127), packed for the one-kernel certified realisation:
+// rows of 128 bytes that hold per = 128 / h products side by side, product r at byte (r % per) * h of row
+// (group, p) of slab r / per.  One thread forms, for one (group, row position) and four consecutive inner indices t,
+// the sums of every product (the same staging as encode_split_kernel).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSplitThreads)
+encode_codes_kernel(const int8_t* __restrict__ codes, int64_t K, int gc, int64_t br, int G, int h,
+                    const CoefTable* __restrict__ d_tab, int8_t* __restrict__ out, int64_t nquad) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R = d_tab->R, ncell = d_tab->ncell;
+  const int total = d_tab->off[R];
+  int* off = reinterpret_cast<int*>(smem_raw);
+  int2* ent = reinterpret_cast<int2*>(smem_raw + ((size_t)(R + 1) * 4 + 15) / 16 * 16);
+  uint32_t* stage = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(ent) + (size_t)total * 8);
+  for (int i = threadIdx.x; i <= R; i += kSplitThreads) off[i] = d_tab->off[i];
+  for (int i = threadIdx.x; i < total; i += kSplitThreads)
+    ent[i] = make_int2(d_tab->cell[i], __float2int_rn(d_tab->coef[i]));
+  stage[ncell * kSplitThreads + threadIdx.x] = 0u;                    // the padding cell
+  const int64_t idx = (int64_t)blockIdx.x * kSplitThreads + threadIdx.x;
+  const bool live = idx < nquad;
+  const int qpr = h / 4;
+  const int64_t rowp = live ? idx / qpr : 0;                          // (group, p)
+  const int t = live ? (int)(idx - rowp * qpr) * 4 : 0;
+  const int64_t g = rowp / br, p = rowp - g * br;
+  for (int c = 0; c < ncell; ++c) {
+    const int gi = c / gc, gj = c - gi * gc;
+    stage[c * kSplitThreads + threadIdx.x] =
+        live ? *reinterpret_cast<const uint32_t*>(codes + ((int64_t)gi * br + p) * K + g * kGroup + gj * h + t) : 0u;
+  }
+  __syncthreads();
+  if (!live) return;
+  const int per = kGroup / h;
+  const int64_t slab = (int64_t)G * br * kGroup;                      // bytes of one slab of `per` products
+  for (int r = 0; r < R; ++r) {
+    int s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+    for (int e = off[r]; e < off[r + 1]; ++e) {
+      const int2 en = ent[e];
+      const uint32_t wv = stage[en.x * kSplitThreads + threadIdx.x];
+      s0 += en.y * (int)(int8_t)(wv & 0xffu);
+      s1 += en.y * (int)(int8_t)((wv >> 8) & 0xffu);
+      s2 += en.y * (int)(int8_t)((wv >> 16) & 0xffu);
+      s3 += en.y * (int)(int8_t)(wv >> 24);
+    }
+    const uint32_t packed = ((uint32_t)s0 & 0xffu) | (((uint32_t)s1 & 0xffu) << 8) | (((uint32_t)s2 & 0xffu) << 16) |
+                            (((uint32_t)s3 & 0xffu) << 24);
+    *reinterpret_cast<uint32_t*>(out + (r / per) * slab + rowp * kGroup + (r % per) * h + t) = packed;
+  }
+}
+
+cudaError_t launch_encode_codes(const int8_t* codes, int64_t K, int gr, int gc, int64_t br, int G, int h,
+                                const CoefTable* d_tab, const CoefTable* h_tab, int8_t* out, cudaStream_t st) {
+  const int64_t nquad = (int64_t)G * br * (h / 4);
+  const size_t smem = ((size_t)(h_tab->R + 1) * 4 + 15) / 16 * 16 + (size_t)h_tab->off[h_tab->R] * 8 +
+                      (size_t)(gr * gc + 1) * kSplitThreads * 4;
+  if (smem > 96 * 1024) return cudaErrorInvalidValue;
+  static unsigned long long smem_ok = 0;
+  cudaError_t e = fmm_allow_dynamic_smem(encode_codes_kernel, 96 * 1024, &smem_ok);
+  if (e != cudaSuccess) return e;
+  const int64_t grid = (nquad + kSplitThreads - 1) / kSplitThreads;
+  if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
+  encode_codes_kernel<<<(unsigned)grid, kSplitThreads, smem, st>>>(codes, K, gc, br, G, h, d_tab, out, nquad);
+  ++fmm_launch_counter();
+  return cudaGetLastError();
+}
+
 int padded_total(const CoefTable& t) { return t.off[t.R]; }
 
 template <typename OutT, int kSplit, int kStages, int kCells, bool kIntAcc = false>
@@ -441,6 +509,12 @@ struct Int8Layout {
   bool trivial;
 };
 
+// Workspace of the one-kernel certified realisation
+struct CertWs {
+  size_t status, tabA, tabB, entries, pass_off, owned, dAt, dBt, ahat, bhat, total;
+  size_t max_entries;
+};
+
 // the classical algorithm <1,1,1;1> as a scheme
 struct TrivialScheme : fmm_scheme {
   TrivialScheme() {
@@ -457,6 +531,27 @@ fmm_status int8_shape_ok(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
   if ((N / s.n) % 8) return FMM_ERR_SHAPE;
   if (M * (K / kGroup) > 0x7fffffffLL / 2 || N * (K / kGroup) > 0x7fffffffLL / 2) return FMM_ERR_SHAPE;
   return FMM_OK;
+}
+
+CertWs cert_layout(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
+  CertWs L{};
+  const int G = (int)(K / kGroup), h = kGroup / s.k, per = kGroup / h;
+  const int64_t bm = M / s.m, bn = N / s.n;
+  const int slabs = (s.R + per - 1) / per;
+  L.max_entries = (size_t)s.R * s.m * s.n;
+  size_t o = 0;
+  L.status = o; o += align_up(sizeof(DeviceStatus));
+  L.tabA = o; o += align_up(sizeof(CoefTable));
+  L.tabB = o; o += align_up(sizeof(CoefTable));
+  L.entries = o; o += align_up(L.max_entries * 8);
+  L.pass_off = o; o += align_up((size_t)(FMM_MAX_R + 1) * FMM_MAX_GRID * FMM_MAX_GRID * 4);
+  L.owned = o; o += align_up(FMM_MAX_GRID * FMM_MAX_GRID * 4);
+  L.dAt = o; o += align_up((size_t)M * G * 4);
+  L.dBt = o; o += align_up((size_t)N * G * 4);
+  L.ahat = o; o += align_up((size_t)slabs * G * bm * kGroup + 128 * kGroup);   // + one tile of rows: boxes may read past the end
+  L.bhat = o; o += align_up((size_t)slabs * G * bn * kGroup + 128 * kGroup);
+  L.total = o;
+  return L;
 }
 
 Int8Layout int8_layout(const fmm_scheme& s, int64_t M, int64_t K, int64_t N) {
@@ -615,7 +710,90 @@ size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N)
   const fmm_scheme& sc = s ? *s : one;
   if (int8_shape_ok(sc, M, K, N) != FMM_OK) return 0;
   if (!s) return fused_layout(M, K, N).total;
+  return cert_layout(sc, M, K, N).total;
+}
+
+size_t int8_gemm_materialised_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N) {
+  TrivialScheme one;
+  const fmm_scheme& sc = s ? *s : one;
+  if (int8_shape_ok(sc, M, K, N) != FMM_OK) return 0;
   return int8_layout(sc, M, K, N).total;
+}
+
+// The certified realisation in one kernel: block sums of the codes as int8 (two launches), scales transposed to
+// group-major (two launches), then int8_certified_kernel.
+static fmm_status int8_certified_one_kernel(const fmm_scheme& sc, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
+                                            const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C,
+                                            int64_t ldc, void* d_ws, size_t ws_bytes, cudaStream_t st) {
+  const CertWs L = cert_layout(sc, M, K, N);
+  if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(d_cA) % 4) || (reinterpret_cast<uintptr_t>(d_cB) % 4)) return FMM_ERR_SHAPE;
+  const int64_t bm = M / sc.m, bn = N / sc.n;
+  const int h = kGroup / sc.k, G = (int)(K / kGroup);
+  FMM_CUDA(cudaMemsetAsync(at<char>(d_ws, L.status), 0, sizeof(DeviceStatus), st));
+  std::unique_ptr<CoefTable> hA(new CoefTable), hB(new CoefTable);
+  std::memset(hA.get(), 0, sizeof(CoefTable)); std::memset(hB.get(), 0, sizeof(CoefTable));
+  fmm_build_tables(sc, hA.get(), hB.get(), nullptr);
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabA), hA.get(), sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.tabB), hB.get(), sizeof(CoefTable), cudaMemcpyHostToDevice, st));
+  // Decode lists.  Every block of C is owned by one of four decode warps (per TMEM lane quarter); the blocks are dealt
+  // out longest list first to the warp with the least work so far that still has a free slot.  The lists are then laid
+  // out by (warp, pass of products, owned block, ascending r); an entry is (TMEM column of the product inside its
+  // pass, integer w).
+  const int blocks = sc.m * sc.n;
+  int passes = 0, pass = 0;
+  int8_certified_passes(sc.R, kGroup / h, &passes, &pass);
+  constexpr int kParts = 4, kOwn = FMM_MAX_GRID * FMM_MAX_GRID / kParts, kBN = 16;
+  std::vector<int> nnz(blocks, 0), order(blocks), owned(kParts * kOwn, -1), load(kParts, 0), used(kParts, 0);
+  for (int d = 0; d < blocks; ++d)
+    for (int r = 0; r < sc.R; ++r) nnz[d] += sc.W[(size_t)r * blocks + d] != 0.0;
+  for (int d = 0; d < blocks; ++d) order[d] = d;
+  std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return nnz[x] > nnz[y]; });
+  for (int d : order) {
+    int best = -1;
+    for (int q = 0; q < kParts; ++q)
+      if (used[q] < kOwn && (best < 0 || load[q] < load[best])) best = q;
+    owned[best * kOwn + used[best]++] = d;
+    load[best] += nnz[d];
+  }
+  std::vector<int2> ent;
+  std::vector<int> poff;
+  for (int q = 0; q < kParts; ++q)
+    for (int ps = 0; ps < passes; ++ps)
+      for (int b = 0; b < kOwn; ++b) {
+        poff.push_back((int)ent.size());
+        const int d = owned[q * kOwn + b];
+        if (d < 0) continue;
+        for (int r = ps * pass; r < (ps == passes - 1 ? sc.R : (ps + 1) * pass); ++r) {
+          const double w = sc.W[(size_t)r * blocks + d];
+          if (w != 0.0) ent.push_back(make_int2((r - ps * pass) * kBN, (int)std::lrint(w)));
+        }
+      }
+  poff.push_back((int)ent.size());
+  if (ent.size() > L.max_entries) return FMM_ERR_LIMIT;
+  if (!ent.empty())
+    FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.entries), ent.data(), ent.size() * sizeof(int2), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.pass_off), poff.data(), poff.size() * sizeof(int), cudaMemcpyHostToDevice, st));
+  FMM_CUDA(cudaMemcpyAsync(at<char>(d_ws, L.owned), owned.data(), owned.size() * sizeof(int), cudaMemcpyHostToDevice, st));
+  {
+    ProfScope ps(0, st);
+    FMM_CUDA(launch_encode_codes(d_cA, K, sc.m, sc.k, bm, G, h, at<CoefTable>(d_ws, L.tabA), hA.get(), at<int8_t>(d_ws, L.ahat), st));
+    FMM_CUDA(launch_encode_codes(d_cB, K, sc.n, sc.k, bn, G, h, at<CoefTable>(d_ws, L.tabB), hB.get(), at<int8_t>(d_ws, L.bhat), st));
+    transpose_scales_kernel<<<stream_blocks(M * G, 256), 256, 0, st>>>(d_dA, M, G, at<float>(d_ws, L.dAt));
+    ++fmm_launch_counter();
+    transpose_scales_kernel<<<stream_blocks(N * G, 256), 256, 0, st>>>(d_dB, N, G, at<float>(d_ws, L.dBt));
+    ++fmm_launch_counter();
+    FMM_CUDA(cudaGetLastError());
+  }
+  Int8CertArgs a{};
+  a.Ahat = at<int8_t>(d_ws, L.ahat); a.Bhat = at<int8_t>(d_ws, L.bhat);
+  a.m = sc.m; a.n = sc.n; a.R = sc.R; a.h = h; a.bm = bm; a.bn = bn; a.G = G; a.M = M; a.N = N;
+  a.dAt = at<float>(d_ws, L.dAt); a.dBt = at<float>(d_ws, L.dBt);
+  a.d_entries = at<int2>(d_ws, L.entries); a.d_pass_off = at<int>(d_ws, L.pass_off); a.d_owned = at<int>(d_ws, L.owned); a.n_entries = (int)ent.size();
+  a.output = output; a.C = d_C; a.ldc = ldc; a.status = at<DeviceStatus>(d_ws, L.status);
+  ProfScope ps(2, st);
+  // the host tables were copied from pageable memory: those copies are complete when cudaMemcpyAsync returns
+  return launch_int8_certified(a, st);
 }
 
 fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
@@ -634,6 +812,25 @@ fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, co
   if (!scheme_certificate(&sc, code_bound, code_bound, kGroup / sc.k, kGroup, 24, nullptr)) return FMM_ERR_CERTIFICATE;
   if (!s)   // the classical operator: one fused tensor-core kernel
     return int8_classical_fused(d_cA, d_dA, d_cB, d_dB, M, K, N, output, d_C, ldc, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
+  return int8_certified_one_kernel(sc, d_cA, d_dA, d_cB, d_dB, M, K, N, output, d_C, ldc, d_ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+// The same operator with every per-group block product written to memory (pack, encode, grouped block products with
+// bf16 operands and fp32 accumulators, grouped decode): the form the one-kernel realisation replaced, kept as an
+// independent implementation to compare against and to time.
+fmm_status int8_gemm_materialised(const fmm_scheme* s, int code_bound, const int8_t* d_cA, const float* d_dA, const int8_t* d_cB,
+                                  const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C, int64_t ldc,
+                                  void* d_ws, size_t ws_bytes, void* stream) {
+  if (!d_cA || !d_dA || !d_cB || !d_dB || !d_C) return FMM_ERR_ARG;
+  if (output != FMM_F32 && output != FMM_BF16) return FMM_ERR_DTYPE;
+  if (code_bound < 1 || code_bound > 127) return FMM_ERR_ARG;
+  TrivialScheme one;
+  const fmm_scheme& sc = s ? *s : one;
+  FMM_TRY(int8_shape_ok(sc, M, K, N));
+  const int eo = output == FMM_F32 ? 4 : 2;
+  if (ldc < N || (ldc * eo) % 16 || (reinterpret_cast<uintptr_t>(d_C) % 16)) return FMM_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(d_cA) % 8) || (reinterpret_cast<uintptr_t>(d_cB) % 8)) return FMM_ERR_SHAPE;
+  if (!scheme_certificate(&sc, code_bound, code_bound, kGroup / sc.k, kGroup, 24, nullptr)) return FMM_ERR_CERTIFICATE;
   const Int8Layout L = int8_layout(sc, M, K, N);
   if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) || ws_bytes < L.total) return FMM_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -201,6 +201,23 @@ fmm_status launch_fp8_group_gemm(const Fp8GroupArgs& a, cudaStream_t st);
 fmm_status launch_int8_group_gemm(const int8_t* cA, const int8_t* cB, const float* dAt, const float* dBt, int64_t M,
                                   int64_t K, int64_t N, int output, void* C, int64_t ldc, DeviceStatus* status, cudaStream_t st);
 
+// The certified int8 realisation in one kernel (tcgen05 kind::i8 block products of the int8 block sums, integer decode
+// and group rescale in the epilogue).  Ahat: int8 [ceil(R / per)][G * bm][128], per = 128 / h products side by side in a
+// row (product r at byte (r % per) * h of row g * bm + p of slab r / per); Bhat likewise with bn.  d_owned: [4][4], the blocks of C
+// (i * n + j, or -1) that each of the four decode warps of a TMEM lane quarter combines; d_entries: decode lists ordered
+// by (decode warp, pass, owned block, r): (TMEM column of the product inside its pass, integer w); d_pass_off: first
+// entry of every such list and one terminal element; passes as int8_certified_passes() gives them.  dAt [G][M],
+// dBt [G][N]: scales, group-major.
+struct Int8CertArgs {
+  const int8_t* Ahat; const int8_t* Bhat;
+  int m, n, R, h; int64_t bm, bn; int G; int64_t M, N;
+  const float* dAt; const float* dBt;
+  const int2* d_entries; const int* d_pass_off; const int* d_owned; int n_entries;
+  int output; void* C; int64_t ldc; DeviceStatus* status;
+};
+void int8_certified_passes(int R, int per, int* passes, int* pass_len);
+fmm_status launch_int8_certified(const Int8CertArgs& a, cudaStream_t st);
+
 // Phase timing (see fmm_profile_enable): RAII bracket of a region of the caller's stream.
 struct ProfScope {
   ProfScope(int kind, cudaStream_t st);

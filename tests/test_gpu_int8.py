@@ -33,12 +33,16 @@ def _quantize(lib, X, b):
     return codes, scales
 
 
-def _gemm(lib, s, b, cA, dA, cB, dB, out_dtype=torch.bfloat16):
+def _gemm(lib, s, b, cA, dA, cB, dB, out_dtype=torch.bfloat16, materialised=False):
     M, K = cA.shape
     N = cB.shape[0]
-    ws = workspace(lib.int8_gemm_workspace(s, M, K, N))
-    C = torch.empty((M, N), dtype=out_dtype, device="cuda")
-    lib.int8_gemm(s, b, cA, dA, cB, dB, C, ws)
+    C = torch.full((M, N), float("nan"), dtype=out_dtype, device="cuda")
+    if materialised:
+        ws = workspace(lib.int8_gemm_materialised_workspace(s, M, K, N))
+        lib.int8_gemm_materialised(s, b, cA, dA, cB, dB, C, ws)
+    else:
+        ws = workspace(lib.int8_gemm_workspace(s, M, K, N))
+        lib.int8_gemm(s, b, cA, dA, cB, dB, C, ws)
     lib.device_status(ws)
     return C.to(torch.float64).cpu().numpy()
 
@@ -57,7 +61,7 @@ def test_quantiser_bit_exact(dtype, b):
     assert np.abs(oc).max() == b and od[3, 1] == 1.0
 
 
-@pytest.mark.parametrize("M,K,N", [(32, 128, 32), (512, 1024, 544), (200, 384, 96)])
+@pytest.mark.parametrize("M,K,N", [(32, 128, 32), (512, 1024, 544), (200, 384, 96), (1040, 256, 2080), (4, 128, 32)])
 def test_classical_and_certified_match_oracle_and_each_other(M, K, N):
     """Same bits from the classical int8 operator, the certified two-level realisation and the oracle."""
     lib = fmm()
@@ -70,10 +74,18 @@ def test_classical_and_certified_match_oracle_and_each_other(M, K, N):
     got_cl = _gemm(lib, None, 31, cA, dA, cB, dB)          # one fused kernel: int8 MMAs, rescale in the epilogue
     assert np.array_equal(got_cl, want)
     one = lib.scheme_load(np.ones((1, 1, 1)), np.ones((1, 1, 1)), np.ones((1, 1, 1)))
-    assert np.array_equal(_gemm(lib, one, 31, cA, dA, cB, dB), want)   # <1,1,1;1> through the materialised pipeline
+    assert np.array_equal(_gemm(lib, one, 31, cA, dA, cB, dB), want)   # <1,1,1;1> through the one-kernel certified path
+    assert np.array_equal(_gemm(lib, one, 31, cA, dA, cB, dB, materialised=True), want)   # and through the materialised pipeline
     s2 = _lib_scheme(lib, S2)
-    got = _gemm(lib, s2, 31, cA, dA, cB, dB)
+    got = _gemm(lib, s2, 31, cA, dA, cB, dB)              # one kernel: 49 int8 products per position in tensor memory
     assert np.array_equal(got, want)
+    assert np.array_equal(_gemm(lib, s2, 31, cA, dA, cB, dB, materialised=True), want)    # every product written to memory
+    if M % 2 == 0:
+        s1 = _lib_scheme(lib, S1)                         # one level: blocks of 64 inner indices, two products per row
+        cA6, dA6 = _quantize(lib, At, 63)
+        cB6, dB6 = _quantize(lib, Bt, 63)
+        ref6 = _gemm(lib, None, 63, cA6, dA6, cB6, dB6)
+        assert np.array_equal(_gemm(lib, s1, 63, cA6, dA6, cB6, dB6), ref6)
     want_cert, mx = oracle.int8_certified(S2, oA, odA, oB, odB)
     assert np.array_equal(want_cert, want) and mx[0] <= 124 and mx[1] <= 124
     # fp32 output: the accumulated value itself, before the cast
