@@ -357,17 +357,16 @@ size_t int8_gemm_workspace(const fmm_scheme* s, int64_t M, int64_t K, int64_t N)
  * computed by one call of s on the group's 128 inner indices split into k blocks of length 128/k (which must be 32,
  * 64 or 128), rows into m and columns into n contiguous blocks — also in one kernel (Figure 3): the block sums of the
  * codes are formed as int8 (certificate (i): they fit), a CTA owns 128 row positions and 16 column positions of every
- * C block, multiplies the R pairs of block sums on the tensor cores (kind::i8, int32 accumulators, one per product, all
- * resident in tensor memory), combines them with the integer w, and applies the group's two scales — no block product
- * leaves the SM.  When the certificate holds the output is bit-identical to the classical operator's for every such s.
+ * C block, multiplies the R pairs of block sums on the tensor cores (kind::i8, one int32 accumulator per product in
+ * tensor memory, at most 16 products at a time), combines them with the integer w, and applies the group's two scales —
+ * no block product leaves the SM.  When the certificate holds the output is bit-identical to the classical operator's for every such s.
  * Returns FMM_ERR_CERTIFICATE, launching nothing, if scheme_certificate(s, code_bound, code_bound, 128/k, 128,
  * 24) fails; the caller vouches that |code| <= code_bound.  Requires M % m == 0, N % n == 0, (N/n) % 8 == 0,
  * K % 128 == 0.  d_ws: DEVICE, >= int8_gemm_workspace bytes, 256-byte aligned; it holds a status word that
  * fmm_device_status reads.  Asynchronous on the stream.
  * int8_gemm_materialised: the same operator with every per-group block product written to memory (pack, encode,
  * grouped block products on bf16 copies of the integers with fp32 accumulators, grouped decode) — an independent
- * implementation of the same bits, an order of magnitude slower at layer sizes (its workspace holds R * K/128 fp32
- * blocks); s == NULL runs the classical algorithm through that pipeline.                                       */
+ * implementation of the same bits, twice as slow at layer sizes and with a workspace of R * K/128 fp32 blocks; s == NULL runs the classical algorithm through that pipeline.                                       */
 fmm_status int8_gemm(const fmm_scheme* s, int code_bound, const int8_t* d_cA, const float* d_dA,
                      const int8_t* d_cB, const float* d_dB, int64_t M, int64_t K, int64_t N, int output, void* d_C,
                      int64_t ldc, void* d_ws, size_t ws_bytes, void* cuda_stream);
