@@ -220,6 +220,14 @@ def test_certificate_on_host_matches_oracle(lib):
     assert lib.int8_gemm_workspace(s2, 64, 100, 64) == 0          # K not a multiple of 128
     assert lib.int8_gemm_workspace(s2, 66, 128, 64) == 0          # M not divisible by m
     assert lib.int8_gemm_workspace(s2, 64, 128, 64) > 0
+    # the one-kernel realisation keeps int8 block sums (49 / 16 of an operand per side), the materialised form every
+    # per-group fp32 product: R * K/128 blocks of bm x bn
+    one = lib.int8_gemm_workspace(s2, 4096, 4096, 4096)
+    mat = lib.int8_gemm_materialised_workspace(s2, 4096, 4096, 4096)
+    sums = 2 * 13 * 32 * 1024 * 128                                # slabs of four products x groups x block rows x 128 bytes
+    assert sums <= one <= sums + (4 << 20)
+    assert mat >= 49 * 32 * 1024 * 1024 * 4
+    assert lib.int8_gemm_materialised_workspace(s2, 64, 100, 64) == 0
 
 
 def test_corrected_certificate_constants(lib):
