@@ -115,6 +115,30 @@ def test_sign_variants_and_one_level_are_bit_identical():
     assert len(outs) == 2                     # b = 31 and b = 63 are different operators
 
 
+def test_integer_weights_other_than_unit_and_undivided_groups():
+    """Algorithms that the unit-weight fast path of the decode does not cover: <1,1,1;2> with C = 2 M1 - M2 (both
+    products the plain one: k = 1, so a call spans the undivided group, h = 128, four MMAs per product) and Strassen
+    with its first product doubled up as 2 M1 - M1' (R = 8, a weight of 2 and an extra product in two decode lists)."""
+    lib = fmm()
+    M, K, N = 200, 384, 96
+    At, A, Bt, B = _inputs(61, M, K, N)
+    one = oracle.Scheme(np.ones((2, 1, 1)), np.ones((2, 1, 1)), np.array([2.0, -1.0]).reshape(2, 1, 1))
+    U = np.concatenate([S1.U, S1.U[:1]]); V = np.concatenate([S1.V, S1.V[:1]])
+    W = np.concatenate([S1.W, -S1.W[:1]]); W[0] *= 2.0
+    dup = oracle.Scheme(U, V, W)
+    for o, b in ((one, 31), (dup, 31)):
+        assert oracle.brent_residual(o) == 0.0
+        cA, dA = _quantize(lib, At, b)
+        cB, dB = _quantize(lib, Bt, b)
+        ref = _gemm(lib, None, b, cA, dA, cB, dB, torch.float32)
+        s = _lib_scheme(lib, o)
+        assert np.array_equal(_gemm(lib, s, b, cA, dA, cB, dB, torch.float32), ref)
+        assert np.array_equal(_gemm(lib, s, b, cA, dA, cB, dB, torch.float32, materialised=True), ref)
+        oA, odA = oracle.quantize_rows(A, b)
+        oB, odB = oracle.quantize_rows(B, b)
+        assert np.array_equal(ref, oracle.int8_classical(oA, odA, oB, odB, od="f32"))
+
+
 def test_certificate_is_enforced():
     lib = fmm()
     M, K, N = 32, 128, 32
