@@ -56,6 +56,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
+// one lane of a converged warp, chosen by the hardware: lets the whole warp run a role's loop with warp-uniform control
+// flow (so that loop state and descriptors can live in uniform registers) while a single lane issues
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -563,7 +571,8 @@ __device__ __forceinline__ void pair_roles(const int warp, const int lane, const
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && leader) {
+    // all 32 lanes run the loop with warp-uniform control flow; one elected lane issues the MMAs and the commits
+    if (leader) {
       // M = 256 across the pair, N = 256
       constexpr uint32_t idesc = (1u << 4) | ((kFp8 ? 0u : 1u) << 7) | ((kFp8 ? 0u : 1u) << 10) |
                                  ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
@@ -573,29 +582,33 @@ __device__ __forceinline__ void pair_roles(const int warp, const int lane, const
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = pair_id; tile < total_tiles && ok; tile += num_pairs) {
-        ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status, tp.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 0x12, status, tp.wait_limit_ns));
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status, tp.wait_limit_ns);
+          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag, 0x11, status, tp.wait_limit_ns));
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = make_smem_desc(sa);
           const uint64_t db = make_smem_desc(sa + L::kABytes);
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BKB / UMMA_KB; ++k)
-            tc_mma_pair<kFp8>(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc,
-                              (kb | k) != 0 ? 1u : 0u);
-          tc_commit_pair(empty_bar(stage));   // frees this stage in both CTAs
+            for (int k = 0; k < BKB / UMMA_KB; ++k)
+              tc_mma_pair<kFp8>(d_tmem, da + (uint64_t)(k * (UMMA_KB >> 4)), db + (uint64_t)(k * (UMMA_KB >> 4)), idesc,
+                                (kb | k) != 0 ? 1u : 0u);
+            tc_commit_pair(empty_bar(stage));   // frees this stage in both CTAs
+          }
+          __syncwarp();
           if (++stage == L::kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit_pair(tfull_bar(acc));       // accumulator complete, visible to both epilogues
+        if (elect_one()) tc_commit_pair(tfull_bar(acc));       // accumulator complete, visible to both epilogues
+        __syncwarp();
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(drain_bar)
                      : "memory");
         const unsigned long long t0 = global_timer_ns();
