@@ -1497,6 +1497,9 @@ fmm_status launch_int8_certified(const Int8CertArgs& a, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? FMM_OK : FMM_ERR_CUDA;
 }
 
+int int8_certified_tile_columns() { return CertLayout::BN; }
+int int8_certified_decode_warps() { return CertLayout::kParts; }
+
 // The R products of a group go through TMEM in ceil(R / kPass) passes of equal length (a multiple of the products per
 // ring stage), the last one taking the remainder, when that fits a buffer; otherwise in passes of kPass.
 void int8_certified_passes(int R, int per, int* passes, int* pass_len) {

@@ -743,7 +743,7 @@ static fmm_status int8_certified_one_kernel(const fmm_scheme& sc, const int8_t* 
   const int blocks = sc.m * sc.n;
   int passes = 0, pass = 0;
   int8_certified_passes(sc.R, kGroup / h, &passes, &pass);
-  constexpr int kParts = 4, kOwn = FMM_MAX_GRID * FMM_MAX_GRID / kParts, kBN = 16;
+  const int kParts = int8_certified_decode_warps(), kOwn = FMM_MAX_GRID * FMM_MAX_GRID / kParts, kBN = int8_certified_tile_columns();
   std::vector<int> nnz(blocks, 0), order(blocks), owned(kParts * kOwn, -1), load(kParts, 0), used(kParts, 0);
   for (int d = 0; d < blocks; ++d)
     for (int r = 0; r < sc.R; ++r) nnz[d] += sc.W[(size_t)r * blocks + d] != 0.0;

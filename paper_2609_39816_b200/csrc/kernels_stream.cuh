@@ -216,6 +216,8 @@ struct Int8CertArgs {
   int output; void* C; int64_t ldc; DeviceStatus* status;
 };
 void int8_certified_passes(int R, int per, int* passes, int* pass_len);
+int int8_certified_tile_columns();   // columns of a tile per block of C = TMEM columns of one product
+int int8_certified_decode_warps();   // decode warps per TMEM lane quarter (each owns 16 / that many blocks of C)
 fmm_status launch_int8_certified(const Int8CertArgs& a, cudaStream_t st);
 
 // Phase timing (see fmm_profile_enable): RAII bracket of a region of the caller's stream.
